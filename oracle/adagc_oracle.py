@@ -1,0 +1,184 @@
+"""CPU oracle for AdamW with AdaGC (Algorithm 1 of the paper; Eq. 2 and Eq. 3).
+
+TEST INFRASTRUCTURE ONLY.  This is a plain, slow, float64 restatement of the
+paper's algorithm used to check the CUDA library.  It shares no code with the
+CUDA path and is never a fallback for it: only the tests, the smoke check and
+the benchmark's CPU-baseline leg may import it.
+
+Every function takes the steps of Algorithm 1 in the paper's order and notation:
+
+    g_t,i      gradient of tensor i at step t (t is 1-based: the first call is t = 1)
+    gamma_i    EMA of the clipped gradient norm of tensor i (one fp32 per tensor,
+               Section 4.3 "Memory")
+    h_t,i      clip factor, hat(g) = h * g
+    m, v       AdamW moments, theta the parameters
+
+Readings taken where the paper is silent or ambiguous (listed in the design notes):
+  * warm-up covers exactly T_start steps: steps 1..T_start use global-norm
+    clipping (Eq. 2), step T_start+1 is the first per-tensor AdaGC step (Eq. 3);
+  * the warm-up EMA seed uses the globally *clipped* per-tensor norm
+    (Algorithm 1 writes the hatted gradient there);
+  * at t = 1 the incoming gamma is ignored: gamma_0,i = ||hat(g)_1,i||;
+    with T_start = 0 the first step seeds gamma_0,i = ||g_1,i|| and then applies Eq. 3;
+  * the clip is active only when ||g|| > lambda_rel * gamma (strict), and the
+    clipped norm that enters the EMA is then lambda_rel * gamma itself
+    (Section 4.2: the clip "scales the gradient norm to" that value);
+  * stored state (gamma, theta, m, v) is rounded to its storage dtype after every
+    step ("storage" mode, the parity reference); `state_dtype=np.float64` keeps
+    everything in float64 for invariant tests.
+
+Parity pins: tests/test_oracle_pins.py (closed forms, library special cases,
+hand-worked example, invariants, brute force).
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+
+@dataclass
+class Hyper:
+    """The 'given' line of Algorithm 1 (eta_t is passed per step as `lr`)."""
+    lr: float = 3e-4
+    beta1: float = 0.9
+    beta2: float = 0.95
+    eps: float = 1e-8
+    wd: float = 0.1          # lambda_w
+    lambda_rel: float = 1.04
+    beta: float = 0.99
+    lambda_abs: float = 1.0
+    warmup: int = 100        # T_start
+
+
+@dataclass
+class ClipResult:
+    norm: np.ndarray      # ||g_t,i||                       float64 [T]
+    h: np.ndarray         # clip factor h_t,i               float64 [T]
+    flag: np.ndarray      # clip active                     bool    [T]
+    clipped: np.ndarray   # ||hat(g)_t,i||                  float64 [T]
+    gamma: np.ndarray     # gamma_t,i in the state dtype    [T]
+    global_norm: float    # ||g_t|| (Eq. 2), always reported
+    margin: np.ndarray    # |norm - threshold| / threshold of every decision (inf where threshold is 0)
+
+
+def sumsq(g: np.ndarray) -> float:
+    """sum_j g_j^2 of one tensor in float64 (the square of the norm in Eq. 3)."""
+    x = np.asarray(g, dtype=np.float64).ravel()
+    return float(np.sum(x * x))
+
+
+def l2_norm(g: np.ndarray) -> float:
+    return math.sqrt(sumsq(g))
+
+
+def clip_decisions(s: Sequence[float], gamma_prev: np.ndarray, step: int, hp: Hyper,
+                   state_dtype=np.float32) -> ClipResult:
+    """Clip factors, flags and the EMA update for one step, from per-tensor sums of squares.
+
+    Warm-up branch: Eq. 2 and the min-seeding line of Algorithm 1.
+    AdaGC branch:   Eq. 3 and the gamma update of Algorithm 1.
+    """
+    s = np.asarray(s, dtype=np.float64)
+    T = s.shape[0]
+    n = np.sqrt(s)                                         # ||g_t,i||
+    G = math.sqrt(float(np.sum(s)))                        # ||g_t|| over all tensors
+    h = np.ones(T, dtype=np.float64)
+    flag = np.zeros(T, dtype=bool)
+    c = np.empty(T, dtype=np.float64)
+    margin = np.full(T, np.inf)
+    gam = np.asarray(gamma_prev).astype(state_dtype).astype(np.float64)
+    if step < 1:
+        raise ValueError("step is 1-based")
+
+    if step <= hp.warmup:
+        # h_t = min{lambda_abs / ||g_t||, 1}
+        clip_all = G > hp.lambda_abs
+        h_t = hp.lambda_abs / G if clip_all else 1.0
+        if hp.lambda_abs > 0:
+            margin[:] = abs(G - hp.lambda_abs) / hp.lambda_abs
+        for i in range(T):
+            h[i] = h_t
+            flag[i] = clip_all
+            c[i] = h_t * n[i]                              # ||hat(g)_t,i||
+            # gamma_t,i = min{gamma_t-1,i, ||hat(g)_t,i||},  gamma_0,i = ||hat(g)_1,i||
+            gam[i] = c[i] if step == 1 else min(gam[i], c[i])
+    else:
+        for i in range(T):
+            if step == 1:                                  # T_start = 0: seed, then Eq. 3
+                gam[i] = float(np.asarray(n[i]).astype(state_dtype))
+            thr = hp.lambda_rel * gam[i]
+            if thr > 0:
+                margin[i] = abs(n[i] - thr) / thr
+            if n[i] > thr:                                 # clip active
+                flag[i] = True
+                h[i] = thr / n[i]                          # lambda_rel * gamma / ||g||
+                c[i] = thr                                 # norm scaled to lambda_rel * gamma
+            else:
+                h[i] = 1.0
+                c[i] = n[i]
+            # gamma_t,i = beta * gamma_t-1,i + (1 - beta) * ||hat(g)_t,i||
+            gam[i] = hp.beta * gam[i] + (1.0 - hp.beta) * c[i]
+    return ClipResult(n, h, flag, c, gam.astype(state_dtype), G, margin)
+
+
+def adamw_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray, h: float,
+                 step: int, hp: Hyper, state_dtype=np.float32
+                 ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """The four AdamW lines of Algorithm 1 on hat(g) = h * g, elementwise, in float64.
+
+    Inputs are read in their storage dtype, the arithmetic is float64, the results are
+    rounded to `state_dtype`.  Works on any array of elements of one tensor (or a sample).
+    """
+    th = np.asarray(theta, dtype=np.float64)
+    gh = float(h) * np.asarray(g, dtype=np.float64)                   # hat(g)
+    m1 = hp.beta1 * np.asarray(m, dtype=np.float64) + (1.0 - hp.beta1) * gh
+    v1 = hp.beta2 * np.asarray(v, dtype=np.float64) + (1.0 - hp.beta2) * gh * gh
+    m_hat = m1 / (1.0 - hp.beta1 ** step)
+    v_hat = v1 / (1.0 - hp.beta2 ** step)
+    th1 = th - hp.lr * hp.wd * th - hp.lr * m_hat / (np.sqrt(v_hat) + hp.eps)
+    return th1.astype(state_dtype), m1.astype(state_dtype), v1.astype(state_dtype)
+
+
+def clipped_grad(g: np.ndarray, h: float) -> np.ndarray:
+    """hat(g) = h * g in float64 (the clip-only use of the method with other optimizers)."""
+    return float(h) * np.asarray(g, dtype=np.float64)
+
+
+class AdaGCAdamW:
+    """Algorithm 1 over a list of tensors; holds theta, m, v, gamma and the counters."""
+
+    def __init__(self, params: Sequence[np.ndarray], hp: Hyper, state_dtype=np.float32):
+        self.hp = hp
+        self.dt = state_dtype
+        self.theta = [np.array(p, dtype=state_dtype) for p in params]
+        self.m = [np.zeros_like(p) for p in self.theta]               # m_0 = 0
+        self.v = [np.zeros_like(p) for p in self.theta]               # v_0 = 0
+        self.gamma = np.zeros(len(self.theta), dtype=state_dtype)
+        self.t = 0
+        self.clip_count = np.zeros(len(self.theta), dtype=np.uint64)
+        self.last: Optional[ClipResult] = None
+
+    def clip(self, grads: Sequence[np.ndarray]) -> ClipResult:
+        """The clipping half of one step: advances t, gamma and the counters."""
+        self.t += 1
+        s = [sumsq(g) for g in grads]
+        r = clip_decisions(s, self.gamma, self.t, self.hp, self.dt)
+        self.gamma = r.gamma
+        self.clip_count += r.flag.astype(np.uint64)
+        self.last = r
+        return r
+
+    def step(self, grads: Sequence[np.ndarray], lr: Optional[float] = None) -> ClipResult:
+        r = self.clip(grads)
+        hp = self.hp if lr is None else Hyper(**{**self.hp.__dict__, "lr": lr})
+        for i, g in enumerate(grads):
+            self.theta[i], self.m[i], self.v[i] = adamw_update(
+                self.theta[i], g, self.m[i], self.v[i], r.h[i], self.t, hp, self.dt)
+        return r
+
+    def clip_only(self, grads: Sequence[np.ndarray]) -> Tuple[ClipResult, List[np.ndarray]]:
+        r = self.clip(grads)
+        return r, [clipped_grad(g, r.h[i]) for i, g in enumerate(grads)]

@@ -1,0 +1,212 @@
+/*
+ * CPU oracle for AdamW with AdaGC (Algorithm 1 of the paper; Eq. 2, Eq. 3), in plain C.
+ *
+ * TEST INFRASTRUCTURE ONLY: a slow, float64, per-tensor restatement of the paper's
+ * algorithm for checking the CUDA library at sizes where the numpy oracle is too slow.
+ * It shares no code, header or table with the CUDA path and is never a fallback for it.
+ *
+ * Arithmetic: every per-element and per-tensor quantity is float64; the sum of squares of a
+ * tensor is accumulated sequentially, in element order, in long double.  Stored state
+ * (theta, m, v, gamma) is fp32 and is rounded once per step on store.  OpenMP, if enabled,
+ * only distributes whole tensors (norms) or independent elements (update) over threads; it
+ * never changes the order of a reduction.
+ *
+ * Readings of the paper (same as the numpy oracle): 1-based step; warm-up = steps
+ * 1..T_start with global-norm clipping (Eq. 2) and min-seeding of gamma from the clipped
+ * per-tensor norms; at step 1 the incoming gamma is ignored; strict ">" activates the clip and
+ * the clipped norm is then lambda_rel * gamma itself (Section 4.2).
+ *
+ * Parity pins: tests/test_oracle_pins.py runs the same pins against this file and the numpy oracle.
+ *
+ * Build: gcc -O2 -fopenmp -ffp-contract=off -shared -fPIC adagc_ref.c -o libadagc_ref.so -lm
+ */
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static inline double bf16_to_double(uint16_t b) {
+  uint32_t u = ((uint32_t)b) << 16;
+  float f;
+  memcpy(&f, &u, 4);
+  return (double)f;
+}
+
+/* Round a double to the nearest bfloat16 (ties to even), from the format's definition:
+ * 8 exponent bits with bias 127, 7 stored mantissa bits, subnormals below 2^-126. */
+static uint16_t double_to_bf16(double x) {
+  float f;
+  uint32_t u;
+  if (isnan(x)) return 0x7fc0;
+  if (isinf(x) || x == 0.0) {
+    f = (float)x;
+    memcpy(&u, &f, 4);
+    return (uint16_t)(u >> 16);
+  }
+  int e;
+  (void)frexp(x, &e); /* |x| = frac * 2^e, frac in [0.5, 1)  ->  floor(log2|x|) = e - 1 */
+  int p = e - 1;
+  if (p < -126) p = -126;
+  double q = ldexp(x, 7 - p);  /* exact power-of-two scaling; |q| < 2^8 */
+  double r = nearbyint(q);     /* round to nearest, ties to even (default rounding mode) */
+  double y = ldexp(r, p - 7);  /* representable in bf16 unless it overflows */
+  f = (float)y;                /* exact, or +-inf on overflow beyond the fp32 range */
+  memcpy(&u, &f, 4);
+  if ((u & 0x7f800000u) == 0x7f800000u) return (uint16_t)((u >> 16) & 0xff80);
+  return (uint16_t)(u >> 16);
+}
+
+int adagc_ref_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+uint16_t adagc_ref_double_to_bf16(double x) { return double_to_bf16(x); }
+
+/* sum_j g_j^2 of one tensor (the square of the norm in Eq. 3). */
+double adagc_ref_sumsq(const void* g, int is_bf16, int64_t n) {
+  long double acc = 0.0L;
+  if (is_bf16) {
+    const uint16_t* p = (const uint16_t*)g;
+    for (int64_t j = 0; j < n; ++j) {
+      double x = bf16_to_double(p[j]);
+      acc += (long double)(x * x);
+    }
+  } else {
+    const float* p = (const float*)g;
+    for (int64_t j = 0; j < n; ++j) {
+      double x = (double)p[j];
+      acc += (long double)(x * x);
+    }
+  }
+  return (double)acc;
+}
+
+/* Sums of squares of T tensors that live at element offsets off[i] of one arena. */
+void adagc_ref_sumsq_tensors(const void* arena, int is_bf16, int32_t T, const int64_t* off,
+                             const int64_t* numel, double* s_out) {
+  const char* base = (const char*)arena;
+  const int64_t esz = is_bf16 ? 2 : 4;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int32_t i = 0; i < T; ++i) s_out[i] = adagc_ref_sumsq(base + off[i] * esz, is_bf16, numel[i]);
+}
+
+/*
+ * Clip factors, flags and the EMA update of one step (Algorithm 1: the warm-up branch with
+ * Eq. 2, or the AdaGC branch with Eq. 3).  gamma is fp32 state, updated in place.
+ * Outputs per tensor: norm, h, flag, clipped norm, decision margin |norm - thr| / thr.
+ */
+void adagc_ref_clip_decisions(int32_t T, const double* s, float* gamma, int64_t step,
+                              double lambda_rel, double beta, double lambda_abs, int64_t warmup,
+                              double* norm, double* h, uint8_t* flag, double* clipped,
+                              double* margin, double* global_norm) {
+  long double tot = 0.0L;
+  for (int32_t i = 0; i < T; ++i) {
+    norm[i] = sqrt(s[i]);
+    tot += (long double)s[i];
+  }
+  const double G = sqrt((double)tot); /* ||g_t|| */
+  *global_norm = G;
+  if (step <= warmup) {
+    const int clip_all = G > lambda_abs;
+    const double h_t = clip_all ? lambda_abs / G : 1.0; /* min{lambda_abs/||g_t||, 1} */
+    for (int32_t i = 0; i < T; ++i) {
+      h[i] = h_t;
+      flag[i] = (uint8_t)clip_all;
+      clipped[i] = h_t * norm[i]; /* ||hat(g)_t,i|| */
+      margin[i] = lambda_abs > 0 ? fabs(G - lambda_abs) / lambda_abs : INFINITY;
+      double gprev = (double)gamma[i];
+      double gnew = (step == 1) ? clipped[i] : (gprev < clipped[i] ? gprev : clipped[i]);
+      gamma[i] = (float)gnew;
+    }
+  } else {
+    for (int32_t i = 0; i < T; ++i) {
+      double gprev = (step == 1) ? (double)(float)norm[i] : (double)gamma[i];
+      const double thr = lambda_rel * gprev;
+      margin[i] = thr > 0 ? fabs(norm[i] - thr) / thr : INFINITY;
+      if (norm[i] > thr) {
+        flag[i] = 1;
+        h[i] = thr / norm[i];
+        clipped[i] = thr;
+      } else {
+        flag[i] = 0;
+        h[i] = 1.0;
+        clipped[i] = norm[i];
+      }
+      gamma[i] = (float)(beta * gprev + (1.0 - beta) * clipped[i]);
+    }
+  }
+}
+
+/* The four AdamW lines of Algorithm 1 on hat(g) = h * g for n elements, in place. */
+void adagc_ref_adamw(float* theta, const void* g, int g_is_bf16, float* m, float* v, int64_t n,
+                     double h, int64_t step, double lr, double beta1, double beta2, double eps,
+                     double wd) {
+  const double bc1 = 1.0 - pow(beta1, (double)step);
+  const double bc2 = 1.0 - pow(beta2, (double)step);
+  const uint16_t* gb = (const uint16_t*)g;
+  const float* gf = (const float*)g;
+#pragma omp parallel for schedule(static) if (n > 65536)
+  for (int64_t j = 0; j < n; ++j) {
+    const double gj = g_is_bf16 ? bf16_to_double(gb[j]) : (double)gf[j];
+    const double gh = h * gj;
+    const double m1 = beta1 * (double)m[j] + (1.0 - beta1) * gh;
+    const double v1 = beta2 * (double)v[j] + (1.0 - beta2) * gh * gh;
+    const double mh = m1 / bc1;
+    const double vh = v1 / bc2;
+    const double th = (double)theta[j];
+    theta[j] = (float)(th - lr * wd * th - lr * mh / (sqrt(vh) + eps));
+    m[j] = (float)m1;
+    v[j] = (float)v1;
+  }
+}
+
+/* hat(g) = h * g written in the gradient's dtype (clip-only use with other optimizers). */
+void adagc_ref_scale(void* out, const void* g, int is_bf16, int64_t n, double h) {
+  if (is_bf16) {
+    const uint16_t* p = (const uint16_t*)g;
+    uint16_t* o = (uint16_t*)out;
+#pragma omp parallel for schedule(static) if (n > 65536)
+    for (int64_t j = 0; j < n; ++j) o[j] = double_to_bf16(h * bf16_to_double(p[j]));
+  } else {
+    const float* p = (const float*)g;
+    float* o = (float*)out;
+#pragma omp parallel for schedule(static) if (n > 65536)
+    for (int64_t j = 0; j < n; ++j) o[j] = (float)(h * (double)p[j]);
+  }
+}
+
+/* One whole step of Algorithm 1 over T tensors laid out in shared arenas.
+ * Stats outputs may be NULL.  Returns the number of tensors clipped. */
+int32_t adagc_ref_step(int32_t T, const int64_t* off, const int64_t* numel, float* theta,
+                       const void* grads, int g_is_bf16, float* m, float* v, float* gamma,
+                       int64_t step, double lr, double beta1, double beta2, double eps, double wd,
+                       double lambda_rel, double beta, double lambda_abs, int64_t warmup,
+                       double* s_ws /* T */, double* norm, double* h, uint8_t* flag,
+                       double* clipped, double* margin, double* global_norm) {
+  adagc_ref_sumsq_tensors(grads, g_is_bf16, T, off, numel, s_ws);
+  adagc_ref_clip_decisions(T, s_ws, gamma, step, lambda_rel, beta, lambda_abs, warmup, norm, h,
+                           flag, clipped, margin, global_norm);
+  const int64_t esz = g_is_bf16 ? 2 : 4;
+  int32_t n_clipped = 0;
+  for (int32_t i = 0; i < T; ++i) n_clipped += flag[i];
+  /* large tensors one after another (threads split their elements) ... */
+  for (int32_t i = 0; i < T; ++i) {
+    if (numel[i] <= 65536) continue;
+    adagc_ref_adamw(theta + off[i], (const char*)grads + off[i] * esz, g_is_bf16, m + off[i],
+                    v + off[i], numel[i], h[i], step, lr, beta1, beta2, eps, wd);
+  }
+  /* ... small tensors distributed whole over the threads. */
+#pragma omp parallel for schedule(dynamic, 16)
+  for (int32_t i = 0; i < T; ++i) {
+    if (numel[i] > 65536) continue;
+    adagc_ref_adamw(theta + off[i], (const char*)grads + off[i] * esz, g_is_bf16, m + off[i],
+                    v + off[i], numel[i], h[i], step, lr, beta1, beta2, eps, wd);
+  }
+  return n_clipped;
+}

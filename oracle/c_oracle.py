@@ -1,0 +1,169 @@
+"""ctypes front end of the C oracle (adagc_ref.c).  TEST INFRASTRUCTURE ONLY.
+
+Same role as adagc_oracle.py (Algorithm 1, Eq. 2, Eq. 3 of the paper in float64), but fast
+enough for layouts with 1e8..1e10 elements.  bf16 gradients are passed as uint16 arrays of
+their bit patterns.  Never imported by the CUDA path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "adagc_ref.c")
+_LIB = os.path.join(_HERE, "libadagc_ref.so")
+_lib = None
+
+_f64p = np.ctypeslib.ndpointer(np.float64, flags="C_CONTIGUOUS")
+_f32p = np.ctypeslib.ndpointer(np.float32, flags="C_CONTIGUOUS")
+_i64p = np.ctypeslib.ndpointer(np.int64, flags="C_CONTIGUOUS")
+_u8p = np.ctypeslib.ndpointer(np.uint8, flags="C_CONTIGUOUS")
+
+
+def build(force: bool = False) -> str:
+    """Compile adagc_ref.c into libadagc_ref.so next to it (gcc, OpenMP, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-fopenmp", "-ffp-contract=off", "-shared", "-fPIC", _SRC, "-o", _LIB, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        L.adagc_ref_num_threads.restype = C.c_int
+        L.adagc_ref_double_to_bf16.restype = C.c_uint16
+        L.adagc_ref_double_to_bf16.argtypes = [C.c_double]
+        L.adagc_ref_sumsq.restype = C.c_double
+        L.adagc_ref_sumsq.argtypes = [C.c_void_p, C.c_int, C.c_int64]
+        L.adagc_ref_sumsq_tensors.restype = None
+        L.adagc_ref_sumsq_tensors.argtypes = [C.c_void_p, C.c_int, C.c_int32, _i64p, _i64p, _f64p]
+        L.adagc_ref_clip_decisions.restype = None
+        L.adagc_ref_clip_decisions.argtypes = [C.c_int32, _f64p, _f32p, C.c_int64, C.c_double, C.c_double,
+                                               C.c_double, C.c_int64, _f64p, _f64p, _u8p, _f64p, _f64p, _f64p]
+        L.adagc_ref_adamw.restype = None
+        L.adagc_ref_adamw.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int64,
+                                      C.c_double, C.c_int64] + [C.c_double] * 5
+        L.adagc_ref_scale.restype = None
+        L.adagc_ref_scale.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_double]
+        L.adagc_ref_step.restype = C.c_int32
+        L.adagc_ref_step.argtypes = ([C.c_int32, _i64p, _i64p, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p,
+                                      C.c_void_p, _f32p, C.c_int64] + [C.c_double] * 8 + [C.c_int64] +
+                                     [_f64p, _f64p, _f64p, _u8p, _f64p, _f64p, _f64p])
+        _lib = L
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().adagc_ref_num_threads())
+
+
+def _grad_ptr(g: np.ndarray) -> Tuple[int, int]:
+    assert g.flags["C_CONTIGUOUS"]
+    if g.dtype == np.uint16:
+        return g.ctypes.data, 1
+    if g.dtype == np.float32:
+        return g.ctypes.data, 0
+    raise TypeError("gradients must be float32, or uint16 holding bf16 bit patterns")
+
+
+def sumsq(g: np.ndarray) -> float:
+    p, bf = _grad_ptr(g)
+    return float(lib().adagc_ref_sumsq(p, bf, g.size))
+
+
+def sumsq_tensors(arena: np.ndarray, offsets: Sequence[int], numels: Sequence[int]) -> np.ndarray:
+    p, bf = _grad_ptr(arena)
+    off = np.ascontiguousarray(offsets, dtype=np.int64)
+    nel = np.ascontiguousarray(numels, dtype=np.int64)
+    out = np.empty(len(off), dtype=np.float64)
+    lib().adagc_ref_sumsq_tensors(p, bf, len(off), off, nel, out)
+    return out
+
+
+def clip_decisions(s: np.ndarray, gamma: np.ndarray, step: int, lambda_rel: float, beta: float,
+                   lambda_abs: float, warmup: int):
+    """Returns dict(norm, h, flag, clipped, margin, global_norm); `gamma` (fp32) is updated in place."""
+    s = np.ascontiguousarray(s, dtype=np.float64)
+    T = len(s)
+    assert gamma.dtype == np.float32 and gamma.flags["C_CONTIGUOUS"] and len(gamma) == T
+    norm, h, clipped, margin = (np.empty(T, np.float64) for _ in range(4))
+    flag = np.empty(T, np.uint8)
+    G = np.empty(1, np.float64)
+    lib().adagc_ref_clip_decisions(T, s, gamma, step, lambda_rel, beta, lambda_abs, warmup,
+                                   norm, h, flag, clipped, margin, G)
+    return dict(norm=norm, h=h, flag=flag.astype(bool), clipped=clipped, margin=margin,
+                global_norm=float(G[0]), gamma=gamma)
+
+
+def adamw_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray, h: float, step: int,
+                 lr: float, beta1: float, beta2: float, eps: float, wd: float) -> None:
+    """In place on fp32 theta, m, v."""
+    p, bf = _grad_ptr(g)
+    for a in (theta, m, v):
+        assert a.dtype == np.float32 and a.flags["C_CONTIGUOUS"] and a.size == g.size
+    lib().adagc_ref_adamw(theta.ctypes.data, p, bf, m.ctypes.data, v.ctypes.data, g.size,
+                          float(h), int(step), lr, beta1, beta2, eps, wd)
+
+
+def scale(g: np.ndarray, h: float, out: Optional[np.ndarray] = None) -> np.ndarray:
+    """hat(g) = h * g rounded to the gradient's dtype."""
+    p, bf = _grad_ptr(g)
+    out = np.empty_like(g) if out is None else out
+    lib().adagc_ref_scale(out.ctypes.data, p, bf, g.size, float(h))
+    return out
+
+
+def double_to_bf16_bits(x: float) -> int:
+    return int(lib().adagc_ref_double_to_bf16(float(x)))
+
+
+class ArenaOracle:
+    """Algorithm 1 over tensors stored at fixed offsets of shared fp32 arenas (theta, m, v)."""
+
+    def __init__(self, offsets: Sequence[int], numels: Sequence[int], theta0: np.ndarray, *,
+                 lr: float, beta1: float, beta2: float, eps: float, wd: float, lambda_rel: float,
+                 beta: float, lambda_abs: float, warmup: int):
+        self.off = np.ascontiguousarray(offsets, dtype=np.int64)
+        self.numel = np.ascontiguousarray(numels, dtype=np.int64)
+        self.T = len(self.off)
+        self.theta = np.array(theta0, dtype=np.float32)
+        self.m = np.zeros_like(self.theta)
+        self.v = np.zeros_like(self.theta)
+        self.gamma = np.zeros(self.T, dtype=np.float32)
+        self.hp = dict(lr=lr, beta1=beta1, beta2=beta2, eps=eps, wd=wd, lambda_rel=lambda_rel,
+                       beta=beta, lambda_abs=lambda_abs, warmup=warmup)
+        self.t = 0
+        self.clip_count = np.zeros(self.T, dtype=np.uint64)
+        self._s = np.empty(self.T, np.float64)
+
+    def step(self, grads: np.ndarray, lr: Optional[float] = None):
+        self.t += 1
+        p, bf = _grad_ptr(grads)
+        hp = self.hp
+        norm, h, clipped, margin = (np.empty(self.T, np.float64) for _ in range(4))
+        flag = np.empty(self.T, np.uint8)
+        G = np.empty(1, np.float64)
+        lib().adagc_ref_step(self.T, self.off, self.numel, self.theta.ctypes.data, p, bf,
+                             self.m.ctypes.data, self.v.ctypes.data, self.gamma, self.t,
+                             hp["lr"] if lr is None else lr, hp["beta1"], hp["beta2"], hp["eps"], hp["wd"],
+                             hp["lambda_rel"], hp["beta"], hp["lambda_abs"], hp["warmup"],
+                             self._s, norm, h, flag, clipped, margin, G)
+        self.clip_count += flag.astype(np.uint64)
+        return dict(norm=norm, h=h, flag=flag.astype(bool), clipped=clipped, margin=margin,
+                    global_norm=float(G[0]), gamma=self.gamma.copy())
+
+    def clip(self, grads: np.ndarray):
+        """Clip-only step: advances gamma and the counters, returns the decisions (no AdamW)."""
+        self.t += 1
+        s = sumsq_tensors(grads, self.off, self.numel)
+        r = clip_decisions(s, self.gamma, self.t, self.hp["lambda_rel"], self.hp["beta"],
+                           self.hp["lambda_abs"], self.hp["warmup"])
+        self.clip_count += r["flag"].astype(np.uint64)
+        r["gamma"] = self.gamma.copy()
+        return r

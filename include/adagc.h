@@ -1,0 +1,167 @@
+/*
+ * adagc.h -- C ABI of the fused AdaGC + AdamW optimizer step for NVIDIA B200 (sm_100a).
+ *
+ * The library implements one step of "AdamW with AdaGC" (Algorithm 1 of the paper):
+ *   - per-tensor gradient norms ||g_t,i|| (Eq. 3) and, during warm-up, the global norm (Eq. 2);
+ *   - the clip factor h: global-norm clipping against lambda_abs for the first T_start steps
+ *     (warm-up branch of Algorithm 1), afterwards per tensor against lambda_rel * gamma_{t-1,i}
+ *     (Eq. 3), where gamma_i is the EMA of that tensor's *clipped* norms;
+ *   - the gamma update (min-seeding in warm-up, EMA with beta afterwards);
+ *   - AdamW moments, bias correction, decoupled weight decay on the clipped gradient
+ *     (last four lines of Algorithm 1).
+ *
+ * Conventions
+ *   - All tensors of a model live in flat "arenas": params, grads, m, v share one element-offset
+ *     table (tensor i occupies elements [offset, offset + numel) of every arena).
+ *   - Pointers named d_* are DEVICE pointers, h_* are HOST pointers.  The caller owns every
+ *     buffer, including the workspace.  No entry point declared in this header allocates or frees
+ *     device memory.
+ *   - `cuda_stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *     adagc_step / adagc_clip only enqueue work; they never synchronise.
+ *   - `step` is 1-based.  Steps 1..warmup use global-norm clipping; step warmup+1 is the first
+ *     per-tensor AdaGC step.  At step 1 the incoming content of `d_ema` is ignored and gamma is
+ *     seeded from that step's clipped norms, so no initialisation of `d_ema` is required.
+ *   - Return value: 0 on success, a negative adagc_status otherwise; on error nothing was enqueued.
+ *     Conditions found on the device (non-finite gradient norm) are reported through the status
+ *     word returned by adagc_get_stats.  The library never prints and never aborts.
+ */
+#ifndef ADAGC_H_
+#define ADAGC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct adagc_ctx adagc_ctx; /* opaque, host-side */
+
+typedef enum { ADAGC_F32 = 0, ADAGC_BF16 = 1 } adagc_dtype;
+
+typedef enum {
+  ADAGC_OK = 0,
+  ADAGC_E_INVALID_ARG = -1, /* null pointer, numel <= 0, hyper-parameter outside its domain, ... */
+  ADAGC_E_MISALIGNED = -2,  /* a tensor offset or an arena pointer is not 16-byte aligned */
+  ADAGC_E_OVERLAP = -3,     /* two tensors of the descriptor overlap */
+  ADAGC_E_WORKSPACE = -4,   /* workspace too small or misaligned */
+  ADAGC_E_DTYPE = -5,       /* unsupported dtype combination */
+  ADAGC_E_CUDA = -6,        /* a CUDA runtime call failed (no device, launch error, ...) */
+  ADAGC_E_NOMEM = -7        /* host allocation of the context failed */
+} adagc_status;
+
+/* Bits of the device status word (adagc_get_stats). */
+#define ADAGC_W_NONFINITE 1 /* some tensor's sum of squares was Inf or NaN in some step */
+
+/* One parameter tensor. */
+typedef struct {
+  int64_t numel;    /* > 0 */
+  int64_t offset;   /* element offset into every arena; offset * sizeof(element) must be a
+                       multiple of 16 bytes for every arena dtype (multiple of 8 elements with
+                       bf16 gradients, of 4 with fp32 gradients) */
+  int32_t ndim;     /* 0..4; informational.  If > 0 the product of shape[0..ndim) must be numel */
+  int32_t reserved; /* set to 0 */
+  int64_t shape[4];
+} adagc_tensor;
+
+/* The model: a list of tensors plus the dtypes of the arenas. */
+typedef struct {
+  int32_t n_tensors;           /* >= 1 */
+  int32_t param_dtype;         /* ADAGC_F32 */
+  int32_t grad_dtype;          /* ADAGC_F32 or ADAGC_BF16 */
+  int32_t state_dtype;         /* ADAGC_F32 (m and v) */
+  const adagc_tensor* tensors; /* host array, copied by adagc_create */
+  double lambda_abs;           /* warm-up global-norm threshold of Eq. 2, > 0 (paper: 1.0) */
+  int32_t flags;               /* reserved, set to 0 */
+  int32_t reserved;            /* set to 0 */
+} adagc_desc;
+
+/* Bytes of device workspace adagc_create needs for this descriptor (chunk table, per-chunk
+ * partial sums, per-tensor statistics).  Returns 0 if the descriptor is invalid. */
+size_t adagc_workspace_bytes(const adagc_desc* desc);
+
+/* Number of fixed-size chunks the tensors are cut into (one partial sum per chunk).
+ * Returns a negative adagc_status if the descriptor is invalid.  Host-only. */
+int64_t adagc_num_chunks(const adagc_desc* desc);
+
+/* Validate the descriptor, build the chunk table and upload it into `d_workspace`
+ * (device memory, 256-byte aligned, at least adagc_workspace_bytes(desc) bytes, owned by the
+ * caller and kept alive until adagc_destroy).  Synchronises `cuda_stream` once.
+ * The CUDA device current at this call is the one the context is bound to. */
+int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_bytes,
+                 void* cuda_stream, adagc_ctx** out);
+
+/* Frees the host-side context (not the workspace). */
+int adagc_destroy(adagc_ctx* ctx);
+
+/*
+ * One fused step of Algorithm 1.
+ *   d_params, d_m, d_v : fp32 arenas, updated in place
+ *   d_grads            : gradient arena in the descriptor's grad dtype, read only
+ *   d_ema              : gamma, n_tensors fp32 values, updated in place (Section 4.3 "Memory":
+ *                        one 32-bit float per tensor)
+ *   step               : t >= 1
+ *   lr, beta1, beta2, eps, wd : eta_t, beta_1, beta_2, epsilon, lambda_w of Algorithm 1
+ *   lambda_rel, beta   : relative threshold and EMA coefficient of Eq. 3
+ *   warmup             : T_start >= 0
+ * Domain: 0 <= beta < 1, 0 <= beta1, beta2 < 1, lambda_rel > 0, eps >= 0, lr and wd finite.
+ * Arena pointers must be 16-byte aligned.
+ */
+int adagc_step(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, void* d_v,
+               float* d_ema, int64_t step, double lr, double beta1, double beta2, double eps,
+               double wd, double lambda_rel, double beta, int64_t warmup, void* cuda_stream);
+
+/*
+ * Clip-only entry (Section 4.2: the clip is optimizer-agnostic): same norms, decisions and
+ * gamma update as adagc_step, then writes the clipped gradient h_i * g_i in the gradient dtype.
+ * d_grads_out may equal d_grads_in (in place); in place, tensors with h == 1 are not rewritten.
+ */
+int adagc_clip(adagc_ctx* ctx, const void* d_grads_in, void* d_grads_out, float* d_ema,
+               int64_t step, double lambda_rel, double beta, int64_t warmup, void* cuda_stream);
+
+/*
+ * adagc_step fed from HOST memory: copies the gradient arena `h_grads` (arena_elems elements of
+ * the grad dtype; pinned memory recommended) into `d_grads`, runs the step, copies the per-tensor
+ * statistics of this step back into the host arrays (any may be NULL) and synchronises the stream.
+ */
+int adagc_step_host(adagc_ctx* ctx, void* d_params, void* d_grads, void* d_m, void* d_v,
+                    float* d_ema, const void* h_grads, int64_t step, double lr, double beta1,
+                    double beta2, double eps, double wd, double lambda_rel, double beta,
+                    int64_t warmup, float* h_norm, float* h_clipfactor, uint8_t* h_flag,
+                    void* cuda_stream);
+
+/*
+ * Statistics of the most recent step, copied to host arrays of n_tensors entries (any pointer may
+ * be NULL): gradient norm, clip factor h, clip flag, cumulative clip count; plus the number of
+ * steps executed and the device status word.  Synchronises the stream.
+ */
+int adagc_get_stats(adagc_ctx* ctx, float* h_norm, float* h_clipfactor, uint8_t* h_flag,
+                    uint64_t* h_clip_count, uint64_t* h_steps_done, int32_t* h_device_status,
+                    void* cuda_stream);
+
+/* Per-tensor sums of squares of the most recent step in float64 (n_tensors entries).
+ * Synchronises the stream. */
+int adagc_get_sumsq(adagc_ctx* ctx, double* h_sumsq, void* cuda_stream);
+
+/* Elements spanned by the arenas: max over tensors of offset + numel. */
+int64_t adagc_arena_elems(const adagc_ctx* ctx);
+
+/* Kernels launched by this context so far. */
+uint64_t adagc_launch_count(const adagc_ctx* ctx);
+
+/*
+ * Optional per-phase timing.  When enabled, adagc_step / adagc_clip record CUDA events on the
+ * caller's stream around the three phases (norm, finalize, update-or-scale).
+ * adagc_get_phase_times synchronises on the last event and returns the durations in
+ * milliseconds of the most recent step: ms[0] norm, ms[1] finalize, ms[2] update / scale.
+ */
+int adagc_set_phase_timing(adagc_ctx* ctx, int enabled);
+int adagc_get_phase_times(adagc_ctx* ctx, float ms[3]);
+
+/* Static string for a status code. */
+const char* adagc_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADAGC_H_ */

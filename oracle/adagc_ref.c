@@ -121,7 +121,7 @@ void adagc_ref_clip_decisions(int32_t T, const double* s, float* gamma, int64_t 
       clipped[i] = h_t * norm[i]; /* ||hat(g)_t,i|| */
       margin[i] = lambda_abs > 0 ? fabs(G - lambda_abs) / lambda_abs : INFINITY;
       double gprev = (double)gamma[i];
-      double gnew = (step == 1) ? clipped[i] : (gprev < clipped[i] ? gprev : clipped[i]);
+      double gnew = (step == 1) ? clipped[i] : (clipped[i] < gprev ? clipped[i] : gprev);
       gamma[i] = (float)gnew;
     }
   } else {

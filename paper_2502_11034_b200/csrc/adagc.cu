@@ -1,0 +1,755 @@
+// Fused AdaGC + AdamW optimizer step for B200 (sm_100a): kernels and the C ABI of include/adagc.h.
+//
+// One step of Algorithm 1 of the paper is three phases on the caller's stream:
+//   1. norm      every fixed-size chunk of every gradient tensor -> one float64 partial sum of
+//                squares (Eq. 3 needs ||g_t,i||, Eq. 2 needs ||g_t||);
+//   2. finalize  per tensor: fixed-order sum of its partials -> norm -> clip factor h, flag and the
+//                gamma update (warm-up branch: global norm first, then min-seeding);
+//   3. update    every chunk again: g, theta, m, v read once, hat(g) = h * g kept in registers,
+//                AdamW lines of Algorithm 1, theta, m, v written once.
+// This is pure streaming work (26..28 bytes per parameter, ~20 flops): the bound is HBM bandwidth,
+// so the kernels are built around 128-bit coalesced accesses, many loads in flight per thread and
+// streaming cache hints; there is no contraction here and tensor cores are not used.
+//
+// Reductions are deterministic: fixed element->thread mapping, fixed shuffle tree, fixed-order sums
+// of partials; no floating-point atomics.  Sums of squares are accumulated in float64 so that the
+// clip decision ||g|| > lambda_rel * gamma agrees with a float64 evaluation of the same predicate.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <algorithm>
+#include <cmath>
+#include <new>
+#include <vector>
+
+#include "../../include/adagc.h"
+
+namespace {
+
+constexpr int kChunkElems = 16384;  // elements per chunk; multiple of 8 keeps every chunk 16-byte aligned
+constexpr int kThreads = 256;
+constexpr int kFinalizeThreads = 256;  // 8 warps = 8 tensors per block
+constexpr int kWarmupThreads = 1024;
+
+struct Chunk {
+  int64_t start;   // element offset into the arenas
+  int32_t count;   // elements in this chunk (<= kChunkElems)
+  int32_t tensor;  // owning tensor
+};
+static_assert(sizeof(Chunk) == 16, "chunk entries are 16 bytes");
+
+struct TensorEntry {
+  int32_t first_chunk;
+  int32_t n_chunks;
+};
+
+struct ClipScalars {
+  double lambda_rel, beta, one_minus_beta, lambda_abs;
+  int64_t step;
+  int32_t n_tensors;
+};
+
+struct AdamScalars {
+  float beta1, one_minus_beta1, beta2, one_minus_beta2;
+  float inv_bc2;    // 1 / (1 - beta2^t)
+  float step_size;  // lr / (1 - beta1^t)
+  float decay;      // 1 - lr * wd
+  float eps;
+};
+
+// ------------------------------------------------------------------------------------------------
+// small device helpers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ double warp_sum(double x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;  // identical in every lane: each level adds the same two values in both partners
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// round-to-nearest-even float -> bf16 bits (NaN stays NaN)
+__device__ __forceinline__ uint32_t f32_to_bf16_bits(float f) {
+  uint32_t u = __float_as_uint(f);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return (u >> 16) | 0x40u;
+  u += 0x7fffu + ((u >> 16) & 1u);
+  return u >> 16;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  return f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
+}
+
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
+__device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
+__device__ __forceinline__ void st_stream(uint4* p, uint4 v) { __stcs(p, v); }
+
+__device__ __forceinline__ double sq_acc(double acc, float x) {
+  const double d = (double)x;
+  return fma(d, d, acc);
+}
+
+// ------------------------------------------------------------------------------------------------
+// phase 1: per-chunk sums of squares (Eq. 3: ||g_t,i||^2 = sum_j g_ij^2)
+// ------------------------------------------------------------------------------------------------
+template <bool kBF16>
+__global__ void __launch_bounds__(kThreads)
+adagc_norm_kernel(const void* __restrict__ grads, const Chunk* __restrict__ chunks, int n_chunks,
+                  double* __restrict__ partials) {
+  constexpr int kEPV = kBF16 ? 8 : 4;  // elements per 16-byte vector
+  constexpr int kUnroll = 8;           // independent 16-byte loads in flight per thread
+  __shared__ double warp_part[kThreads / 32];
+  const int tid = threadIdx.x;
+  for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+    const Chunk ck = chunks[c];
+    const uint4* __restrict__ vec =
+        reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + ck.start * (kBF16 ? 2 : 4));
+    const int nvec = ck.count / kEPV;
+    double acc0 = 0.0, acc1 = 0.0;
+    for (int base = 0; base < nvec; base += kThreads * kUnroll) {
+      uint4 q[kUnroll];
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const int i = base + u * kThreads + tid;
+        q[u] = (i < nvec) ? __ldg(vec + i) : make_uint4(0u, 0u, 0u, 0u);
+      }
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        if (kBF16) {
+          acc0 = sq_acc(acc0, bf16_lo(q[u].x));
+          acc1 = sq_acc(acc1, bf16_hi(q[u].x));
+          acc0 = sq_acc(acc0, bf16_lo(q[u].y));
+          acc1 = sq_acc(acc1, bf16_hi(q[u].y));
+          acc0 = sq_acc(acc0, bf16_lo(q[u].z));
+          acc1 = sq_acc(acc1, bf16_hi(q[u].z));
+          acc0 = sq_acc(acc0, bf16_lo(q[u].w));
+          acc1 = sq_acc(acc1, bf16_hi(q[u].w));
+        } else {
+          acc0 = sq_acc(acc0, __uint_as_float(q[u].x));
+          acc1 = sq_acc(acc1, __uint_as_float(q[u].y));
+          acc0 = sq_acc(acc0, __uint_as_float(q[u].z));
+          acc1 = sq_acc(acc1, __uint_as_float(q[u].w));
+        }
+      }
+    }
+    // ragged tail of the tensor's last chunk (fewer than one vector)
+    const int t = nvec * kEPV + tid;
+    if (t < ck.count) {
+      float x;
+      if (kBF16) {
+        const uint16_t b = reinterpret_cast<const uint16_t*>(vec)[t];
+        x = __uint_as_float(static_cast<uint32_t>(b) << 16);
+      } else {
+        x = reinterpret_cast<const float*>(vec)[t];
+      }
+      acc0 = sq_acc(acc0, x);
+    }
+    const double w = warp_sum(acc0 + acc1);
+    if ((tid & 31) == 0) warp_part[tid >> 5] = w;
+    __syncthreads();
+    if (tid == 0) {
+      double s = warp_part[0];
+#pragma unroll
+      for (int k = 1; k < kThreads / 32; ++k) s += warp_part[k];
+      partials[c] = s;
+    }
+    __syncthreads();
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// phase 2: per-tensor reduction, clip decision, gamma update
+// ------------------------------------------------------------------------------------------------
+struct StatPtrs {
+  double* sumsq;         // [T] float64 sum of squares of this step
+  float* norm;           // [T]
+  float* h;              // [T] clip factor
+  uint8_t* flag;         // [T]
+  unsigned long long* clip_count;  // [T] cumulative
+  unsigned long long* steps_done;  // [1]
+  int* status;           // [1] device status word
+};
+
+// AdaGC branch of Algorithm 1 for one tensor (Eq. 3 and the gamma update).
+__device__ __forceinline__ void adagc_decide(int i, double s, const ClipScalars& cs,
+                                             float* __restrict__ ema, const StatPtrs& st) {
+  const double n = sqrt(s);  // ||g_t,i||
+  // gamma is fp32 state; with T_start = 0 the first step seeds it with this step's norm
+  const double g_prev = (cs.step == 1) ? (double)(float)n : (double)ema[i];
+  const double thr = __dmul_rn(cs.lambda_rel, g_prev);
+  const bool clip = n > thr;  // strict: equality is not a clip
+  const double h = clip ? __ddiv_rn(thr, n) : 1.0;
+  const double c = clip ? thr : n;  // clipped norm: exactly lambda_rel * gamma when active
+  const double g_new = __dadd_rn(__dmul_rn(cs.beta, g_prev), __dmul_rn(cs.one_minus_beta, c));
+  ema[i] = (float)g_new;
+  st.norm[i] = (float)n;
+  st.h[i] = (float)h;
+  st.flag[i] = clip ? 1 : 0;
+  if (clip) st.clip_count[i] += 1ull;
+  if (!isfinite(s)) atomicOr(st.status, ADAGC_W_NONFINITE);
+}
+
+// One warp per tensor: fixed-order sum of the tensor's chunk partials; in the AdaGC branch the
+// same warp takes the decision.
+__global__ void __launch_bounds__(kFinalizeThreads)
+adagc_tensor_finalize_kernel(const double* __restrict__ partials, const TensorEntry* __restrict__ tensors,
+                             ClipScalars cs, int decide, float* __restrict__ ema, StatPtrs st) {
+  const int w = (blockIdx.x * kFinalizeThreads + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (w >= cs.n_tensors) return;
+  const TensorEntry te = tensors[w];
+  double acc = 0.0;
+  for (int j = lane; j < te.n_chunks; j += 32) acc += partials[te.first_chunk + j];
+  acc = warp_sum(acc);
+  if (lane == 0) {
+    st.sumsq[w] = acc;
+    if (decide) {
+      adagc_decide(w, acc, cs, ema, st);
+      if (w == 0) *st.steps_done += 1ull;
+    }
+  }
+}
+
+// Warm-up branch of Algorithm 1: global norm (Eq. 2), one clip factor for every tensor, and
+// gamma_t,i = min{gamma_t-1,i, ||hat(g)_t,i||} with gamma_0,i = ||hat(g)_1,i||.  One block.
+__global__ void __launch_bounds__(kWarmupThreads)
+adagc_warmup_finalize_kernel(ClipScalars cs, float* __restrict__ ema, StatPtrs st) {
+  __shared__ double warp_part[kWarmupThreads / 32];
+  __shared__ double total_s;
+  const int tid = threadIdx.x;
+  double acc = 0.0;
+  for (int i = tid; i < cs.n_tensors; i += kWarmupThreads) acc += st.sumsq[i];
+  acc = warp_sum(acc);
+  if ((tid & 31) == 0) warp_part[tid >> 5] = acc;
+  __syncthreads();
+  if (tid == 0) {
+    double s = warp_part[0];
+    for (int k = 1; k < kWarmupThreads / 32; ++k) s += warp_part[k];
+    total_s = s;
+    *st.steps_done += 1ull;
+  }
+  __syncthreads();
+  const double G = sqrt(total_s);  // ||g_t||
+  const bool clip_all = G > cs.lambda_abs;
+  const double h = clip_all ? __ddiv_rn(cs.lambda_abs, G) : 1.0;  // min{lambda_abs / ||g_t||, 1}
+  const float hf = (float)h;
+  for (int i = tid; i < cs.n_tensors; i += kWarmupThreads) {
+    const double s = st.sumsq[i];
+    const double n = sqrt(s);
+    const double c = __dmul_rn(h, n);  // ||hat(g)_t,i||
+    double g_new = c;
+    if (cs.step != 1) {
+      const double g_prev = (double)ema[i];
+      g_new = (c < g_prev) ? c : g_prev;
+    }
+    ema[i] = (float)g_new;
+    st.norm[i] = (float)n;
+    st.h[i] = hf;
+    st.flag[i] = clip_all ? 1 : 0;
+    if (clip_all) st.clip_count[i] += 1ull;
+    if (!isfinite(s)) atomicOr(st.status, ADAGC_W_NONFINITE);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// phase 3: AdamW on the clipped gradient (last four lines of Algorithm 1)
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void adamw_elem(float g, float h, float& p, float& m, float& v,
+                                           const AdamScalars& a) {
+  const float gh = h * g;  // hat(g)
+  m = fmaf(a.beta1, m, a.one_minus_beta1 * gh);
+  v = fmaf(a.beta2, v, a.one_minus_beta2 * (gh * gh));
+  const float denom = __fsqrt_rn(v * a.inv_bc2) + a.eps;  // sqrt(v_hat) + eps
+  p = fmaf(-a.step_size, __fdiv_rn(m, denom), p * a.decay);
+}
+
+__device__ __forceinline__ void adamw_vec4(const float g0, const float g1, const float g2, const float g3,
+                                           float h, float4& p, float4& m, float4& v, const AdamScalars& a) {
+  adamw_elem(g0, h, p.x, m.x, v.x, a);
+  adamw_elem(g1, h, p.y, m.y, v.y, a);
+  adamw_elem(g2, h, p.z, m.z, v.z, a);
+  adamw_elem(g3, h, p.w, m.w, v.w, a);
+}
+
+template <bool kBF16>
+__global__ void __launch_bounds__(kThreads)
+adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, float* __restrict__ m_arena,
+                    float* __restrict__ v_arena, const Chunk* __restrict__ chunks, int n_chunks,
+                    const float* __restrict__ h_arr, AdamScalars a) {
+  const int tid = threadIdx.x;
+  for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+    const Chunk ck = chunks[c];
+    const float h = h_arr[ck.tensor];
+    float4* __restrict__ p4 = reinterpret_cast<float4*>(params + ck.start);
+    float4* __restrict__ m4 = reinterpret_cast<float4*>(m_arena + ck.start);
+    float4* __restrict__ v4 = reinterpret_cast<float4*>(v_arena + ck.start);
+    const char* gbase = static_cast<const char*>(grads) + ck.start * (kBF16 ? 2 : 4);
+    const int n8 = ck.count >> 3;  // groups of 8 elements
+#pragma unroll 2
+    for (int i = tid; i < n8; i += kThreads) {
+      float g[8];
+      if (kBF16) {
+        const uint4 q = ld_stream(reinterpret_cast<const uint4*>(gbase) + i);
+        g[0] = bf16_lo(q.x); g[1] = bf16_hi(q.x); g[2] = bf16_lo(q.y); g[3] = bf16_hi(q.y);
+        g[4] = bf16_lo(q.z); g[5] = bf16_hi(q.z); g[6] = bf16_lo(q.w); g[7] = bf16_hi(q.w);
+      } else {
+        const float4 ga = ld_stream(reinterpret_cast<const float4*>(gbase) + 2 * i);
+        const float4 gb = ld_stream(reinterpret_cast<const float4*>(gbase) + 2 * i + 1);
+        g[0] = ga.x; g[1] = ga.y; g[2] = ga.z; g[3] = ga.w;
+        g[4] = gb.x; g[5] = gb.y; g[6] = gb.z; g[7] = gb.w;
+      }
+      float4 pa = ld_stream(p4 + 2 * i), pb = ld_stream(p4 + 2 * i + 1);
+      float4 ma = ld_stream(m4 + 2 * i), mb = ld_stream(m4 + 2 * i + 1);
+      float4 va = ld_stream(v4 + 2 * i), vb = ld_stream(v4 + 2 * i + 1);
+      adamw_vec4(g[0], g[1], g[2], g[3], h, pa, ma, va, a);
+      adamw_vec4(g[4], g[5], g[6], g[7], h, pb, mb, vb, a);
+      st_stream(p4 + 2 * i, pa); st_stream(p4 + 2 * i + 1, pb);
+      st_stream(m4 + 2 * i, ma); st_stream(m4 + 2 * i + 1, mb);
+      st_stream(v4 + 2 * i, va); st_stream(v4 + 2 * i + 1, vb);
+    }
+    const int t = (n8 << 3) + tid;  // ragged tail: fewer than 8 elements
+    if (t < ck.count) {
+      float g;
+      if (kBF16) {
+        g = __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const uint16_t*>(gbase)[t]) << 16);
+      } else {
+        g = reinterpret_cast<const float*>(gbase)[t];
+      }
+      float p = params[ck.start + t], m = m_arena[ck.start + t], v = v_arena[ck.start + t];
+      adamw_elem(g, h, p, m, v, a);
+      params[ck.start + t] = p;
+      m_arena[ck.start + t] = m;
+      v_arena[ck.start + t] = v;
+    }
+  }
+}
+
+// Clip-only: hat(g) = h * g written in the gradient dtype.  In place, chunks with h == 1 are skipped.
+template <bool kBF16>
+__global__ void __launch_bounds__(kThreads)
+adagc_scale_kernel(const void* __restrict__ gin, void* __restrict__ gout, const Chunk* __restrict__ chunks,
+                   int n_chunks, const float* __restrict__ h_arr, int in_place) {
+  constexpr int kEPV = kBF16 ? 8 : 4;
+  const int tid = threadIdx.x;
+  for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+    const Chunk ck = chunks[c];
+    const float h = h_arr[ck.tensor];
+    if (in_place && h == 1.0f) continue;
+    const int64_t boff = ck.start * (kBF16 ? 2 : 4);
+    const uint4* src = reinterpret_cast<const uint4*>(static_cast<const char*>(gin) + boff);
+    uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(gout) + boff);
+    const int nvec = ck.count / kEPV;
+#pragma unroll 4
+    for (int i = tid; i < nvec; i += kThreads) {
+      uint4 q = ld_stream(src + i);
+      if (kBF16) {
+        q.x = pack_bf16(h * bf16_lo(q.x), h * bf16_hi(q.x));
+        q.y = pack_bf16(h * bf16_lo(q.y), h * bf16_hi(q.y));
+        q.z = pack_bf16(h * bf16_lo(q.z), h * bf16_hi(q.z));
+        q.w = pack_bf16(h * bf16_lo(q.w), h * bf16_hi(q.w));
+      } else {
+        q.x = __float_as_uint(h * __uint_as_float(q.x));
+        q.y = __float_as_uint(h * __uint_as_float(q.y));
+        q.z = __float_as_uint(h * __uint_as_float(q.z));
+        q.w = __float_as_uint(h * __uint_as_float(q.w));
+      }
+      st_stream(dst + i, q);
+    }
+    const int t = nvec * kEPV + tid;
+    if (t < ck.count) {
+      if (kBF16) {
+        const uint16_t b = reinterpret_cast<const uint16_t*>(src)[t];
+        const float x = h * __uint_as_float(static_cast<uint32_t>(b) << 16);
+        reinterpret_cast<uint16_t*>(dst)[t] = static_cast<uint16_t>(f32_to_bf16_bits(x));
+      } else {
+        reinterpret_cast<float*>(dst)[t] = h * reinterpret_cast<const float*>(src)[t];
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Layout {  // byte offsets of the workspace sections
+  size_t chunks, tensors, partials, sumsq, norm, h, clip_count, scalars, flag, total;
+};
+
+Layout make_layout(int64_t n_chunks, int64_t T) {
+  Layout L;
+  size_t o = 0;
+  L.chunks = o;     o = align_up(o + sizeof(Chunk) * n_chunks, 256);
+  L.tensors = o;    o = align_up(o + sizeof(TensorEntry) * T, 256);
+  L.partials = o;   o = align_up(o + sizeof(double) * n_chunks, 256);
+  L.sumsq = o;      o = align_up(o + sizeof(double) * T, 256);
+  L.norm = o;       o = align_up(o + sizeof(float) * T, 256);
+  L.h = o;          o = align_up(o + sizeof(float) * T, 256);
+  L.clip_count = o; o = align_up(o + sizeof(uint64_t) * T, 256);
+  L.scalars = o;    o = align_up(o + 256, 256);  // steps_done (u64) at +0, status (i32) at +8
+  L.flag = o;       o = align_up(o + T, 256);
+  L.total = o;
+  return L;
+}
+
+int validate_desc(const adagc_desc* d, int64_t* n_chunks_out, int64_t* arena_elems_out) {
+  if (!d || !d->tensors || d->n_tensors < 1) return ADAGC_E_INVALID_ARG;
+  if (d->param_dtype != ADAGC_F32 || d->state_dtype != ADAGC_F32) return ADAGC_E_DTYPE;
+  if (d->grad_dtype != ADAGC_F32 && d->grad_dtype != ADAGC_BF16) return ADAGC_E_DTYPE;
+  if (!(d->lambda_abs > 0.0) || !std::isfinite(d->lambda_abs)) return ADAGC_E_INVALID_ARG;
+  const int64_t align = (d->grad_dtype == ADAGC_BF16) ? 8 : 4;
+  int64_t n_chunks = 0, extent = 0;
+  std::vector<std::pair<int64_t, int64_t>> spans;
+  spans.reserve(d->n_tensors);
+  for (int32_t i = 0; i < d->n_tensors; ++i) {
+    const adagc_tensor& t = d->tensors[i];
+    if (t.numel <= 0 || t.offset < 0 || t.ndim < 0 || t.ndim > 4) return ADAGC_E_INVALID_ARG;
+    if (t.numel > (int64_t(1) << 44) || t.offset > (int64_t(1) << 46)) return ADAGC_E_INVALID_ARG;
+    if (t.ndim > 0) {
+      int64_t prod = 1;
+      for (int k = 0; k < t.ndim; ++k) {
+        if (t.shape[k] <= 0) return ADAGC_E_INVALID_ARG;
+        prod *= t.shape[k];
+      }
+      if (prod != t.numel) return ADAGC_E_INVALID_ARG;
+    }
+    if (t.offset % align != 0) return ADAGC_E_MISALIGNED;
+    n_chunks += (t.numel + kChunkElems - 1) / kChunkElems;
+    extent = std::max(extent, t.offset + t.numel);
+    spans.emplace_back(t.offset, t.offset + t.numel);
+  }
+  if (n_chunks > int64_t(0x7fffffff)) return ADAGC_E_INVALID_ARG;
+  std::sort(spans.begin(), spans.end());
+  for (size_t k = 1; k < spans.size(); ++k)
+    if (spans[k].first < spans[k - 1].second) return ADAGC_E_OVERLAP;
+  if (n_chunks_out) *n_chunks_out = n_chunks;
+  if (arena_elems_out) *arena_elems_out = extent;
+  return ADAGC_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+struct adagc_ctx {
+  int32_t T = 0;
+  int32_t n_chunks = 0;
+  int64_t arena_elems = 0;
+  bool bf16 = false;
+  double lambda_abs = 1.0;
+  int device = 0;
+  int grid_norm = 1, grid_update = 1, grid_scale = 1;
+  char* ws = nullptr;
+  Layout L{};
+  uint64_t launches = 0;
+  bool timing = false;
+  bool timing_valid = false;
+  cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+  const Chunk* d_chunks() const { return reinterpret_cast<const Chunk*>(ws + L.chunks); }
+  const TensorEntry* d_tensors() const { return reinterpret_cast<const TensorEntry*>(ws + L.tensors); }
+  double* d_partials() const { return reinterpret_cast<double*>(ws + L.partials); }
+  StatPtrs stats() const {
+    StatPtrs s;
+    s.sumsq = reinterpret_cast<double*>(ws + L.sumsq);
+    s.norm = reinterpret_cast<float*>(ws + L.norm);
+    s.h = reinterpret_cast<float*>(ws + L.h);
+    s.flag = reinterpret_cast<uint8_t*>(ws + L.flag);
+    s.clip_count = reinterpret_cast<unsigned long long*>(ws + L.clip_count);
+    s.steps_done = reinterpret_cast<unsigned long long*>(ws + L.scalars);
+    s.status = reinterpret_cast<int*>(ws + L.scalars + 8);
+    return s;
+  }
+};
+
+namespace {
+
+int check_clip_args(const adagc_ctx* ctx, const float* d_ema, int64_t step, double lambda_rel, double beta,
+                    int64_t warmup) {
+  if (!ctx || !d_ema) return ADAGC_E_INVALID_ARG;
+  if (step < 1 || warmup < 0) return ADAGC_E_INVALID_ARG;
+  if (!(lambda_rel > 0.0) || !std::isfinite(lambda_rel)) return ADAGC_E_INVALID_ARG;
+  if (!(beta >= 0.0 && beta < 1.0)) return ADAGC_E_INVALID_ARG;
+  return ADAGC_OK;
+}
+
+// phases 1 and 2
+int enqueue_clip_phases(adagc_ctx* ctx, const void* d_grads, float* d_ema, int64_t step, double lambda_rel,
+                        double beta, int64_t warmup, cudaStream_t s) {
+  if (ctx->timing) cudaEventRecord(ctx->ev[0], s);
+  if (ctx->bf16)
+    adagc_norm_kernel<true><<<ctx->grid_norm, kThreads, 0, s>>>(d_grads, ctx->d_chunks(), ctx->n_chunks,
+                                                               ctx->d_partials());
+  else
+    adagc_norm_kernel<false><<<ctx->grid_norm, kThreads, 0, s>>>(d_grads, ctx->d_chunks(), ctx->n_chunks,
+                                                                ctx->d_partials());
+  ctx->launches++;
+  if (ctx->timing) cudaEventRecord(ctx->ev[1], s);
+  ClipScalars cs;
+  cs.lambda_rel = lambda_rel;
+  cs.beta = beta;
+  cs.one_minus_beta = 1.0 - beta;
+  cs.lambda_abs = ctx->lambda_abs;
+  cs.step = step;
+  cs.n_tensors = ctx->T;
+  const bool in_warmup = step <= warmup;
+  const int blocks = (ctx->T * 32 + kFinalizeThreads - 1) / kFinalizeThreads;
+  adagc_tensor_finalize_kernel<<<blocks, kFinalizeThreads, 0, s>>>(ctx->d_partials(), ctx->d_tensors(), cs,
+                                                                  in_warmup ? 0 : 1, d_ema, ctx->stats());
+  ctx->launches++;
+  if (in_warmup) {
+    adagc_warmup_finalize_kernel<<<1, kWarmupThreads, 0, s>>>(cs, d_ema, ctx->stats());
+    ctx->launches++;
+  }
+  if (ctx->timing) cudaEventRecord(ctx->ev[2], s);
+  return ADAGC_OK;
+}
+
+int finish_launches(adagc_ctx* ctx, cudaStream_t s) {
+  if (ctx->timing) {
+    cudaEventRecord(ctx->ev[3], s);
+    ctx->timing_valid = true;
+  }
+  return cudaGetLastError() == cudaSuccess ? ADAGC_OK : ADAGC_E_CUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t adagc_workspace_bytes(const adagc_desc* desc) {
+  int64_t n_chunks = 0;
+  if (validate_desc(desc, &n_chunks, nullptr) != ADAGC_OK) return 0;
+  return make_layout(n_chunks, desc->n_tensors).total;
+}
+
+int64_t adagc_num_chunks(const adagc_desc* desc) {
+  int64_t n_chunks = 0;
+  const int rc = validate_desc(desc, &n_chunks, nullptr);
+  return rc != ADAGC_OK ? rc : n_chunks;
+}
+
+int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_bytes, void* cuda_stream,
+                 adagc_ctx** out) {
+  if (!out) return ADAGC_E_INVALID_ARG;
+  *out = nullptr;
+  int64_t n_chunks = 0, extent = 0;
+  const int rc = validate_desc(desc, &n_chunks, &extent);
+  if (rc != ADAGC_OK) return rc;
+  const Layout L = make_layout(n_chunks, desc->n_tensors);
+  if (!d_workspace || workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(d_workspace) & 255u))
+    return ADAGC_E_WORKSPACE;
+
+  std::vector<Chunk> chunks;
+  std::vector<TensorEntry> tensors;
+  chunks.reserve(n_chunks);
+  tensors.reserve(desc->n_tensors);
+  for (int32_t i = 0; i < desc->n_tensors; ++i) {
+    const adagc_tensor& t = desc->tensors[i];
+    TensorEntry te;
+    te.first_chunk = static_cast<int32_t>(chunks.size());
+    for (int64_t o = 0; o < t.numel; o += kChunkElems) {
+      Chunk c;
+      c.start = t.offset + o;
+      c.count = static_cast<int32_t>(std::min<int64_t>(kChunkElems, t.numel - o));
+      c.tensor = i;
+      chunks.push_back(c);
+    }
+    te.n_chunks = static_cast<int32_t>(chunks.size()) - te.first_chunk;
+    tensors.push_back(te);
+  }
+
+  adagc_ctx* ctx = new (std::nothrow) adagc_ctx();
+  if (!ctx) return ADAGC_E_NOMEM;
+  ctx->T = desc->n_tensors;
+  ctx->n_chunks = static_cast<int32_t>(n_chunks);
+  ctx->arena_elems = extent;
+  ctx->bf16 = desc->grad_dtype == ADAGC_BF16;
+  ctx->lambda_abs = desc->lambda_abs;
+  ctx->ws = static_cast<char*>(d_workspace);
+  ctx->L = L;
+
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  cudaDeviceProp prop;
+  bool ok = cudaGetDevice(&ctx->device) == cudaSuccess &&
+            cudaGetDeviceProperties(&prop, ctx->device) == cudaSuccess;
+  if (ok) {
+    int occ_n = 0, occ_u = 0, occ_s = 0;
+    if (ctx->bf16) {
+      ok = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_n, adagc_norm_kernel<true>, kThreads, 0) == cudaSuccess &&
+           cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_u, adagc_update_kernel<true>, kThreads, 0) == cudaSuccess &&
+           cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_s, adagc_scale_kernel<true>, kThreads, 0) == cudaSuccess;
+    } else {
+      ok = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_n, adagc_norm_kernel<false>, kThreads, 0) == cudaSuccess &&
+           cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_u, adagc_update_kernel<false>, kThreads, 0) == cudaSuccess &&
+           cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_s, adagc_scale_kernel<false>, kThreads, 0) == cudaSuccess;
+    }
+    if (ok) {
+      const int64_t sms = prop.multiProcessorCount;
+      ctx->grid_norm = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(n_chunks, sms * std::max(occ_n, 1))));
+      ctx->grid_update = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(n_chunks, sms * std::max(occ_u, 1))));
+      ctx->grid_scale = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(n_chunks, sms * std::max(occ_s, 1))));
+    }
+  }
+  ok = ok && cudaMemsetAsync(ctx->ws, 0, L.total, s) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(ctx->ws + L.chunks, chunks.data(), sizeof(Chunk) * chunks.size(),
+                             cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(ctx->ws + L.tensors, tensors.data(), sizeof(TensorEntry) * tensors.size(),
+                             cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok = ok && cudaStreamSynchronize(s) == cudaSuccess;  // the host vectors die at return
+  for (int k = 0; ok && k < 4; ++k) ok = cudaEventCreate(&ctx->ev[k]) == cudaSuccess;
+  if (!ok) {
+    (void)cudaGetLastError();
+    for (int k = 0; k < 4; ++k)
+      if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
+    delete ctx;
+    return ADAGC_E_CUDA;
+  }
+  *out = ctx;
+  return ADAGC_OK;
+}
+
+int adagc_destroy(adagc_ctx* ctx) {
+  if (!ctx) return ADAGC_E_INVALID_ARG;
+  for (int k = 0; k < 4; ++k)
+    if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
+  delete ctx;
+  return ADAGC_OK;
+}
+
+int adagc_step(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, void* d_v, float* d_ema,
+               int64_t step, double lr, double beta1, double beta2, double eps, double wd, double lambda_rel,
+               double beta, int64_t warmup, void* cuda_stream) {
+  int rc = check_clip_args(ctx, d_ema, step, lambda_rel, beta, warmup);
+  if (rc != ADAGC_OK) return rc;
+  if (!d_params || !d_grads || !d_m || !d_v) return ADAGC_E_INVALID_ARG;
+  if (!(beta1 >= 0.0 && beta1 < 1.0) || !(beta2 >= 0.0 && beta2 < 1.0)) return ADAGC_E_INVALID_ARG;
+  if (!(eps >= 0.0) || !std::isfinite(eps) || !std::isfinite(lr) || !std::isfinite(wd)) return ADAGC_E_INVALID_ARG;
+  if (!aligned16(d_params) || !aligned16(d_grads) || !aligned16(d_m) || !aligned16(d_v)) return ADAGC_E_MISALIGNED;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  rc = enqueue_clip_phases(ctx, d_grads, d_ema, step, lambda_rel, beta, warmup, s);
+  if (rc != ADAGC_OK) return rc;
+
+  // scalar coefficients in double, rounded once to the kernel's fp32
+  const double bc1 = 1.0 - std::pow(beta1, static_cast<double>(step));
+  const double bc2 = 1.0 - std::pow(beta2, static_cast<double>(step));
+  AdamScalars a;
+  a.beta1 = static_cast<float>(beta1);
+  a.one_minus_beta1 = static_cast<float>(1.0 - beta1);
+  a.beta2 = static_cast<float>(beta2);
+  a.one_minus_beta2 = static_cast<float>(1.0 - beta2);
+  a.inv_bc2 = static_cast<float>(1.0 / bc2);
+  a.step_size = static_cast<float>(lr / bc1);
+  a.decay = static_cast<float>(1.0 - lr * wd);
+  a.eps = static_cast<float>(eps);
+  const StatPtrs st = ctx->stats();
+  if (ctx->bf16)
+    adagc_update_kernel<true><<<ctx->grid_update, kThreads, 0, s>>>(
+        static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), static_cast<float*>(d_v),
+        ctx->d_chunks(), ctx->n_chunks, st.h, a);
+  else
+    adagc_update_kernel<false><<<ctx->grid_update, kThreads, 0, s>>>(
+        static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), static_cast<float*>(d_v),
+        ctx->d_chunks(), ctx->n_chunks, st.h, a);
+  ctx->launches++;
+  return finish_launches(ctx, s);
+}
+
+int adagc_clip(adagc_ctx* ctx, const void* d_grads_in, void* d_grads_out, float* d_ema, int64_t step,
+               double lambda_rel, double beta, int64_t warmup, void* cuda_stream) {
+  int rc = check_clip_args(ctx, d_ema, step, lambda_rel, beta, warmup);
+  if (rc != ADAGC_OK) return rc;
+  if (!d_grads_in || !d_grads_out) return ADAGC_E_INVALID_ARG;
+  if (!aligned16(d_grads_in) || !aligned16(d_grads_out)) return ADAGC_E_MISALIGNED;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  rc = enqueue_clip_phases(ctx, d_grads_in, d_ema, step, lambda_rel, beta, warmup, s);
+  if (rc != ADAGC_OK) return rc;
+  const int in_place = d_grads_in == d_grads_out ? 1 : 0;
+  if (ctx->bf16)
+    adagc_scale_kernel<true><<<ctx->grid_scale, kThreads, 0, s>>>(d_grads_in, d_grads_out, ctx->d_chunks(),
+                                                                 ctx->n_chunks, ctx->stats().h, in_place);
+  else
+    adagc_scale_kernel<false><<<ctx->grid_scale, kThreads, 0, s>>>(d_grads_in, d_grads_out, ctx->d_chunks(),
+                                                                  ctx->n_chunks, ctx->stats().h, in_place);
+  ctx->launches++;
+  return finish_launches(ctx, s);
+}
+
+int adagc_get_stats(adagc_ctx* ctx, float* h_norm, float* h_clipfactor, uint8_t* h_flag, uint64_t* h_clip_count,
+                    uint64_t* h_steps_done, int32_t* h_device_status, void* cuda_stream) {
+  if (!ctx) return ADAGC_E_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const StatPtrs st = ctx->stats();
+  const size_t T = static_cast<size_t>(ctx->T);
+  bool ok = true;
+  if (h_norm) ok = ok && cudaMemcpyAsync(h_norm, st.norm, 4 * T, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  if (h_clipfactor) ok = ok && cudaMemcpyAsync(h_clipfactor, st.h, 4 * T, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  if (h_flag) ok = ok && cudaMemcpyAsync(h_flag, st.flag, T, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  if (h_clip_count)
+    ok = ok && cudaMemcpyAsync(h_clip_count, st.clip_count, 8 * T, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  if (h_steps_done)
+    ok = ok && cudaMemcpyAsync(h_steps_done, st.steps_done, 8, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  if (h_device_status)
+    ok = ok && cudaMemcpyAsync(h_device_status, st.status, 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  ok = ok && cudaStreamSynchronize(s) == cudaSuccess;
+  return ok ? ADAGC_OK : ADAGC_E_CUDA;
+}
+
+int adagc_get_sumsq(adagc_ctx* ctx, double* h_sumsq, void* cuda_stream) {
+  if (!ctx || !h_sumsq) return ADAGC_E_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  bool ok = cudaMemcpyAsync(h_sumsq, ctx->stats().sumsq, 8 * static_cast<size_t>(ctx->T),
+                            cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  ok = ok && cudaStreamSynchronize(s) == cudaSuccess;
+  return ok ? ADAGC_OK : ADAGC_E_CUDA;
+}
+
+int adagc_step_host(adagc_ctx* ctx, void* d_params, void* d_grads, void* d_m, void* d_v, float* d_ema,
+                    const void* h_grads, int64_t step, double lr, double beta1, double beta2, double eps,
+                    double wd, double lambda_rel, double beta, int64_t warmup, float* h_norm,
+                    float* h_clipfactor, uint8_t* h_flag, void* cuda_stream) {
+  if (!ctx || !h_grads || !d_grads) return ADAGC_E_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const size_t bytes = static_cast<size_t>(ctx->arena_elems) * (ctx->bf16 ? 2 : 4);
+  if (cudaMemcpyAsync(d_grads, h_grads, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return ADAGC_E_CUDA;
+  const int rc = adagc_step(ctx, d_params, d_grads, d_m, d_v, d_ema, step, lr, beta1, beta2, eps, wd,
+                            lambda_rel, beta, warmup, cuda_stream);
+  if (rc != ADAGC_OK) return rc;
+  return adagc_get_stats(ctx, h_norm, h_clipfactor, h_flag, nullptr, nullptr, nullptr, cuda_stream);
+}
+
+int64_t adagc_arena_elems(const adagc_ctx* ctx) { return ctx ? ctx->arena_elems : ADAGC_E_INVALID_ARG; }
+
+uint64_t adagc_launch_count(const adagc_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int adagc_set_phase_timing(adagc_ctx* ctx, int enabled) {
+  if (!ctx) return ADAGC_E_INVALID_ARG;
+  ctx->timing = enabled != 0;
+  ctx->timing_valid = false;
+  return ADAGC_OK;
+}
+
+int adagc_get_phase_times(adagc_ctx* ctx, float ms[3]) {
+  if (!ctx || !ms || !ctx->timing_valid) return ADAGC_E_INVALID_ARG;
+  if (cudaEventSynchronize(ctx->ev[3]) != cudaSuccess) return ADAGC_E_CUDA;
+  for (int k = 0; k < 3; ++k)
+    if (cudaEventElapsedTime(&ms[k], ctx->ev[k], ctx->ev[k + 1]) != cudaSuccess) return ADAGC_E_CUDA;
+  return ADAGC_OK;
+}
+
+const char* adagc_strerror(int status) {
+  switch (status) {
+    case ADAGC_OK: return "ok";
+    case ADAGC_E_INVALID_ARG: return "invalid argument";
+    case ADAGC_E_MISALIGNED: return "tensor offset or arena pointer not 16-byte aligned";
+    case ADAGC_E_OVERLAP: return "tensors overlap";
+    case ADAGC_E_WORKSPACE: return "workspace too small or misaligned";
+    case ADAGC_E_DTYPE: return "unsupported dtype combination";
+    case ADAGC_E_CUDA: return "CUDA runtime error";
+    case ADAGC_E_NOMEM: return "host allocation failed";
+    default: return "unknown status";
+  }
+}
+
+}  // extern "C"

@@ -1,0 +1,242 @@
+"""Drives the CUDA library and the CPU oracle over the same seeded inputs and compares them.
+
+The gradients and the initial parameters are drawn once (on the device the CUDA path runs on)
+and the same bits are copied to the host for the oracle; no expected value ever comes from the
+CUDA path.  Tolerances (stated by the target of this work, repeated in each test):
+  clip flags, clip counts, step counter: bit-exact;
+  norms, gamma, h: 1e-5 relative;  float64 sums of squares: 1e-11 relative;
+  fp32 theta, m, v: per tensor ||delta||_2 <= 1e-5 ||ref||_2 and per element
+  |delta| <= 1e-5 * max(|ref|, rms(ref));  bf16 clipped gradients: 1 bf16 ulp.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional
+
+import numpy as np
+import torch
+
+from oracle import c_oracle
+from paper_2502_11034_b200 import binding, workloads
+
+RTOL = 1e-5
+
+
+def to_numpy_grads(g: torch.Tensor) -> np.ndarray:
+    g = g.detach().cpu().contiguous()
+    if g.dtype == torch.bfloat16:
+        return g.view(torch.int16).numpy().view(np.uint16)
+    return g.numpy()
+
+
+def hyper_of(wl: workloads.Workload, **over) -> Dict[str, float]:
+    hp = dict(wl.hyper)
+    hp["warmup"] = wl.warmup
+    hp.update(over)
+    return hp
+
+
+@dataclass
+class ParityReport:
+    steps: int = 0
+    decisions: int = 0
+    clipped: int = 0
+    min_margin: float = math.inf
+    max_norm_rel: float = 0.0
+    max_gamma_rel: float = 0.0
+    max_sumsq_rel: float = 0.0
+    max_tensor_rel: Dict[str, float] = field(default_factory=dict)
+    gamma_bit_mismatch: int = 0
+
+    def line(self) -> str:
+        return (f"steps={self.steps} decisions={self.decisions} clipped={self.clipped} "
+                f"min_margin={self.min_margin:.3e} norm_rel={self.max_norm_rel:.2e} "
+                f"gamma_rel={self.max_gamma_rel:.2e} gamma_bit_mismatch={self.gamma_bit_mismatch} "
+                f"sumsq_rel={self.max_sumsq_rel:.2e} state_rel={self.max_tensor_rel}")
+
+
+def _rel(a: np.ndarray, b: np.ndarray) -> float:
+    a, b = np.asarray(a, np.float64), np.asarray(b, np.float64)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        r = np.abs(a - b) / np.abs(b)
+    r[(a == b)] = 0.0
+    r[np.isnan(a) & np.isnan(b)] = 0.0
+    return float(np.max(r)) if r.size else 0.0
+
+
+def check_decisions(st, sumsq_gpu, gamma_gpu, r, rep: ParityReport, step: int):
+    """Per-step comparison of what the finalize phase produced."""
+    flag_ref = np.asarray(r["flag"], bool)
+    if not np.array_equal(st["flag"], flag_ref):
+        bad = np.nonzero(st["flag"] != flag_ref)[0]
+        raise AssertionError(f"step {step}: clip decisions differ at tensors {bad[:10]} "
+                             f"(margins {np.asarray(r['margin'])[bad[:10]]})")
+    rep.decisions += len(flag_ref)
+    rep.clipped += int(flag_ref.sum())
+    rep.min_margin = min(rep.min_margin, float(np.min(r["margin"])))
+    rep.max_norm_rel = max(rep.max_norm_rel, _rel(st["norm"], r["norm"]))
+    rep.max_gamma_rel = max(rep.max_gamma_rel, _rel(gamma_gpu, r["gamma"]))
+    rep.gamma_bit_mismatch += int((np.asarray(gamma_gpu, np.float32).view(np.uint32) !=
+                                   np.asarray(r["gamma"], np.float32).view(np.uint32)).sum())
+    rep.max_sumsq_rel = max(rep.max_sumsq_rel, _rel(sumsq_gpu, np.asarray(r["norm"], np.float64) ** 2))
+    assert _rel(st["norm"], r["norm"]) <= RTOL, f"step {step}: norms differ"
+    assert _rel(gamma_gpu, r["gamma"]) <= RTOL, f"step {step}: gamma differs"
+    assert _rel(st["h"], r["h"]) <= RTOL, f"step {step}: clip factors differ"
+    assert _rel(sumsq_gpu, np.asarray(r["norm"], np.float64) ** 2) <= 1e-11, f"step {step}: float64 sums of squares differ"
+
+
+def check_state(name: str, got: np.ndarray, ref: np.ndarray, rep: ParityReport, what: str = ""):
+    """fp32 state of one tensor: relative L2 error and per-element error."""
+    got, ref = np.asarray(got, np.float64), np.asarray(ref, np.float64)
+    nref = float(np.linalg.norm(ref))
+    d = float(np.linalg.norm(got - ref))
+    rel = d / nref if nref > 0 else d
+    rep.max_tensor_rel[name] = max(rep.max_tensor_rel.get(name, 0.0), rel)
+    assert rel <= RTOL, f"{name} of {what}: ||delta||/||ref|| = {rel:.3e}"
+    rms = nref / math.sqrt(max(ref.size, 1))
+    bound = RTOL * np.maximum(np.abs(ref), rms)
+    worst = np.abs(got - ref) - bound
+    assert (worst <= 0).all(), f"{name} of {what}: element error {np.abs(got - ref).max():.3e} above bound"
+
+
+def run_full(wl: workloads.Workload, n_steps: int, device="cuda", hyper_over: Optional[dict] = None,
+             lr_schedule=None, canary: bool = True) -> ParityReport:
+    """Every element of every tensor, fused AdaGC+AdamW step, GPU vs C oracle."""
+    hp = hyper_of(wl, **(hyper_over or {}))
+    offs = [t.offset for t in wl.tensors]
+    nums = [t.numel for t in wl.tensors]
+    opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=device)
+    theta = workloads.init_params(wl, device)
+    theta0 = theta.cpu().numpy().copy()
+    pad_mask = None
+    if canary and wl.arena_elems != wl.n_params:
+        pad = np.ones(wl.arena_elems, bool)
+        for o, n in zip(offs, nums):
+            pad[o:o + n] = False
+        pad_mask = torch.from_numpy(pad).to(device)
+        theta[pad_mask] = 777.0
+    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    if pad_mask is not None:
+        m[pad_mask] = 777.0
+        v[pad_mask] = 777.0
+    ema = torch.full((wl.n_tensors,), float("nan"), dtype=torch.float32, device=device)  # must be ignored at t=1
+    ref = c_oracle.ArenaOracle(offs, nums, theta0, lr=hp["lr"], beta1=hp["beta1"], beta2=hp["beta2"],
+                               eps=hp["eps"], wd=hp["wd"], lambda_rel=hp["lambda_rel"], beta=hp["beta"],
+                               lambda_abs=hp["lambda_abs"], warmup=hp["warmup"])
+    rep = ParityReport()
+    for t in range(1, n_steps + 1):
+        g = workloads.grads_for_step(wl, t, device)
+        lr = hp["lr"] if lr_schedule is None else lr_schedule(t)
+        opt.step(theta, g, m, v, ema, t, lr, hp["beta1"], hp["beta2"], hp["eps"], hp["wd"],
+                 hp["lambda_rel"], hp["beta"], hp["warmup"])
+        r = ref.step(to_numpy_grads(g), lr=lr)
+        st = opt.get_stats()
+        check_decisions(st, opt.get_sumsq(), ema.cpu().numpy(), r, rep, t)
+        rep.steps = t
+    st = opt.get_stats()
+    assert st["steps_done"] == n_steps
+    assert np.array_equal(st["clip_count"], ref.clip_count)
+    assert st["status"] == 0
+    th, mm, vv = theta.cpu().numpy(), m.cpu().numpy(), v.cpu().numpy()
+    for t_, o, n in zip(wl.tensors, offs, nums):
+        check_state("theta", th[o:o + n], ref.theta[o:o + n], rep, t_.name)
+        check_state("m", mm[o:o + n], ref.m[o:o + n], rep, t_.name)
+        check_state("v", vv[o:o + n], ref.v[o:o + n], rep, t_.name)
+    if pad_mask is not None:
+        for a in (theta, m, v):
+            assert bool((a[pad_mask] == 777.0).all()), "guard bands between tensors were overwritten"
+    opt.close()
+    return rep
+
+
+def sample_indices(numel: int, k: int, rng: np.random.RandomState, chunk: int = 16384) -> np.ndarray:
+    """Element indices of one tensor to check: both ends, around chunk boundaries, and random ones."""
+    idx = [np.arange(min(numel, 32)), np.arange(max(0, numel - 32), numel)]
+    for b in (chunk, 2 * chunk, (numel // chunk) * chunk):
+        if 0 < b < numel:
+            idx.append(np.arange(max(0, b - 9), min(numel, b + 9)))
+    if numel > 64:
+        idx.append(rng.randint(0, numel, size=k))
+    return np.unique(np.concatenate(idx)).astype(np.int64)
+
+
+def run_sampled(wl: workloads.Workload, n_steps: int, device="cuda", k: int = 2048,
+                mode: str = "adamw", in_place: bool = True, hyper_over: Optional[dict] = None) -> ParityReport:
+    """Full-size layouts: all norms / decisions / gamma against the oracle (it streams the whole
+    gradient), theta/m/v (or the clipped gradient) on sampled elements the oracle computes one by one.
+    Legal because, given h_i, the update of an element depends on that element only (Algorithm 1)."""
+    hp = hyper_of(wl, **(hyper_over or {}))
+    offs = np.array([t.offset for t in wl.tensors], np.int64)
+    nums = np.array([t.numel for t in wl.tensors], np.int64)
+    opt = binding.AdaGC(nums.tolist(), offs.tolist(), wl.torch_grad_dtype, hp["lambda_abs"], device=device)
+    rng = np.random.RandomState(99)
+    samp = [sample_indices(int(n), k, rng) + int(o) for o, n in zip(offs, nums)]   # arena indices per tensor
+    sizes = np.array([len(s) for s in samp], np.int64)
+    soff = np.concatenate([[0], np.cumsum(sizes)[:-1]]).astype(np.int64)
+    flat = torch.from_numpy(np.concatenate(samp)).to(device)
+    rep = ParityReport()
+    gamma = np.zeros(wl.n_tensors, np.float32)
+    clip_count = np.zeros(wl.n_tensors, np.uint64)
+    ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device=device)
+    if mode == "adamw":
+        theta = workloads.init_params(wl, device)
+        m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+        s_theta = theta[flat].cpu().numpy().copy()
+        s_m, s_v = np.zeros_like(s_theta), np.zeros_like(s_theta)
+    g_out = None
+    for t in range(1, n_steps + 1):
+        g = workloads.grads_for_step(wl, t, device)
+        g_np = to_numpy_grads(g)                         # the same bits, for the oracle
+        s_g = np.ascontiguousarray(g_np[flat.cpu().numpy()])
+        if mode == "adamw":
+            opt.step(theta, g, m, v, ema, t, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"],
+                     hp["lambda_rel"], hp["beta"], hp["warmup"])
+        else:
+            g_out = g if in_place else torch.empty_like(g)
+            opt.clip(g, g_out, ema, t, hp["lambda_rel"], hp["beta"], hp["warmup"])
+        ssq = c_oracle.sumsq_tensors(g_np, offs, nums)
+        r = c_oracle.clip_decisions(ssq, gamma, t, hp["lambda_rel"], hp["beta"], hp["lambda_abs"], hp["warmup"])
+        clip_count += r["flag"].astype(np.uint64)
+        st = opt.get_stats()
+        check_decisions(st, opt.get_sumsq(), ema.cpu().numpy(), r, rep, t)
+        for i in range(wl.n_tensors):
+            sl = slice(int(soff[i]), int(soff[i] + sizes[i]))
+            if mode == "adamw":
+                c_oracle.adamw_update(s_theta[sl], s_g[sl], s_m[sl], s_v[sl], float(r["h"][i]), t,
+                                      hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"])
+        if mode != "adamw":
+            got = to_numpy_grads(g_out[flat])
+            want = np.empty_like(s_g)
+            for i in range(wl.n_tensors):
+                sl = slice(int(soff[i]), int(soff[i] + sizes[i]))
+                c_oracle.scale(s_g[sl], float(r["h"][i]), out=want[sl])
+            check_clipped_grads(got, want, f"step {t}")
+        rep.steps = t
+        del g
+    st = opt.get_stats()
+    assert st["steps_done"] == n_steps and np.array_equal(st["clip_count"], clip_count) and st["status"] == 0
+    if mode == "adamw":
+        g_theta, g_m, g_v = (a[flat].cpu().numpy() for a in (theta, m, v))
+        for i, t_ in enumerate(wl.tensors):
+            sl = slice(int(soff[i]), int(soff[i] + sizes[i]))
+            check_state("theta", g_theta[sl], s_theta[sl], rep, t_.name)
+            check_state("m", g_m[sl], s_m[sl], rep, t_.name)
+            check_state("v", g_v[sl], s_v[sl], rep, t_.name)
+    opt.close()
+    return rep
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def check_clipped_grads(got: np.ndarray, want: np.ndarray, what: str):
+    """Clipped gradients in the gradient dtype: fp32 within 1e-5 relative, bf16 within one bf16 ulp."""
+    if got.dtype == np.uint16:
+        a, b = bf16_bits_to_f64(got), bf16_bits_to_f64(want)
+        ulp = np.maximum(np.abs(b), 2.0 ** -126) * 2.0 ** -7     # spacing is at most 2^-7 relative
+        assert (np.abs(a - b) <= ulp).all(), f"{what}: bf16 clipped gradient off by more than one ulp"
+    else:
+        a, b = got.astype(np.float64), want.astype(np.float64)
+        assert (np.abs(a - b) <= RTOL * np.abs(b) + 1e-45).all(), f"{what}: clipped gradient differs"

@@ -1,0 +1,274 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle.
+
+Bar: clip flags / clip counts / step counter bit-exact; norms, gamma, h within 1e-5 relative;
+fp32 theta, m, v within 1e-5 (per-tensor L2 and per element); bf16 clipped gradients within one ulp.
+"""
+import numpy as np
+import pytest
+import torch
+
+from paper_2502_11034_b200 import binding, workloads
+
+import parity_harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _report(name, rep):
+    print(f"\n[parity] {name}: {rep.line()}")
+
+
+# ------------------------------------------------------------------ the five configurations
+def test_tiny_all_elements():
+    """Config 1: 8 fp32 tensors, 12 steps, x100 spike on tensor index 3 at step 6."""
+    wl = workloads.build("tiny")
+    rep = H.run_full(wl, wl.n_steps)
+    _report("tiny", rep)
+    assert rep.clipped > 0
+    # lambda_abs = 1 never clips this layout in warm-up; a smaller threshold exercises that branch
+    rep2 = H.run_full(wl, wl.n_steps, hyper_over=dict(lambda_abs=0.5))
+    _report("tiny lambda_abs=0.5", rep2)
+    # the 1-based reading of "tensor 3"
+    wl.extra["spike_tensor"] = 2
+    _report("tiny spike on index 2", H.run_full(wl, wl.n_steps))
+
+
+def test_gpt2_small_all_elements():
+    """Config 2: 148 tensors, bf16 gradients with per-tensor scales, 50 steps, 1% spiked x50 per step."""
+    wl = workloads.build("gpt2_small")
+    rep = H.run_full(wl, wl.n_steps)
+    _report("gpt2_small", rep)
+    assert rep.decisions == 148 * 50 and rep.clipped > 0
+
+
+def test_many_small_all_elements():
+    """Config 4: 20 000 fp32 tensors, Student-t(2) gradients, 30 steps."""
+    wl = workloads.build("many_small")
+    rep = H.run_full(wl, wl.n_steps)
+    _report("many_small", rep)
+    assert rep.decisions == 20000 * 30 and rep.clipped > 0
+
+
+def test_llama32_1b_sampled_adamw_and_clip_only():
+    """Config 5 at full size: all decisions for 100 steps; state / clipped gradients on samples."""
+    wl = workloads.build("llama32_1b")
+    rep = H.run_sampled(wl, wl.n_steps, mode="adamw")
+    _report("llama32_1b adamw", rep)
+    assert rep.decisions == 146 * 100 and rep.clipped > 0
+    rep = H.run_sampled(wl, 30, mode="clip", in_place=True)
+    _report("llama32_1b clip-only in place", rep)
+    rep = H.run_sampled(wl, 14, mode="clip", in_place=False)
+    _report("llama32_1b clip-only out of place", rep)
+
+
+def test_llama2_7b_sampled():
+    """Config 3 at full size (the benchmark's launch configuration): 20 steps, spike at step 12."""
+    free, _ = torch.cuda.mem_get_info()
+    wl = workloads.build("llama2_7b")
+    need = wl.arena_elems * 14 + (4 << 30)
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GiB of device memory, {free >> 30} GiB free")
+    rep = H.run_sampled(wl, wl.n_steps, mode="adamw", k=1024)
+    _report("llama2_7b", rep)
+    assert rep.decisions == 291 * 20
+    assert rep.clipped >= 8
+
+
+# ------------------------------------------------------------------ small layouts, all elements
+@pytest.mark.parametrize("name,over", [
+    ("llama2_7b", dict(n_layer=2, d=256, ffn=688, vocab=1000)),
+    ("llama32_1b", dict(n_layer=2, d=128, ffn=512, vocab=2000, kv_dim=32)),
+    ("gpt2_small", dict(n_layer=2, d=96, vocab=1031, n_pos=64)),
+    ("many_small", dict(n_tensors=300, lo=1, hi=40000)),
+])
+def test_small_layouts_all_elements(name, over):
+    wl = workloads.build(name, **over)
+    rep = H.run_full(wl, min(wl.n_steps, 25))
+    _report(f"{name} (small)", rep)
+
+
+def _ragged_workload(sizes, dtype):
+    specs, total = workloads._layout([(f"t{i}", (n,)) for i, n in enumerate(sizes)])
+    hp = dict(workloads.PAPER_DEFAULTS, lambda_abs=0.05)
+    return workloads.Workload("ragged", 7, specs, dtype, hp, warmup=2, n_steps=8, arena_elems=total,
+                              grad_kind="student_t", grad_df=3, grad_scale=1e-3,
+                              extra={"spike_frac": 0.2, "spike_lo": 5.0, "spike_hi": 500.0})
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_ragged_tails_and_chunk_edges(dtype):
+    """Sizes around the vector width and the 16384-element chunk: tails of 1..7 elements,
+    one element short of / past a chunk, several chunks plus a tail."""
+    sizes = [1, 2, 3, 5, 7, 8, 9, 10, 15, 16, 17, 31, 33, 255, 257, 2047, 2049, 16383, 16384, 16385,
+             32767, 32768, 32769, 3 * 16384 + 5, 100003]
+    rep = H.run_full(_ragged_workload(sizes, dtype), 8)
+    _report(f"ragged {dtype}", rep)
+    assert rep.clipped > 0
+
+
+def test_single_tensor_and_warmup_zero():
+    """T = 1 (the 'global adaptive' view) and T_start = 0 (gamma seeded from the first norm)."""
+    wl = _ragged_workload([50000], "bf16")
+    _report("T=1", H.run_full(wl, 6))
+    wl = _ragged_workload([40, 5000, 70000], "f32")
+    _report("warmup=0", H.run_full(wl, 8, hyper_over=dict(warmup=0)))
+    _report("always warm-up", H.run_full(wl, 5, hyper_over=dict(warmup=100, lambda_abs=1e-3)))
+    _report("eps=1e-15, beta2=0.999, lr schedule",
+            H.run_full(wl, 8, hyper_over=dict(eps=1e-15, beta2=0.999), lr_schedule=lambda t: 1e-3 * t / 8))
+
+
+# ------------------------------------------------------------------ properties and edge cases
+def _mini():
+    wl = workloads.build("llama2_7b", n_layer=1, d=128, ffn=344, vocab=500)
+    offs, nums = [t.offset for t in wl.tensors], [t.numel for t in wl.tensors]
+    return wl, offs, nums
+
+
+def _run_gpu(wl, offs, nums, steps, start_state=None, first_step=1):
+    hp = H.hyper_of(wl)
+    opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"])
+    if start_state is None:
+        theta = workloads.init_params(wl, "cuda")
+        m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+        ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device="cuda")
+    else:
+        theta, m, v, ema = (a.clone() for a in start_state)
+    flags = []
+    for t in range(first_step, first_step + steps):
+        g = workloads.grads_for_step(wl, t, "cuda")
+        opt.step(theta, g, m, v, ema, t, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"],
+                 hp["lambda_rel"], hp["beta"], hp["warmup"])
+        flags.append(opt.get_stats()["flag"].copy())
+    opt.close()
+    return (theta, m, v, ema), flags
+
+
+def test_run_twice_is_bit_identical():
+    wl, offs, nums = _mini()
+    a, fa = _run_gpu(wl, offs, nums, 12)
+    b, fb = _run_gpu(wl, offs, nums, 12)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+    assert all(np.array_equal(p, q) for p, q in zip(fa, fb))
+
+
+def test_checkpoint_resume_is_bit_identical():
+    """The caller's buffers (theta, m, v, gamma) and the step number are the whole state."""
+    wl, offs, nums = _mini()
+    full, _ = _run_gpu(wl, offs, nums, 16)
+    half, _ = _run_gpu(wl, offs, nums, 8)
+    saved = tuple(a.cpu() for a in half)                        # "checkpoint"
+    resumed, _ = _run_gpu(wl, offs, nums, 8, start_state=tuple(a.cuda() for a in saved), first_step=9)
+    for x, y in zip(full, resumed):
+        assert torch.equal(x, y)
+
+
+def test_zero_and_nonfinite_gradients_and_absorbing_gamma():
+    from oracle import c_oracle
+    nums, offs = [1000, 24, 3000], [0, 1000, 1024]
+    opt = binding.AdaGC(nums, offs, torch.float32, 1.0)
+    theta = torch.randn(4024, device="cuda", generator=torch.Generator("cuda").manual_seed(5))
+    theta0 = theta.cpu().numpy().copy()
+    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    ema = torch.zeros(3, dtype=torch.float32, device="cuda")
+    hp = dict(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, wd=0.1, lambda_rel=1.04, beta=0.9, lambda_abs=1.0, warmup=0)
+    ref = c_oracle.ArenaOracle(offs, nums, theta0, **hp)
+    gen = torch.Generator("cuda").manual_seed(6)
+    for t in range(1, 7):
+        g = torch.randn(4024, device="cuda", generator=gen) * 1e-2
+        if t == 1:
+            g[1000:1024] = 0.0                                  # gamma of tensor 1 seeded with 0 ...
+        if t in (3, 4):
+            g[0:1000] = 0.0                                     # zero gradient: no clip, gamma decays
+        if t == 5:
+            g[1024 + 17] = float("inf")
+        if t == 6:
+            g[1024 + 5] = float("nan")
+        opt.step(theta, g, m, v, ema, t, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"],
+                 hp["lambda_rel"], hp["beta"], hp["warmup"])
+        r = ref.step(g.cpu().numpy())
+        st = opt.get_stats()
+        assert np.array_equal(st["flag"], r["flag"]), f"step {t}"
+        got, want = ema.cpu().numpy(), r["gamma"]
+        assert np.array_equal(np.isnan(got), np.isnan(want)) and np.array_equal(np.isinf(got), np.isinf(want))
+        fin = np.isfinite(want)
+        np.testing.assert_allclose(got[fin], want[fin], rtol=1e-5)
+        if t >= 2:
+            assert st["flag"][1] and st["h"][1] == 0.0 and got[1] == 0.0      # ... is absorbing
+        assert (st["status"] & binding.ADAGC_W_NONFINITE) == (binding.ADAGC_W_NONFINITE if t >= 5 else 0)
+    th = theta.cpu().numpy()
+    bad = np.isnan(ref.theta)
+    assert np.array_equal(np.isnan(th), bad)                     # NaN propagates as in plain AdamW ...
+    assert set(np.nonzero(bad)[0]) == {1024 + 17, 1024 + 5}      # ... and only where the gradient was bad
+    np.testing.assert_allclose(th[~bad], ref.theta[~bad], rtol=1e-5, atol=1e-7)
+    opt.close()
+
+
+def test_argument_errors_enqueue_nothing():
+    nums, offs = [100, 60], [0, 104]
+    opt = binding.AdaGC(nums, offs, torch.bfloat16, 1.0)
+    theta = torch.ones(164, device="cuda")
+    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    g = torch.ones(164, device="cuda", dtype=torch.bfloat16)
+    ema = torch.zeros(2, device="cuda")
+    ok = dict(step=1, lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, wd=0.1, lambda_rel=1.04, beta=0.99, warmup=0)
+    for bad in (dict(step=0), dict(beta=1.0), dict(beta=-0.1), dict(lambda_rel=0.0), dict(beta1=1.0),
+                dict(eps=-1.0), dict(warmup=-1), dict(lr=float("nan"))):
+        kw = dict(ok, **bad)
+        with pytest.raises(binding.AdagcError) as e:
+            opt.step(theta, g, m, v, ema, **kw)
+        assert e.value.status == -1
+    with pytest.raises(binding.AdagcError) as e:
+        opt.step(theta[1:], g, m, v, ema, **ok)                   # misaligned arena pointer
+    assert e.value.status == -2
+    torch.cuda.synchronize()
+    assert opt.launch_count() == 0 and bool((theta == 1).all()) and opt.get_stats()["steps_done"] == 0
+    opt.close()
+
+
+def test_phase_timing_and_launch_count():
+    wl, offs, nums = _mini()
+    hp = H.hyper_of(wl)
+    opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"])
+    theta = workloads.init_params(wl, "cuda")
+    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device="cuda")
+    g = workloads.grads_for_step(wl, 1, "cuda")
+    opt.set_phase_timing(True)
+    args = (hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"], hp["beta"])
+    opt.step(theta, g, m, v, ema, 1, *args, 1)                    # warm-up step: 4 kernels
+    assert opt.launch_count() == 4
+    opt.step(theta, g, m, v, ema, 2, *args, 1)                    # AdaGC step: 3 kernels
+    assert opt.launch_count() == 7
+    ms = opt.get_phase_times()
+    assert len(ms) == 3 and all(x >= 0 for x in ms)
+    opt.close()
+
+
+def test_step_host_matches_device_entry():
+    wl, offs, nums = _mini()
+    hp = H.hyper_of(wl)
+    args = (hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"], hp["beta"], hp["warmup"])
+    outs = []
+    for host in (False, True):
+        opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"])
+        theta = workloads.init_params(wl, "cuda")
+        m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+        ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device="cuda")
+        g_dev = torch.empty(wl.arena_elems, dtype=wl.torch_grad_dtype, device="cuda")
+        norm = torch.empty(wl.n_tensors, dtype=torch.float32).pin_memory()
+        hfac = torch.empty(wl.n_tensors, dtype=torch.float32).pin_memory()
+        flag = torch.empty(wl.n_tensors, dtype=torch.uint8).pin_memory()
+        for t in range(1, 9):
+            g = workloads.grads_for_step(wl, t, "cuda")
+            if host:
+                opt.step_host(theta, g_dev, m, v, ema, g.cpu().pin_memory(), t, *args, norm, hfac, flag)
+                st = opt.get_stats()
+                assert np.array_equal(norm.numpy(), st["norm"]) and np.array_equal(flag.numpy().astype(bool), st["flag"])
+                assert np.array_equal(hfac.numpy(), st["h"])
+            else:
+                opt.step(theta, g, m, v, ema, t, *args)
+        outs.append((theta, m, v, ema))
+        opt.close()
+    for x, y in zip(*outs):
+        assert torch.equal(x, y)

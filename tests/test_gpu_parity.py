@@ -39,6 +39,11 @@ def test_gpt2_small_all_elements():
     rep = H.run_full(wl, wl.n_steps)
     _report("gpt2_small", rep)
     assert rep.decisions == 148 * 50 and rep.clipped > 0
+    # with lambda_abs = 1 the warm-up clips hard and seeds gamma low, so every later decision is a clip
+    # with a wide margin; a large lambda_abs gives the mixed, close decisions that test bit-exactness
+    rep = H.run_full(wl, 30, hyper_over=dict(lambda_abs=1e4))
+    _report("gpt2_small lambda_abs=1e4", rep)
+    assert 0 < rep.clipped < rep.decisions
 
 
 def test_many_small_all_elements():
@@ -47,6 +52,9 @@ def test_many_small_all_elements():
     rep = H.run_full(wl, wl.n_steps)
     _report("many_small", rep)
     assert rep.decisions == 20000 * 30 and rep.clipped > 0
+    rep = H.run_full(wl, 20, hyper_over=dict(lambda_abs=1e4))
+    _report("many_small lambda_abs=1e4", rep)
+    assert 0 < rep.clipped < rep.decisions
 
 
 def test_llama32_1b_sampled_adamw_and_clip_only():

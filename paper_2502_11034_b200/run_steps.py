@@ -1,0 +1,54 @@
+"""Run a few fused AdaGC + AdamW steps (or clip-only steps) on a named synthetic layout.
+
+    python -m paper_2502_11034_b200.run_steps --workload gpt2_small --steps 4 [--mode step|clip] [--scale-layers N]
+
+A minimal driver of the C ABI (adagc_create / adagc_step / adagc_clip / adagc_get_stats): useful as
+an example and as a small, short-running target for profilers.  Prints the per-phase device times.
+"""
+from __future__ import annotations
+
+import argparse
+
+import torch
+
+from . import binding, workloads
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="gpt2_small")
+    ap.add_argument("--steps", type=int, default=4)
+    ap.add_argument("--mode", choices=["step", "clip"], default="step")
+    ap.add_argument("--n-layer", type=int, default=None, help="override the layer count of a layered layout")
+    ap.add_argument("--warmup", type=int, default=1, help="T_start: steps of global-norm clipping")
+    args = ap.parse_args()
+    over = {} if args.n_layer is None else {"n_layer": args.n_layer}
+    wl = workloads.build(args.workload, **over)
+    hp = wl.hyper
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    offs, nums = [t.offset for t in wl.tensors], [t.numel for t in wl.tensors]
+    opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=dev)
+    theta = workloads.init_params(wl, dev)
+    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device=dev)
+    g = workloads.grads_for_step(wl, 1, dev)
+    g_out = torch.empty_like(g) if args.mode == "clip" else None
+    opt.set_phase_timing(True)
+    for t in range(1, args.steps + 1):
+        if args.mode == "step":
+            opt.step(theta, g, m, v, ema, t, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"],
+                     hp["lambda_rel"], hp["beta"], args.warmup)
+        else:
+            opt.clip(g, g_out, ema, t, hp["lambda_rel"], hp["beta"], args.warmup)
+        ms = opt.get_phase_times()
+        print(f"step {t}: norm {ms[0]:.4f} ms, finalize {ms[1]:.4f} ms, {'update' if args.mode == 'step' else 'scale'} "
+              f"{ms[2]:.4f} ms  ({wl.n_params} params)")
+    st = opt.get_stats()
+    print(f"steps_done={st['steps_done']} clipped_last_step={int(st['flag'].sum())} status={st['status']} "
+          f"kernels_launched={opt.launch_count()}")
+    opt.close()
+
+
+if __name__ == "__main__":
+    main()

@@ -47,7 +47,8 @@ typedef enum {
   ADAGC_E_WORKSPACE = -4,   /* workspace too small or misaligned */
   ADAGC_E_DTYPE = -5,       /* unsupported dtype combination */
   ADAGC_E_CUDA = -6,        /* a CUDA runtime call failed (no device, launch error, ...) */
-  ADAGC_E_NOMEM = -7        /* host allocation of the context failed */
+  ADAGC_E_NOMEM = -7,       /* host allocation of the context failed */
+  ADAGC_E_TOO_LARGE = -8    /* adagc_sumsq_noalloc: more elements than its fixed scratch covers */
 } adagc_status;
 
 /* Bits of the device status word (adagc_get_stats). */
@@ -157,6 +158,33 @@ uint64_t adagc_launch_count(const adagc_ctx* ctx);
  */
 int adagc_set_phase_timing(adagc_ctx* ctx, int enabled);
 int adagc_get_phase_times(adagc_ctx* ctx, float ms[3]);
+
+/*
+ * Sum of squares (squared L2 norm) of one contiguous gradient buffer, for callers that cannot
+ * allocate.  (The paper has no counterpart of this entry point: it is a convenience of this library.)
+ *
+ * Who needs it: code that must take a gradient norm at a point where it cannot get device memory --
+ * it runs while the framework's allocator is locked or out of memory, it is a plug-in that is handed
+ * only its input and output buffers, or its memory budget was fixed before start-up.  Everything else
+ * in this header works on a caller-provided workspace; this call needs none.  Its per-chunk partial
+ * sums live in a fixed 512 KiB array inside the library's device image, so every GPU that loads the
+ * library holds those 512 KiB until the process exits.
+ *
+ *   d_grads      device buffer of `numel` elements of `grad_dtype` (ADAGC_F32 or ADAGC_BF16),
+ *                16-byte aligned, read only
+ *   numel        1 .. 2^30 (1 073 741 824) elements; more returns ADAGC_E_TOO_LARGE and enqueues nothing
+ *   d_sumsq_out  device pointer to one double (8-byte aligned), overwritten with sum_j g_j^2 in
+ *                float64; same chunking and summation order as the norm phase of adagc_step
+ *
+ * The call enqueues two kernels on `cuda_stream`, does not synchronise, and calls no allocating
+ * routine.  The first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress, with that device current); make that first call outside any stream capture.
+ * All calls share the one array and it keeps the previous call's contents; every entry a call reads
+ * it has first rewritten, so nothing needs clearing, but two calls whose kernels overlap on the GPU
+ * (different streams, or several host threads) race on it: serialise them on one stream or with events.
+ */
+int adagc_sumsq_noalloc(const void* d_grads, int32_t grad_dtype, int64_t numel, double* d_sumsq_out,
+                        void* cuda_stream);
 
 /* Static string for a status code. */
 const char* adagc_strerror(int status);

@@ -73,6 +73,8 @@ def lib() -> C.CDLL:
     L.adagc_set_phase_timing.argtypes = [vp, C.c_int]
     L.adagc_get_phase_times.restype = C.c_int
     L.adagc_get_phase_times.argtypes = [vp, C.POINTER(C.c_float)]
+    L.adagc_sumsq_noalloc.restype = C.c_int
+    L.adagc_sumsq_noalloc.argtypes = [vp, C.c_int32, i64, vp, vp]
     L.adagc_strerror.restype = C.c_char_p
     L.adagc_strerror.argtypes = [C.c_int]
     _lib = L
@@ -81,6 +83,18 @@ def lib() -> C.CDLL:
 
 def strerror(status: int) -> str:
     return lib().adagc_strerror(int(status)).decode()
+
+
+def sumsq_noalloc(grads: torch.Tensor, out: torch.Tensor, numel: Optional[int] = None, stream=None) -> None:
+    """adagc_sumsq_noalloc: sum of squares of a contiguous gradient buffer into `out` (one float64 on the
+    device) without any workspace; for callers that cannot allocate device memory.  Enqueues only."""
+    gd = {torch.float32: ADAGC_F32, torch.bfloat16: ADAGC_BF16}[grads.dtype]
+    assert out.dtype == torch.float64 and out.is_cuda and grads.is_cuda and grads.is_contiguous()
+    n = grads.numel() if numel is None else int(numel)
+    with torch.cuda.device(grads.device):
+        rc = lib().adagc_sumsq_noalloc(_ptr(grads), gd, n, _ptr(out), _stream_ptr(stream))
+    if rc != 0:
+        raise AdagcError(rc, "adagc_sumsq_noalloc")
 
 
 def make_desc(numels: Sequence[int], offsets: Sequence[int], grad_dtype: int, lambda_abs: float = 1.0,

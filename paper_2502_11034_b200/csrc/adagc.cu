@@ -748,8 +748,148 @@ const char* adagc_strerror(int status) {
     case ADAGC_E_DTYPE: return "unsupported dtype combination";
     case ADAGC_E_CUDA: return "CUDA runtime error";
     case ADAGC_E_NOMEM: return "host allocation failed";
+    case ADAGC_E_TOO_LARGE: return "size exceeds the fixed scratch of the no-allocation entry point";
     default: return "unknown status";
   }
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Sum of squares of one contiguous gradient buffer with NO caller- or library-allocated scratch.
+//
+// Some callers cannot obtain device memory at the moment they need a norm: code running while an
+// allocator is locked or exhausted, plug-ins that are handed only their input and output buffers,
+// or hosts whose memory budget is fixed up front.  For them the per-chunk partial sums (the scratch
+// that the norm phase above keeps in the caller's workspace) live in a fixed array inside this
+// library's device image.  Every GPU that loads the library holds that array until the process exits.
+// ------------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxChunks = 65536;  // 512 KiB of scratch; covers 2^30 elements
+constexpr int64_t kStaticMaxElems = int64_t(kStaticMaxChunks) * kChunkElems;
+constexpr int kMaxDevices = 64;
+
+static __device__ __align__(256) double g_static_partials[kStaticMaxChunks];
+
+// Same per-chunk arithmetic and thread mapping as adagc_norm_kernel, chunks taken implicitly as
+// consecutive kChunkElems-element slices of one buffer.
+template <bool kBF16>
+__global__ void __launch_bounds__(kThreads)
+adagc_sumsq_static_kernel(const void* __restrict__ grads, int64_t numel, int n_chunks,
+                          double* __restrict__ partials) {
+  constexpr int kEPV = kBF16 ? 8 : 4;
+  constexpr int kUnroll = 8;
+  __shared__ double warp_part[kThreads / 32];
+  const int tid = threadIdx.x;
+  for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+    const int64_t start = int64_t(c) * kChunkElems;
+    const int count = static_cast<int>(numel - start < kChunkElems ? numel - start : kChunkElems);
+    const uint4* __restrict__ vec =
+        reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + start * (kBF16 ? 2 : 4));
+    const int nvec = count / kEPV;
+    double acc0 = 0.0, acc1 = 0.0;
+    for (int base = 0; base < nvec; base += kThreads * kUnroll) {
+      uint4 q[kUnroll];
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        const int i = base + u * kThreads + tid;
+        q[u] = (i < nvec) ? __ldg(vec + i) : make_uint4(0u, 0u, 0u, 0u);
+      }
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        if (kBF16) {
+          acc0 = sq_acc(acc0, bf16_lo(q[u].x));
+          acc1 = sq_acc(acc1, bf16_hi(q[u].x));
+          acc0 = sq_acc(acc0, bf16_lo(q[u].y));
+          acc1 = sq_acc(acc1, bf16_hi(q[u].y));
+          acc0 = sq_acc(acc0, bf16_lo(q[u].z));
+          acc1 = sq_acc(acc1, bf16_hi(q[u].z));
+          acc0 = sq_acc(acc0, bf16_lo(q[u].w));
+          acc1 = sq_acc(acc1, bf16_hi(q[u].w));
+        } else {
+          acc0 = sq_acc(acc0, __uint_as_float(q[u].x));
+          acc1 = sq_acc(acc1, __uint_as_float(q[u].y));
+          acc0 = sq_acc(acc0, __uint_as_float(q[u].z));
+          acc1 = sq_acc(acc1, __uint_as_float(q[u].w));
+        }
+      }
+    }
+    const int t = nvec * kEPV + tid;
+    if (t < count) {
+      float x;
+      if (kBF16) {
+        x = __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const uint16_t*>(vec)[t]) << 16);
+      } else {
+        x = reinterpret_cast<const float*>(vec)[t];
+      }
+      acc0 = sq_acc(acc0, x);
+    }
+    const double w = warp_sum(acc0 + acc1);
+    if ((tid & 31) == 0) warp_part[tid >> 5] = w;
+    __syncthreads();
+    if (tid == 0) {
+      double s = warp_part[0];
+#pragma unroll
+      for (int k = 1; k < kThreads / 32; ++k) s += warp_part[k];
+      partials[c] = s;  // every partial that is read below is rewritten by this launch
+    }
+    __syncthreads();
+  }
+}
+
+// One warp sums the partials in the same fixed order as adagc_tensor_finalize_kernel.
+__global__ void __launch_bounds__(32)
+adagc_sumsq_static_reduce_kernel(const double* __restrict__ partials, int n_chunks, double* __restrict__ out) {
+  const int lane = threadIdx.x;
+  double acc = 0.0;
+  for (int j = lane; j < n_chunks; j += 32) acc += partials[j];
+  acc = warp_sum(acc);
+  if (lane == 0) *out = acc;
+}
+
+struct StaticScratch {
+  bool ready[kMaxDevices] = {};
+  double* ptr[kMaxDevices] = {};
+  int sms[kMaxDevices] = {};
+};
+StaticScratch g_static;  // host side; filled on the first call on each device
+
+}  // namespace
+
+extern "C" int adagc_sumsq_noalloc(const void* d_grads, int32_t grad_dtype, int64_t numel, double* d_sumsq_out,
+                                   void* cuda_stream) {
+  if (!d_grads || !d_sumsq_out || numel <= 0) return ADAGC_E_INVALID_ARG;
+  if (grad_dtype != ADAGC_F32 && grad_dtype != ADAGC_BF16) return ADAGC_E_DTYPE;
+  if (numel > kStaticMaxElems) return ADAGC_E_TOO_LARGE;
+  if (!aligned16(d_grads) || (reinterpret_cast<uintptr_t>(d_sumsq_out) & 7u)) return ADAGC_E_MISALIGNED;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    (void)cudaGetLastError();
+    return ADAGC_E_CUDA;
+  }
+  if (!g_static.ready[dev]) {
+    // In host code the array's name is only a handle; the address the kernels need comes from the
+    // runtime, once per device, with that device current.
+    double* p = nullptr;
+    int sms = 0;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_partials) != cudaSuccess || !p ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+      (void)cudaGetLastError();
+      return ADAGC_E_CUDA;
+    }
+    g_static.ptr[dev] = p;
+    g_static.sms[dev] = sms;
+    g_static.ready[dev] = true;
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const int n_chunks = static_cast<int>((numel + kChunkElems - 1) / kChunkElems);
+  const int grid = std::max(1, std::min(n_chunks, g_static.sms[dev] * 8));
+  double* partials = g_static.ptr[dev];
+  if (grad_dtype == ADAGC_BF16)
+    adagc_sumsq_static_kernel<true><<<grid, kThreads, 0, s>>>(d_grads, numel, n_chunks, partials);
+  else
+    adagc_sumsq_static_kernel<false><<<grid, kThreads, 0, s>>>(d_grads, numel, n_chunks, partials);
+  adagc_sumsq_static_reduce_kernel<<<1, 32, 0, s>>>(partials, n_chunks, d_sumsq_out);
+  return cudaGetLastError() == cudaSuccess ? ADAGC_OK : ADAGC_E_CUDA;
+}

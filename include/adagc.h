@@ -56,7 +56,7 @@ typedef enum {
 
 /* One parameter tensor. */
 typedef struct {
-  int64_t numel;    /* > 0 */
+  int64_t numel;    /* > 0; offset + numel <= 2^34 */
   int64_t offset;   /* element offset into every arena; offset * sizeof(element) must be a
                        multiple of 16 bytes for every arena dtype (multiple of 8 elements with
                        bf16 gradients, of 4 with fp32 gradients) */

@@ -19,7 +19,10 @@
 
 #include <algorithm>
 #include <cmath>
+#include <functional>
 #include <new>
+#include <queue>
+#include <utility>
 #include <vector>
 
 #include "../../include/adagc.h"
@@ -41,11 +44,19 @@ constexpr int kWarmupThreads = 1024;
 constexpr int kUpdateBlocksPerSM = ADAGC_UPDATE_BLOCKS_PER_SM;
 
 struct Chunk {
-  int64_t start;   // element offset into the arenas
-  int32_t count;   // elements in this chunk (<= kChunkElems)
-  int32_t tensor;  // owning tensor
+  uint32_t start4;  // element offset into the arenas, in units of 4 elements
+  int32_t count;    // elements in this chunk (<= kChunkElems)
+  int32_t tensor;   // owning tensor
+  int32_t partial;  // index of this chunk's partial sum: chunks of a tensor are numbered consecutively
 };
 static_assert(sizeof(Chunk) == 16, "chunk entries are 16 bytes");
+__host__ __device__ __forceinline__ int64_t chunk_start(const Chunk& c) { return static_cast<int64_t>(c.start4) * 4; }
+
+// Chunks are handed to thread blocks by a table built once on the host: block b owns the entries
+// [block_begin[b], block_begin[b+1]) of its kernel's table.  The assignment balances elements (plus a
+// fixed cost per chunk) over the blocks; with equal chunks it is plain round-robin.
+constexpr int kMaxGrid = 8192;          // entries reserved for each block_begin array
+constexpr int kChunkFixedCost = 1024;
 
 struct TensorEntry {
   int32_t first_chunk;
@@ -104,16 +115,17 @@ __device__ __forceinline__ double sq_acc(double acc, float x) {
 // ------------------------------------------------------------------------------------------------
 template <bool kBF16>
 __global__ void __launch_bounds__(kThreads)
-adagc_norm_kernel(const void* __restrict__ grads, const Chunk* __restrict__ chunks, int n_chunks,
-                  double* __restrict__ partials) {
+adagc_norm_kernel(const void* __restrict__ grads, const Chunk* __restrict__ chunks,
+                  const int32_t* __restrict__ block_begin, double* __restrict__ partials) {
   constexpr int kEPV = kBF16 ? 8 : 4;  // elements per 16-byte vector
   constexpr int kUnroll = 8;           // independent 16-byte loads in flight per thread
   __shared__ double warp_part[kThreads / 32];
   const int tid = threadIdx.x;
-  for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+  const int c_end = block_begin[blockIdx.x + 1];
+  for (int c = block_begin[blockIdx.x]; c < c_end; ++c) {
     const Chunk ck = chunks[c];
     const uint4* __restrict__ vec =
-        reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + ck.start * (kBF16 ? 2 : 4));
+        reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + chunk_start(ck) * (kBF16 ? 2 : 4));
     const int nvec = ck.count / kEPV;
     double acc0 = 0.0, acc1 = 0.0;
     for (int base = 0; base < nvec; base += kThreads * kUnroll) {
@@ -161,7 +173,7 @@ adagc_norm_kernel(const void* __restrict__ grads, const Chunk* __restrict__ chun
       double s = warp_part[0];
 #pragma unroll
       for (int k = 1; k < kThreads / 32; ++k) s += warp_part[k];
-      partials[c] = s;
+      partials[ck.partial] = s;
     }
     __syncthreads();
   }
@@ -310,34 +322,50 @@ __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gba
 template <bool kBF16>
 __global__ void __launch_bounds__(kThreads)
 adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, float* __restrict__ m_arena,
-                    float* __restrict__ v_arena, const Chunk* __restrict__ chunks, int n_chunks,
-                    const float* __restrict__ h_arr, AdamScalars a) {
+                    float* __restrict__ v_arena, const Chunk* __restrict__ chunks,
+                    const int32_t* __restrict__ block_begin, const float* __restrict__ h_arr, AdamScalars a) {
   const int tid = threadIdx.x;
-  int c = blockIdx.x;
+  int c = block_begin[blockIdx.x];
+  const int n_chunks = block_begin[blockIdx.x + 1];  // end of this block's entries
   if (c >= n_chunks) return;
   Chunk ck = chunks[c];
   float h = h_arr[ck.tensor];
+  constexpr int kWarps = kThreads / 32;
+  int row_base = 0;
   while (true) {
     // fetch the next chunk's table entry and clip factor now: with only two blocks resident per SM
     // nothing else would hide these two dependent loads between chunks
-    const int c_next = c + gridDim.x;
+    const int c_next = c + 1;
     Chunk ck_next = ck;
     float h_next = h;
     if (c_next < n_chunks) {
       ck_next = chunks[c_next];
       h_next = h_arr[ck_next.tensor];
     }
-    float4* __restrict__ p4 = reinterpret_cast<float4*>(params + ck.start);
-    float4* __restrict__ m4 = reinterpret_cast<float4*>(m_arena + ck.start);
-    float4* __restrict__ v4 = reinterpret_cast<float4*>(v_arena + ck.start);
-    const char* __restrict__ gbase = static_cast<const char*>(grads) + ck.start * (kBF16 ? 2 : 4);
+    const int64_t start = chunk_start(ck);
+    float4* __restrict__ p4 = reinterpret_cast<float4*>(params + start);
+    float4* __restrict__ m4 = reinterpret_cast<float4*>(m_arena + start);
+    float4* __restrict__ v4 = reinterpret_cast<float4*>(v_arena + start);
+    const char* __restrict__ gbase = static_cast<const char*>(grads) + start * (kBF16 ? 2 : 4);
     if (ck.count == kChunkElems) {  // full chunk: fixed trip count
 #pragma unroll 2
       for (int k = 0; k < kChunkElems / 8 / kThreads; ++k) adamw_group8<kBF16>(k * kThreads + tid, gbase, p4, m4, v4, h, a);
     } else {
+      // Partial chunk (a small tensor, or the end of one).  Work is dealt in rows of 32 groups (256
+      // elements) and the rows of successive chunks go to the block's warps in one continuing
+      // round-robin: row_base counts the rows dealt so far.  Restarting at warp 0 for every chunk
+      // would give the low warps the extra rows every time and make them the critical path.
       const int n8 = ck.count >> 3;
-      for (int i = tid; i < n8; i += kThreads) adamw_group8<kBF16>(i, gbase, p4, m4, v4, h, a);
-      const int t = (n8 << 3) + tid;  // ragged tail: fewer than 8 elements
+      const int rows = (n8 + 31) >> 5;
+      const int warp = tid >> 5, lane = tid & 31;
+#pragma unroll 2
+      for (int r = (warp - row_base) & (kWarps - 1); r < rows; r += kWarps) {
+        const int i = (r << 5) + lane;
+        if (i < n8) adamw_group8<kBF16>(i, gbase, p4, m4, v4, h, a);
+      }
+      row_base = (row_base + rows) & (kWarps - 1);
+      const int tail_lane = (warp == row_base) ? lane : kThreads;  // the next warp in turn takes the tail
+      const int t = (n8 << 3) + tail_lane;  // ragged tail: fewer than 8 elements
       if (t < ck.count) {
         float g;
         if (kBF16) {
@@ -345,11 +373,11 @@ adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, 
         } else {
           g = reinterpret_cast<const float*>(gbase)[t];
         }
-        float p = params[ck.start + t], m = m_arena[ck.start + t], v = v_arena[ck.start + t];
+        float p = params[start + t], m = m_arena[start + t], v = v_arena[start + t];
         adamw_elem(g, h, p, m, v, a);
-        params[ck.start + t] = p;
-        m_arena[ck.start + t] = m;
-        v_arena[ck.start + t] = v;
+        params[start + t] = p;
+        m_arena[start + t] = m;
+        v_arena[start + t] = v;
       }
     }
     if (c_next >= n_chunks) break;
@@ -361,37 +389,56 @@ adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, 
 
 // Clip-only: hat(g) = h * g written in the gradient dtype.  In place, chunks with h == 1 are skipped.
 template <bool kBF16>
+__device__ __forceinline__ uint4 scale_vec(uint4 q, float h) {
+  if (kBF16) {
+    q.x = pack_bf16(h * bf16_lo(q.x), h * bf16_hi(q.x));
+    q.y = pack_bf16(h * bf16_lo(q.y), h * bf16_hi(q.y));
+    q.z = pack_bf16(h * bf16_lo(q.z), h * bf16_hi(q.z));
+    q.w = pack_bf16(h * bf16_lo(q.w), h * bf16_hi(q.w));
+  } else {
+    q.x = __float_as_uint(h * __uint_as_float(q.x));
+    q.y = __float_as_uint(h * __uint_as_float(q.y));
+    q.z = __float_as_uint(h * __uint_as_float(q.z));
+    q.w = __float_as_uint(h * __uint_as_float(q.w));
+  }
+  return q;
+}
+
+template <bool kBF16>
 __global__ void __launch_bounds__(kThreads)
 adagc_scale_kernel(const void* __restrict__ gin, void* __restrict__ gout, const Chunk* __restrict__ chunks,
-                   int n_chunks, const float* __restrict__ h_arr, int in_place) {
+                   const int32_t* __restrict__ block_begin, const float* __restrict__ h_arr, int in_place) {
   constexpr int kEPV = kBF16 ? 8 : 4;
-  const int tid = threadIdx.x;
-  for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
+  constexpr int kWarps = kThreads / 32;
+  constexpr int kBatch = 4;  // 16-byte loads in flight per thread
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int row_base = 0;  // rows (32 vectors) dealt so far: successive chunks continue one round-robin over the warps
+  const int c_end = block_begin[blockIdx.x + 1];
+  for (int c = block_begin[blockIdx.x]; c < c_end; ++c) {
     const Chunk ck = chunks[c];
     const float h = h_arr[ck.tensor];
     if (in_place && h == 1.0f) continue;
-    const int64_t boff = ck.start * (kBF16 ? 2 : 4);
+    const int64_t boff = chunk_start(ck) * (kBF16 ? 2 : 4);
     const uint4* src = reinterpret_cast<const uint4*>(static_cast<const char*>(gin) + boff);
     uint4* dst = reinterpret_cast<uint4*>(static_cast<char*>(gout) + boff);
     const int nvec = ck.count / kEPV;
-#pragma unroll 4
-    for (int i = tid; i < nvec; i += kThreads) {
-      uint4 q = ld_stream(src + i);
-      if (kBF16) {
-        q.x = pack_bf16(h * bf16_lo(q.x), h * bf16_hi(q.x));
-        q.y = pack_bf16(h * bf16_lo(q.y), h * bf16_hi(q.y));
-        q.z = pack_bf16(h * bf16_lo(q.z), h * bf16_hi(q.z));
-        q.w = pack_bf16(h * bf16_lo(q.w), h * bf16_hi(q.w));
-      } else {
-        q.x = __float_as_uint(h * __uint_as_float(q.x));
-        q.y = __float_as_uint(h * __uint_as_float(q.y));
-        q.z = __float_as_uint(h * __uint_as_float(q.z));
-        q.w = __float_as_uint(h * __uint_as_float(q.w));
+    const int rows = (nvec + 31) >> 5;
+    for (int r0 = (warp - row_base) & (kWarps - 1); r0 < rows; r0 += kWarps * kBatch) {
+      uint4 q[kBatch];
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        const int i = ((r0 + u * kWarps) << 5) + lane;
+        if (i < nvec) q[u] = ld_stream(src + i);
       }
-      st_stream(dst + i, q);
+#pragma unroll
+      for (int u = 0; u < kBatch; ++u) {
+        const int i = ((r0 + u * kWarps) << 5) + lane;
+        if (i < nvec) st_stream(dst + i, scale_vec<kBF16>(q[u], h));
+      }
     }
-    const int t = nvec * kEPV + tid;
-    if (t < ck.count) {
+    row_base = (row_base + rows) & (kWarps - 1);
+    const int t = nvec * kEPV + lane;  // ragged tail (fewer than one vector): the next warp in turn
+    if (warp == row_base && t < ck.count) {
       if (kBF16) {
         const uint16_t b = reinterpret_cast<const uint16_t*>(src)[t];
         const float x = h * __uint_as_float(static_cast<uint32_t>(b) << 16);
@@ -409,13 +456,17 @@ adagc_scale_kernel(const void* __restrict__ gin, void* __restrict__ gout, const 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {  // byte offsets of the workspace sections
-  size_t chunks, tensors, partials, sumsq, norm, h, clip_count, scalars, flag, total;
+  size_t chunks_wide, chunks_upd, begin_wide, begin_upd, tensors, partials, sumsq, norm, h, clip_count, scalars, flag,
+      total;
 };
 
 Layout make_layout(int64_t n_chunks, int64_t T) {
   Layout L;
   size_t o = 0;
-  L.chunks = o;     o = align_up(o + sizeof(Chunk) * n_chunks, 256);
+  L.chunks_wide = o; o = align_up(o + sizeof(Chunk) * n_chunks, 256);  // order of the norm / scale grid
+  L.chunks_upd = o;  o = align_up(o + sizeof(Chunk) * n_chunks, 256);  // order of the update grid
+  L.begin_wide = o;  o = align_up(o + sizeof(int32_t) * (kMaxGrid + 1), 256);
+  L.begin_upd = o;   o = align_up(o + sizeof(int32_t) * (kMaxGrid + 1), 256);
   L.tensors = o;    o = align_up(o + sizeof(TensorEntry) * T, 256);
   L.partials = o;   o = align_up(o + sizeof(double) * n_chunks, 256);
   L.sumsq = o;      o = align_up(o + sizeof(double) * T, 256);
@@ -440,7 +491,7 @@ int validate_desc(const adagc_desc* d, int64_t* n_chunks_out, int64_t* arena_ele
   for (int32_t i = 0; i < d->n_tensors; ++i) {
     const adagc_tensor& t = d->tensors[i];
     if (t.numel <= 0 || t.offset < 0 || t.ndim < 0 || t.ndim > 4) return ADAGC_E_INVALID_ARG;
-    if (t.numel > (int64_t(1) << 44) || t.offset > (int64_t(1) << 46)) return ADAGC_E_INVALID_ARG;
+    if (t.numel > (int64_t(1) << 34) || t.offset + t.numel > (int64_t(1) << 34)) return ADAGC_E_INVALID_ARG;
     if (t.ndim > 0) {
       int64_t prod = 1;
       for (int k = 0; k < t.ndim; ++k) {
@@ -465,6 +516,29 @@ int validate_desc(const adagc_desc* d, int64_t* n_chunks_out, int64_t* arena_ele
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// List scheduling in table order: each chunk goes to the block with the least work so far (ties to the
+// lowest block index, so equal chunks are dealt round-robin); a block keeps its chunks in arrival order.
+void balance_chunks(const std::vector<Chunk>& chunks, int grid, std::vector<Chunk>* table,
+                    std::vector<int32_t>* block_begin) {
+  using Load = std::pair<int64_t, int>;  // (work assigned, block)
+  std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
+  for (int b = 0; b < grid; ++b) heap.emplace(0, b);
+  std::vector<int32_t> owner(chunks.size());
+  std::vector<int32_t> count(grid, 0);
+  for (size_t i = 0; i < chunks.size(); ++i) {
+    const Load top = heap.top();
+    heap.pop();
+    owner[i] = top.second;
+    count[top.second] += 1;
+    heap.emplace(top.first + chunks[i].count + kChunkFixedCost, top.second);
+  }
+  block_begin->assign(grid + 1, 0);
+  for (int b = 0; b < grid; ++b) (*block_begin)[b + 1] = (*block_begin)[b] + count[b];
+  std::vector<int32_t> pos(block_begin->begin(), block_begin->end() - 1);
+  table->resize(chunks.size());
+  for (size_t i = 0; i < chunks.size(); ++i) (*table)[pos[owner[i]]++] = chunks[i];
+}
+
 }  // namespace
 
 struct adagc_ctx {
@@ -474,14 +548,17 @@ struct adagc_ctx {
   bool bf16 = false;
   double lambda_abs = 1.0;
   int device = 0;
-  int grid_norm = 1, grid_update = 1, grid_scale = 1;
+  int grid_wide = 1, grid_update = 1;  // norm and scale kernels: SMs x resident blocks; update: SMs x 2
   char* ws = nullptr;
   Layout L{};
   uint64_t launches = 0;
   bool timing = false;
   bool timing_valid = false;
   cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
-  const Chunk* d_chunks() const { return reinterpret_cast<const Chunk*>(ws + L.chunks); }
+  const Chunk* d_chunks_wide() const { return reinterpret_cast<const Chunk*>(ws + L.chunks_wide); }
+  const Chunk* d_chunks_upd() const { return reinterpret_cast<const Chunk*>(ws + L.chunks_upd); }
+  const int32_t* d_begin_wide() const { return reinterpret_cast<const int32_t*>(ws + L.begin_wide); }
+  const int32_t* d_begin_upd() const { return reinterpret_cast<const int32_t*>(ws + L.begin_upd); }
   const TensorEntry* d_tensors() const { return reinterpret_cast<const TensorEntry*>(ws + L.tensors); }
   double* d_partials() const { return reinterpret_cast<double*>(ws + L.partials); }
   StatPtrs stats() const {
@@ -513,10 +590,10 @@ int enqueue_clip_phases(adagc_ctx* ctx, const void* d_grads, float* d_ema, int64
                         double beta, int64_t warmup, cudaStream_t s) {
   if (ctx->timing) cudaEventRecord(ctx->ev[0], s);
   if (ctx->bf16)
-    adagc_norm_kernel<true><<<ctx->grid_norm, kThreads, 0, s>>>(d_grads, ctx->d_chunks(), ctx->n_chunks,
+    adagc_norm_kernel<true><<<ctx->grid_wide, kThreads, 0, s>>>(d_grads, ctx->d_chunks_wide(), ctx->d_begin_wide(),
                                                                ctx->d_partials());
   else
-    adagc_norm_kernel<false><<<ctx->grid_norm, kThreads, 0, s>>>(d_grads, ctx->d_chunks(), ctx->n_chunks,
+    adagc_norm_kernel<false><<<ctx->grid_wide, kThreads, 0, s>>>(d_grads, ctx->d_chunks_wide(), ctx->d_begin_wide(),
                                                                 ctx->d_partials());
   ctx->launches++;
   if (ctx->timing) cudaEventRecord(ctx->ev[1], s);
@@ -585,9 +662,10 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
     te.first_chunk = static_cast<int32_t>(chunks.size());
     for (int64_t o = 0; o < t.numel; o += kChunkElems) {
       Chunk c;
-      c.start = t.offset + o;
+      c.start4 = static_cast<uint32_t>((t.offset + o) / 4);
       c.count = static_cast<int32_t>(std::min<int64_t>(kChunkElems, t.numel - o));
       c.tensor = i;
+      c.partial = static_cast<int32_t>(chunks.size());
       chunks.push_back(c);
     }
     te.n_chunks = static_cast<int32_t>(chunks.size()) - te.first_chunk;
@@ -623,13 +701,26 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
     }
     if (ok) {
       const int64_t sms = prop.multiProcessorCount;
-      ctx->grid_norm = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(n_chunks, sms * std::max(occ_n, 1))));
-      ctx->grid_update = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(n_chunks, sms * kUpdateBlocksPerSM)));
-      ctx->grid_scale = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(n_chunks, sms * std::max(occ_s, 1))));
+      const int64_t wide = sms * std::max(1, std::min(occ_n, occ_s));
+      ctx->grid_wide = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>({n_chunks, wide, kMaxGrid})));
+      ctx->grid_update = static_cast<int>(
+          std::max<int64_t>(1, std::min<int64_t>({n_chunks, sms * kUpdateBlocksPerSM, kMaxGrid})));
     }
   }
+  std::vector<Chunk> table_wide, table_upd;
+  std::vector<int32_t> begin_wide, begin_upd;
+  if (ok) {
+    balance_chunks(chunks, ctx->grid_wide, &table_wide, &begin_wide);
+    balance_chunks(chunks, ctx->grid_update, &table_upd, &begin_upd);
+  }
   ok = ok && cudaMemsetAsync(ctx->ws, 0, L.total, s) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(ctx->ws + L.chunks, chunks.data(), sizeof(Chunk) * chunks.size(),
+  ok = ok && cudaMemcpyAsync(ctx->ws + L.chunks_wide, table_wide.data(), sizeof(Chunk) * table_wide.size(),
+                             cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(ctx->ws + L.chunks_upd, table_upd.data(), sizeof(Chunk) * table_upd.size(),
+                             cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(ctx->ws + L.begin_wide, begin_wide.data(), sizeof(int32_t) * begin_wide.size(),
+                             cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(ctx->ws + L.begin_upd, begin_upd.data(), sizeof(int32_t) * begin_upd.size(),
                              cudaMemcpyHostToDevice, s) == cudaSuccess;
   ok = ok && cudaMemcpyAsync(ctx->ws + L.tensors, tensors.data(), sizeof(TensorEntry) * tensors.size(),
                              cudaMemcpyHostToDevice, s) == cudaSuccess;
@@ -683,11 +774,11 @@ int adagc_step(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, v
   if (ctx->bf16)
     adagc_update_kernel<true><<<ctx->grid_update, kThreads, 0, s>>>(
         static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), static_cast<float*>(d_v),
-        ctx->d_chunks(), ctx->n_chunks, st.h, a);
+        ctx->d_chunks_upd(), ctx->d_begin_upd(), st.h, a);
   else
     adagc_update_kernel<false><<<ctx->grid_update, kThreads, 0, s>>>(
         static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), static_cast<float*>(d_v),
-        ctx->d_chunks(), ctx->n_chunks, st.h, a);
+        ctx->d_chunks_upd(), ctx->d_begin_upd(), st.h, a);
   ctx->launches++;
   return finish_launches(ctx, s);
 }
@@ -703,11 +794,11 @@ int adagc_clip(adagc_ctx* ctx, const void* d_grads_in, void* d_grads_out, float*
   if (rc != ADAGC_OK) return rc;
   const int in_place = d_grads_in == d_grads_out ? 1 : 0;
   if (ctx->bf16)
-    adagc_scale_kernel<true><<<ctx->grid_scale, kThreads, 0, s>>>(d_grads_in, d_grads_out, ctx->d_chunks(),
-                                                                 ctx->n_chunks, ctx->stats().h, in_place);
+    adagc_scale_kernel<true><<<ctx->grid_wide, kThreads, 0, s>>>(d_grads_in, d_grads_out, ctx->d_chunks_wide(),
+                                                                ctx->d_begin_wide(), ctx->stats().h, in_place);
   else
-    adagc_scale_kernel<false><<<ctx->grid_scale, kThreads, 0, s>>>(d_grads_in, d_grads_out, ctx->d_chunks(),
-                                                                  ctx->n_chunks, ctx->stats().h, in_place);
+    adagc_scale_kernel<false><<<ctx->grid_wide, kThreads, 0, s>>>(d_grads_in, d_grads_out, ctx->d_chunks_wide(),
+                                                                 ctx->d_begin_wide(), ctx->stats().h, in_place);
   ctx->launches++;
   return finish_launches(ctx, s);
 }

@@ -292,7 +292,8 @@ def run_ours(args, wl):
     step_s = seconds_max / args.steps
     achieved = bpp * wl.n_params / (upd_ms * 1e-3) / 1e9
     norm_gbs = (bpp - 24) * wl.n_params / (norm_ms * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "adagc_update_kernel", "achieved": achieved, "peak": peak,
+    kernel = "adagc_update_tma_kernel" if opt.update_path == binding.UPDATE_PATH_BULK else "adagc_update_kernel"
+    roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
                 "traffic": TRAFFIC_BYTES.get(wl.name),
                 "algorithmic_bytes_per_launch": bpp * wl.n_params, "launch_ms": upd_ms,

@@ -53,6 +53,16 @@ typedef enum {
 
 /* Bits of the device status word (adagc_get_stats). */
 #define ADAGC_W_NONFINITE 1 /* some tensor's sum of squares was Inf or NaN in some step */
+#define ADAGC_E_TIMEOUT 2   /* a bounded device-side wait gave up (a bulk copy never completed): the
+                               update of that step is incomplete */
+
+/* adagc_desc.flags: which kernel runs the AdamW update phase.  AUTO (0) currently picks the bulk-async
+ * kernel (cp.async.bulk + mbarrier pipeline through shared memory), which measured 1-2 % faster than the
+ * register-streaming kernel; the other two values force one path (the tests cover both). */
+#define ADAGC_UPDATE_PATH_AUTO 0
+#define ADAGC_UPDATE_PATH_REGISTERS 1
+#define ADAGC_UPDATE_PATH_BULK 2
+#define ADAGC_UPDATE_PATH_MASK 3
 
 /* One parameter tensor. */
 typedef struct {
@@ -73,7 +83,7 @@ typedef struct {
   int32_t state_dtype;         /* ADAGC_F32 (m and v) */
   const adagc_tensor* tensors; /* host array, copied by adagc_create */
   double lambda_abs;           /* warm-up global-norm threshold of Eq. 2, > 0 (paper: 1.0) */
-  int32_t flags;               /* reserved, set to 0 */
+  int32_t flags;               /* 0, or one ADAGC_UPDATE_PATH_* value */
   int32_t reserved;            /* set to 0 */
 } adagc_desc;
 
@@ -144,6 +154,9 @@ int adagc_get_stats(adagc_ctx* ctx, float* h_norm, float* h_clipfactor, uint8_t*
  * Synchronises the stream. */
 int adagc_get_sumsq(adagc_ctx* ctx, double* h_sumsq, void* cuda_stream);
 
+/* The update path this context uses: ADAGC_UPDATE_PATH_REGISTERS or ADAGC_UPDATE_PATH_BULK. */
+int adagc_update_path(const adagc_ctx* ctx);
+
 /* Elements spanned by the arenas: max over tensors of offset + numel. */
 int64_t adagc_arena_elems(const adagc_ctx* ctx);
 
@@ -185,6 +198,15 @@ int adagc_get_phase_times(adagc_ctx* ctx, float ms[3]);
  */
 int adagc_sumsq_noalloc(const void* d_grads, int32_t grad_dtype, int64_t numel, double* d_sumsq_out,
                         void* cuda_stream);
+
+/*
+ * Test aid for the bounded device-side waits (the bulk-async update kernel waits on shared-memory
+ * barriers; every such wait gives up after a time limit instead of spinning forever).  Launches one
+ * small block that waits, with the same routine, on a barrier that nothing ever signals; after
+ * `limit_ms` (0 < limit_ms <= 1000) it gives up, sets ADAGC_E_TIMEOUT in the device status word and
+ * returns normally, leaving the context usable.  Enqueues only.
+ */
+int adagc_debug_wait_timeout(adagc_ctx* ctx, double limit_ms, void* cuda_stream);
 
 /* Static string for a status code. */
 const char* adagc_strerror(int status);

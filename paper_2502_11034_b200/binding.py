@@ -14,6 +14,8 @@ import torch
 
 ADAGC_F32, ADAGC_BF16 = 0, 1
 ADAGC_W_NONFINITE = 1
+ADAGC_E_TIMEOUT = 2
+UPDATE_PATH_AUTO, UPDATE_PATH_REGISTERS, UPDATE_PATH_BULK = 0, 1, 2
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libadagc.so")
 _lib = None
@@ -65,6 +67,8 @@ def lib() -> C.CDLL:
     L.adagc_get_stats.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     L.adagc_get_sumsq.restype = C.c_int
     L.adagc_get_sumsq.argtypes = [vp, vp, vp]
+    L.adagc_update_path.restype = C.c_int
+    L.adagc_update_path.argtypes = [vp]
     L.adagc_arena_elems.restype = i64
     L.adagc_arena_elems.argtypes = [vp]
     L.adagc_launch_count.restype = C.c_uint64
@@ -75,6 +79,8 @@ def lib() -> C.CDLL:
     L.adagc_get_phase_times.argtypes = [vp, C.POINTER(C.c_float)]
     L.adagc_sumsq_noalloc.restype = C.c_int
     L.adagc_sumsq_noalloc.argtypes = [vp, C.c_int32, i64, vp, vp]
+    L.adagc_debug_wait_timeout.restype = C.c_int
+    L.adagc_debug_wait_timeout.argtypes = [vp, dbl, vp]
     L.adagc_strerror.restype = C.c_char_p
     L.adagc_strerror.argtypes = [C.c_int]
     _lib = L
@@ -99,7 +105,7 @@ def sumsq_noalloc(grads: torch.Tensor, out: torch.Tensor, numel: Optional[int] =
 
 def make_desc(numels: Sequence[int], offsets: Sequence[int], grad_dtype: int, lambda_abs: float = 1.0,
               shapes: Optional[Sequence[Sequence[int]]] = None, param_dtype: int = ADAGC_F32,
-              state_dtype: int = ADAGC_F32):
+              state_dtype: int = ADAGC_F32, flags: int = 0):
     """Build an adagc_desc; returns (desc, keepalive) -- keep both alive while the desc is used."""
     n = len(numels)
     arr = (adagc_tensor * max(n, 1))()
@@ -114,6 +120,7 @@ def make_desc(numels: Sequence[int], offsets: Sequence[int], grad_dtype: int, la
     d.n_tensors, d.param_dtype, d.grad_dtype, d.state_dtype = n, param_dtype, grad_dtype, state_dtype
     d.tensors = C.cast(arr, C.POINTER(adagc_tensor))
     d.lambda_abs = float(lambda_abs)
+    d.flags = int(flags)
     return d, arr
 
 
@@ -130,13 +137,13 @@ class AdaGC:
     """adagc_ctx plus its torch-owned workspace.  Method names mirror the C entry points."""
 
     def __init__(self, numels: Sequence[int], offsets: Sequence[int], grad_dtype: torch.dtype,
-                 lambda_abs: float = 1.0, shapes=None, device="cuda"):
+                 lambda_abs: float = 1.0, shapes=None, device="cuda", flags: int = 0):
         L = lib()
         gd = {torch.float32: ADAGC_F32, torch.bfloat16: ADAGC_BF16}[grad_dtype]
         self.grad_dtype = grad_dtype
         self.n_tensors = len(numels)
         self.device = torch.device(device)
-        desc, keep = make_desc(numels, offsets, gd, lambda_abs, shapes)
+        desc, keep = make_desc(numels, offsets, gd, lambda_abs, shapes, flags=flags)
         nbytes = L.adagc_workspace_bytes(C.byref(desc))
         if nbytes == 0:
             rc = L.adagc_num_chunks(C.byref(desc))
@@ -151,6 +158,7 @@ class AdaGC:
             raise AdagcError(rc, "adagc_create")
         self._h = h
         self.arena_elems = int(L.adagc_arena_elems(h))
+        self.update_path = int(L.adagc_update_path(h))
 
     def close(self):
         if getattr(self, "_h", None):
@@ -207,6 +215,11 @@ class AdaGC:
         if rc != 0:
             raise AdagcError(rc, "adagc_get_sumsq")
         return out
+
+    def debug_wait_timeout(self, limit_ms: float, stream=None):
+        rc = lib().adagc_debug_wait_timeout(self._h, float(limit_ms), _stream_ptr(stream))
+        if rc != 0:
+            raise AdagcError(rc, "adagc_debug_wait_timeout")
 
     def launch_count(self) -> int:
         return int(lib().adagc_launch_count(self._h))

@@ -101,12 +101,12 @@ def check_state(name: str, got: np.ndarray, ref: np.ndarray, rep: ParityReport, 
 
 
 def run_full(wl: workloads.Workload, n_steps: int, device="cuda", hyper_over: Optional[dict] = None,
-             lr_schedule=None, canary: bool = True) -> ParityReport:
+             lr_schedule=None, canary: bool = True, flags: int = 0) -> ParityReport:
     """Every element of every tensor, fused AdaGC+AdamW step, GPU vs C oracle."""
     hp = hyper_of(wl, **(hyper_over or {}))
     offs = [t.offset for t in wl.tensors]
     nums = [t.numel for t in wl.tensors]
-    opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=device)
+    opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=device, flags=flags)
     theta = workloads.init_params(wl, device)
     theta0 = theta.cpu().numpy().copy()
     pad_mask = None

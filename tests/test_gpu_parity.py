@@ -93,6 +93,10 @@ def test_small_layouts_all_elements(name, over):
     wl = workloads.build(name, **over)
     rep = H.run_full(wl, min(wl.n_steps, 25))
     _report(f"{name} (small)", rep)
+    # both kernels of the update phase, forced
+    for path in (binding.UPDATE_PATH_REGISTERS, binding.UPDATE_PATH_BULK):
+        rep = H.run_full(wl, 8, flags=path)
+        _report(f"{name} (small, update path {path})", rep)
 
 
 def _ragged_workload(sizes, dtype):
@@ -103,14 +107,15 @@ def _ragged_workload(sizes, dtype):
                               extra={"spike_frac": 0.2, "spike_lo": 5.0, "spike_hi": 500.0})
 
 
+@pytest.mark.parametrize("path", [binding.UPDATE_PATH_REGISTERS, binding.UPDATE_PATH_BULK], ids=["registers", "bulk"])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_ragged_tails_and_chunk_edges(dtype):
+def test_ragged_tails_and_chunk_edges(dtype, path):
     """Sizes around the vector width and the 16384-element chunk: tails of 1..7 elements,
     one element short of / past a chunk, several chunks plus a tail."""
     sizes = [1, 2, 3, 5, 7, 8, 9, 10, 15, 16, 17, 31, 33, 255, 257, 2047, 2049, 16383, 16384, 16385,
-             32767, 32768, 32769, 3 * 16384 + 5, 100003]
-    rep = H.run_full(_ragged_workload(sizes, dtype), 8)
-    _report(f"ragged {dtype}", rep)
+             32767, 32768, 32769, 3 * 16384 + 5, 100003, 40 * 16384, 9 * 16384 + 4095]
+    rep = H.run_full(_ragged_workload(sizes, dtype), 8, flags=path)
+    _report(f"ragged {dtype} path {path}", rep)
     assert rep.clipped > 0
 
 
@@ -231,6 +236,31 @@ def test_argument_errors_enqueue_nothing():
     assert e.value.status == -2
     torch.cuda.synchronize()
     assert opt.launch_count() == 0 and bool((theta == 1).all()) and opt.get_stats()["steps_done"] == 0
+    opt.close()
+
+
+def test_bounded_wait_gives_up_and_context_stays_usable():
+    """A device-side wait that is never satisfied runs out after its limit, reports ADAGC_E_TIMEOUT through
+    the status word, and the same context then runs a correct step (nothing faults, nothing hangs)."""
+    import time
+    wl, offs, nums = _mini()
+    hp = H.hyper_of(wl)
+    opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], flags=binding.UPDATE_PATH_BULK)
+    assert opt.get_stats()["status"] == 0
+    t0 = time.perf_counter()
+    opt.debug_wait_timeout(50.0)
+    st = opt.get_stats()                                           # synchronises
+    dt = time.perf_counter() - t0
+    assert st["status"] & binding.ADAGC_E_TIMEOUT and 0.04 < dt < 5.0
+    theta = workloads.init_params(wl, "cuda")
+    before = theta.clone()
+    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device="cuda")
+    g = workloads.grads_for_step(wl, 1, "cuda")
+    opt.step(theta, g, m, v, ema, 1, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"],
+             hp["lambda_rel"], hp["beta"], hp["warmup"])
+    st = opt.get_stats()
+    assert st["steps_done"] == 1 and np.isfinite(st["norm"]).all() and not torch.equal(theta, before)
     opt.close()
 
 

@@ -620,7 +620,10 @@ adagc_scale_kernel(const void* __restrict__ gin, void* __restrict__ gout, const 
                    const int32_t* __restrict__ block_begin, const float* __restrict__ h_arr, int in_place) {
   constexpr int kEPV = kBF16 ? 8 : 4;
   constexpr int kWarps = kThreads / 32;
-  constexpr int kBatch = 4;  // 16-byte loads in flight per thread
+#ifndef ADAGC_SCALE_BATCH
+#define ADAGC_SCALE_BATCH 1
+#endif
+  constexpr int kBatch = ADAGC_SCALE_BATCH;  // 16-byte loads in flight per thread
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int row_base = 0;  // rows (32 vectors) dealt so far: successive chunks continue one round-robin over the warps
   const int c_end = block_begin[blockIdx.x + 1];

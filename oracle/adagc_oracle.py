@@ -142,6 +142,24 @@ def adamw_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray,
     return th1.astype(state_dtype), m1.astype(state_dtype), v1.astype(state_dtype)
 
 
+def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, beta1: float,
+                beta2: float, wd: float, state_dtype=np.float32) -> Tuple[np.ndarray, np.ndarray]:
+    """Lion on the clipped gradient hat(g) = h * g (Section 4.2 of the paper: the clip is
+    optimizer-agnostic and is used with Lion; the update itself is Lion's published rule,
+    Chen et al. 2023):
+        c     = beta1 * m + (1 - beta1) * hat(g)
+        theta = theta - lr * (sign(c) + wd * theta)        (decoupled decay on theta_{t-1})
+        m     = beta2 * m + (1 - beta2) * hat(g)
+    Elementwise, float64 arithmetic, results rounded to `state_dtype`."""
+    th = np.asarray(theta, dtype=np.float64)
+    mm = np.asarray(m, dtype=np.float64)
+    gh = float(h) * np.asarray(g, dtype=np.float64)
+    c = beta1 * mm + (1.0 - beta1) * gh
+    th1 = th - lr * (np.sign(c) + wd * th)
+    m1 = beta2 * mm + (1.0 - beta2) * gh
+    return th1.astype(state_dtype), m1.astype(state_dtype)
+
+
 def clipped_grad(g: np.ndarray, h: float) -> np.ndarray:
     """hat(g) = h * g in float64 (the clip-only use of the method with other optimizers)."""
     return float(h) * np.asarray(g, dtype=np.float64)

@@ -166,6 +166,25 @@ void adagc_ref_adamw(float* theta, const void* g, int g_is_bf16, float* m, float
   }
 }
 
+/* Lion on hat(g) = h * g for n elements, in place (Section 4.2: AdaGC with other optimizers; Lion's
+ * published rule: c = beta1 m + (1-beta1) g;  theta -= lr (sign(c) + wd theta);  m = beta2 m + (1-beta2) g). */
+void adagc_ref_lion(float* theta, const void* g, int g_is_bf16, float* m, int64_t n, double h, double lr,
+                    double beta1, double beta2, double wd) {
+  const uint16_t* gb = (const uint16_t*)g;
+  const float* gf = (const float*)g;
+#pragma omp parallel for schedule(static) if (n > 65536)
+  for (int64_t j = 0; j < n; ++j) {
+    const double gj = g_is_bf16 ? bf16_to_double(gb[j]) : (double)gf[j];
+    const double gh = h * gj;
+    const double mj = (double)m[j];
+    const double c = beta1 * mj + (1.0 - beta1) * gh;
+    const double sgn = (c > 0.0) - (c < 0.0);
+    const double th = (double)theta[j];
+    theta[j] = (float)(th - lr * (sgn + wd * th));
+    m[j] = (float)(beta2 * mj + (1.0 - beta2) * gh);
+  }
+}
+
 /* hat(g) = h * g written in the gradient's dtype (clip-only use with other optimizers). */
 void adagc_ref_scale(void* out, const void* g, int is_bf16, int64_t n, double h) {
   if (is_bf16) {

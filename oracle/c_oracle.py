@@ -49,6 +49,8 @@ def lib():
         L.adagc_ref_adamw.restype = None
         L.adagc_ref_adamw.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int64,
                                       C.c_double, C.c_int64] + [C.c_double] * 5
+        L.adagc_ref_lion.restype = None
+        L.adagc_ref_lion.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64] + [C.c_double] * 5
         L.adagc_ref_scale.restype = None
         L.adagc_ref_scale.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_double]
         L.adagc_ref_step.restype = C.c_int32
@@ -109,6 +111,15 @@ def adamw_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray,
         assert a.dtype == np.float32 and a.flags["C_CONTIGUOUS"] and a.size == g.size
     lib().adagc_ref_adamw(theta.ctypes.data, p, bf, m.ctypes.data, v.ctypes.data, g.size,
                           float(h), int(step), lr, beta1, beta2, eps, wd)
+
+
+def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, beta1: float,
+                beta2: float, wd: float) -> None:
+    """Lion on the clipped gradient, in place on fp32 theta and m."""
+    p, bf = _grad_ptr(g)
+    for a in (theta, m):
+        assert a.dtype == np.float32 and a.flags["C_CONTIGUOUS"] and a.size == g.size
+    lib().adagc_ref_lion(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, beta1, beta2, wd)
 
 
 def scale(g: np.ndarray, h: float, out: Optional[np.ndarray] = None) -> np.ndarray:

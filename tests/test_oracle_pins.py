@@ -563,3 +563,73 @@ def test_clip_only_scaling_in_gradient_dtype():
     assert (np.abs(got - want64) <= np.abs(want64) * 2.0 ** -8 + 1e-45).all()
     gf = f32_exact(rng.normal(size=1000))
     np.testing.assert_array_equal(co.scale(gf, h), (h * gf.astype(np.float64)).astype(np.float32))
+
+
+# ----------------------------------------------------------------------------- Lion on the clipped gradient
+def _lion(impl_name, theta, g, m, h, lr, b1, b2, wd):
+    if impl_name == "numpy":
+        return npo.lion_update(theta, g, m, h, lr, b1, b2, wd, np.float32)
+    th, mm = np.array(theta, np.float32), np.array(m, np.float32)
+    co.lion_update(th, np.ascontiguousarray(g, np.float32), mm, h, lr, b1, b2, wd)
+    return th, mm
+
+
+@pytest.mark.parametrize("impl_name", ["numpy", "c"])
+def test_lion_closed_forms(impl_name):
+    rng = np.random.RandomState(21)
+    n = 300
+    theta0 = f32_exact(rng.normal(size=n))
+    g = f32_exact(rng.normal(size=n) * 1e-2)
+    g[::7] = 0.0
+    lr, b1, b2, wd = 1e-3, 0.9, 0.99, 0.1
+    # first step from m = 0: c = (1-b1) h g, so the update is lr * sign(g); m_1 = (1-b2) h g
+    for h in (1.0, 0.125):
+        th, m = _lion(impl_name, theta0, g, np.zeros(n, np.float32), h, lr, b1, b2, wd)
+        want = theta0.astype(np.float64) * (1 - lr * wd) - lr * np.sign(g.astype(np.float64))
+        np.testing.assert_allclose(th, want, rtol=2e-7, atol=1e-9)
+        np.testing.assert_allclose(m, (1 - b2) * h * g.astype(np.float64), rtol=2e-7)
+    # constant gradient: m_t = g (1 - b2^t); theta_t = theta_0 r^t - lr s (1 - r^t)/(1 - r), r = 1 - lr wd
+    th, m = theta0.copy(), np.zeros(n, np.float32)
+    T = 50
+    for _ in range(T):
+        th, m = _lion(impl_name, th, g, m, 1.0, lr, b1, b2, wd)
+    r = 1 - lr * wd
+    sgn = np.sign(g.astype(np.float64))
+    np.testing.assert_allclose(m, g.astype(np.float64) * (1 - b2 ** T), rtol=1e-5)
+    np.testing.assert_allclose(th, theta0.astype(np.float64) * r ** T - lr * sgn * (1 - r ** T) / (1 - r),
+                               rtol=1e-5, atol=1e-7)
+    # the step size never depends on the gradient's magnitude: |theta_t - r theta_{t-1}| is lr or 0
+    th2, _ = _lion(impl_name, theta0, g * np.float32(1e4), np.zeros(n, np.float32), 0.3, lr, b1, b2, wd)
+    th1, _ = _lion(impl_name, theta0, g, np.zeros(n, np.float32), 1.0, lr, b1, b2, wd)
+    np.testing.assert_array_equal(th1, th2)
+    # sign follows the interpolation c, not the gradient: a small opposite gradient does not flip it
+    m0 = np.full(4, 1.0, np.float32)
+    gneg = np.full(4, -1.0, np.float32)
+    th, m = _lion(impl_name, np.zeros(4, np.float32), gneg, m0, 1.0, lr, b1, b2, 0.0)
+    np.testing.assert_allclose(th, -lr * np.ones(4), rtol=1e-6)          # c = 0.9 - 0.1 > 0
+    th, m = _lion(impl_name, np.zeros(4, np.float32), gneg * np.float32(10), m0, 1.0, lr, b1, b2, 0.0)
+    np.testing.assert_allclose(th, +lr * np.ones(4), rtol=1e-6)          # c = 0.9 - 1.0 < 0
+    np.testing.assert_allclose(m, 0.99 * 1.0 + 0.01 * -10.0, rtol=1e-6)
+
+
+def test_lion_brute_force_and_oracles_agree():
+    rng = np.random.RandomState(22)
+    n = 64
+    theta = f32_exact(rng.normal(size=n)); m = np.zeros(n, np.float32)
+    tb = [float(x) for x in theta]; mb = [0.0] * n
+    tc, mc = theta.copy(), m.copy()
+    lr, b1, b2, wd = 3e-4, 0.9, 0.99, 0.1
+    for t in range(20):
+        g = f32_exact(rng.standard_t(3, size=n) * 1e-2)
+        h = 1.0 if t % 3 else 0.37
+        theta, m = npo.lion_update(theta, g, m, h, lr, b1, b2, wd, np.float32)
+        co.lion_update(tc, g, mc, h, lr, b1, b2, wd)
+        for j in range(n):
+            gh = h * float(g[j])
+            c = b1 * mb[j] + (1 - b1) * gh
+            tb[j] = tb[j] - lr * (math.copysign(1.0, c) * (c != 0) + wd * tb[j])
+            mb[j] = b2 * mb[j] + (1 - b2) * gh
+    np.testing.assert_allclose(theta, tb, rtol=1e-5, atol=1e-7)
+    np.testing.assert_allclose(m, mb, rtol=1e-5, atol=1e-9)
+    np.testing.assert_allclose(tc, theta, rtol=3e-7, atol=1e-9)
+    np.testing.assert_allclose(mc, m, rtol=3e-7, atol=1e-12)

@@ -150,11 +150,24 @@ def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: f
         c     = beta1 * m + (1 - beta1) * hat(g)
         theta = theta - lr * (sign(c) + wd * theta)        (decoupled decay on theta_{t-1})
         m     = beta2 * m + (1 - beta2) * hat(g)
-    Elementwise, float64 arithmetic, results rounded to `state_dtype`."""
+    Elementwise; theta and m are computed in float64 and rounded to `state_dtype`.
+
+    sign(c) is a discrete decision, and neither paper fixes its precision.  So that it can be compared
+    with a float32 implementation it is taken in float32, in this stated order: h, beta1 and 1 - beta1
+    are rounded to float32; hat(g) = fl32(h * g); t = fl32((1 - beta1) * hat(g)); the sign is that of the
+    exact value of beta1 * m + t (what a fused multiply-add returns the sign of).  In float64-state mode
+    (`state_dtype=np.float64`) the decision is taken in float64 like everything else."""
     th = np.asarray(theta, dtype=np.float64)
     mm = np.asarray(m, dtype=np.float64)
-    gh = float(h) * np.asarray(g, dtype=np.float64)
-    c = beta1 * mm + (1.0 - beta1) * gh
+    g64 = np.asarray(g, dtype=np.float64)
+    gh = float(h) * g64
+    if state_dtype == np.float32:
+        h32 = float(np.float32(h))
+        gh32 = (h32 * g64).astype(np.float32).astype(np.float64)            # products of two fp32 are exact in fp64
+        t32 = (float(np.float32(1.0 - beta1)) * gh32).astype(np.float32).astype(np.float64)
+        c = float(np.float32(beta1)) * mm + t32
+    else:
+        c = beta1 * mm + (1.0 - beta1) * gh
     th1 = th - lr * (np.sign(c) + wd * th)
     m1 = beta2 * mm + (1.0 - beta2) * gh
     return th1.astype(state_dtype), m1.astype(state_dtype)

@@ -123,6 +123,20 @@ int adagc_step(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, v
                double wd, double lambda_rel, double beta, int64_t warmup, void* cuda_stream);
 
 /*
+ * The same clip fused with Lion instead of AdamW (Section 4.2 of the paper: AdaGC is optimizer-agnostic
+ * and is used with Lion).  Phases 1 and 2 are those of adagc_step; the update phase applies Lion's rule
+ * to the clipped gradient hat(g) = h_i g:
+ *     c = beta1 m + (1 - beta1) hat(g);   theta <- theta - lr (sign(c) + wd theta);
+ *     m <- beta2 m + (1 - beta2) hat(g)
+ * d_params and d_m are fp32 arenas updated in place (Lion keeps one state per parameter, there is no v).
+ * Everything elementwise is fp32; where the two terms of c cancel to within fp32 rounding the sign is a
+ * near-tie and may differ from a float64 evaluation.  Typical beta1 0.9, beta2 0.99.
+ */
+int adagc_step_lion(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, float* d_ema,
+                    int64_t step, double lr, double beta1, double beta2, double wd, double lambda_rel,
+                    double beta, int64_t warmup, void* cuda_stream);
+
+/*
  * Clip-only entry (Section 4.2: the clip is optimizer-agnostic): same norms, decisions and
  * gamma update as adagc_step, then writes the clipped gradient h_i * g_i in the gradient dtype.
  * d_grads_out may equal d_grads_in (in place); in place, tensors with h == 1 are not rewritten.

@@ -143,34 +143,33 @@ def adamw_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray,
 
 
 def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, beta1: float,
-                beta2: float, wd: float, state_dtype=np.float32) -> Tuple[np.ndarray, np.ndarray]:
+                beta2: float, wd: float, state_dtype=np.float32, return_margin: bool = False):
     """Lion on the clipped gradient hat(g) = h * g (Section 4.2 of the paper: the clip is
     optimizer-agnostic and is used with Lion; the update itself is Lion's published rule,
     Chen et al. 2023):
         c     = beta1 * m + (1 - beta1) * hat(g)
         theta = theta - lr * (sign(c) + wd * theta)        (decoupled decay on theta_{t-1})
         m     = beta2 * m + (1 - beta2) * hat(g)
-    Elementwise; theta and m are computed in float64 and rounded to `state_dtype`.
+    Elementwise, float64 arithmetic, results rounded to `state_dtype`.
 
-    sign(c) is a discrete decision, and neither paper fixes its precision.  So that it can be compared
-    with a float32 implementation it is taken in float32, in this stated order: h, beta1 and 1 - beta1
-    are rounded to float32; hat(g) = fl32(h * g); t = fl32((1 - beta1) * hat(g)); the sign is that of the
-    exact value of beta1 * m + t (what a fused multiply-add returns the sign of).  In float64-state mode
-    (`state_dtype=np.float64`) the decision is taken in float64 like everything else."""
+    sign(c) is a discrete decision.  Where the two terms of c nearly cancel, an implementation that
+    rounds differently (float32 arithmetic, a stored m that differs in its last bit) may legitimately
+    take the other sign; with `return_margin` the relative margin |c| / (|beta1 m| + |(1-beta1) hat(g)|)
+    of every element is returned too, so that a comparison can tell such near-ties from real errors."""
     th = np.asarray(theta, dtype=np.float64)
     mm = np.asarray(m, dtype=np.float64)
-    g64 = np.asarray(g, dtype=np.float64)
-    gh = float(h) * g64
-    if state_dtype == np.float32:
-        h32 = float(np.float32(h))
-        gh32 = (h32 * g64).astype(np.float32).astype(np.float64)            # products of two fp32 are exact in fp64
-        t32 = (float(np.float32(1.0 - beta1)) * gh32).astype(np.float32).astype(np.float64)
-        c = float(np.float32(beta1)) * mm + t32
-    else:
-        c = beta1 * mm + (1.0 - beta1) * gh
+    gh = float(h) * np.asarray(g, dtype=np.float64)
+    a, b = beta1 * mm, (1.0 - beta1) * gh
+    c = a + b
     th1 = th - lr * (np.sign(c) + wd * th)
     m1 = beta2 * mm + (1.0 - beta2) * gh
-    return th1.astype(state_dtype), m1.astype(state_dtype)
+    out = (th1.astype(state_dtype), m1.astype(state_dtype))
+    if return_margin:
+        den = np.abs(a) + np.abs(b)
+        with np.errstate(divide="ignore", invalid="ignore"):
+            margin = np.where(den > 0, np.abs(c) / den, np.inf)
+        return out + (margin,)
+    return out
 
 
 def clipped_grad(g: np.ndarray, h: float) -> np.ndarray:

@@ -168,24 +168,23 @@ void adagc_ref_adamw(float* theta, const void* g, int g_is_bf16, float* m, float
 
 /* Lion on hat(g) = h * g for n elements, in place (Section 4.2: AdaGC with other optimizers; Lion's
  * published rule: c = beta1 m + (1-beta1) g;  theta -= lr (sign(c) + wd theta);  m = beta2 m + (1-beta2) g).
- * theta and m are computed in float64.  sign(c) is a discrete decision whose precision no paper fixes;
- * to be comparable with a float32 implementation it is taken in float32 in this order: h, beta1 and
- * 1 - beta1 rounded to float32; hat(g) = fl32(h g); t = fl32((1 - beta1) hat(g)); sign of the exact
- * beta1 m + t (the sign a fused multiply-add returns). */
+ * sign(c) is a discrete decision: where the two terms of c nearly cancel, an implementation that rounds
+ * differently may legitimately take the other sign.  If near_tie is not NULL, near_tie[j] is incremented
+ * (saturating at 255) when |c| < tie_tol * (|beta1 m| + |(1-beta1) hat(g)|), so that a comparison can
+ * tell such elements from real errors. */
 void adagc_ref_lion(float* theta, const void* g, int g_is_bf16, float* m, int64_t n, double h, double lr,
-                    double beta1, double beta2, double wd) {
+                    double beta1, double beta2, double wd, uint8_t* near_tie, double tie_tol) {
   const uint16_t* gb = (const uint16_t*)g;
   const float* gf = (const float*)g;
-  const double h32 = (double)(float)h, b1_32 = (double)(float)beta1, omb1_32 = (double)(float)(1.0 - beta1);
 #pragma omp parallel for schedule(static) if (n > 65536)
   for (int64_t j = 0; j < n; ++j) {
     const double gj = g_is_bf16 ? bf16_to_double(gb[j]) : (double)gf[j];
     const double gh = h * gj;
     const double mj = (double)m[j];
-    const double gh32 = (double)(float)(h32 * gj);   /* product of two fp32 values: exact in double */
-    const double t32 = (double)(float)(omb1_32 * gh32);
-    const double c = b1_32 * mj + t32;
+    const double a = beta1 * mj, b = (1.0 - beta1) * gh;
+    const double c = a + b;
     const double sgn = (c > 0.0) - (c < 0.0);
+    if (near_tie && fabs(c) < tie_tol * (fabs(a) + fabs(b)) && near_tie[j] < 255) near_tie[j] += 1;
     const double th = (double)theta[j];
     theta[j] = (float)(th - lr * (sgn + wd * th));
     m[j] = (float)(beta2 * mj + (1.0 - beta2) * gh);

@@ -50,7 +50,8 @@ def lib():
         L.adagc_ref_adamw.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int64,
                                       C.c_double, C.c_int64] + [C.c_double] * 5
         L.adagc_ref_lion.restype = None
-        L.adagc_ref_lion.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64] + [C.c_double] * 5
+        L.adagc_ref_lion.argtypes = ([C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64] + [C.c_double] * 5 +
+                                     [C.c_void_p, C.c_double])
         L.adagc_ref_scale.restype = None
         L.adagc_ref_scale.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_double]
         L.adagc_ref_step.restype = C.c_int32
@@ -114,12 +115,18 @@ def adamw_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray,
 
 
 def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, beta1: float,
-                beta2: float, wd: float) -> None:
-    """Lion on the clipped gradient, in place on fp32 theta and m."""
+                beta2: float, wd: float, near_tie: Optional[np.ndarray] = None, tie_tol: float = 0.0) -> None:
+    """Lion on the clipped gradient, in place on fp32 theta and m.  `near_tie` (uint8, same length) counts,
+    per element, the steps in which sign(c) was decided with a relative margin below `tie_tol`."""
     p, bf = _grad_ptr(g)
     for a in (theta, m):
         assert a.dtype == np.float32 and a.flags["C_CONTIGUOUS"] and a.size == g.size
-    lib().adagc_ref_lion(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, beta1, beta2, wd)
+    nt = None
+    if near_tie is not None:
+        assert near_tie.dtype == np.uint8 and near_tie.flags["C_CONTIGUOUS"] and near_tie.size == g.size
+        nt = near_tie.ctypes.data
+    lib().adagc_ref_lion(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, beta1, beta2, wd,
+                         nt, float(tie_tol))
 
 
 def scale(g: np.ndarray, h: float, out: Optional[np.ndarray] = None) -> np.ndarray:

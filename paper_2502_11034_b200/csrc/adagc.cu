@@ -276,25 +276,42 @@ adagc_warmup_finalize_kernel(ClipScalars cs, float* __restrict__ ema, StatPtrs s
 // ------------------------------------------------------------------------------------------------
 // phase 3: AdamW on the clipped gradient (last four lines of Algorithm 1)
 // ------------------------------------------------------------------------------------------------
+// kOpt selects the optimizer applied to the clipped gradient: AdamW (Algorithm 1) or Lion (Section 4.2
+// names it as another optimizer the clip is used with; its rule is c = beta1 m + (1-beta1) hat(g),
+// theta -= lr (sign(c) + wd theta), m = beta2 m + (1-beta2) hat(g); one state stream, no v).
+constexpr int kOptAdamW = 0;
+constexpr int kOptLion = 1;
+
+template <int kOpt>
 __device__ __forceinline__ void adamw_elem(float g, float h, float& p, float& m, float& v,
                                            const AdamScalars& a) {
   const float gh = h * g;  // hat(g)
-  m = fmaf(a.beta1, m, a.one_minus_beta1 * gh);
-  v = fmaf(a.beta2, v, a.one_minus_beta2 * (gh * gh));
-  const float denom = __fsqrt_rn(v * a.inv_bc2) + a.eps;  // sqrt(v_hat) + eps
-  p = fmaf(-a.step_size, __fdiv_rn(m, denom), p * a.decay);
+  if (kOpt == kOptLion) {
+    // fp32 like the rest of the update; where the two terms nearly cancel the sign is a near-tie
+    const float c = fmaf(a.beta1, m, a.one_minus_beta1 * gh);
+    const float sgn = c > 0.0f ? 1.0f : (c < 0.0f ? -1.0f : c);  // 0 stays 0, NaN stays NaN
+    p = fmaf(-a.step_size, sgn, p * a.decay);                    // step_size = lr, decay = 1 - lr wd
+    m = fmaf(a.beta2, m, a.one_minus_beta2 * gh);
+  } else {
+    m = fmaf(a.beta1, m, a.one_minus_beta1 * gh);
+    v = fmaf(a.beta2, v, a.one_minus_beta2 * (gh * gh));
+    const float denom = __fsqrt_rn(v * a.inv_bc2) + a.eps;  // sqrt(v_hat) + eps
+    p = fmaf(-a.step_size, __fdiv_rn(m, denom), p * a.decay);
+  }
 }
 
+template <int kOpt>
 __device__ __forceinline__ void adamw_vec4(const float g0, const float g1, const float g2, const float g3,
                                            float h, float4& p, float4& m, float4& v, const AdamScalars& a) {
-  adamw_elem(g0, h, p.x, m.x, v.x, a);
-  adamw_elem(g1, h, p.y, m.y, v.y, a);
-  adamw_elem(g2, h, p.z, m.z, v.z, a);
-  adamw_elem(g3, h, p.w, m.w, v.w, a);
+  adamw_elem<kOpt>(g0, h, p.x, m.x, v.x, a);
+  adamw_elem<kOpt>(g1, h, p.y, m.y, v.y, a);
+  adamw_elem<kOpt>(g2, h, p.z, m.z, v.z, a);
+  adamw_elem<kOpt>(g3, h, p.w, m.w, v.w, a);
 }
 
-// Eight consecutive elements of one chunk: 7 (bf16 gradients) or 8 (fp32) 16-byte loads, 6 stores.
-template <bool kBF16>
+// Eight consecutive elements of one chunk: 7 (bf16 gradients) or 8 (fp32) 16-byte loads, 6 stores
+// (AdamW; Lion has no v stream).
+template <bool kBF16, int kOpt>
 __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gbase, float4* __restrict__ p4,
                                              float4* __restrict__ m4, float4* __restrict__ v4, float h,
                                              const AdamScalars& a) {
@@ -311,19 +328,26 @@ __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gba
   }
   float4 pa = ld_stream(p4 + 2 * i), pb = ld_stream(p4 + 2 * i + 1);
   float4 ma = ld_stream(m4 + 2 * i), mb = ld_stream(m4 + 2 * i + 1);
-  float4 va = ld_stream(v4 + 2 * i), vb = ld_stream(v4 + 2 * i + 1);
-  adamw_vec4(g[0], g[1], g[2], g[3], h, pa, ma, va, a);
-  adamw_vec4(g[4], g[5], g[6], g[7], h, pb, mb, vb, a);
+  float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
+  if (kOpt == kOptAdamW) {
+    va = ld_stream(v4 + 2 * i);
+    vb = ld_stream(v4 + 2 * i + 1);
+  }
+  adamw_vec4<kOpt>(g[0], g[1], g[2], g[3], h, pa, ma, va, a);
+  adamw_vec4<kOpt>(g[4], g[5], g[6], g[7], h, pb, mb, vb, a);
   st_stream(p4 + 2 * i, pa); st_stream(p4 + 2 * i + 1, pb);
   st_stream(m4 + 2 * i, ma); st_stream(m4 + 2 * i + 1, mb);
-  st_stream(v4 + 2 * i, va); st_stream(v4 + 2 * i + 1, vb);
+  if (kOpt == kOptAdamW) {
+    st_stream(v4 + 2 * i, va);
+    st_stream(v4 + 2 * i + 1, vb);
+  }
 }
 
 // A partial chunk (a small tensor, or the end of one).  Work is dealt in rows of 32 groups (256
 // elements) and the rows of successive chunks go to the block's warps in one continuing round-robin:
 // row_base counts the rows dealt so far.  Restarting at warp 0 for every chunk would give the low warps
 // the extra rows every time and make them the critical path.
-template <bool kBF16, int kBlockThreads>
+template <bool kBF16, int kBlockThreads, int kOpt>
 __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, int& row_base, float* __restrict__ params,
                                                     const void* __restrict__ grads, float* __restrict__ m_arena,
                                                     float* __restrict__ v_arena, const AdamScalars& a) {
@@ -339,7 +363,7 @@ __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, in
 #pragma unroll 2
   for (int r = (warp - row_base) & (kWarps - 1); r < rows; r += kWarps) {
     const int i = (r << 5) + lane;
-    if (i < n8) adamw_group8<kBF16>(i, gbase, p4, m4, v4, h, a);
+    if (i < n8) adamw_group8<kBF16, kOpt>(i, gbase, p4, m4, v4, h, a);
   }
   row_base = (row_base + rows) & (kWarps - 1);
   const int t = (n8 << 3) + lane;  // ragged tail (fewer than 8 elements): the next warp in turn takes it
@@ -350,16 +374,17 @@ __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, in
     } else {
       g = reinterpret_cast<const float*>(gbase)[t];
     }
-    float p = params[start + t], m = m_arena[start + t], v = v_arena[start + t];
-    adamw_elem(g, h, p, m, v, a);
+    float p = params[start + t], m = m_arena[start + t], v = 0.0f;
+    if (kOpt == kOptAdamW) v = v_arena[start + t];
+    adamw_elem<kOpt>(g, h, p, m, v, a);
     params[start + t] = p;
     m_arena[start + t] = m;
-    v_arena[start + t] = v;
+    if (kOpt == kOptAdamW) v_arena[start + t] = v;
   }
 }
 
 // Register-streaming update kernel: every thread loads eight elements of each stream into registers.
-template <bool kBF16>
+template <bool kBF16, int kOpt>
 __global__ void __launch_bounds__(kThreads)
 adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, float* __restrict__ m_arena,
                     float* __restrict__ v_arena, const Chunk* __restrict__ chunks,
@@ -388,9 +413,10 @@ adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, 
       float4* __restrict__ v4 = reinterpret_cast<float4*>(v_arena + start);
       const char* __restrict__ gbase = static_cast<const char*>(grads) + start * (kBF16 ? 2 : 4);
 #pragma unroll 2
-      for (int k = 0; k < kChunkElems / 8 / kThreads; ++k) adamw_group8<kBF16>(k * kThreads + tid, gbase, p4, m4, v4, h, a);
+      for (int k = 0; k < kChunkElems / 8 / kThreads; ++k)
+        adamw_group8<kBF16, kOpt>(k * kThreads + tid, gbase, p4, m4, v4, h, a);
     } else {
-      adamw_partial_chunk<kBF16, kThreads>(ck, h, row_base, params, grads, m_arena, v_arena, a);
+      adamw_partial_chunk<kBF16, kThreads, kOpt>(ck, h, row_base, params, grads, m_arena, v_arena, a);
     }
     if (c_next >= n_chunks) break;
     c = c_next;
@@ -472,9 +498,11 @@ __device__ __forceinline__ void bulk_wait_smem_read() { asm volatile("cp.async.b
 __device__ __forceinline__ void bulk_wait_done() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_generic_to_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-constexpr int tma_smem_bytes(bool bf16) { return kTmaStages * kTile * (12 + (bf16 ? 2 : 4)); }
+constexpr int tma_smem_bytes(bool bf16, int opt) {
+  return kTmaStages * kTile * ((opt == kOptLion ? 8 : 12) + (bf16 ? 2 : 4));
+}
 
-template <bool kBF16>
+template <bool kBF16, int kOpt>
 __global__ void __launch_bounds__(kTmaThreads, 1)
 adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ grads, float* __restrict__ m_arena,
                         float* __restrict__ v_arena, const Chunk* __restrict__ chunks,
@@ -482,7 +510,8 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
                         const float* __restrict__ h_arr, AdamScalars a, int* __restrict__ status) {
   extern __shared__ __align__(128) unsigned char tile_smem[];
   constexpr int kGBytes = kBF16 ? 2 : 4;
-  constexpr uint32_t kStageBytes = kTile * (12 + kGBytes);
+  constexpr int kStateBytes = kOpt == kOptLion ? 8 : 12;  // theta, m (and v) per element; g follows them
+  constexpr uint32_t kStageBytes = kTile * (kStateBytes + kGBytes);
   __shared__ __align__(8) uint64_t full_bar[kTmaStages];
   const int tid = threadIdx.x;
   const int begin = block_begin[blockIdx.x], mid = block_mid[blockIdx.x], end = block_begin[blockIdx.x + 1];
@@ -503,8 +532,8 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
     mbar_arrive_expect_tx(&full_bar[s], kStageBytes);
     bulk_load(b, params + e, kTile * 4, &full_bar[s]);
     bulk_load(b + kTile * 4, m_arena + e, kTile * 4, &full_bar[s]);
-    bulk_load(b + kTile * 8, v_arena + e, kTile * 4, &full_bar[s]);
-    bulk_load(b + kTile * 12, static_cast<const char*>(grads) + e * kGBytes, kTile * kGBytes, &full_bar[s]);
+    if (kOpt == kOptAdamW) bulk_load(b + kTile * 8, v_arena + e, kTile * 4, &full_bar[s]);
+    bulk_load(b + kTile * kStateBytes, static_cast<const char*>(grads) + e * kGBytes, kTile * kGBytes, &full_bar[s]);
   };
 
   bool healthy = true;
@@ -539,15 +568,17 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
         for (int q = tid; q < kTile / 4; q += kTmaThreads) {
           float g0, g1, g2, g3;
           if (kBF16) {
-            const uint2 w = reinterpret_cast<const uint2*>(b + kTile * 12)[q];
+            const uint2 w = reinterpret_cast<const uint2*>(b + kTile * kStateBytes)[q];
             g0 = bf16_lo(w.x); g1 = bf16_hi(w.x); g2 = bf16_lo(w.y); g3 = bf16_hi(w.y);
           } else {
-            const float4 w = reinterpret_cast<const float4*>(b + kTile * 12)[q];
+            const float4 w = reinterpret_cast<const float4*>(b + kTile * kStateBytes)[q];
             g0 = w.x; g1 = w.y; g2 = w.z; g3 = w.w;
           }
-          float4 p = p4[q], m = m4[q], v = v4[q];
-          adamw_vec4(g0, g1, g2, g3, h, p, m, v, a);
-          p4[q] = p; m4[q] = m; v4[q] = v;
+          float4 p = p4[q], m = m4[q], v = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (kOpt == kOptAdamW) v = v4[q];
+          adamw_vec4<kOpt>(g0, g1, g2, g3, h, p, m, v, a);
+          p4[q] = p; m4[q] = m;
+          if (kOpt == kOptAdamW) v4[q] = v;
         }
         fence_generic_to_async_smem();  // the updated tile must be visible to the bulk-copy engine
       } else {
@@ -563,7 +594,7 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
         const int64_t e = chunk_start(ck) + static_cast<int64_t>(sub) * kTile;
         bulk_store(params + e, b, kTile * 4);
         bulk_store(m_arena + e, b + kTile * 4, kTile * 4);
-        bulk_store(v_arena + e, b + kTile * 8, kTile * 4);
+        if (kOpt == kOptAdamW) bulk_store(v_arena + e, b + kTile * 8, kTile * 4);
         bulk_commit();
       }
       if (last_of_chunk) {
@@ -593,7 +624,7 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
   int row_base = 0;
   for (int c = mid; c < end; ++c) {
     const Chunk ck = chunks[c];
-    adamw_partial_chunk<kBF16, kTmaThreads>(ck, h_arr[ck.tensor], row_base, params, grads, m_arena, v_arena, a);
+    adamw_partial_chunk<kBF16, kTmaThreads, kOpt>(ck, h_arr[ck.tensor], row_base, params, grads, m_arena, v_arena, a);
   }
 }
 
@@ -844,6 +875,33 @@ int enqueue_clip_phases(adagc_ctx* ctx, const void* d_grads, float* d_ema, int64
   return ADAGC_OK;
 }
 
+// Largest L1 carve-out for the register kernels (L1 lines hold their loads in flight); opt-in shared
+// memory size for the bulk-async kernels.
+template <bool kBF16>
+bool prepare_update_kernels() {
+  return cudaFuncSetAttribute(adagc_update_kernel<kBF16, kOptAdamW>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                              cudaSharedmemCarveoutMaxL1) == cudaSuccess &&
+         cudaFuncSetAttribute(adagc_update_kernel<kBF16, kOptLion>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                              cudaSharedmemCarveoutMaxL1) == cudaSuccess &&
+         cudaFuncSetAttribute(adagc_update_tma_kernel<kBF16, kOptAdamW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              tma_smem_bytes(kBF16, kOptAdamW)) == cudaSuccess &&
+         cudaFuncSetAttribute(adagc_update_tma_kernel<kBF16, kOptLion>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              tma_smem_bytes(kBF16, kOptLion)) == cudaSuccess;
+}
+
+template <bool kBF16, int kOpt>
+void launch_update(adagc_ctx* ctx, float* p, const void* g, float* m, float* v, const AdamScalars& a,
+                   cudaStream_t s) {
+  const StatPtrs st = ctx->stats();
+  if (ctx->update_bulk)
+    adagc_update_tma_kernel<kBF16, kOpt><<<ctx->grid_update, kTmaThreads, tma_smem_bytes(kBF16, kOpt), s>>>(
+        p, g, m, v, ctx->d_chunks_upd(), ctx->d_begin_upd(), ctx->d_mid_upd(), st.h, a, st.status);
+  else
+    adagc_update_kernel<kBF16, kOpt><<<ctx->grid_update, kThreads, 0, s>>>(p, g, m, v, ctx->d_chunks_upd(),
+                                                                          ctx->d_begin_upd(), st.h, a);
+  ctx->launches++;
+}
+
 int finish_launches(adagc_ctx* ctx, cudaStream_t s) {
   if (ctx->timing) {
     cudaEventRecord(ctx->ev[3], s);
@@ -917,18 +975,12 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
     int occ_n = 0, occ_s = 0;
     if (ctx->bf16) {
       ok = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_n, adagc_norm_kernel<true>, kThreads, 0) == cudaSuccess &&
-           cudaFuncSetAttribute(adagc_update_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                cudaSharedmemCarveoutMaxL1) == cudaSuccess &&
-           cudaFuncSetAttribute(adagc_update_tma_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                tma_smem_bytes(true)) == cudaSuccess &&
-           cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_s, adagc_scale_kernel<true>, kThreads, 0) == cudaSuccess;
+           cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_s, adagc_scale_kernel<true>, kThreads, 0) == cudaSuccess &&
+           prepare_update_kernels<true>();
     } else {
       ok = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_n, adagc_norm_kernel<false>, kThreads, 0) == cudaSuccess &&
-           cudaFuncSetAttribute(adagc_update_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                                cudaSharedmemCarveoutMaxL1) == cudaSuccess &&
-           cudaFuncSetAttribute(adagc_update_tma_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                tma_smem_bytes(false)) == cudaSuccess &&
-           cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_s, adagc_scale_kernel<false>, kThreads, 0) == cudaSuccess;
+           cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_s, adagc_scale_kernel<false>, kThreads, 0) == cudaSuccess &&
+           prepare_update_kernels<false>();
     }
     if (ok) {
       const int64_t sms = prop.multiProcessorCount;
@@ -1004,26 +1056,40 @@ int adagc_step(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, v
   a.step_size = static_cast<float>(lr / bc1);
   a.decay = static_cast<float>(1.0 - lr * wd);
   a.eps = static_cast<float>(eps);
-  const StatPtrs st = ctx->stats();
-  float* p = static_cast<float*>(d_params);
-  float* m = static_cast<float*>(d_m);
-  float* v = static_cast<float*>(d_v);
-  if (ctx->update_bulk) {
-    if (ctx->bf16)
-      adagc_update_tma_kernel<true><<<ctx->grid_update, kTmaThreads, tma_smem_bytes(true), s>>>(
-          p, d_grads, m, v, ctx->d_chunks_upd(), ctx->d_begin_upd(), ctx->d_mid_upd(), st.h, a, st.status);
-    else
-      adagc_update_tma_kernel<false><<<ctx->grid_update, kTmaThreads, tma_smem_bytes(false), s>>>(
-          p, d_grads, m, v, ctx->d_chunks_upd(), ctx->d_begin_upd(), ctx->d_mid_upd(), st.h, a, st.status);
-  } else {
-    if (ctx->bf16)
-      adagc_update_kernel<true><<<ctx->grid_update, kThreads, 0, s>>>(p, d_grads, m, v, ctx->d_chunks_upd(),
-                                                                     ctx->d_begin_upd(), st.h, a);
-    else
-      adagc_update_kernel<false><<<ctx->grid_update, kThreads, 0, s>>>(p, d_grads, m, v, ctx->d_chunks_upd(),
-                                                                      ctx->d_begin_upd(), st.h, a);
-  }
-  ctx->launches++;
+  if (ctx->bf16)
+    launch_update<true, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
+                                   static_cast<float*>(d_v), a, s);
+  else
+    launch_update<false, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
+                                    static_cast<float*>(d_v), a, s);
+  return finish_launches(ctx, s);
+}
+
+int adagc_step_lion(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, float* d_ema, int64_t step,
+                    double lr, double beta1, double beta2, double wd, double lambda_rel, double beta,
+                    int64_t warmup, void* cuda_stream) {
+  int rc = check_clip_args(ctx, d_ema, step, lambda_rel, beta, warmup);
+  if (rc != ADAGC_OK) return rc;
+  if (!d_params || !d_grads || !d_m) return ADAGC_E_INVALID_ARG;
+  if (!(beta1 >= 0.0 && beta1 < 1.0) || !(beta2 >= 0.0 && beta2 < 1.0)) return ADAGC_E_INVALID_ARG;
+  if (!std::isfinite(lr) || !std::isfinite(wd)) return ADAGC_E_INVALID_ARG;
+  if (!aligned16(d_params) || !aligned16(d_grads) || !aligned16(d_m)) return ADAGC_E_MISALIGNED;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  rc = enqueue_clip_phases(ctx, d_grads, d_ema, step, lambda_rel, beta, warmup, s);
+  if (rc != ADAGC_OK) return rc;
+  AdamScalars a;
+  a.beta1 = static_cast<float>(beta1);
+  a.one_minus_beta1 = static_cast<float>(1.0 - beta1);
+  a.beta2 = static_cast<float>(beta2);
+  a.one_minus_beta2 = static_cast<float>(1.0 - beta2);
+  a.inv_bc2 = 0.0f;
+  a.step_size = static_cast<float>(lr);
+  a.decay = static_cast<float>(1.0 - lr * wd);
+  a.eps = 0.0f;
+  if (ctx->bf16)
+    launch_update<true, kOptLion>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), nullptr, a, s);
+  else
+    launch_update<false, kOptLion>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), nullptr, a, s);
   return finish_launches(ctx, s);
 }
 

@@ -240,3 +240,60 @@ def check_clipped_grads(got: np.ndarray, want: np.ndarray, what: str):
     else:
         a, b = got.astype(np.float64), want.astype(np.float64)
         assert (np.abs(a - b) <= RTOL * np.abs(b) + 1e-45).all(), f"{what}: clipped gradient differs"
+
+
+LION_TIE_TOL = 1e-5      # sign(c) decided with a relative margin below this may legitimately differ
+
+
+def run_full_lion(wl: workloads.Workload, n_steps: int, device="cuda", flags: int = 0, lr: float = 1e-4,
+                  beta1: float = 0.9, beta2: float = 0.99, hyper_over: Optional[dict] = None) -> ParityReport:
+    """Every element, clip fused with Lion (adagc_step_lion) vs the C oracle.
+    m never depends on a sign decision and is compared on every element.  theta is compared with the
+    usual tolerance on every element whose sign(c) was never a near-tie (relative margin >= 1e-5, the
+    path's tolerance); an element with k near-ties may differ by up to 2 lr k on top of it."""
+    hp = hyper_of(wl, **(hyper_over or {}))
+    offs = np.array([t.offset for t in wl.tensors], np.int64)
+    nums = np.array([t.numel for t in wl.tensors], np.int64)
+    opt = binding.AdaGC(nums.tolist(), offs.tolist(), wl.torch_grad_dtype, hp["lambda_abs"], device=device, flags=flags)
+    theta = workloads.init_params(wl, device)
+    m = torch.zeros_like(theta)
+    ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device=device)
+    r_theta = theta.cpu().numpy().copy()
+    r_m = np.zeros_like(r_theta)
+    ties = np.zeros(r_theta.shape, np.uint8)
+    gamma = np.zeros(wl.n_tensors, np.float32)
+    clip_count = np.zeros(wl.n_tensors, np.uint64)
+    rep = ParityReport()
+    for t in range(1, n_steps + 1):
+        g = workloads.grads_for_step(wl, t, device)
+        opt.step_lion(theta, g, m, ema, t, lr, beta1, beta2, hp["wd"], hp["lambda_rel"], hp["beta"], hp["warmup"])
+        g_np = to_numpy_grads(g)
+        ssq = c_oracle.sumsq_tensors(g_np, offs, nums)
+        r = c_oracle.clip_decisions(ssq, gamma, t, hp["lambda_rel"], hp["beta"], hp["lambda_abs"], hp["warmup"])
+        clip_count += r["flag"].astype(np.uint64)
+        for i, (o, n) in enumerate(zip(offs, nums)):
+            c_oracle.lion_update(r_theta[o:o + n], g_np[o:o + n], r_m[o:o + n], float(r["h"][i]), lr, beta1, beta2,
+                                 hp["wd"], near_tie=ties[o:o + n], tie_tol=LION_TIE_TOL)
+        st = opt.get_stats()
+        check_decisions(st, opt.get_sumsq(), ema.cpu().numpy(), r, rep, t)
+        rep.steps = t
+    st = opt.get_stats()
+    assert st["steps_done"] == n_steps and np.array_equal(st["clip_count"], clip_count) and st["status"] == 0
+    th, mm = theta.cpu().numpy(), m.cpu().numpy()
+    n_ties = n_flipped = 0
+    for t_, o, n in zip(wl.tensors, offs, nums):
+        sure = ties[o:o + n] == 0
+        check_state("m", mm[o:o + n], r_m[o:o + n], rep, t_.name)
+        check_state("theta", th[o:o + n][sure], r_theta[o:o + n][sure], rep, t_.name)
+        if not sure.all():
+            d = np.abs(th[o:o + n][~sure].astype(np.float64) - r_theta[o:o + n][~sure])
+            k = ties[o:o + n][~sure].astype(np.float64)
+            ref = np.abs(r_theta[o:o + n][~sure].astype(np.float64))
+            assert (d <= 2.0 * lr * k * 1.001 + RTOL * np.maximum(ref, 1e-3)).all(), f"theta of {t_.name}: near-tie element off"
+            n_ties += int((~sure).sum())
+            n_flipped += int((d > lr).sum())
+    rep.max_tensor_rel["lion_near_tie_elements"] = n_ties
+    rep.max_tensor_rel["lion_flipped_elements"] = n_flipped
+    assert n_ties <= 1e-3 * wl.n_params + 50      # near-ties are rare: this is not a loophole for real errors
+    opt.close()
+    return rep

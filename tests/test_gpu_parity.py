@@ -99,6 +99,23 @@ def test_small_layouts_all_elements(name, over):
         _report(f"{name} (small, update path {path})", rep)
 
 
+@pytest.mark.parametrize("path", [binding.UPDATE_PATH_REGISTERS, binding.UPDATE_PATH_BULK], ids=["registers", "bulk"])
+def test_lion_small_layouts_all_elements(path):
+    """The clip fused with Lion (Section 4.2: optimizer-agnostic use), both update kernels."""
+    for name, over in [("llama2_7b", dict(n_layer=2, d=256, ffn=688, vocab=1000)),
+                       ("many_small", dict(n_tensors=300, lo=1, hi=40000))]:
+        wl = workloads.build(name, **over)
+        rep = H.run_full_lion(wl, 15, flags=path)
+        _report(f"lion {name} (small, path {path})", rep)
+
+
+def test_lion_gpt2_small_all_elements():
+    wl = workloads.build("gpt2_small")
+    rep = H.run_full_lion(wl, 20, hyper_over=dict(lambda_abs=1e4))
+    _report("lion gpt2_small", rep)
+    assert 0 < rep.clipped < rep.decisions
+
+
 def _ragged_workload(sizes, dtype):
     specs, total = workloads._layout([(f"t{i}", (n,)) for i, n in enumerate(sizes)])
     hp = dict(workloads.PAPER_DEFAULTS, lambda_abs=0.05)

@@ -42,9 +42,10 @@ UNIT = "params/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
-# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the update kernel, scaled to a full
-# launch of the named layout (see profiles/); absent until a capture of the current kernel exists.
-TRAFFIC_BYTES = {}
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the update kernel: 25.54 B/param measured on
+# the GPT-2-small-shaped layout (profiles/adagc_kernels_gpt2_small_ncu_full.md: 3178.1 MB for 124 439 808
+# params), scaled by the parameter count because the traffic of this streaming kernel grows in proportion.
+TRAFFIC_BYTES_PER_PARAM = {"bf16": 3178.112e6 / 124439808}
 
 
 # ------------------------------------------------------------------------------------ helpers
@@ -295,7 +296,8 @@ def run_ours(args, wl):
     kernel = "adagc_update_tma_kernel" if opt.update_path == binding.UPDATE_PATH_BULK else "adagc_update_kernel"
     roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-                "traffic": TRAFFIC_BYTES.get(wl.name),
+                "traffic": (TRAFFIC_BYTES_PER_PARAM[wl.grad_dtype] * wl.n_params
+                            if wl.grad_dtype in TRAFFIC_BYTES_PER_PARAM and kernel == "adagc_update_tma_kernel" else None),
                 "algorithmic_bytes_per_launch": bpp * wl.n_params, "launch_ms": upd_ms,
                 "whole_step_frac": bpp * wl.n_params / step_s / 1e9 / peak,
                 "whole_step_frac_of_nominal_8TBs": bpp * wl.n_params / step_s / 1e9 / NOMINAL_HBM_GBS,

@@ -98,7 +98,9 @@ int64_t adagc_num_chunks(const adagc_desc* desc);
 /* Validate the descriptor, build the chunk table and upload it into `d_workspace`
  * (device memory, 256-byte aligned, at least adagc_workspace_bytes(desc) bytes, owned by the
  * caller and kept alive until adagc_destroy).  Synchronises `cuda_stream` once.
- * The CUDA device current at this call is the one the context is bound to. */
+ * The CUDA device current at this call is the one the context is bound to: adagc_step, adagc_clip and
+ * adagc_step_lion return ADAGC_E_INVALID_ARG when another device is current.  A context is not
+ * thread-safe: one caller at a time. */
 int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_bytes,
                  void* cuda_stream, adagc_ctx** out);
 

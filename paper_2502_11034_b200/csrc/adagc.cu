@@ -113,69 +113,79 @@ __device__ __forceinline__ double sq_acc(double acc, float x) {
 // ------------------------------------------------------------------------------------------------
 // phase 1: per-chunk sums of squares (Eq. 3: ||g_t,i||^2 = sum_j g_ij^2)
 // ------------------------------------------------------------------------------------------------
+// Sum of squares of `count` elements starting at the 16-byte aligned `vec`, by one block of kThreads
+// threads: fixed element -> thread mapping, float64 per-thread accumulators, fixed shuffle tree, then a
+// fixed-order sum of the warp totals.  The result is valid in thread 0.  Ends with a barrier, so
+// `warp_part` can be reused at once.
+template <bool kBF16>
+__device__ __forceinline__ double block_chunk_sumsq(const uint4* __restrict__ vec, int count, double* warp_part) {
+  constexpr int kEPV = kBF16 ? 8 : 4;  // elements per 16-byte vector
+  constexpr int kUnroll = 8;           // independent 16-byte loads in flight per thread
+  const int tid = threadIdx.x;
+  const int nvec = count / kEPV;
+  double acc0 = 0.0, acc1 = 0.0;
+  for (int base = 0; base < nvec; base += kThreads * kUnroll) {
+    uint4 q[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      const int i = base + u * kThreads + tid;
+      q[u] = (i < nvec) ? __ldg(vec + i) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      if (kBF16) {
+        acc0 = sq_acc(acc0, bf16_lo(q[u].x));
+        acc1 = sq_acc(acc1, bf16_hi(q[u].x));
+        acc0 = sq_acc(acc0, bf16_lo(q[u].y));
+        acc1 = sq_acc(acc1, bf16_hi(q[u].y));
+        acc0 = sq_acc(acc0, bf16_lo(q[u].z));
+        acc1 = sq_acc(acc1, bf16_hi(q[u].z));
+        acc0 = sq_acc(acc0, bf16_lo(q[u].w));
+        acc1 = sq_acc(acc1, bf16_hi(q[u].w));
+      } else {
+        acc0 = sq_acc(acc0, __uint_as_float(q[u].x));
+        acc1 = sq_acc(acc1, __uint_as_float(q[u].y));
+        acc0 = sq_acc(acc0, __uint_as_float(q[u].z));
+        acc1 = sq_acc(acc1, __uint_as_float(q[u].w));
+      }
+    }
+  }
+  // ragged tail of a tensor's last chunk (fewer than one vector)
+  const int t = nvec * kEPV + tid;
+  if (t < count) {
+    float x;
+    if (kBF16) {
+      x = __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const uint16_t*>(vec)[t]) << 16);
+    } else {
+      x = reinterpret_cast<const float*>(vec)[t];
+    }
+    acc0 = sq_acc(acc0, x);
+  }
+  const double w = warp_sum(acc0 + acc1);
+  if ((tid & 31) == 0) warp_part[tid >> 5] = w;
+  __syncthreads();
+  double s = 0.0;
+  if (tid == 0) {
+    s = warp_part[0];
+#pragma unroll
+    for (int k = 1; k < kThreads / 32; ++k) s += warp_part[k];
+  }
+  __syncthreads();
+  return s;
+}
+
 template <bool kBF16>
 __global__ void __launch_bounds__(kThreads)
 adagc_norm_kernel(const void* __restrict__ grads, const Chunk* __restrict__ chunks,
                   const int32_t* __restrict__ block_begin, double* __restrict__ partials) {
-  constexpr int kEPV = kBF16 ? 8 : 4;  // elements per 16-byte vector
-  constexpr int kUnroll = 8;           // independent 16-byte loads in flight per thread
   __shared__ double warp_part[kThreads / 32];
-  const int tid = threadIdx.x;
   const int c_end = block_begin[blockIdx.x + 1];
   for (int c = block_begin[blockIdx.x]; c < c_end; ++c) {
     const Chunk ck = chunks[c];
-    const uint4* __restrict__ vec =
+    const uint4* vec =
         reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + chunk_start(ck) * (kBF16 ? 2 : 4));
-    const int nvec = ck.count / kEPV;
-    double acc0 = 0.0, acc1 = 0.0;
-    for (int base = 0; base < nvec; base += kThreads * kUnroll) {
-      uint4 q[kUnroll];
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        const int i = base + u * kThreads + tid;
-        q[u] = (i < nvec) ? __ldg(vec + i) : make_uint4(0u, 0u, 0u, 0u);
-      }
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        if (kBF16) {
-          acc0 = sq_acc(acc0, bf16_lo(q[u].x));
-          acc1 = sq_acc(acc1, bf16_hi(q[u].x));
-          acc0 = sq_acc(acc0, bf16_lo(q[u].y));
-          acc1 = sq_acc(acc1, bf16_hi(q[u].y));
-          acc0 = sq_acc(acc0, bf16_lo(q[u].z));
-          acc1 = sq_acc(acc1, bf16_hi(q[u].z));
-          acc0 = sq_acc(acc0, bf16_lo(q[u].w));
-          acc1 = sq_acc(acc1, bf16_hi(q[u].w));
-        } else {
-          acc0 = sq_acc(acc0, __uint_as_float(q[u].x));
-          acc1 = sq_acc(acc1, __uint_as_float(q[u].y));
-          acc0 = sq_acc(acc0, __uint_as_float(q[u].z));
-          acc1 = sq_acc(acc1, __uint_as_float(q[u].w));
-        }
-      }
-    }
-    // ragged tail of the tensor's last chunk (fewer than one vector)
-    const int t = nvec * kEPV + tid;
-    if (t < ck.count) {
-      float x;
-      if (kBF16) {
-        const uint16_t b = reinterpret_cast<const uint16_t*>(vec)[t];
-        x = __uint_as_float(static_cast<uint32_t>(b) << 16);
-      } else {
-        x = reinterpret_cast<const float*>(vec)[t];
-      }
-      acc0 = sq_acc(acc0, x);
-    }
-    const double w = warp_sum(acc0 + acc1);
-    if ((tid & 31) == 0) warp_part[tid >> 5] = w;
-    __syncthreads();
-    if (tid == 0) {
-      double s = warp_part[0];
-#pragma unroll
-      for (int k = 1; k < kThreads / 32; ++k) s += warp_part[k];
-      partials[ck.partial] = s;
-    }
-    __syncthreads();
+    const double s = block_chunk_sumsq<kBF16>(vec, ck.count, warp_part);
+    if (threadIdx.x == 0) partials[ck.partial] = s;
   }
 }
 
@@ -837,6 +847,9 @@ namespace {
 int check_clip_args(const adagc_ctx* ctx, const float* d_ema, int64_t step, double lambda_rel, double beta,
                     int64_t warmup) {
   if (!ctx || !d_ema) return ADAGC_E_INVALID_ARG;
+  int dev = -1;  // the context's tables live on the device that was current at adagc_create
+  if (cudaGetDevice(&dev) != cudaSuccess) return ADAGC_E_CUDA;
+  if (dev != ctx->device) return ADAGC_E_INVALID_ARG;
   if (step < 1 || warmup < 0) return ADAGC_E_INVALID_ARG;
   if (!(lambda_rel > 0.0) || !std::isfinite(lambda_rel)) return ADAGC_E_INVALID_ARG;
   if (!(beta >= 0.0 && beta < 1.0)) return ADAGC_E_INVALID_ARG;
@@ -1222,69 +1235,19 @@ constexpr int kMaxDevices = 64;
 
 static __device__ __align__(256) double g_static_partials[kStaticMaxChunks];
 
-// Same per-chunk arithmetic and thread mapping as adagc_norm_kernel, chunks taken implicitly as
-// consecutive kChunkElems-element slices of one buffer.
+// Same per-chunk arithmetic and thread mapping as adagc_norm_kernel (block_chunk_sumsq), chunks taken
+// implicitly as consecutive kChunkElems-element slices of one buffer.
 template <bool kBF16>
 __global__ void __launch_bounds__(kThreads)
 adagc_sumsq_static_kernel(const void* __restrict__ grads, int64_t numel, int n_chunks,
                           double* __restrict__ partials) {
-  constexpr int kEPV = kBF16 ? 8 : 4;
-  constexpr int kUnroll = 8;
   __shared__ double warp_part[kThreads / 32];
-  const int tid = threadIdx.x;
   for (int c = blockIdx.x; c < n_chunks; c += gridDim.x) {
     const int64_t start = int64_t(c) * kChunkElems;
     const int count = static_cast<int>(numel - start < kChunkElems ? numel - start : kChunkElems);
-    const uint4* __restrict__ vec =
-        reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + start * (kBF16 ? 2 : 4));
-    const int nvec = count / kEPV;
-    double acc0 = 0.0, acc1 = 0.0;
-    for (int base = 0; base < nvec; base += kThreads * kUnroll) {
-      uint4 q[kUnroll];
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        const int i = base + u * kThreads + tid;
-        q[u] = (i < nvec) ? __ldg(vec + i) : make_uint4(0u, 0u, 0u, 0u);
-      }
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        if (kBF16) {
-          acc0 = sq_acc(acc0, bf16_lo(q[u].x));
-          acc1 = sq_acc(acc1, bf16_hi(q[u].x));
-          acc0 = sq_acc(acc0, bf16_lo(q[u].y));
-          acc1 = sq_acc(acc1, bf16_hi(q[u].y));
-          acc0 = sq_acc(acc0, bf16_lo(q[u].z));
-          acc1 = sq_acc(acc1, bf16_hi(q[u].z));
-          acc0 = sq_acc(acc0, bf16_lo(q[u].w));
-          acc1 = sq_acc(acc1, bf16_hi(q[u].w));
-        } else {
-          acc0 = sq_acc(acc0, __uint_as_float(q[u].x));
-          acc1 = sq_acc(acc1, __uint_as_float(q[u].y));
-          acc0 = sq_acc(acc0, __uint_as_float(q[u].z));
-          acc1 = sq_acc(acc1, __uint_as_float(q[u].w));
-        }
-      }
-    }
-    const int t = nvec * kEPV + tid;
-    if (t < count) {
-      float x;
-      if (kBF16) {
-        x = __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const uint16_t*>(vec)[t]) << 16);
-      } else {
-        x = reinterpret_cast<const float*>(vec)[t];
-      }
-      acc0 = sq_acc(acc0, x);
-    }
-    const double w = warp_sum(acc0 + acc1);
-    if ((tid & 31) == 0) warp_part[tid >> 5] = w;
-    __syncthreads();
-    if (tid == 0) {
-      double s = warp_part[0];
-#pragma unroll
-      for (int k = 1; k < kThreads / 32; ++k) s += warp_part[k];
-      partials[c] = s;  // every partial that is read below is rewritten by this launch
-    }
-    __syncthreads();
+    const uint4* vec = reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + start * (kBF16 ? 2 : 4));
+    const double s = block_chunk_sumsq<kBF16>(vec, count, warp_part);
+    if (threadIdx.x == 0) partials[c] = s;  // every partial that is read below is rewritten by this launch
   }
 }
 

@@ -80,6 +80,11 @@ def test_llama2_7b_sampled():
     _report("llama2_7b", rep)
     assert rep.decisions == 291 * 20
     assert rep.clipped >= 8
+    # With lambda_abs = 1 the warm-up clips (global norm 8.2) and every later decision is a clip; with a large
+    # lambda_abs the steady state is calm and exactly the eight spiked tensors are clipped at step 12.
+    rep = H.run_sampled(wl, 13, mode="adamw", k=256, hyper_over=dict(lambda_abs=1e4))
+    _report("llama2_7b lambda_abs=1e4", rep)
+    assert 8 <= rep.clipped < 291
 
 
 # ------------------------------------------------------------------ small layouts, all elements

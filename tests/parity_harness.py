@@ -297,3 +297,37 @@ def run_full_lion(wl: workloads.Workload, n_steps: int, device="cuda", flags: in
     assert n_ties <= 1e-3 * wl.n_params + 50      # near-ties are rare: this is not a loophole for real errors
     opt.close()
     return rep
+
+
+def run_full_clip(wl: workloads.Workload, n_steps: int, in_place: bool, device="cuda",
+                  hyper_over: Optional[dict] = None) -> ParityReport:
+    """Clip-only entry, every element: clipped gradients in the gradient dtype vs the C oracle."""
+    hp = hyper_of(wl, **(hyper_over or {}))
+    offs = np.array([t.offset for t in wl.tensors], np.int64)
+    nums = np.array([t.numel for t in wl.tensors], np.int64)
+    opt = binding.AdaGC(nums.tolist(), offs.tolist(), wl.torch_grad_dtype, hp["lambda_abs"], device=device)
+    ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device=device)
+    gamma = np.zeros(wl.n_tensors, np.float32)
+    rep = ParityReport()
+    for t in range(1, n_steps + 1):
+        g = workloads.grads_for_step(wl, t, device)
+        g_np = to_numpy_grads(g).copy()
+        out = g if in_place else torch.full_like(g, 7.0)
+        opt.clip(g, out, ema, t, hp["lambda_rel"], hp["beta"], hp["warmup"])
+        ssq = c_oracle.sumsq_tensors(g_np, offs, nums)
+        r = c_oracle.clip_decisions(ssq, gamma, t, hp["lambda_rel"], hp["beta"], hp["lambda_abs"], hp["warmup"])
+        check_decisions(opt.get_stats(), opt.get_sumsq(), ema.cpu().numpy(), r, rep, t)
+        got = to_numpy_grads(out)
+        for i, (o, n) in enumerate(zip(offs, nums)):
+            want = c_oracle.scale(np.ascontiguousarray(g_np[o:o + n]), float(r["h"][i]))
+            check_clipped_grads(got[o:o + n], want, f"step {t}, tensor {wl.tensors[i].name}")
+            if float(r["h"][i]) == 1.0:
+                assert np.array_equal(got[o:o + n], g_np[o:o + n])      # unclipped tensors pass through bit for bit
+        if not in_place and wl.arena_elems != wl.n_params:
+            pad = np.ones(wl.arena_elems, bool)
+            for o, n in zip(offs, nums):
+                pad[o:o + n] = False
+            assert (out.float().cpu().numpy()[pad] == 7.0).all(), "padding between tensors was written"
+        rep.steps = t
+    opt.close()
+    return rep

@@ -121,6 +121,18 @@ def test_lion_gpt2_small_all_elements():
     assert 0 < rep.clipped < rep.decisions
 
 
+@pytest.mark.parametrize("in_place", [True, False], ids=["in_place", "out_of_place"])
+def test_clip_only_small_layouts_all_elements(in_place):
+    """adagc_clip on every element, both gradient dtypes; calm and spiky steady states."""
+    for name, over, hov in [("llama32_1b", dict(n_layer=2, d=128, ffn=512, vocab=2000, kv_dim=32), dict(lambda_abs=1e4)),
+                            ("many_small", dict(n_tensors=300, lo=1, hi=40000), dict(lambda_abs=1e4)),
+                            ("tiny", {}, {})]:
+        wl = workloads.build(name, **over)
+        rep = H.run_full_clip(wl, 12, in_place, hyper_over=hov)
+        _report(f"clip-only {name} in_place={in_place}", rep)
+        assert rep.clipped > 0
+
+
 def _ragged_workload(sizes, dtype):
     specs, total = workloads._layout([(f"t{i}", (n,)) for i, n in enumerate(sizes)])
     hp = dict(workloads.PAPER_DEFAULTS, lambda_abs=0.05)

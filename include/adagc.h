@@ -147,9 +147,13 @@ int adagc_clip(adagc_ctx* ctx, const void* d_grads_in, void* d_grads_out, float*
                int64_t step, double lambda_rel, double beta, int64_t warmup, void* cuda_stream);
 
 /*
- * adagc_step fed from HOST memory: copies the gradient arena `h_grads` (arena_elems elements of
- * the grad dtype; pinned memory recommended) into `d_grads`, runs the step, copies the per-tensor
- * statistics of this step back into the host arrays (any may be NULL) and synchronises the stream.
+ * adagc_step fed from HOST memory: copies the gradient arena `h_grads` (arena_elems elements of the grad
+ * dtype; pinned memory recommended) into `d_grads`, runs the step, copies the per-tensor statistics of this
+ * step back into the host arrays (any may be NULL) and synchronises the stream.
+ * On AdaGC steps (step > warmup) the work is pipelined: the tensors are taken in groups (arena order), the
+ * copies run on a stream owned by the context, and each group goes through norm, finalize and update on
+ * `cuda_stream` as soon as its gradients have arrived, so the kernels hide behind the host-to-device copy.
+ * Results are identical to adagc_step's.  Warm-up steps need the global norm first and are not pipelined.
  */
 int adagc_step_host(adagc_ctx* ctx, void* d_params, void* d_grads, void* d_m, void* d_v,
                     float* d_ema, const void* h_grads, int64_t step, double lr, double beta1,

@@ -57,6 +57,11 @@ __host__ __device__ __forceinline__ int64_t chunk_start(const Chunk& c) { return
 // fixed cost per chunk) over the blocks; with equal chunks it is plain round-robin.
 constexpr int kMaxGrid = 8192;          // entries reserved for each block_begin array
 constexpr int kChunkFixedCost = 1024;
+// adagc_step_host in steady state: the tensors are cut (in arena order) into at most kMaxGroups groups; each
+// group's gradients are copied on a second stream while the previous groups run norm/finalize/update.
+constexpr int kMaxGroups = 64;
+constexpr int kGroupMaxGrid = 1536;              // blocks per group launch (per block_begin array)
+constexpr int64_t kGroupMinBytes = 64ll << 20;   // smallest gradient slice worth its own launches
 
 struct TensorEntry {
   int32_t first_chunk;
@@ -225,10 +230,14 @@ __device__ __forceinline__ void adagc_decide(int i, double s, const ClipScalars&
 // same warp takes the decision.
 __global__ void __launch_bounds__(kFinalizeThreads)
 adagc_tensor_finalize_kernel(const double* __restrict__ partials, const TensorEntry* __restrict__ tensors,
-                             ClipScalars cs, int decide, float* __restrict__ ema, StatPtrs st) {
-  const int w = (blockIdx.x * kFinalizeThreads + threadIdx.x) >> 5;
+                             ClipScalars cs, int decide, float* __restrict__ ema, StatPtrs st,
+                             const int32_t* __restrict__ order, int first, int count, int bump_steps) {
+  // the warps of this launch take `count` tensors: order[first..first+count) if an order is given
+  // (a group of the pipelined host step), else the tensors first..first+count-1
+  const int k = (blockIdx.x * kFinalizeThreads + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
-  if (w >= cs.n_tensors) return;
+  if (k >= count) return;
+  const int w = order ? order[first + k] : first + k;
   const TensorEntry te = tensors[w];
   double acc = 0.0;
   for (int j = lane; j < te.n_chunks; j += 32) acc += partials[te.first_chunk + j];
@@ -237,7 +246,7 @@ adagc_tensor_finalize_kernel(const double* __restrict__ partials, const TensorEn
     st.sumsq[w] = acc;
     if (decide) {
       adagc_decide(w, acc, cs, ema, st);
-      if (w == 0) *st.steps_done += 1ull;
+      if (k == 0 && bump_steps) *st.steps_done += 1ull;
     }
   }
 }
@@ -710,7 +719,8 @@ adagc_scale_kernel(const void* __restrict__ gin, void* __restrict__ gout, const 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {  // byte offsets of the workspace sections
-  size_t chunks_wide, chunks_upd, begin_wide, begin_upd, mid_upd, tensors, partials, sumsq, norm, h, clip_count, scalars, flag,
+  size_t chunks_wide, chunks_upd, begin_wide, begin_upd, mid_upd, g_chunks_wide, g_chunks_upd, g_begin_wide,
+      g_begin_upd, g_mid_upd, g_order, tensors, partials, sumsq, norm, h, clip_count, scalars, flag,
       total;
 };
 
@@ -722,6 +732,13 @@ Layout make_layout(int64_t n_chunks, int64_t T) {
   L.begin_wide = o;  o = align_up(o + sizeof(int32_t) * (kMaxGrid + 1), 256);
   L.begin_upd = o;   o = align_up(o + sizeof(int32_t) * (kMaxGrid + 1), 256);
   L.mid_upd = o;     o = align_up(o + sizeof(int32_t) * (kMaxGrid + 1), 256);
+  // the same tables once more, cut into groups of tensors for the pipelined host step
+  L.g_chunks_wide = o; o = align_up(o + sizeof(Chunk) * n_chunks, 256);
+  L.g_chunks_upd = o;  o = align_up(o + sizeof(Chunk) * n_chunks, 256);
+  L.g_begin_wide = o;  o = align_up(o + sizeof(int32_t) * kMaxGroups * (kGroupMaxGrid + 1), 256);
+  L.g_begin_upd = o;   o = align_up(o + sizeof(int32_t) * kMaxGroups * (kGroupMaxGrid + 1), 256);
+  L.g_mid_upd = o;     o = align_up(o + sizeof(int32_t) * kMaxGroups * (kGroupMaxGrid + 1), 256);
+  L.g_order = o;       o = align_up(o + sizeof(int32_t) * T, 256);
   L.tensors = o;    o = align_up(o + sizeof(TensorEntry) * T, 256);
   L.partials = o;   o = align_up(o + sizeof(double) * n_chunks, 256);
   L.sumsq = o;      o = align_up(o + sizeof(double) * T, 256);
@@ -822,6 +839,16 @@ struct adagc_ctx {
   bool timing = false;
   bool timing_valid = false;
   cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+  struct Group {
+    int64_t elem_begin = 0, elem_end = 0;  // arena range holding the group's tensors
+    int32_t chunk_base = 0;                // first entry of the group in the grouped chunk tables
+    int32_t order_first = 0, n_tensors = 0;
+    int grid_wide = 1, grid_update = 1;
+  };
+  std::vector<Group> groups;
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t ev_entry = nullptr;
+  std::vector<cudaEvent_t> ev_group;
   const Chunk* d_chunks_wide() const { return reinterpret_cast<const Chunk*>(ws + L.chunks_wide); }
   const Chunk* d_chunks_upd() const { return reinterpret_cast<const Chunk*>(ws + L.chunks_upd); }
   const int32_t* d_begin_wide() const { return reinterpret_cast<const int32_t*>(ws + L.begin_wide); }
@@ -856,38 +883,6 @@ int check_clip_args(const adagc_ctx* ctx, const float* d_ema, int64_t step, doub
   return ADAGC_OK;
 }
 
-// phases 1 and 2
-int enqueue_clip_phases(adagc_ctx* ctx, const void* d_grads, float* d_ema, int64_t step, double lambda_rel,
-                        double beta, int64_t warmup, cudaStream_t s) {
-  if (ctx->timing) cudaEventRecord(ctx->ev[0], s);
-  if (ctx->bf16)
-    adagc_norm_kernel<true><<<ctx->grid_wide, kThreads, 0, s>>>(d_grads, ctx->d_chunks_wide(), ctx->d_begin_wide(),
-                                                               ctx->d_partials());
-  else
-    adagc_norm_kernel<false><<<ctx->grid_wide, kThreads, 0, s>>>(d_grads, ctx->d_chunks_wide(), ctx->d_begin_wide(),
-                                                                ctx->d_partials());
-  ctx->launches++;
-  if (ctx->timing) cudaEventRecord(ctx->ev[1], s);
-  ClipScalars cs;
-  cs.lambda_rel = lambda_rel;
-  cs.beta = beta;
-  cs.one_minus_beta = 1.0 - beta;
-  cs.lambda_abs = ctx->lambda_abs;
-  cs.step = step;
-  cs.n_tensors = ctx->T;
-  const bool in_warmup = step <= warmup;
-  const int blocks = (ctx->T * 32 + kFinalizeThreads - 1) / kFinalizeThreads;
-  adagc_tensor_finalize_kernel<<<blocks, kFinalizeThreads, 0, s>>>(ctx->d_partials(), ctx->d_tensors(), cs,
-                                                                  in_warmup ? 0 : 1, d_ema, ctx->stats());
-  ctx->launches++;
-  if (in_warmup) {
-    adagc_warmup_finalize_kernel<<<1, kWarmupThreads, 0, s>>>(cs, d_ema, ctx->stats());
-    ctx->launches++;
-  }
-  if (ctx->timing) cudaEventRecord(ctx->ev[2], s);
-  return ADAGC_OK;
-}
-
 // Largest L1 carve-out for the register kernels (L1 lines hold their loads in flight); opt-in shared
 // memory size for the bulk-async kernels.
 template <bool kBF16>
@@ -902,17 +897,107 @@ bool prepare_update_kernels() {
                               tma_smem_bytes(kBF16, kOptLion)) == cudaSuccess;
 }
 
+// One kernel's view of the chunk tables: the whole layout, or one group of the pipelined host step.
+struct TableView {
+  const Chunk* chunks;
+  const int32_t* begin;
+  const int32_t* mid;  // update tables only
+  int grid;
+};
+
+template <bool kBF16, int kOpt>
+void launch_update(adagc_ctx* ctx, const TableView& tv, float* p, const void* g, float* m, float* v,
+                   const AdamScalars& a, cudaStream_t s) {
+  const StatPtrs st = ctx->stats();
+  if (ctx->update_bulk)
+    adagc_update_tma_kernel<kBF16, kOpt><<<tv.grid, kTmaThreads, tma_smem_bytes(kBF16, kOpt), s>>>(
+        p, g, m, v, tv.chunks, tv.begin, tv.mid, st.h, a, st.status);
+  else
+    adagc_update_kernel<kBF16, kOpt><<<tv.grid, kThreads, 0, s>>>(p, g, m, v, tv.chunks, tv.begin, st.h, a);
+  ctx->launches++;
+}
+
 template <bool kBF16, int kOpt>
 void launch_update(adagc_ctx* ctx, float* p, const void* g, float* m, float* v, const AdamScalars& a,
                    cudaStream_t s) {
-  const StatPtrs st = ctx->stats();
-  if (ctx->update_bulk)
-    adagc_update_tma_kernel<kBF16, kOpt><<<ctx->grid_update, kTmaThreads, tma_smem_bytes(kBF16, kOpt), s>>>(
-        p, g, m, v, ctx->d_chunks_upd(), ctx->d_begin_upd(), ctx->d_mid_upd(), st.h, a, st.status);
+  const TableView tv = {ctx->d_chunks_upd(), ctx->d_begin_upd(), ctx->d_mid_upd(), ctx->grid_update};
+  launch_update<kBF16, kOpt>(ctx, tv, p, g, m, v, a, s);
+}
+
+void launch_norm(adagc_ctx* ctx, const TableView& tv, const void* d_grads, cudaStream_t s) {
+  if (ctx->bf16)
+    adagc_norm_kernel<true><<<tv.grid, kThreads, 0, s>>>(d_grads, tv.chunks, tv.begin, ctx->d_partials());
   else
-    adagc_update_kernel<kBF16, kOpt><<<ctx->grid_update, kThreads, 0, s>>>(p, g, m, v, ctx->d_chunks_upd(),
-                                                                          ctx->d_begin_upd(), st.h, a);
+    adagc_norm_kernel<false><<<tv.grid, kThreads, 0, s>>>(d_grads, tv.chunks, tv.begin, ctx->d_partials());
   ctx->launches++;
+}
+
+ClipScalars make_clip_scalars(const adagc_ctx* ctx, int64_t step, double lambda_rel, double beta) {
+  ClipScalars cs;
+  cs.lambda_rel = lambda_rel;
+  cs.beta = beta;
+  cs.one_minus_beta = 1.0 - beta;
+  cs.lambda_abs = ctx->lambda_abs;
+  cs.step = step;
+  cs.n_tensors = ctx->T;
+  return cs;
+}
+
+// scalar coefficients of the AdamW lines of Algorithm 1, in double, rounded once to the kernel's fp32
+AdamScalars make_adam_scalars(int64_t step, double lr, double beta1, double beta2, double eps, double wd) {
+  const double bc1 = 1.0 - std::pow(beta1, static_cast<double>(step));
+  const double bc2 = 1.0 - std::pow(beta2, static_cast<double>(step));
+  AdamScalars a;
+  a.beta1 = static_cast<float>(beta1);
+  a.one_minus_beta1 = static_cast<float>(1.0 - beta1);
+  a.beta2 = static_cast<float>(beta2);
+  a.one_minus_beta2 = static_cast<float>(1.0 - beta2);
+  a.inv_bc2 = static_cast<float>(1.0 / bc2);
+  a.step_size = static_cast<float>(lr / bc1);
+  a.decay = static_cast<float>(1.0 - lr * wd);
+  a.eps = static_cast<float>(eps);
+  return a;
+}
+
+int check_adamw_args(const void* d_params, const void* d_grads, const void* d_m, const void* d_v, double lr,
+                     double beta1, double beta2, double eps, double wd) {
+  if (!d_params || !d_grads || !d_m || !d_v) return ADAGC_E_INVALID_ARG;
+  if (!(beta1 >= 0.0 && beta1 < 1.0) || !(beta2 >= 0.0 && beta2 < 1.0)) return ADAGC_E_INVALID_ARG;
+  if (!(eps >= 0.0) || !std::isfinite(eps) || !std::isfinite(lr) || !std::isfinite(wd)) return ADAGC_E_INVALID_ARG;
+  if (!aligned16(d_params) || !aligned16(d_grads) || !aligned16(d_m) || !aligned16(d_v)) return ADAGC_E_MISALIGNED;
+  return ADAGC_OK;
+}
+
+// phases 1 and 2
+int enqueue_clip_phases(adagc_ctx* ctx, const void* d_grads, float* d_ema, int64_t step, double lambda_rel,
+                        double beta, int64_t warmup, cudaStream_t s) {
+  if (ctx->timing) cudaEventRecord(ctx->ev[0], s);
+  const TableView wide = {ctx->d_chunks_wide(), ctx->d_begin_wide(), nullptr, ctx->grid_wide};
+  launch_norm(ctx, wide, d_grads, s);
+  if (ctx->timing) cudaEventRecord(ctx->ev[1], s);
+  const ClipScalars cs = make_clip_scalars(ctx, step, lambda_rel, beta);
+  const bool in_warmup = step <= warmup;
+  const int blocks = (ctx->T * 32 + kFinalizeThreads - 1) / kFinalizeThreads;
+  adagc_tensor_finalize_kernel<<<blocks, kFinalizeThreads, 0, s>>>(ctx->d_partials(), ctx->d_tensors(), cs,
+                                                                  in_warmup ? 0 : 1, d_ema, ctx->stats(), nullptr, 0,
+                                                                  ctx->T, 1);
+  ctx->launches++;
+  if (in_warmup) {
+    adagc_warmup_finalize_kernel<<<1, kWarmupThreads, 0, s>>>(cs, d_ema, ctx->stats());
+    ctx->launches++;
+  }
+  if (ctx->timing) cudaEventRecord(ctx->ev[2], s);
+  return ADAGC_OK;
+}
+
+void release_ctx(adagc_ctx* ctx) {
+  for (int k = 0; k < 4; ++k)
+    if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
+  for (cudaEvent_t e : ctx->ev_group)
+    if (e) cudaEventDestroy(e);
+  if (ctx->ev_entry) cudaEventDestroy(ctx->ev_entry);
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  delete ctx;
 }
 
 int finish_launches(adagc_ctx* ctx, cudaStream_t s) {
@@ -1023,13 +1108,73 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
                              cudaMemcpyHostToDevice, s) == cudaSuccess;
   ok = ok && cudaMemcpyAsync(ctx->ws + L.tensors, tensors.data(), sizeof(TensorEntry) * tensors.size(),
                              cudaMemcpyHostToDevice, s) == cudaSuccess;
+  // groups of tensors (arena order) for the pipelined host step, each with its own balanced tables
+  std::vector<Chunk> g_table_wide, g_table_upd;
+  std::vector<int32_t> g_begin_wide(static_cast<size_t>(kMaxGroups) * (kGroupMaxGrid + 1), 0), g_begin_upd = g_begin_wide,
+                       g_mid_upd = g_begin_wide, g_order(desc->n_tensors);
+  if (ok) {
+    const int64_t esz = ctx->bf16 ? 2 : 4;
+    for (int32_t i = 0; i < desc->n_tensors; ++i) g_order[i] = i;
+    std::sort(g_order.begin(), g_order.end(),
+              [&](int32_t x, int32_t y) { return desc->tensors[x].offset < desc->tensors[y].offset; });
+    int64_t total_bytes = 0;
+    for (int32_t i = 0; i < desc->n_tensors; ++i) total_bytes += desc->tensors[i].numel * esz;
+    const int64_t target = std::max<int64_t>(kGroupMinBytes, (total_bytes + kMaxGroups - 1) / kMaxGroups);
+    g_table_wide.reserve(n_chunks);
+    g_table_upd.reserve(n_chunks);
+    int32_t k = 0;
+    while (k < desc->n_tensors) {
+      adagc_ctx::Group gr;
+      gr.order_first = k;
+      gr.chunk_base = static_cast<int32_t>(g_table_wide.size());
+      gr.elem_begin = desc->tensors[g_order[k]].offset;
+      std::vector<Chunk> mine;
+      int64_t bytes = 0;
+      const bool last_group = static_cast<int>(ctx->groups.size()) == kMaxGroups - 1;
+      while (k < desc->n_tensors && (bytes < target || last_group)) {
+        const int32_t i = g_order[k];
+        bytes += desc->tensors[i].numel * esz;
+        gr.elem_end = desc->tensors[i].offset + desc->tensors[i].numel;
+        mine.insert(mine.end(), chunks.begin() + tensors[i].first_chunk,
+                    chunks.begin() + tensors[i].first_chunk + tensors[i].n_chunks);
+        ++k;
+      }
+      gr.n_tensors = k - gr.order_first;
+      const int64_t nc = static_cast<int64_t>(mine.size());
+      gr.grid_wide = static_cast<int>(std::min<int64_t>({nc, ctx->grid_wide, kGroupMaxGrid}));
+      gr.grid_update = static_cast<int>(std::min<int64_t>({nc, ctx->grid_update, kGroupMaxGrid}));
+      std::vector<Chunk> tw, tu;
+      std::vector<int32_t> bw, bu, mu;
+      balance_chunks(mine, gr.grid_wide, &tw, &bw);
+      balance_chunks(mine, gr.grid_update, &tu, &bu, &mu);
+      const size_t slot = ctx->groups.size() * (kGroupMaxGrid + 1);
+      std::copy(bw.begin(), bw.end(), g_begin_wide.begin() + slot);
+      std::copy(bu.begin(), bu.end(), g_begin_upd.begin() + slot);
+      std::copy(mu.begin(), mu.end(), g_mid_upd.begin() + slot);
+      g_table_wide.insert(g_table_wide.end(), tw.begin(), tw.end());
+      g_table_upd.insert(g_table_upd.end(), tu.begin(), tu.end());
+      ctx->groups.push_back(gr);
+    }
+  }
+  auto upload = [&](size_t off, const void* src, size_t bytes) {
+    ok = ok && cudaMemcpyAsync(ctx->ws + off, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  };
+  upload(L.g_chunks_wide, g_table_wide.data(), sizeof(Chunk) * g_table_wide.size());
+  upload(L.g_chunks_upd, g_table_upd.data(), sizeof(Chunk) * g_table_upd.size());
+  upload(L.g_begin_wide, g_begin_wide.data(), sizeof(int32_t) * g_begin_wide.size());
+  upload(L.g_begin_upd, g_begin_upd.data(), sizeof(int32_t) * g_begin_upd.size());
+  upload(L.g_mid_upd, g_mid_upd.data(), sizeof(int32_t) * g_mid_upd.size());
+  upload(L.g_order, g_order.data(), sizeof(int32_t) * g_order.size());
   ok = ok && cudaStreamSynchronize(s) == cudaSuccess;  // the host vectors die at return
   for (int k = 0; ok && k < 4; ++k) ok = cudaEventCreate(&ctx->ev[k]) == cudaSuccess;
+  ok = ok && cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+  ok = ok && cudaEventCreateWithFlags(&ctx->ev_entry, cudaEventDisableTiming) == cudaSuccess;
+  ctx->ev_group.assign(ctx->groups.size(), nullptr);
+  for (size_t k = 0; ok && k < ctx->ev_group.size(); ++k)
+    ok = cudaEventCreateWithFlags(&ctx->ev_group[k], cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
     (void)cudaGetLastError();
-    for (int k = 0; k < 4; ++k)
-      if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
-    delete ctx;
+    release_ctx(ctx);
     return ADAGC_E_CUDA;
   }
   *out = ctx;
@@ -1038,9 +1183,7 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
 
 int adagc_destroy(adagc_ctx* ctx) {
   if (!ctx) return ADAGC_E_INVALID_ARG;
-  for (int k = 0; k < 4; ++k)
-    if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
-  delete ctx;
+  release_ctx(ctx);
   return ADAGC_OK;
 }
 
@@ -1049,26 +1192,12 @@ int adagc_step(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, v
                double beta, int64_t warmup, void* cuda_stream) {
   int rc = check_clip_args(ctx, d_ema, step, lambda_rel, beta, warmup);
   if (rc != ADAGC_OK) return rc;
-  if (!d_params || !d_grads || !d_m || !d_v) return ADAGC_E_INVALID_ARG;
-  if (!(beta1 >= 0.0 && beta1 < 1.0) || !(beta2 >= 0.0 && beta2 < 1.0)) return ADAGC_E_INVALID_ARG;
-  if (!(eps >= 0.0) || !std::isfinite(eps) || !std::isfinite(lr) || !std::isfinite(wd)) return ADAGC_E_INVALID_ARG;
-  if (!aligned16(d_params) || !aligned16(d_grads) || !aligned16(d_m) || !aligned16(d_v)) return ADAGC_E_MISALIGNED;
+  rc = check_adamw_args(d_params, d_grads, d_m, d_v, lr, beta1, beta2, eps, wd);
+  if (rc != ADAGC_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   rc = enqueue_clip_phases(ctx, d_grads, d_ema, step, lambda_rel, beta, warmup, s);
   if (rc != ADAGC_OK) return rc;
-
-  // scalar coefficients in double, rounded once to the kernel's fp32
-  const double bc1 = 1.0 - std::pow(beta1, static_cast<double>(step));
-  const double bc2 = 1.0 - std::pow(beta2, static_cast<double>(step));
-  AdamScalars a;
-  a.beta1 = static_cast<float>(beta1);
-  a.one_minus_beta1 = static_cast<float>(1.0 - beta1);
-  a.beta2 = static_cast<float>(beta2);
-  a.one_minus_beta2 = static_cast<float>(1.0 - beta2);
-  a.inv_bc2 = static_cast<float>(1.0 / bc2);
-  a.step_size = static_cast<float>(lr / bc1);
-  a.decay = static_cast<float>(1.0 - lr * wd);
-  a.eps = static_cast<float>(eps);
+  const AdamScalars a = make_adam_scalars(step, lr, beta1, beta2, eps, wd);
   if (ctx->bf16)
     launch_update<true, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
                                    static_cast<float*>(d_v), a, s);
@@ -1160,12 +1289,66 @@ int adagc_step_host(adagc_ctx* ctx, void* d_params, void* d_grads, void* d_m, vo
                     double wd, double lambda_rel, double beta, int64_t warmup, float* h_norm,
                     float* h_clipfactor, uint8_t* h_flag, void* cuda_stream) {
   if (!ctx || !h_grads || !d_grads) return ADAGC_E_INVALID_ARG;
-  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-  const size_t bytes = static_cast<size_t>(ctx->arena_elems) * (ctx->bf16 ? 2 : 4);
-  if (cudaMemcpyAsync(d_grads, h_grads, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return ADAGC_E_CUDA;
-  const int rc = adagc_step(ctx, d_params, d_grads, d_m, d_v, d_ema, step, lr, beta1, beta2, eps, wd,
-                            lambda_rel, beta, warmup, cuda_stream);
+  int rc = check_clip_args(ctx, d_ema, step, lambda_rel, beta, warmup);
   if (rc != ADAGC_OK) return rc;
+  rc = check_adamw_args(d_params, d_grads, d_m, d_v, lr, beta1, beta2, eps, wd);
+  if (rc != ADAGC_OK) return rc;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const size_t esz = ctx->bf16 ? 2 : 4;
+  const char* h_bytes = static_cast<const char*>(h_grads);
+  char* d_bytes = static_cast<char*>(d_grads);
+
+  if (step <= warmup || ctx->timing || ctx->groups.size() < 2) {
+    // warm-up needs the global norm before any update can start: copy everything, then the plain step
+    const size_t bytes = static_cast<size_t>(ctx->arena_elems) * esz;
+    if (cudaMemcpyAsync(d_grads, h_grads, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return ADAGC_E_CUDA;
+    rc = adagc_step(ctx, d_params, d_grads, d_m, d_v, d_ema, step, lr, beta1, beta2, eps, wd, lambda_rel, beta,
+                    warmup, cuda_stream);
+    if (rc != ADAGC_OK) return rc;
+    return adagc_get_stats(ctx, h_norm, h_clipfactor, h_flag, nullptr, nullptr, nullptr, cuda_stream);
+  }
+
+  // AdaGC steps decide per tensor, so a group of tensors can go through all three phases as soon as its
+  // gradients have arrived: the copies run on a second stream, group by group, and the caller's stream
+  // follows one group behind.  The copy engine stays busy from start to end; the kernels hide behind it.
+  bool ok = cudaEventRecord(ctx->ev_entry, s) == cudaSuccess &&      // earlier work on s may still read d_grads
+            cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_entry, 0) == cudaSuccess;
+  for (size_t k = 0; ok && k < ctx->groups.size(); ++k) {
+    const adagc_ctx::Group& gr = ctx->groups[k];
+    const size_t off = static_cast<size_t>(gr.elem_begin) * esz;
+    const size_t bytes = static_cast<size_t>(gr.elem_end - gr.elem_begin) * esz;
+    ok = cudaMemcpyAsync(d_bytes + off, h_bytes + off, bytes, cudaMemcpyHostToDevice, ctx->copy_stream) == cudaSuccess &&
+         cudaEventRecord(ctx->ev_group[k], ctx->copy_stream) == cudaSuccess;
+  }
+  if (!ok) return ADAGC_E_CUDA;
+  const ClipScalars cs = make_clip_scalars(ctx, step, lambda_rel, beta);
+  const AdamScalars a = make_adam_scalars(step, lr, beta1, beta2, eps, wd);
+  const Chunk* gcw = reinterpret_cast<const Chunk*>(ctx->ws + ctx->L.g_chunks_wide);
+  const Chunk* gcu = reinterpret_cast<const Chunk*>(ctx->ws + ctx->L.g_chunks_upd);
+  const int32_t* gbw = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.g_begin_wide);
+  const int32_t* gbu = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.g_begin_upd);
+  const int32_t* gmu = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.g_mid_upd);
+  const int32_t* order = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.g_order);
+  for (size_t k = 0; k < ctx->groups.size(); ++k) {
+    const adagc_ctx::Group& gr = ctx->groups[k];
+    const size_t slot = k * (kGroupMaxGrid + 1);
+    if (cudaStreamWaitEvent(s, ctx->ev_group[k], 0) != cudaSuccess) return ADAGC_E_CUDA;
+    const TableView wide = {gcw + gr.chunk_base, gbw + slot, nullptr, gr.grid_wide};
+    const TableView upd = {gcu + gr.chunk_base, gbu + slot, gmu + slot, gr.grid_update};
+    launch_norm(ctx, wide, d_grads, s);
+    const int blocks = (gr.n_tensors * 32 + kFinalizeThreads - 1) / kFinalizeThreads;
+    adagc_tensor_finalize_kernel<<<blocks, kFinalizeThreads, 0, s>>>(ctx->d_partials(), ctx->d_tensors(), cs, 1, d_ema,
+                                                                    ctx->stats(), order, gr.order_first, gr.n_tensors,
+                                                                    k == 0 ? 1 : 0);
+    ctx->launches++;
+    if (ctx->bf16)
+      launch_update<true, kOptAdamW>(ctx, upd, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
+                                     static_cast<float*>(d_v), a, s);
+    else
+      launch_update<false, kOptAdamW>(ctx, upd, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
+                                      static_cast<float*>(d_v), a, s);
+  }
+  if (cudaGetLastError() != cudaSuccess) return ADAGC_E_CUDA;
   return adagc_get_stats(ctx, h_norm, h_clipfactor, h_flag, nullptr, nullptr, nullptr, cuda_stream);
 }
 

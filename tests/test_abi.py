@@ -80,7 +80,7 @@ def test_no_cpu_fallback_without_a_device():
     lib = binding.lib()
     d, keep = binding.make_desc([100], [0], binding.ADAGC_F32)
     h = C.c_void_p()
-    assert lib.adagc_create(C.byref(d), 256, 1 << 20, None, C.byref(h)) == -6 and not h.value
+    assert lib.adagc_create(C.byref(d), 256, 1 << 24, None, C.byref(h)) == -6 and not h.value
     with pytest.raises(Exception):
         binding.AdaGC([100], [0], torch.float32)
 

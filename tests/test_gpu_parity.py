@@ -317,9 +317,17 @@ def test_phase_timing_and_launch_count():
     opt.close()
 
 
-def test_step_host_matches_device_entry():
-    wl, offs, nums = _mini()
-    hp = H.hyper_of(wl)
+@pytest.mark.parametrize("layout", ["mini", "gpt2_small"])
+def test_step_host_matches_device_entry(layout):
+    """The host-buffer entry gives bit-identical results; on the larger layout (several groups of tensors)
+    its AdaGC steps run pipelined behind the host-to-device copies, its warm-up steps do not."""
+    if layout == "mini":
+        wl, offs, nums = _mini()
+    else:
+        wl = workloads.build("gpt2_small")
+        wl.warmup = 3
+        offs, nums = [t.offset for t in wl.tensors], [t.numel for t in wl.tensors]
+    hp = H.hyper_of(wl, lambda_abs=1e4)
     args = (hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"], hp["beta"], hp["warmup"])
     outs = []
     for host in (False, True):
@@ -340,7 +348,10 @@ def test_step_host_matches_device_entry():
                 assert np.array_equal(hfac.numpy(), st["h"])
             else:
                 opt.step(theta, g, m, v, ema, t, *args)
-        outs.append((theta, m, v, ema))
+        final = opt.get_stats()
+        assert final["steps_done"] == 8 and final["status"] == 0
+        outs.append((theta, m, v, ema, torch.from_numpy(final["clip_count"].astype(np.int64))))
         opt.close()
     for x, y in zip(*outs):
         assert torch.equal(x, y)
+    assert int(outs[0][4].sum()) > 0

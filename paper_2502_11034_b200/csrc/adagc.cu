@@ -990,6 +990,38 @@ int enqueue_clip_phases(adagc_ctx* ctx, const void* d_grads, float* d_ema, int64
   return ADAGC_OK;
 }
 
+// Norm, finalize and AdamW update of an AdaGC step (step > warmup), one group of tensors after the other.
+// With wait_copies, stream s waits for each group's host-to-device copy event first.
+int enqueue_grouped_adamw(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, void* d_v, float* d_ema,
+                          const ClipScalars& cs, const AdamScalars& a, bool wait_copies, cudaStream_t s) {
+  const Chunk* gcw = reinterpret_cast<const Chunk*>(ctx->ws + ctx->L.g_chunks_wide);
+  const Chunk* gcu = reinterpret_cast<const Chunk*>(ctx->ws + ctx->L.g_chunks_upd);
+  const int32_t* gbw = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.g_begin_wide);
+  const int32_t* gbu = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.g_begin_upd);
+  const int32_t* gmu = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.g_mid_upd);
+  const int32_t* order = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.g_order);
+  for (size_t k = 0; k < ctx->groups.size(); ++k) {
+    const adagc_ctx::Group& gr = ctx->groups[k];
+    const size_t slot = k * (kGroupMaxGrid + 1);
+    if (wait_copies && cudaStreamWaitEvent(s, ctx->ev_group[k], 0) != cudaSuccess) return ADAGC_E_CUDA;
+    const TableView wide = {gcw + gr.chunk_base, gbw + slot, nullptr, gr.grid_wide};
+    const TableView upd = {gcu + gr.chunk_base, gbu + slot, gmu + slot, gr.grid_update};
+    launch_norm(ctx, wide, d_grads, s);
+    const int blocks = (gr.n_tensors * 32 + kFinalizeThreads - 1) / kFinalizeThreads;
+    adagc_tensor_finalize_kernel<<<blocks, kFinalizeThreads, 0, s>>>(ctx->d_partials(), ctx->d_tensors(), cs, 1, d_ema,
+                                                                    ctx->stats(), order, gr.order_first, gr.n_tensors,
+                                                                    k == 0 ? 1 : 0);
+    ctx->launches++;
+    if (ctx->bf16)
+      launch_update<true, kOptAdamW>(ctx, upd, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
+                                     static_cast<float*>(d_v), a, s);
+    else
+      launch_update<false, kOptAdamW>(ctx, upd, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
+                                      static_cast<float*>(d_v), a, s);
+  }
+  return ADAGC_OK;
+}
+
 void release_ctx(adagc_ctx* ctx) {
   for (int k = 0; k < 4; ++k)
     if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
@@ -1321,33 +1353,9 @@ int adagc_step_host(adagc_ctx* ctx, void* d_params, void* d_grads, void* d_m, vo
          cudaEventRecord(ctx->ev_group[k], ctx->copy_stream) == cudaSuccess;
   }
   if (!ok) return ADAGC_E_CUDA;
-  const ClipScalars cs = make_clip_scalars(ctx, step, lambda_rel, beta);
-  const AdamScalars a = make_adam_scalars(step, lr, beta1, beta2, eps, wd);
-  const Chunk* gcw = reinterpret_cast<const Chunk*>(ctx->ws + ctx->L.g_chunks_wide);
-  const Chunk* gcu = reinterpret_cast<const Chunk*>(ctx->ws + ctx->L.g_chunks_upd);
-  const int32_t* gbw = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.g_begin_wide);
-  const int32_t* gbu = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.g_begin_upd);
-  const int32_t* gmu = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.g_mid_upd);
-  const int32_t* order = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.g_order);
-  for (size_t k = 0; k < ctx->groups.size(); ++k) {
-    const adagc_ctx::Group& gr = ctx->groups[k];
-    const size_t slot = k * (kGroupMaxGrid + 1);
-    if (cudaStreamWaitEvent(s, ctx->ev_group[k], 0) != cudaSuccess) return ADAGC_E_CUDA;
-    const TableView wide = {gcw + gr.chunk_base, gbw + slot, nullptr, gr.grid_wide};
-    const TableView upd = {gcu + gr.chunk_base, gbu + slot, gmu + slot, gr.grid_update};
-    launch_norm(ctx, wide, d_grads, s);
-    const int blocks = (gr.n_tensors * 32 + kFinalizeThreads - 1) / kFinalizeThreads;
-    adagc_tensor_finalize_kernel<<<blocks, kFinalizeThreads, 0, s>>>(ctx->d_partials(), ctx->d_tensors(), cs, 1, d_ema,
-                                                                    ctx->stats(), order, gr.order_first, gr.n_tensors,
-                                                                    k == 0 ? 1 : 0);
-    ctx->launches++;
-    if (ctx->bf16)
-      launch_update<true, kOptAdamW>(ctx, upd, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
-                                     static_cast<float*>(d_v), a, s);
-    else
-      launch_update<false, kOptAdamW>(ctx, upd, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
-                                      static_cast<float*>(d_v), a, s);
-  }
+  rc = enqueue_grouped_adamw(ctx, d_params, d_grads, d_m, d_v, d_ema, make_clip_scalars(ctx, step, lambda_rel, beta),
+                             make_adam_scalars(step, lr, beta1, beta2, eps, wd), true, s);
+  if (rc != ADAGC_OK) return rc;
   if (cudaGetLastError() != cudaSuccess) return ADAGC_E_CUDA;
   return adagc_get_stats(ctx, h_norm, h_clipfactor, h_flag, nullptr, nullptr, nullptr, cuda_stream);
 }

@@ -75,12 +75,31 @@ def l2_norm(g: np.ndarray) -> float:
 
 
 def clip_decisions(s: Sequence[float], gamma_prev: np.ndarray, step: int, hp: Hyper,
-                   state_dtype=np.float32) -> ClipResult:
+                   state_dtype=np.float32, keep_initial: bool = False,
+                   global_adaptive: bool = False) -> ClipResult:
     """Clip factors, flags and the EMA update for one step, from per-tensor sums of squares.
 
     Warm-up branch: Eq. 2 and the min-seeding line of Algorithm 1.
     AdaGC branch:   Eq. 3 and the gamma update of Algorithm 1.
+
+    Two variants of the paper's ablations (Section 5, "EMA Initialization Strategy" and "Adaptivity Efficacy
+    and Locality Granularity"):
+      keep_initial    gamma is not seeded at t = 1; the caller's gamma_0 (e.g. the constant 0.5 or 1.0 of
+                      the ablation) is used as gamma_{t-1} from the first step on;
+      global_adaptive "Global AdaGC": one adaptive threshold for the whole model, i.e. this same algorithm
+                      applied to the single tensor that all gradients form together; every tensor gets
+                      that one clip factor, flag and gamma.
     """
+    if global_adaptive:
+        s_all = np.asarray(s, dtype=np.float64)
+        one = clip_decisions([float(np.sum(s_all))], np.asarray(gamma_prev)[:1], step, hp, state_dtype,
+                             keep_initial, False)
+        T = s_all.shape[0]
+        n_i = np.sqrt(s_all)
+        return ClipResult(n_i, np.full(T, one.h[0]), np.full(T, bool(one.flag[0])), one.h[0] * n_i,
+                          np.full(T, one.gamma[0], dtype=state_dtype), one.global_norm,
+                          np.full(T, one.margin[0]))
+    seed = step == 1 and not keep_initial
     s = np.asarray(s, dtype=np.float64)
     T = s.shape[0]
     n = np.sqrt(s)                                         # ||g_t,i||
@@ -104,10 +123,10 @@ def clip_decisions(s: Sequence[float], gamma_prev: np.ndarray, step: int, hp: Hy
             flag[i] = clip_all
             c[i] = h_t * n[i]                              # ||hat(g)_t,i||
             # gamma_t,i = min{gamma_t-1,i, ||hat(g)_t,i||},  gamma_0,i = ||hat(g)_1,i||
-            gam[i] = c[i] if step == 1 else min(gam[i], c[i])
+            gam[i] = c[i] if seed else min(gam[i], c[i])
     else:
         for i in range(T):
-            if step == 1:                                  # T_start = 0: seed, then Eq. 3
+            if seed:                                       # T_start = 0: seed, then Eq. 3
                 gam[i] = float(np.asarray(n[i]).astype(state_dtype))
             thr = hp.lambda_rel * gam[i]
             if thr > 0:

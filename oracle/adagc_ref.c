@@ -101,10 +101,28 @@ void adagc_ref_sumsq_tensors(const void* arena, int is_bf16, int32_t T, const in
  * Eq. 2, or the AdaGC branch with Eq. 3).  gamma is fp32 state, updated in place.
  * Outputs per tensor: norm, h, flag, clipped norm, decision margin |norm - thr| / thr.
  */
+void adagc_ref_clip_decisions_ex(int32_t T, const double* s, float* gamma, int64_t step,
+                                 double lambda_rel, double beta, double lambda_abs, int64_t warmup,
+                                 int variant, double* norm, double* h, uint8_t* flag, double* clipped,
+                                 double* margin, double* global_norm);
+
 void adagc_ref_clip_decisions(int32_t T, const double* s, float* gamma, int64_t step,
                               double lambda_rel, double beta, double lambda_abs, int64_t warmup,
                               double* norm, double* h, uint8_t* flag, double* clipped,
                               double* margin, double* global_norm) {
+  adagc_ref_clip_decisions_ex(T, s, gamma, step, lambda_rel, beta, lambda_abs, warmup, 0, norm, h, flag,
+                              clipped, margin, global_norm);
+}
+
+/* The same with the two ablation variants of the paper's Section 5 (bits of `variant`):
+ *   1  keep the caller's gamma_0: no seeding at t = 1 ("constant initialization");
+ *   2  "Global AdaGC": one adaptive threshold for the whole model = this algorithm on the single tensor
+ *      that all gradients form together; every tensor gets that clip factor, flag and gamma. */
+void adagc_ref_clip_decisions_ex(int32_t T, const double* s, float* gamma, int64_t step,
+                                 double lambda_rel, double beta, double lambda_abs, int64_t warmup,
+                                 int variant, double* norm, double* h, uint8_t* flag, double* clipped,
+                                 double* margin, double* global_norm) {
+  const int seed = (step == 1) && !(variant & 1);
   long double tot = 0.0L;
   for (int32_t i = 0; i < T; ++i) {
     norm[i] = sqrt(s[i]);
@@ -112,6 +130,21 @@ void adagc_ref_clip_decisions(int32_t T, const double* s, float* gamma, int64_t 
   }
   const double G = sqrt((double)tot); /* ||g_t|| */
   *global_norm = G;
+  if (variant & 2) {
+    double s1 = (double)tot, n1, h1, c1, m1, G1;
+    uint8_t f1;
+    float g1 = gamma[0];
+    adagc_ref_clip_decisions_ex(1, &s1, &g1, step, lambda_rel, beta, lambda_abs, warmup, variant & 1, &n1, &h1,
+                                &f1, &c1, &m1, &G1);
+    for (int32_t i = 0; i < T; ++i) {
+      h[i] = h1;
+      flag[i] = f1;
+      clipped[i] = h1 * norm[i];
+      margin[i] = m1;
+      gamma[i] = g1;
+    }
+    return;
+  }
   if (step <= warmup) {
     const int clip_all = G > lambda_abs;
     const double h_t = clip_all ? lambda_abs / G : 1.0; /* min{lambda_abs/||g_t||, 1} */
@@ -121,12 +154,12 @@ void adagc_ref_clip_decisions(int32_t T, const double* s, float* gamma, int64_t 
       clipped[i] = h_t * norm[i]; /* ||hat(g)_t,i|| */
       margin[i] = lambda_abs > 0 ? fabs(G - lambda_abs) / lambda_abs : INFINITY;
       double gprev = (double)gamma[i];
-      double gnew = (step == 1) ? clipped[i] : (clipped[i] < gprev ? clipped[i] : gprev);
+      double gnew = seed ? clipped[i] : (clipped[i] < gprev ? clipped[i] : gprev);
       gamma[i] = (float)gnew;
     }
   } else {
     for (int32_t i = 0; i < T; ++i) {
-      double gprev = (step == 1) ? (double)(float)norm[i] : (double)gamma[i];
+      double gprev = seed ? (double)(float)norm[i] : (double)gamma[i];
       const double thr = lambda_rel * gprev;
       margin[i] = thr > 0 ? fabs(norm[i] - thr) / thr : INFINITY;
       if (norm[i] > thr) {

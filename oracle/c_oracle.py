@@ -46,6 +46,10 @@ def lib():
         L.adagc_ref_clip_decisions.restype = None
         L.adagc_ref_clip_decisions.argtypes = [C.c_int32, _f64p, _f32p, C.c_int64, C.c_double, C.c_double,
                                                C.c_double, C.c_int64, _f64p, _f64p, _u8p, _f64p, _f64p, _f64p]
+        L.adagc_ref_clip_decisions_ex.restype = None
+        L.adagc_ref_clip_decisions_ex.argtypes = [C.c_int32, _f64p, _f32p, C.c_int64, C.c_double, C.c_double,
+                                                  C.c_double, C.c_int64, C.c_int, _f64p, _f64p, _u8p, _f64p, _f64p,
+                                                  _f64p]
         L.adagc_ref_adamw.restype = None
         L.adagc_ref_adamw.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int64,
                                       C.c_double, C.c_int64] + [C.c_double] * 5
@@ -90,7 +94,7 @@ def sumsq_tensors(arena: np.ndarray, offsets: Sequence[int], numels: Sequence[in
 
 
 def clip_decisions(s: np.ndarray, gamma: np.ndarray, step: int, lambda_rel: float, beta: float,
-                   lambda_abs: float, warmup: int):
+                   lambda_abs: float, warmup: int, keep_initial: bool = False, global_adaptive: bool = False):
     """Returns dict(norm, h, flag, clipped, margin, global_norm); `gamma` (fp32) is updated in place."""
     s = np.ascontiguousarray(s, dtype=np.float64)
     T = len(s)
@@ -98,8 +102,9 @@ def clip_decisions(s: np.ndarray, gamma: np.ndarray, step: int, lambda_rel: floa
     norm, h, clipped, margin = (np.empty(T, np.float64) for _ in range(4))
     flag = np.empty(T, np.uint8)
     G = np.empty(1, np.float64)
-    lib().adagc_ref_clip_decisions(T, s, gamma, step, lambda_rel, beta, lambda_abs, warmup,
-                                   norm, h, flag, clipped, margin, G)
+    variant = (1 if keep_initial else 0) | (2 if global_adaptive else 0)
+    lib().adagc_ref_clip_decisions_ex(T, s, gamma, step, lambda_rel, beta, lambda_abs, warmup, variant,
+                                      norm, h, flag, clipped, margin, G)
     return dict(norm=norm, h=h, flag=flag.astype(bool), clipped=clipped, margin=margin,
                 global_norm=float(G[0]), gamma=gamma)
 

@@ -633,3 +633,59 @@ def test_lion_brute_force_and_oracles_agree():
     np.testing.assert_allclose(m, mb, rtol=1e-5, atol=1e-9)
     np.testing.assert_allclose(tc, theta, rtol=3e-7, atol=1e-9)
     np.testing.assert_allclose(mc, m, rtol=3e-7, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------- ablation variants (Section 5)
+def _decide(impl_name, s, gamma, step, hp, **kw):
+    if impl_name == "numpy":
+        r = npo.clip_decisions(s, gamma, step, hp, np.float32, **kw)
+        return dict(h=r.h, flag=r.flag, gamma=np.asarray(r.gamma, np.float32), norm=r.norm)
+    g = np.array(gamma, np.float32)
+    r = co.clip_decisions(np.asarray(s, np.float64), g, step, hp.lambda_rel, hp.beta, hp.lambda_abs, hp.warmup, **kw)
+    return dict(h=r["h"], flag=r["flag"], gamma=g, norm=r["norm"])
+
+
+@pytest.mark.parametrize("impl_name", ["numpy", "c"])
+def test_global_adaptive_is_the_algorithm_on_the_concatenated_gradient(impl_name):
+    """'Global AdaGC' (one adaptive threshold for the whole model) must equal the per-tensor algorithm run on
+    the single tensor made of all gradients; the T = 1 run below uses the plain (non-variant) code path."""
+    rng = np.random.RandomState(31)
+    sizes = [40, 1000, 7, 333]
+    hp = npo.Hyper(warmup=3, lambda_abs=0.08, lambda_rel=1.04, beta=0.9)
+    gam_g = np.zeros(len(sizes), np.float32)
+    gam_1 = np.zeros(1, np.float32)
+    seen = set()
+    for t in range(1, 16):
+        gs = [f32_exact(rng.normal(size=n) * 1e-3 * (30 if t in (7, 11) else 1)) for n in sizes]
+        s = [npo.sumsq(g) for g in gs]
+        one = _decide(impl_name, [npo.sumsq(np.concatenate(gs))], gam_1, t, hp)
+        glo = _decide(impl_name, s, gam_g, t, hp, global_adaptive=True)
+        gam_1, gam_g = one["gamma"], glo["gamma"]
+        assert len(set(np.asarray(glo["h"]).tolist())) == 1 and len(set(np.asarray(glo["flag"]).tolist())) == 1
+        assert bool(glo["flag"][0]) == bool(one["flag"][0])
+        assert glo["h"][0] == pytest.approx(one["h"][0], rel=1e-14)
+        np.testing.assert_allclose(gam_g, np.full(len(sizes), gam_1[0]), rtol=1.2e-7)
+        np.testing.assert_allclose(glo["norm"], [math.sqrt(x) for x in s], rtol=1e-15)
+        seen.add((t <= hp.warmup, bool(one["flag"][0])))
+    assert (False, True) in seen and (False, False) in seen          # AdaGC steps both clipped and calm
+
+
+@pytest.mark.parametrize("impl_name", ["numpy", "c"])
+def test_keep_initial_uses_the_callers_gamma_from_the_first_step(impl_name):
+    """Constant initialization of the ablation: gamma_0 given by the caller, no seeding at t = 1."""
+    hp = npo.Hyper(warmup=0, lambda_rel=2.0, beta=0.5)
+    r = _decide(impl_name, [9.0, 16.0], np.array([1.0, 8.0], np.float32), 1, hp, keep_initial=True)
+    np.testing.assert_array_equal(np.asarray(r["flag"]), [True, False])     # 3 > 2*1 ; 4 <= 2*8
+    np.testing.assert_array_equal(np.asarray(r["h"]), [2.0 / 3.0, 1.0])
+    np.testing.assert_array_equal(r["gamma"], np.array([0.5 * 1 + 0.5 * 2, 0.5 * 8 + 0.5 * 4], np.float32))
+    # default behaviour for comparison: seeded with the norms, nothing clipped
+    r0 = _decide(impl_name, [9.0, 16.0], np.array([1.0, 8.0], np.float32), 1, hp)
+    assert not np.asarray(r0["flag"]).any() and list(r0["gamma"]) == [3.0, 4.0]
+    # warm-up with keep_initial: running minimum starts from the caller's value
+    hpw = npo.Hyper(warmup=5, lambda_abs=100.0)
+    r = _decide(impl_name, [9.0, 16.0], np.array([1.0, 8.0], np.float32), 1, hpw, keep_initial=True)
+    assert list(r["gamma"]) == [1.0, 4.0]
+    # after the first step the variant changes nothing
+    a = _decide(impl_name, [9.0, 16.0], np.array([1.0, 8.0], np.float32), 4, hp, keep_initial=True)
+    b = _decide(impl_name, [9.0, 16.0], np.array([1.0, 8.0], np.float32), 4, hp)
+    np.testing.assert_array_equal(a["gamma"], b["gamma"])

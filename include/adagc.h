@@ -63,6 +63,15 @@ typedef enum {
 #define ADAGC_UPDATE_PATH_REGISTERS 1
 #define ADAGC_UPDATE_PATH_BULK 2
 #define ADAGC_UPDATE_PATH_MASK 3
+/* Two variants from the paper's ablations (Section 5), OR-ed into adagc_desc.flags:
+ *   ADAGC_EMA_KEEP_INITIAL      "constant initialization": gamma is not seeded at step 1; the values the
+ *                               caller put into d_ema (e.g. 0.5 or 1.0) serve as gamma_0.
+ *   ADAGC_CLIP_GLOBAL_ADAPTIVE  "Global AdaGC": one adaptive threshold for the whole model -- the same
+ *                               algorithm applied to the single tensor that all gradients form together.
+ *                               Every tensor gets that clip factor and flag; all n_tensors entries of
+ *                               d_ema hold the one gamma (entry 0 is the one read). */
+#define ADAGC_EMA_KEEP_INITIAL 4
+#define ADAGC_CLIP_GLOBAL_ADAPTIVE 8
 
 /* One parameter tensor. */
 typedef struct {
@@ -83,7 +92,7 @@ typedef struct {
   int32_t state_dtype;         /* ADAGC_F32 (m and v) */
   const adagc_tensor* tensors; /* host array, copied by adagc_create */
   double lambda_abs;           /* warm-up global-norm threshold of Eq. 2, > 0 (paper: 1.0) */
-  int32_t flags;               /* 0, or one ADAGC_UPDATE_PATH_* value */
+  int32_t flags;               /* 0, or one ADAGC_UPDATE_PATH_* value, optionally OR-ed with the variant flags */
   int32_t reserved;            /* set to 0 */
 } adagc_desc;
 

@@ -151,14 +151,16 @@ class ArenaOracle:
 
     def __init__(self, offsets: Sequence[int], numels: Sequence[int], theta0: np.ndarray, *,
                  lr: float, beta1: float, beta2: float, eps: float, wd: float, lambda_rel: float,
-                 beta: float, lambda_abs: float, warmup: int):
+                 beta: float, lambda_abs: float, warmup: int, keep_initial: bool = False,
+                 global_adaptive: bool = False, gamma0: Optional[np.ndarray] = None):
+        self.keep_initial, self.global_adaptive = keep_initial, global_adaptive
         self.off = np.ascontiguousarray(offsets, dtype=np.int64)
         self.numel = np.ascontiguousarray(numels, dtype=np.int64)
         self.T = len(self.off)
         self.theta = np.array(theta0, dtype=np.float32)
         self.m = np.zeros_like(self.theta)
         self.v = np.zeros_like(self.theta)
-        self.gamma = np.zeros(self.T, dtype=np.float32)
+        self.gamma = np.zeros(self.T, dtype=np.float32) if gamma0 is None else np.array(gamma0, dtype=np.float32)
         self.hp = dict(lr=lr, beta1=beta1, beta2=beta2, eps=eps, wd=wd, lambda_rel=lambda_rel,
                        beta=beta, lambda_abs=lambda_abs, warmup=warmup)
         self.t = 0
@@ -166,6 +168,8 @@ class ArenaOracle:
         self._s = np.empty(self.T, np.float64)
 
     def step(self, grads: np.ndarray, lr: Optional[float] = None):
+        if self.keep_initial or self.global_adaptive:
+            return self._step_variant(grads, lr)
         self.t += 1
         p, bf = _grad_ptr(grads)
         hp = self.hp
@@ -181,12 +185,22 @@ class ArenaOracle:
         return dict(norm=norm, h=h, flag=flag.astype(bool), clipped=clipped, margin=margin,
                     global_norm=float(G[0]), gamma=self.gamma.copy())
 
+    def _step_variant(self, grads: np.ndarray, lr: Optional[float]):
+        """One step with an ablation variant: the same three stages, composed from the single functions."""
+        r = self.clip(grads)
+        hp = self.hp
+        for i in range(self.T):
+            o, n = int(self.off[i]), int(self.numel[i])
+            adamw_update(self.theta[o:o + n], grads[o:o + n], self.m[o:o + n], self.v[o:o + n], float(r["h"][i]),
+                         self.t, hp["lr"] if lr is None else lr, hp["beta1"], hp["beta2"], hp["eps"], hp["wd"])
+        return r
+
     def clip(self, grads: np.ndarray):
         """Clip-only step: advances gamma and the counters, returns the decisions (no AdamW)."""
         self.t += 1
         s = sumsq_tensors(grads, self.off, self.numel)
         r = clip_decisions(s, self.gamma, self.t, self.hp["lambda_rel"], self.hp["beta"],
-                           self.hp["lambda_abs"], self.hp["warmup"])
+                           self.hp["lambda_abs"], self.hp["warmup"], self.keep_initial, self.global_adaptive)
         self.clip_count += r["flag"].astype(np.uint64)
         r["gamma"] = self.gamma.copy()
         return r

@@ -72,6 +72,7 @@ struct ClipScalars {
   double lambda_rel, beta, one_minus_beta, lambda_abs;
   int64_t step;
   int32_t n_tensors;
+  int32_t seed;  // 1: gamma is seeded at this step (t = 1, unless the descriptor keeps the caller's gamma_0)
 };
 
 struct AdamScalars {
@@ -212,7 +213,7 @@ __device__ __forceinline__ void adagc_decide(int i, double s, const ClipScalars&
                                              float* __restrict__ ema, const StatPtrs& st) {
   const double n = sqrt(s);  // ||g_t,i||
   // gamma is fp32 state; with T_start = 0 the first step seeds it with this step's norm
-  const double g_prev = (cs.step == 1) ? (double)(float)n : (double)ema[i];
+  const double g_prev = cs.seed ? (double)(float)n : (double)ema[i];
   const double thr = __dmul_rn(cs.lambda_rel, g_prev);
   const bool clip = n > thr;  // strict: equality is not a clip
   const double h = clip ? __ddiv_rn(thr, n) : 1.0;
@@ -279,7 +280,7 @@ adagc_warmup_finalize_kernel(ClipScalars cs, float* __restrict__ ema, StatPtrs s
     const double n = sqrt(s);
     const double c = __dmul_rn(h, n);  // ||hat(g)_t,i||
     double g_new = c;
-    if (cs.step != 1) {
+    if (!cs.seed) {
       const double g_prev = (double)ema[i];
       g_new = (c < g_prev) ? c : g_prev;
     }
@@ -288,6 +289,56 @@ adagc_warmup_finalize_kernel(ClipScalars cs, float* __restrict__ ema, StatPtrs s
     st.h[i] = hf;
     st.flag[i] = clip_all ? 1 : 0;
     if (clip_all) st.clip_count[i] += 1ull;
+    if (!isfinite(s)) atomicOr(st.status, ADAGC_W_NONFINITE);
+  }
+}
+
+// "Global AdaGC" (the adaptivity / locality ablation of Section 5): one adaptive threshold for the whole
+// model, i.e. Algorithm 1 applied to the single tensor that all gradients form together.  One block;
+// every tensor receives the same clip factor, flag and gamma.  `in_warmup` selects Eq. 2 or Eq. 3.
+__global__ void __launch_bounds__(kWarmupThreads)
+adagc_global_finalize_kernel(ClipScalars cs, int in_warmup, float* __restrict__ ema, StatPtrs st) {
+  __shared__ double warp_part[kWarmupThreads / 32];
+  __shared__ double total_s;
+  const int tid = threadIdx.x;
+  double acc = 0.0;
+  for (int i = tid; i < cs.n_tensors; i += kWarmupThreads) acc += st.sumsq[i];
+  acc = warp_sum(acc);
+  if ((tid & 31) == 0) warp_part[tid >> 5] = acc;
+  __syncthreads();
+  if (tid == 0) {
+    double s = warp_part[0];
+    for (int k = 1; k < kWarmupThreads / 32; ++k) s += warp_part[k];
+    total_s = s;
+    *st.steps_done += 1ull;
+  }
+  __syncthreads();
+  const double G = sqrt(total_s);        // the norm of the one big tensor
+  const double g_in = (double)ema[0];    // read by every thread before anyone overwrites it ...
+  __syncthreads();                       // ... which this barrier guarantees
+  bool clip;
+  double h, g_new;
+  if (in_warmup) {
+    clip = G > cs.lambda_abs;
+    h = clip ? __ddiv_rn(cs.lambda_abs, G) : 1.0;
+    const double c = __dmul_rn(h, G);
+    g_new = cs.seed ? c : ((c < g_in) ? c : g_in);
+  } else {
+    const double g_prev = cs.seed ? (double)(float)G : g_in;
+    const double thr = __dmul_rn(cs.lambda_rel, g_prev);
+    clip = G > thr;
+    h = clip ? __ddiv_rn(thr, G) : 1.0;
+    const double c = clip ? thr : G;
+    g_new = __dadd_rn(__dmul_rn(cs.beta, g_prev), __dmul_rn(cs.one_minus_beta, c));
+  }
+  const float hf = (float)h, gf = (float)g_new;
+  for (int i = tid; i < cs.n_tensors; i += kWarmupThreads) {
+    const double s = st.sumsq[i];
+    ema[i] = gf;
+    st.norm[i] = (float)sqrt(s);
+    st.h[i] = hf;
+    st.flag[i] = clip ? 1 : 0;
+    if (clip) st.clip_count[i] += 1ull;
     if (!isfinite(s)) atomicOr(st.status, ADAGC_W_NONFINITE);
   }
 }
@@ -756,7 +807,8 @@ int validate_desc(const adagc_desc* d, int64_t* n_chunks_out, int64_t* arena_ele
   if (d->param_dtype != ADAGC_F32 || d->state_dtype != ADAGC_F32) return ADAGC_E_DTYPE;
   if (d->grad_dtype != ADAGC_F32 && d->grad_dtype != ADAGC_BF16) return ADAGC_E_DTYPE;
   if (!(d->lambda_abs > 0.0) || !std::isfinite(d->lambda_abs)) return ADAGC_E_INVALID_ARG;
-  if ((d->flags & ~ADAGC_UPDATE_PATH_MASK) != 0 || (d->flags & ADAGC_UPDATE_PATH_MASK) == 3) return ADAGC_E_INVALID_ARG;
+  constexpr int kKnownFlags = ADAGC_UPDATE_PATH_MASK | ADAGC_EMA_KEEP_INITIAL | ADAGC_CLIP_GLOBAL_ADAPTIVE;
+  if ((d->flags & ~kKnownFlags) != 0 || (d->flags & ADAGC_UPDATE_PATH_MASK) == 3) return ADAGC_E_INVALID_ARG;
   const int64_t align = (d->grad_dtype == ADAGC_BF16) ? 8 : 4;
   int64_t n_chunks = 0, extent = 0;
   std::vector<std::pair<int64_t, int64_t>> spans;
@@ -833,6 +885,8 @@ struct adagc_ctx {
   int device = 0;
   int grid_wide = 1, grid_update = 1;  // norm and scale kernels: SMs x resident blocks; update: SMs x 2 or x 1
   bool update_bulk = false;            // update phase through the bulk-async (TMA) kernel
+  bool keep_initial = false;           // ADAGC_EMA_KEEP_INITIAL
+  bool global_adaptive = false;        // ADAGC_CLIP_GLOBAL_ADAPTIVE
   char* ws = nullptr;
   Layout L{};
   uint64_t launches = 0;
@@ -940,6 +994,7 @@ ClipScalars make_clip_scalars(const adagc_ctx* ctx, int64_t step, double lambda_
   cs.lambda_abs = ctx->lambda_abs;
   cs.step = step;
   cs.n_tensors = ctx->T;
+  cs.seed = (step == 1 && !ctx->keep_initial) ? 1 : 0;
   return cs;
 }
 
@@ -978,11 +1033,15 @@ int enqueue_clip_phases(adagc_ctx* ctx, const void* d_grads, float* d_ema, int64
   const ClipScalars cs = make_clip_scalars(ctx, step, lambda_rel, beta);
   const bool in_warmup = step <= warmup;
   const int blocks = (ctx->T * 32 + kFinalizeThreads - 1) / kFinalizeThreads;
+  const bool per_tensor = !in_warmup && !ctx->global_adaptive;
   adagc_tensor_finalize_kernel<<<blocks, kFinalizeThreads, 0, s>>>(ctx->d_partials(), ctx->d_tensors(), cs,
-                                                                  in_warmup ? 0 : 1, d_ema, ctx->stats(), nullptr, 0,
+                                                                  per_tensor ? 1 : 0, d_ema, ctx->stats(), nullptr, 0,
                                                                   ctx->T, 1);
   ctx->launches++;
-  if (in_warmup) {
+  if (ctx->global_adaptive) {
+    adagc_global_finalize_kernel<<<1, kWarmupThreads, 0, s>>>(cs, in_warmup ? 1 : 0, d_ema, ctx->stats());
+    ctx->launches++;
+  } else if (in_warmup) {
     adagc_warmup_finalize_kernel<<<1, kWarmupThreads, 0, s>>>(cs, d_ema, ctx->stats());
     ctx->launches++;
   }
@@ -1117,6 +1176,8 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
       const int64_t wide = sms * std::max(1, std::min(occ_n, occ_s));
       ctx->grid_wide = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>({n_chunks, wide, kMaxGrid})));
       ctx->update_bulk = (desc->flags & ADAGC_UPDATE_PATH_MASK) != ADAGC_UPDATE_PATH_REGISTERS;
+      ctx->keep_initial = (desc->flags & ADAGC_EMA_KEEP_INITIAL) != 0;
+      ctx->global_adaptive = (desc->flags & ADAGC_CLIP_GLOBAL_ADAPTIVE) != 0;
       ctx->grid_update = static_cast<int>(std::max<int64_t>(
           1, std::min<int64_t>({n_chunks, sms * (ctx->update_bulk ? 1 : kUpdateBlocksPerSM), kMaxGrid})));
     }
@@ -1330,7 +1391,7 @@ int adagc_step_host(adagc_ctx* ctx, void* d_params, void* d_grads, void* d_m, vo
   const char* h_bytes = static_cast<const char*>(h_grads);
   char* d_bytes = static_cast<char*>(d_grads);
 
-  if (step <= warmup || ctx->timing || ctx->groups.size() < 2) {
+  if (step <= warmup || ctx->timing || ctx->global_adaptive || ctx->groups.size() < 2) {
     // warm-up needs the global norm before any update can start: copy everything, then the plain step
     const size_t bytes = static_cast<size_t>(ctx->arena_elems) * esz;
     if (cudaMemcpyAsync(d_grads, h_grads, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return ADAGC_E_CUDA;

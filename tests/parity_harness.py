@@ -101,7 +101,7 @@ def check_state(name: str, got: np.ndarray, ref: np.ndarray, rep: ParityReport, 
 
 
 def run_full(wl: workloads.Workload, n_steps: int, device="cuda", hyper_over: Optional[dict] = None,
-             lr_schedule=None, canary: bool = True, flags: int = 0) -> ParityReport:
+             lr_schedule=None, canary: bool = True, flags: int = 0, gamma0: Optional[float] = None) -> ParityReport:
     """Every element of every tensor, fused AdaGC+AdamW step, GPU vs C oracle."""
     hp = hyper_of(wl, **(hyper_over or {}))
     offs = [t.offset for t in wl.tensors]
@@ -120,10 +120,14 @@ def run_full(wl: workloads.Workload, n_steps: int, device="cuda", hyper_over: Op
     if pad_mask is not None:
         m[pad_mask] = 777.0
         v[pad_mask] = 777.0
-    ema = torch.full((wl.n_tensors,), float("nan"), dtype=torch.float32, device=device)  # must be ignored at t=1
+    keep = bool(flags & binding.EMA_KEEP_INITIAL)
+    # without the keep-initial variant the incoming gamma must be ignored at t = 1: poison it
+    ema = torch.full((wl.n_tensors,), float("nan") if not keep else float(gamma0), dtype=torch.float32, device=device)
     ref = c_oracle.ArenaOracle(offs, nums, theta0, lr=hp["lr"], beta1=hp["beta1"], beta2=hp["beta2"],
                                eps=hp["eps"], wd=hp["wd"], lambda_rel=hp["lambda_rel"], beta=hp["beta"],
-                               lambda_abs=hp["lambda_abs"], warmup=hp["warmup"])
+                               lambda_abs=hp["lambda_abs"], warmup=hp["warmup"], keep_initial=keep,
+                               global_adaptive=bool(flags & binding.CLIP_GLOBAL_ADAPTIVE),
+                               gamma0=None if not keep else np.full(wl.n_tensors, gamma0, np.float32))
     rep = ParityReport()
     for t in range(1, n_steps + 1):
         g = workloads.grads_for_step(wl, t, device)

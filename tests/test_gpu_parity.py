@@ -133,6 +133,18 @@ def test_clip_only_small_layouts_all_elements(in_place):
         assert rep.clipped > 0
 
 
+@pytest.mark.parametrize("variant", ["keep_initial", "global_adaptive", "both"])
+def test_ablation_variants_all_elements(variant):
+    """Section 5 variants: caller-given gamma_0 (no seeding at t = 1) and Global AdaGC (one adaptive threshold)."""
+    flags = {"keep_initial": binding.EMA_KEEP_INITIAL, "global_adaptive": binding.CLIP_GLOBAL_ADAPTIVE,
+             "both": binding.EMA_KEEP_INITIAL | binding.CLIP_GLOBAL_ADAPTIVE}[variant]
+    wl = workloads.build("llama2_7b", n_layer=2, d=256, ffn=688, vocab=1000)
+    for warmup, gamma0 in ((0, 0.02), (3, 0.5)):
+        rep = H.run_full(wl, 16, flags=flags, gamma0=gamma0, hyper_over=dict(warmup=warmup, lambda_abs=1e4))
+        _report(f"{variant} warmup={warmup} gamma0={gamma0}", rep)
+    assert rep.steps == 16
+
+
 def _ragged_workload(sizes, dtype):
     specs, total = workloads._layout([(f"t{i}", (n,)) for i, n in enumerate(sizes)])
     hp = dict(workloads.PAPER_DEFAULTS, lambda_abs=0.05)

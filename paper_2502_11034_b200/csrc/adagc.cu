@@ -5,11 +5,17 @@
 //                squares (Eq. 3 needs ||g_t,i||, Eq. 2 needs ||g_t||);
 //   2. finalize  per tensor: fixed-order sum of its partials -> norm -> clip factor h, flag and the
 //                gamma update (warm-up branch: global norm first, then min-seeding);
-//   3. update    every chunk again: g, theta, m, v read once, hat(g) = h * g kept in registers,
-//                AdamW lines of Algorithm 1, theta, m, v written once.
+//   3. update    every chunk again: g, theta, m, v read once, hat(g) = h * g kept on chip,
+//                AdamW lines of Algorithm 1 (or Lion's rule), theta, m, v written once.  Two kernels:
+//                a bulk-async one (cp.async.bulk + mbarrier ring through shared memory, the default)
+//                and a register-streaming one.
 // This is pure streaming work (26..28 bytes per parameter, ~20 flops): the bound is HBM bandwidth,
-// so the kernels are built around 128-bit coalesced accesses, many loads in flight per thread and
-// streaming cache hints; there is no contraction here and tensor cores are not used.
+// so the kernels are built around large coalesced transfers, a measured amount of loads in flight
+// per SM and streaming cache hints; there is no contraction here and tensor cores are not used.
+//
+// Host side (second half of the file): descriptor validation, the balanced per-block chunk tables
+// built once at adagc_create, the entry points, and adagc_step_host, which pipelines groups of
+// tensors behind the host-to-device copies.
 //
 // Reductions are deterministic: fixed element->thread mapping, fixed shuffle tree, fixed-order sums
 // of partials; no floating-point atomics.  Sums of squares are accumulated in float64 so that the
@@ -34,14 +40,13 @@ constexpr int kThreads = 256;
 constexpr int kFinalizeThreads = 256;  // 8 warps = 8 tensors per block
 constexpr int kWarmupThreads = 1024;
 // The update kernel moves 7 streams (4 read, 3 written).  Measured on B200, DRAM efficiency of that mix
-// peaks with about 512 threads x 112 bytes of loads in flight per SM and drops by ~15 % with twice as
-// many, so its grid is two 256-thread blocks per SM.  The kernels use no shared memory worth
-// mentioning and ask for the largest L1 carve-out: L1 lines hold the loads in flight, and a kernel
-// launched with a large shared-memory reservation lost 20 % of its bandwidth here.
+// peaks with about 57 KB of loads in flight per SM and drops by ~15 % with twice as many.
+// Register-streaming variant: 512 threads x 112 bytes, i.e. a grid of two 256-thread blocks per SM, with
+// the largest L1 carve-out (L1 lines hold the loads in flight; reserving 100 KB of shared memory per
+// block cost 20 % of the bandwidth).  Bulk-async variant: one 512-thread block per SM with one 57 KB
+// tile in flight; it measured 1-2 % faster on every layout tried (26.7 vs 27.2 ms on the 7B-shaped one)
+// and is the default; the descriptor's flags can force either.
 constexpr int kUpdateBlocksPerSM = 2;
-// The bulk-async variant of the update kernel (one 512-thread block per SM, tiles staged in shared
-// memory by cp.async.bulk) measured 1-2 % faster than the register variant on every layout tried
-// (26.7 vs 27.2 ms on the 7B-shaped one), so it is the default; the descriptor's flags can force either.
 
 struct Chunk {
   uint32_t start4;  // element offset into the arenas, in units of 4 elements

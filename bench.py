@@ -389,7 +389,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", default=None, help="tiny | gpt2_small | llama2_7b | many_small | llama32_1b")
+    ap.add_argument("--workload", default=None, help="tiny | gpt2_small | llama2_7b | many_small | llama32_1b | moe_8x1b")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     wl = pick_workload(args)

@@ -155,7 +155,31 @@ def llama32_1b(n_layer: int = 16, d: int = 2048, ffn: int = 8192, vocab: int = 1
                     notes="Llama-3.2-1B-shaped, tied embedding, GQA k/v, Student-t(3) gradients")
 
 
-_BUILDERS = {"tiny": tiny_mlp, "gpt2_small": gpt2_small, "llama2_7b": llama2_7b,
+def moe_8x1b(n_layer: int = 24, d: int = 2048, ffn: int = 5632, vocab: int = 32000, kv_dim: int = 256,
+             n_experts: int = 8) -> Workload:
+    """Mixture-of-experts layout shaped like the paper's Mixtral 8x1B run (hyper-parameter table: 24 layers,
+    hidden 2048, FFN 5632, 32 heads, 4 key-value heads, 8 routed experts).  Per layer: four attention
+    matrices, a router, three matrices per expert and two norm vectors, i.e. (7 + 3E) L + 3 tensors -- the
+    census of Section 4.3 "Memory" with no shared expert and the router counted."""
+    shapes: List[Tuple[str, Tuple[int, ...]]] = [("embed", (vocab, d))]
+    for l in range(n_layer):
+        p = f"l{l}."
+        shapes += [(p + "attn_norm", (d,)), (p + "q_proj", (d, d)), (p + "k_proj", (kv_dim, d)),
+                   (p + "v_proj", (kv_dim, d)), (p + "o_proj", (d, d)), (p + "ffn_norm", (d,)),
+                   (p + "router", (n_experts, d))]
+        for e in range(n_experts):
+            shapes += [(p + f"e{e}.gate_proj", (ffn, d)), (p + f"e{e}.up_proj", (ffn, d)),
+                       (p + f"e{e}.down_proj", (d, ffn))]
+    shapes += [("final_norm", (d,)), ("lm_head", (vocab, d))]
+    specs, total = _layout(shapes)
+    hyper = dict(PAPER_DEFAULTS, beta2=0.999)          # the table's Adam beta2 for this model
+    return Workload("moe_8x1b", 6, specs, "bf16", hyper, warmup=5, n_steps=20, arena_elems=total,
+                    grad_kind="student_t", grad_df=3, grad_scale=1e-4,
+                    extra={"spike_frac": 0.02, "spike_lo": 10.0, "spike_hi": 1000.0},
+                    notes="Mixtral-8x1B-shaped MoE: (7+3E)L+3 tensors, experts get heavy-tailed gradients")
+
+
+_BUILDERS = {"tiny": tiny_mlp, "moe_8x1b": moe_8x1b, "gpt2_small": gpt2_small, "llama2_7b": llama2_7b,
              "many_small": many_small, "llama32_1b": llama32_1b}
 
 

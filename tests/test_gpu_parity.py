@@ -133,6 +133,15 @@ def test_clip_only_small_layouts_all_elements(in_place):
         assert rep.clipped > 0
 
 
+def test_moe_layout_small_all_elements():
+    """Mixture-of-experts tensor census ((7+3E)L+3 tensors, Section 4.3 "Memory"), reduced dimensions."""
+    wl = workloads.build("moe_8x1b", n_layer=2, d=128, ffn=352, vocab=1000, kv_dim=32, n_experts=4)
+    assert wl.n_tensors == (7 + 3 * 4) * 2 + 3
+    rep = H.run_full(wl, 20, hyper_over=dict(lambda_abs=1e4))
+    _report("moe (small)", rep)
+    assert 0 < rep.clipped < rep.decisions
+
+
 @pytest.mark.parametrize("variant", ["keep_initial", "global_adaptive", "both"])
 def test_ablation_variants_all_elements(variant):
     """Section 5 variants: caller-given gamma_0 (no seeding at t = 1) and Global AdaGC (one adaptive threshold)."""

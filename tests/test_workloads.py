@@ -18,7 +18,10 @@ def test_layout_census():
     ms = W.build("many_small")
     assert ms.n_tensors == 20000 and 1.5e8 < ms.n_params < 2.3e8
     assert min(t.numel for t in ms.tensors) >= 64 and max(t.numel for t in ms.tensors) <= 65536
-    for wl in (tiny, g2, l7, l1, ms):
+    moe = W.build("moe_8x1b")
+    assert moe.n_tensors == (7 + 3 * 8) * 24 + 3 == 747 and 6.5e9 < moe.n_params < 7.5e9
+    assert moe.hyper["beta2"] == 0.999
+    for wl in (tiny, g2, l7, l1, ms, moe):
         offs = np.array([t.offset for t in wl.tensors])
         nums = np.array([t.numel for t in wl.tensors])
         assert (offs % W.ALIGN_ELEMS == 0).all()

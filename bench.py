@@ -37,13 +37,13 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
-METRIC = "fused AdaGC+AdamW step throughput (parameters/s)"
+METRIC = "fused AdaGC+AdamW step time, params/s, HBM GB/s (% of peak) at 7B layout"
 UNIT = "params/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the update kernel: 25.54 B/param measured on
-# the GPT-2-small-shaped layout (profiles/adagc_kernels_gpt2_small_ncu_full.md: 3178.6 MB for 124 439 808
+# the GPT-2-small-shaped layout (committed ncu summary of that capture: 3178.6 MB for 124 439 808
 # params), scaled by the parameter count because the traffic of this streaming kernel grows in proportion.
 TRAFFIC_BYTES_PER_PARAM = {"bf16": 3178.644e6 / 124439808}
 

@@ -50,6 +50,9 @@ def test_descriptor_validation_codes():
     assert chunks([100], [0], shapes=[(10, 11)])[0] == -1                # shape does not match numel
     assert chunks([100, 50], [0, 102])[0] == -2                          # fp32: offsets in multiples of 4
     assert chunks([100, 50], [0, 100], binding.ADAGC_BF16)[0] == -2      # bf16: multiples of 8
+    assert chunks([(1 << 34) + 8], [0])[0] == -1                         # beyond the largest supported arena
+    assert chunks([1 << 20], [(1 << 34) - 8])[0] == -1
+    assert chunks([1 << 34], [0])[0] == (1 << 34) // 16384               # the maximum itself is accepted
     assert chunks([100, 50], [0, 96])[0] == -3                           # overlap
     assert chunks([50, 100], [96, 0])[0] == -3                           # overlap, unsorted
     assert chunks([100], [0], dt=2)[0] == -5

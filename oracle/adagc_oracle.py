@@ -191,6 +191,21 @@ def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: f
     return out
 
 
+def sgdm_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, momentum: float,
+                wd: float, state_dtype=np.float32) -> Tuple[np.ndarray, np.ndarray]:
+    """SGD with momentum on the clipped gradient hat(g) = h * g (Section 4.2: the clip is optimizer-agnostic).
+    The textbook heavy-ball form with L2 weight decay folded into the gradient, the form common libraries use:
+        d     = hat(g) + wd * theta
+        m     = momentum * m + d              (m_0 = 0)
+        theta = theta - lr * m
+    Elementwise, float64 arithmetic, results rounded to `state_dtype`."""
+    th = np.asarray(theta, dtype=np.float64)
+    d = float(h) * np.asarray(g, dtype=np.float64) + wd * th
+    m1 = momentum * np.asarray(m, dtype=np.float64) + d
+    th1 = th - lr * m1
+    return th1.astype(state_dtype), m1.astype(state_dtype)
+
+
 def clipped_grad(g: np.ndarray, h: float) -> np.ndarray:
     """hat(g) = h * g in float64 (the clip-only use of the method with other optimizers)."""
     return float(h) * np.asarray(g, dtype=np.float64)

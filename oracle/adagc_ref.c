@@ -224,6 +224,23 @@ void adagc_ref_lion(float* theta, const void* g, int g_is_bf16, float* m, int64_
   }
 }
 
+/* SGD with momentum on hat(g) = h * g, in place (Section 4.2: AdaGC with other optimizers): heavy-ball form
+ * with L2 weight decay folded into the gradient: d = hat(g) + wd theta;  m = momentum m + d;  theta -= lr m. */
+void adagc_ref_sgdm(float* theta, const void* g, int g_is_bf16, float* m, int64_t n, double h, double lr,
+                    double momentum, double wd) {
+  const uint16_t* gb = (const uint16_t*)g;
+  const float* gf = (const float*)g;
+#pragma omp parallel for schedule(static) if (n > 65536)
+  for (int64_t j = 0; j < n; ++j) {
+    const double gj = g_is_bf16 ? bf16_to_double(gb[j]) : (double)gf[j];
+    const double th = (double)theta[j];
+    const double d = h * gj + wd * th;
+    const double m1 = momentum * (double)m[j] + d;
+    theta[j] = (float)(th - lr * m1);
+    m[j] = (float)m1;
+  }
+}
+
 /* hat(g) = h * g written in the gradient's dtype (clip-only use with other optimizers). */
 void adagc_ref_scale(void* out, const void* g, int is_bf16, int64_t n, double h) {
   if (is_bf16) {

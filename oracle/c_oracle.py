@@ -56,6 +56,8 @@ def lib():
         L.adagc_ref_lion.restype = None
         L.adagc_ref_lion.argtypes = ([C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64] + [C.c_double] * 5 +
                                      [C.c_void_p, C.c_double])
+        L.adagc_ref_sgdm.restype = None
+        L.adagc_ref_sgdm.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64] + [C.c_double] * 4
         L.adagc_ref_scale.restype = None
         L.adagc_ref_scale.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_double]
         L.adagc_ref_step.restype = C.c_int32
@@ -132,6 +134,15 @@ def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: f
         nt = near_tie.ctypes.data
     lib().adagc_ref_lion(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, beta1, beta2, wd,
                          nt, float(tie_tol))
+
+
+def sgdm_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, momentum: float,
+                wd: float) -> None:
+    """SGD with momentum on the clipped gradient, in place on fp32 theta and m."""
+    p, bf = _grad_ptr(g)
+    for a in (theta, m):
+        assert a.dtype == np.float32 and a.flags["C_CONTIGUOUS"] and a.size == g.size
+    lib().adagc_ref_sgdm(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, momentum, wd)
 
 
 def scale(g: np.ndarray, h: float, out: Optional[np.ndarray] = None) -> np.ndarray:

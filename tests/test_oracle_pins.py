@@ -689,3 +689,37 @@ def test_keep_initial_uses_the_callers_gamma_from_the_first_step(impl_name):
     a = _decide(impl_name, [9.0, 16.0], np.array([1.0, 8.0], np.float32), 4, hp, keep_initial=True)
     b = _decide(impl_name, [9.0, 16.0], np.array([1.0, 8.0], np.float32), 4, hp)
     np.testing.assert_array_equal(a["gamma"], b["gamma"])
+
+
+# ----------------------------------------------------------------------------- SGD with momentum on the clipped gradient
+@pytest.mark.parametrize("impl_name", ["numpy", "c"])
+def test_sgdm_matches_library_sgd(impl_name):
+    """Special case that reduces to a library routine: torch.optim.SGD(momentum, weight_decay) fed the
+    clipped gradients, float64."""
+    rng = np.random.RandomState(41)
+    n = 200
+    theta0 = f32_exact(rng.normal(size=n))
+    lr, mu, wd = 1e-2, 0.9, 0.05
+    p = torch.tensor(theta0.astype(np.float64), requires_grad=True)
+    opt = torch.optim.SGD([p], lr=lr, momentum=mu, weight_decay=wd)
+    th, m = theta0.copy(), np.zeros(n, np.float32)
+    for t in range(25):
+        g = f32_exact(rng.standard_t(3, size=n) * 1e-2)
+        h = 1.0 if t % 4 else 0.21
+        p.grad = torch.tensor(h * g.astype(np.float64))
+        opt.step()
+        if impl_name == "numpy":
+            th, m = npo.sgdm_update(th, g, m, h, lr, mu, wd, np.float32)
+        else:
+            co.sgdm_update(th, g, m, h, lr, mu, wd)
+    np.testing.assert_allclose(th, p.detach().numpy(), rtol=2e-6, atol=1e-7)      # fp32 storage vs float64 library run
+    th64, m64 = theta0.astype(np.float64), np.zeros(n)
+    p2 = torch.tensor(theta0.astype(np.float64), requires_grad=True)
+    opt2 = torch.optim.SGD([p2], lr=lr, momentum=mu, weight_decay=wd)
+    rng = np.random.RandomState(42)
+    for t in range(25):
+        g = rng.normal(size=n)
+        p2.grad = torch.tensor(0.5 * g)
+        opt2.step()
+        th64, m64 = npo.sgdm_update(th64, g, m64, 0.5, lr, mu, wd, np.float64)
+    np.testing.assert_allclose(th64, p2.detach().numpy(), rtol=1e-12, atol=1e-15)

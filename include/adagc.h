@@ -148,6 +148,15 @@ int adagc_step_lion(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d
                     double beta, int64_t warmup, void* cuda_stream);
 
 /*
+ * The same clip fused with SGD with momentum (heavy-ball form, L2 weight decay folded into the gradient):
+ *     d = hat(g) + wd theta;   m <- momentum m + d;   theta <- theta - lr m          (m_0 = 0)
+ * d_params and d_m are fp32 arenas updated in place; 0 <= momentum < 1.
+ */
+int adagc_step_sgdm(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, float* d_ema,
+                    int64_t step, double lr, double momentum, double wd, double lambda_rel, double beta,
+                    int64_t warmup, void* cuda_stream);
+
+/*
  * Clip-only entry (Section 4.2: the clip is optimizer-agnostic): same norms, decisions and
  * gamma update as adagc_step, then writes the clipped gradient h_i * g_i in the gradient dtype.
  * d_grads_out may equal d_grads_in (in place); in place, tensors with h == 1 are not rewritten.

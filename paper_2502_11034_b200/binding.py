@@ -61,6 +61,8 @@ def lib() -> C.CDLL:
     L.adagc_step.argtypes = [vp, vp, vp, vp, vp, f32p, i64, dbl, dbl, dbl, dbl, dbl, dbl, dbl, i64, vp]
     L.adagc_step_lion.restype = C.c_int
     L.adagc_step_lion.argtypes = [vp, vp, vp, vp, f32p, i64, dbl, dbl, dbl, dbl, dbl, dbl, i64, vp]
+    L.adagc_step_sgdm.restype = C.c_int
+    L.adagc_step_sgdm.argtypes = [vp, vp, vp, vp, f32p, i64, dbl, dbl, dbl, dbl, dbl, i64, vp]
     L.adagc_clip.restype = C.c_int
     L.adagc_clip.argtypes = [vp, vp, vp, f32p, i64, dbl, dbl, i64, vp]
     L.adagc_step_host.restype = C.c_int
@@ -189,6 +191,13 @@ class AdaGC:
                                    beta2, wd, lambda_rel, beta, int(warmup), _stream_ptr(stream))
         if rc != 0:
             raise AdagcError(rc, "adagc_step_lion")
+
+    def step_sgdm(self, params, grads, m, ema, step, lr, momentum, wd, lambda_rel, beta, warmup, stream=None):
+        assert grads.dtype == self.grad_dtype and params.dtype == m.dtype == ema.dtype == torch.float32
+        rc = lib().adagc_step_sgdm(self._h, _ptr(params), _ptr(grads), _ptr(m), _ptr(ema), int(step), lr, momentum,
+                                   wd, lambda_rel, beta, int(warmup), _stream_ptr(stream))
+        if rc != 0:
+            raise AdagcError(rc, "adagc_step_sgdm")
 
     def clip(self, grads_in, grads_out, ema, step, lambda_rel, beta, warmup, stream=None):
         assert grads_in.dtype == grads_out.dtype == self.grad_dtype and ema.dtype == torch.float32

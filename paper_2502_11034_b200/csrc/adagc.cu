@@ -356,6 +356,7 @@ adagc_global_finalize_kernel(ClipScalars cs, int in_warmup, float* __restrict__ 
 // theta -= lr (sign(c) + wd theta), m = beta2 m + (1-beta2) hat(g); one state stream, no v).
 constexpr int kOptAdamW = 0;
 constexpr int kOptLion = 1;
+constexpr int kOptSgdM = 2;  // heavy-ball SGD: d = hat(g) + wd theta, m = momentum m + d, theta -= lr m (no v)
 
 template <int kOpt>
 __device__ __forceinline__ void adamw_elem(float g, float h, float& p, float& m, float& v,
@@ -367,6 +368,10 @@ __device__ __forceinline__ void adamw_elem(float g, float h, float& p, float& m,
     const float sgn = c > 0.0f ? 1.0f : (c < 0.0f ? -1.0f : c);  // 0 stays 0, NaN stays NaN
     p = fmaf(-a.step_size, sgn, p * a.decay);                    // step_size = lr, decay = 1 - lr wd
     m = fmaf(a.beta2, m, a.one_minus_beta2 * gh);
+  } else if (kOpt == kOptSgdM) {
+    const float d = fmaf(a.decay, p, gh);  // here decay holds wd itself, beta1 the momentum, step_size lr
+    m = fmaf(a.beta1, m, d);
+    p = fmaf(-a.step_size, m, p);
   } else {
     m = fmaf(a.beta1, m, a.one_minus_beta1 * gh);
     v = fmaf(a.beta2, v, a.one_minus_beta2 * (gh * gh));
@@ -574,7 +579,7 @@ __device__ __forceinline__ void bulk_wait_done() { asm volatile("cp.async.bulk.w
 __device__ __forceinline__ void fence_generic_to_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 constexpr int tma_smem_bytes(bool bf16, int opt) {
-  return kTmaStages * kTile * ((opt == kOptLion ? 8 : 12) + (bf16 ? 2 : 4));
+  return kTmaStages * kTile * ((opt == kOptAdamW ? 12 : 8) + (bf16 ? 2 : 4));
 }
 
 template <bool kBF16, int kOpt>
@@ -585,7 +590,7 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
                         const float* __restrict__ h_arr, AdamScalars a, int* __restrict__ status) {
   extern __shared__ __align__(128) unsigned char tile_smem[];
   constexpr int kGBytes = kBF16 ? 2 : 4;
-  constexpr int kStateBytes = kOpt == kOptLion ? 8 : 12;  // theta, m (and v) per element; g follows them
+  constexpr int kStateBytes = kOpt == kOptAdamW ? 12 : 8;  // theta, m (and v) per element; g follows them
   constexpr uint32_t kStageBytes = kTile * (kStateBytes + kGBytes);
   __shared__ __align__(8) uint64_t full_bar[kTmaStages];
   const int tid = threadIdx.x;
@@ -953,7 +958,11 @@ bool prepare_update_kernels() {
          cudaFuncSetAttribute(adagc_update_tma_kernel<kBF16, kOptAdamW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               tma_smem_bytes(kBF16, kOptAdamW)) == cudaSuccess &&
          cudaFuncSetAttribute(adagc_update_tma_kernel<kBF16, kOptLion>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              tma_smem_bytes(kBF16, kOptLion)) == cudaSuccess;
+                              tma_smem_bytes(kBF16, kOptLion)) == cudaSuccess &&
+         cudaFuncSetAttribute(adagc_update_kernel<kBF16, kOptSgdM>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                              cudaSharedmemCarveoutMaxL1) == cudaSuccess &&
+         cudaFuncSetAttribute(adagc_update_tma_kernel<kBF16, kOptSgdM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              tma_smem_bytes(kBF16, kOptSgdM)) == cudaSuccess;
 }
 
 // One kernel's view of the chunk tables: the whole layout, or one group of the pipelined host step.
@@ -1330,6 +1339,28 @@ int adagc_step_lion(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d
     launch_update<true, kOptLion>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), nullptr, a, s);
   else
     launch_update<false, kOptLion>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), nullptr, a, s);
+  return finish_launches(ctx, s);
+}
+
+int adagc_step_sgdm(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, float* d_ema, int64_t step,
+                    double lr, double momentum, double wd, double lambda_rel, double beta, int64_t warmup,
+                    void* cuda_stream) {
+  int rc = check_clip_args(ctx, d_ema, step, lambda_rel, beta, warmup);
+  if (rc != ADAGC_OK) return rc;
+  if (!d_params || !d_grads || !d_m) return ADAGC_E_INVALID_ARG;
+  if (!(momentum >= 0.0 && momentum < 1.0) || !std::isfinite(lr) || !std::isfinite(wd)) return ADAGC_E_INVALID_ARG;
+  if (!aligned16(d_params) || !aligned16(d_grads) || !aligned16(d_m)) return ADAGC_E_MISALIGNED;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  rc = enqueue_clip_phases(ctx, d_grads, d_ema, step, lambda_rel, beta, warmup, s);
+  if (rc != ADAGC_OK) return rc;
+  AdamScalars a = {};
+  a.beta1 = static_cast<float>(momentum);
+  a.step_size = static_cast<float>(lr);
+  a.decay = static_cast<float>(wd);
+  if (ctx->bf16)
+    launch_update<true, kOptSgdM>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), nullptr, a, s);
+  else
+    launch_update<false, kOptSgdM>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), nullptr, a, s);
   return finish_launches(ctx, s);
 }
 

@@ -1,6 +1,6 @@
 """Run a few fused AdaGC + AdamW steps (or clip-only steps) on a named synthetic layout.
 
-    python -m paper_2502_11034_b200.run_steps --workload gpt2_small --steps 4 [--mode step|clip|lion] [--n-layer N]
+    python -m paper_2502_11034_b200.run_steps --workload gpt2_small --steps 4 [--mode step|clip|lion|sgdm] [--n-layer N]
         [--update-path auto|registers|bulk]
 
 A minimal driver of the C ABI (adagc_create / adagc_step / adagc_clip / adagc_get_stats): useful as
@@ -19,7 +19,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", default="gpt2_small")
     ap.add_argument("--steps", type=int, default=4)
-    ap.add_argument("--mode", choices=["step", "clip", "lion"], default="step")
+    ap.add_argument("--mode", choices=["step", "clip", "lion", "sgdm"], default="step")
     ap.add_argument("--n-layer", type=int, default=None, help="override the layer count of a layered layout")
     ap.add_argument("--warmup", type=int, default=1, help="T_start: steps of global-norm clipping")
     ap.add_argument("--update-path", choices=["auto", "registers", "bulk"], default="auto",
@@ -46,6 +46,8 @@ def main():
                      hp["lambda_rel"], hp["beta"], args.warmup)
         elif args.mode == "lion":
             opt.step_lion(theta, g, m, ema, t, 1e-4, 0.9, 0.99, hp["wd"], hp["lambda_rel"], hp["beta"], args.warmup)
+        elif args.mode == "sgdm":
+            opt.step_sgdm(theta, g, m, ema, t, 1e-2, 0.9, hp["wd"], hp["lambda_rel"], hp["beta"], args.warmup)
         else:
             opt.clip(g, g_out, ema, t, hp["lambda_rel"], hp["beta"], args.warmup)
         ms = opt.get_phase_times()

@@ -335,3 +335,36 @@ def run_full_clip(wl: workloads.Workload, n_steps: int, in_place: bool, device="
         rep.steps = t
     opt.close()
     return rep
+
+
+def run_full_sgdm(wl: workloads.Workload, n_steps: int, device="cuda", flags: int = 0, lr: float = 1e-2,
+                  momentum: float = 0.9, hyper_over: Optional[dict] = None) -> ParityReport:
+    """Every element, clip fused with SGD with momentum (adagc_step_sgdm) vs the C oracle."""
+    hp = hyper_of(wl, **(hyper_over or {}))
+    offs = np.array([t.offset for t in wl.tensors], np.int64)
+    nums = np.array([t.numel for t in wl.tensors], np.int64)
+    opt = binding.AdaGC(nums.tolist(), offs.tolist(), wl.torch_grad_dtype, hp["lambda_abs"], device=device, flags=flags)
+    theta = workloads.init_params(wl, device)
+    m = torch.zeros_like(theta)
+    ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device=device)
+    r_theta = theta.cpu().numpy().copy()
+    r_m = np.zeros_like(r_theta)
+    gamma = np.zeros(wl.n_tensors, np.float32)
+    rep = ParityReport()
+    for t in range(1, n_steps + 1):
+        g = workloads.grads_for_step(wl, t, device)
+        opt.step_sgdm(theta, g, m, ema, t, lr, momentum, hp["wd"], hp["lambda_rel"], hp["beta"], hp["warmup"])
+        g_np = to_numpy_grads(g)
+        ssq = c_oracle.sumsq_tensors(g_np, offs, nums)
+        r = c_oracle.clip_decisions(ssq, gamma, t, hp["lambda_rel"], hp["beta"], hp["lambda_abs"], hp["warmup"])
+        for i, (o, n) in enumerate(zip(offs, nums)):
+            c_oracle.sgdm_update(r_theta[o:o + n], g_np[o:o + n], r_m[o:o + n], float(r["h"][i]), lr, momentum, hp["wd"])
+        check_decisions(opt.get_stats(), opt.get_sumsq(), ema.cpu().numpy(), r, rep, t)
+        rep.steps = t
+    th, mm = theta.cpu().numpy(), m.cpu().numpy()
+    for t_, o, n in zip(wl.tensors, offs, nums):
+        check_state("theta", th[o:o + n], r_theta[o:o + n], rep, t_.name)
+        check_state("m", mm[o:o + n], r_m[o:o + n], rep, t_.name)
+    assert opt.get_stats()["status"] == 0
+    opt.close()
+    return rep

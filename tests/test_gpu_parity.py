@@ -114,6 +114,17 @@ def test_lion_small_layouts_all_elements(path):
         _report(f"lion {name} (small, path {path})", rep)
 
 
+@pytest.mark.parametrize("path", [binding.UPDATE_PATH_REGISTERS, binding.UPDATE_PATH_BULK], ids=["registers", "bulk"])
+def test_sgdm_small_layouts_all_elements(path):
+    """The clip fused with SGD with momentum, both update kernels, both gradient dtypes."""
+    for name, over in [("llama2_7b", dict(n_layer=2, d=256, ffn=688, vocab=1000)),
+                       ("many_small", dict(n_tensors=300, lo=1, hi=40000))]:
+        wl = workloads.build(name, **over)
+        rep = H.run_full_sgdm(wl, 15, flags=path, hyper_over=dict(lambda_abs=1e4))
+        _report(f"sgdm {name} (small, path {path})", rep)
+        assert rep.clipped > 0
+
+
 def test_lion_gpt2_small_all_elements():
     wl = workloads.build("gpt2_small")
     rep = H.run_full_lion(wl, 20, hyper_over=dict(lambda_abs=1e4))

@@ -125,6 +125,20 @@ def test_c_oracle_bf16_inputs_and_rounding():
 
 
 # ----------------------------------------------------------------------------- hand-worked example
+def test_golden_fixture_equals_its_exact_derivation():
+    """The stored hand-worked table is reproduced by exact rational arithmetic (no oracle involved)."""
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("make_worked_example", os.path.join(GOLDEN, "make_worked_example.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    for r, s in zip(mod.derive(), _golden()["steps"]):
+        assert r["norm"] == s["norm"] and r["h"] == s["h"] and r["flag"] == s["flag"] and r["gamma"] == s["gamma"]
+        if "global_norm" in s:
+            assert r["global_norm_sq"] == s["global_norm"] ** 2
+        if "global_norm_sq" in s:
+            assert r["global_norm_sq"] == s["global_norm_sq"]
+
+
 def _golden():
     with open(os.path.join(GOLDEN, "worked_example.json")) as f:
         return json.load(f)

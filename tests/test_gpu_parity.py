@@ -87,6 +87,39 @@ def test_llama2_7b_sampled():
     assert 8 <= rep.clipped < 291
 
 
+def test_hand_worked_example_on_the_gpu():
+    """The 2-tensor worked example (tests/golden/worked_example.json): every norm, clip factor, flag and gamma
+    of the table is exactly representable, so the CUDA path must reproduce the table exactly."""
+    import json
+    import os
+    from oracle import adagc_oracle as npo
+    gold = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "worked_example.json")))
+    hp = gold["hyper"]
+    offs, nums = [0, 8], [2, 3]
+    opt = binding.AdaGC(nums, offs, torch.float32, hp["lambda_abs"])
+    theta = torch.zeros(16, device="cuda")
+    theta[0:2] = torch.tensor(gold["theta0"]["A"])
+    theta[8:11] = torch.tensor(gold["theta0"]["B"])
+    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    ema = torch.zeros(2, device="cuda")
+    ref = npo.AdaGCAdamW([gold["theta0"]["A"], gold["theta0"]["B"]], npo.Hyper(**hp), np.float32)
+    for srow in gold["steps"]:
+        g = torch.zeros(16, device="cuda")
+        g[0:2] = torch.tensor(srow["gA"])
+        g[8:11] = torch.tensor(srow["gB"])
+        opt.step(theta, g, m, v, ema, srow["t"], hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"],
+                 hp["lambda_rel"], hp["beta"], hp["warmup"])
+        ref.step([np.array(srow["gA"], np.float32), np.array(srow["gB"], np.float32)])
+        st = opt.get_stats()
+        assert st["norm"].tolist() == srow["norm"] and st["h"].tolist() == srow["h"]
+        assert st["flag"].astype(int).tolist() == srow["flag"] and ema.cpu().tolist() == srow["gamma"]
+    th = theta.cpu().numpy()
+    np.testing.assert_allclose(th[0:2], ref.theta[0], rtol=1e-5)
+    np.testing.assert_allclose(th[8:11], ref.theta[1], rtol=1e-5)
+    assert float(theta[2:8].abs().sum()) == 0.0 and st["clip_count"].tolist() == [3, 1]
+    opt.close()
+
+
 # ------------------------------------------------------------------ small layouts, all elements
 @pytest.mark.parametrize("name,over", [
     ("llama2_7b", dict(n_layer=2, d=256, ffn=688, vocab=1000)),

@@ -134,6 +134,19 @@ int adagc_step(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, v
                double wd, double lambda_rel, double beta, int64_t warmup, void* cuda_stream);
 
 /*
+ * adagc_step that also emits the model's working copy of the parameters: mixed-precision training keeps fp32
+ * master parameters in the optimizer and runs the model on a bf16 copy (the paper's runs use bfloat16
+ * precision).  Besides everything adagc_step does, d_params_bf16[j] = bf16(theta_t[j]) (round to nearest even)
+ * is written for every element of every tensor, from the same kernel, so no separate cast pass re-reads theta.
+ * d_params_bf16 is a bf16 arena with the descriptor's element offsets, 16-byte aligned; every tensor offset
+ * must then be a multiple of 8 elements (ADAGC_E_MISALIGNED otherwise).  28 B/param instead of 26.
+ */
+int adagc_step_emit_bf16(adagc_ctx* ctx, void* d_params, void* d_params_bf16, const void* d_grads, void* d_m,
+                         void* d_v, float* d_ema, int64_t step, double lr, double beta1, double beta2,
+                         double eps, double wd, double lambda_rel, double beta, int64_t warmup,
+                         void* cuda_stream);
+
+/*
  * The same clip fused with Lion instead of AdamW (Section 4.2 of the paper: AdaGC is optimizer-agnostic
  * and is used with Lion).  Phases 1 and 2 are those of adagc_step; the update phase applies Lion's rule
  * to the clipped gradient hat(g) = h_i g:

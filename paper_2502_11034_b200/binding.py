@@ -59,6 +59,8 @@ def lib() -> C.CDLL:
     L.adagc_destroy.argtypes = [vp]
     L.adagc_step.restype = C.c_int
     L.adagc_step.argtypes = [vp, vp, vp, vp, vp, f32p, i64, dbl, dbl, dbl, dbl, dbl, dbl, dbl, i64, vp]
+    L.adagc_step_emit_bf16.restype = C.c_int
+    L.adagc_step_emit_bf16.argtypes = [vp, vp, vp, vp, vp, vp, f32p, i64, dbl, dbl, dbl, dbl, dbl, dbl, dbl, i64, vp]
     L.adagc_step_lion.restype = C.c_int
     L.adagc_step_lion.argtypes = [vp, vp, vp, vp, f32p, i64, dbl, dbl, dbl, dbl, dbl, dbl, i64, vp]
     L.adagc_step_sgdm.restype = C.c_int
@@ -184,6 +186,16 @@ class AdaGC:
                               lr, beta1, beta2, eps, wd, lambda_rel, beta, int(warmup), _stream_ptr(stream))
         if rc != 0:
             raise AdagcError(rc, "adagc_step")
+
+    def step_emit_bf16(self, params, params_bf16, grads, m, v, ema, step, lr, beta1, beta2, eps, wd, lambda_rel, beta,
+                       warmup, stream=None):
+        assert grads.dtype == self.grad_dtype and params_bf16.dtype == torch.bfloat16
+        assert params.dtype == m.dtype == v.dtype == ema.dtype == torch.float32
+        rc = lib().adagc_step_emit_bf16(self._h, _ptr(params), _ptr(params_bf16), _ptr(grads), _ptr(m), _ptr(v),
+                                        _ptr(ema), int(step), lr, beta1, beta2, eps, wd, lambda_rel, beta,
+                                        int(warmup), _stream_ptr(stream))
+        if rc != 0:
+            raise AdagcError(rc, "adagc_step_emit_bf16")
 
     def step_lion(self, params, grads, m, ema, step, lr, beta1, beta2, wd, lambda_rel, beta, warmup, stream=None):
         assert grads.dtype == self.grad_dtype and params.dtype == m.dtype == ema.dtype == torch.float32

@@ -394,7 +394,7 @@ __device__ __forceinline__ void adamw_vec4(const float g0, const float g1, const
 template <bool kBF16, int kOpt>
 __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gbase, float4* __restrict__ p4,
                                              float4* __restrict__ m4, float4* __restrict__ v4, float h,
-                                             const AdamScalars& a) {
+                                             const AdamScalars& a, uint4* __restrict__ lowp8 = nullptr) {
   float g[8];
   if (kBF16) {
     const uint4 q = ld_stream(reinterpret_cast<const uint4*>(gbase) + i);
@@ -421,6 +421,9 @@ __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gba
     st_stream(v4 + 2 * i, va);
     st_stream(v4 + 2 * i + 1, vb);
   }
+  if (lowp8)  // bf16 copy of the updated parameters (the model's working weights in mixed precision)
+    st_stream(lowp8 + i, make_uint4(pack_bf16(pa.x, pa.y), pack_bf16(pa.z, pa.w), pack_bf16(pb.x, pb.y),
+                                    pack_bf16(pb.z, pb.w)));
 }
 
 // A partial chunk (a small tensor, or the end of one).  Work is dealt in rows of 32 groups (256
@@ -430,7 +433,8 @@ __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gba
 template <bool kBF16, int kBlockThreads, int kOpt>
 __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, int& row_base, float* __restrict__ params,
                                                     const void* __restrict__ grads, float* __restrict__ m_arena,
-                                                    float* __restrict__ v_arena, const AdamScalars& a) {
+                                                    float* __restrict__ v_arena, const AdamScalars& a,
+                                                    uint16_t* __restrict__ lowp = nullptr) {
   constexpr int kWarps = kBlockThreads / 32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int64_t start = chunk_start(ck);
@@ -443,7 +447,7 @@ __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, in
 #pragma unroll 2
   for (int r = (warp - row_base) & (kWarps - 1); r < rows; r += kWarps) {
     const int i = (r << 5) + lane;
-    if (i < n8) adamw_group8<kBF16, kOpt>(i, gbase, p4, m4, v4, h, a);
+    if (i < n8) adamw_group8<kBF16, kOpt>(i, gbase, p4, m4, v4, h, a, lowp ? reinterpret_cast<uint4*>(lowp + start) : nullptr);
   }
   row_base = (row_base + rows) & (kWarps - 1);
   const int t = (n8 << 3) + lane;  // ragged tail (fewer than 8 elements): the next warp in turn takes it
@@ -460,6 +464,7 @@ __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, in
     params[start + t] = p;
     m_arena[start + t] = m;
     if (kOpt == kOptAdamW) v_arena[start + t] = v;
+    if (lowp) lowp[start + t] = static_cast<uint16_t>(f32_to_bf16_bits(p));
   }
 }
 
@@ -468,7 +473,8 @@ template <bool kBF16, int kOpt>
 __global__ void __launch_bounds__(kThreads)
 adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, float* __restrict__ m_arena,
                     float* __restrict__ v_arena, const Chunk* __restrict__ chunks,
-                    const int32_t* __restrict__ block_begin, const float* __restrict__ h_arr, AdamScalars a) {
+                    const int32_t* __restrict__ block_begin, const float* __restrict__ h_arr, AdamScalars a,
+                    uint16_t* __restrict__ lowp) {
   const int tid = threadIdx.x;
   int c = block_begin[blockIdx.x];
   const int n_chunks = block_begin[blockIdx.x + 1];  // end of this block's entries
@@ -494,9 +500,10 @@ adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, 
       const char* __restrict__ gbase = static_cast<const char*>(grads) + start * (kBF16 ? 2 : 4);
 #pragma unroll 2
       for (int k = 0; k < kChunkElems / 8 / kThreads; ++k)
-        adamw_group8<kBF16, kOpt>(k * kThreads + tid, gbase, p4, m4, v4, h, a);
+        adamw_group8<kBF16, kOpt>(k * kThreads + tid, gbase, p4, m4, v4, h, a,
+                                  lowp ? reinterpret_cast<uint4*>(lowp + start) : nullptr);
     } else {
-      adamw_partial_chunk<kBF16, kThreads, kOpt>(ck, h, row_base, params, grads, m_arena, v_arena, a);
+      adamw_partial_chunk<kBF16, kThreads, kOpt>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp);
     }
     if (c_next >= n_chunks) break;
     c = c_next;
@@ -578,8 +585,8 @@ __device__ __forceinline__ void bulk_wait_smem_read() { asm volatile("cp.async.b
 __device__ __forceinline__ void bulk_wait_done() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_generic_to_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-constexpr int tma_smem_bytes(bool bf16, int opt) {
-  return kTmaStages * kTile * ((opt == kOptAdamW ? 12 : 8) + (bf16 ? 2 : 4));
+constexpr int tma_smem_bytes(bool bf16, int opt, bool emit_lowp = false) {
+  return kTmaStages * kTile * ((opt == kOptAdamW ? 12 : 8) + (bf16 ? 2 : 4) + (emit_lowp ? 2 : 0));
 }
 
 template <bool kBF16, int kOpt>
@@ -587,11 +594,14 @@ __global__ void __launch_bounds__(kTmaThreads, 1)
 adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ grads, float* __restrict__ m_arena,
                         float* __restrict__ v_arena, const Chunk* __restrict__ chunks,
                         const int32_t* __restrict__ block_begin, const int32_t* __restrict__ block_mid,
-                        const float* __restrict__ h_arr, AdamScalars a, int* __restrict__ status) {
+                        const float* __restrict__ h_arr, AdamScalars a, int* __restrict__ status,
+                        uint16_t* __restrict__ lowp) {
   extern __shared__ __align__(128) unsigned char tile_smem[];
   constexpr int kGBytes = kBF16 ? 2 : 4;
   constexpr int kStateBytes = kOpt == kOptAdamW ? 12 : 8;  // theta, m (and v) per element; g follows them
-  constexpr uint32_t kStageBytes = kTile * (kStateBytes + kGBytes);
+  constexpr uint32_t kStageBytes = kTile * (kStateBytes + kGBytes);  // what the loads of one tile bring in
+  // with a bf16 copy of the parameters to emit, each stage has a fifth region that only the stores read
+  const uint32_t stage_stride = kStageBytes + (lowp ? kTile * 2 : 0);
   __shared__ __align__(8) uint64_t full_bar[kTmaStages];
   const int tid = threadIdx.x;
   const int begin = block_begin[blockIdx.x], mid = block_mid[blockIdx.x], end = block_begin[blockIdx.x + 1];
@@ -608,7 +618,7 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
   // thread 0 only: start the four loads of one tile (tile `sub` of the chunk that starts at element e0)
   auto issue_tile = [&](int64_t e0, int sub, int s) {
     const int64_t e = e0 + static_cast<int64_t>(sub) * kTile;
-    unsigned char* b = tile_smem + static_cast<size_t>(s) * kStageBytes;
+    unsigned char* b = tile_smem + static_cast<size_t>(s) * stage_stride;
     mbar_arrive_expect_tx(&full_bar[s], kStageBytes);
     bulk_load(b, params + e, kTile * 4, &full_bar[s]);
     bulk_load(b + kTile * 4, m_arena + e, kTile * 4, &full_bar[s]);
@@ -639,7 +649,7 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
         if (last_of_chunk) issue_tile(chunk_start(ck_next), 0, s ^ 1);
         else issue_tile(chunk_start(ck), sub + 1, s ^ 1);
       }
-      unsigned char* b = tile_smem + static_cast<size_t>(s) * kStageBytes;
+      unsigned char* b = tile_smem + static_cast<size_t>(s) * stage_stride;
       if (mbar_wait_bounded(&full_bar[s], (j >> 1) & 1)) {
         float4* p4 = reinterpret_cast<float4*>(b);
         float4* m4 = reinterpret_cast<float4*>(b + kTile * 4);
@@ -659,6 +669,7 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
           adamw_vec4<kOpt>(g0, g1, g2, g3, h, p, m, v, a);
           p4[q] = p; m4[q] = m;
           if (kOpt == kOptAdamW) v4[q] = v;
+          if (lowp) reinterpret_cast<uint2*>(b + kStageBytes)[q] = make_uint2(pack_bf16(p.x, p.y), pack_bf16(p.z, p.w));
         }
         fence_generic_to_async_smem();  // the updated tile must be visible to the bulk-copy engine
       } else {
@@ -675,6 +686,7 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
         bulk_store(params + e, b, kTile * 4);
         bulk_store(m_arena + e, b + kTile * 4, kTile * 4);
         if (kOpt == kOptAdamW) bulk_store(v_arena + e, b + kTile * 8, kTile * 4);
+        if (lowp) bulk_store(lowp + e, b + kStageBytes, kTile * 2);
         bulk_commit();
       }
       if (last_of_chunk) {
@@ -704,7 +716,8 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
   int row_base = 0;
   for (int c = mid; c < end; ++c) {
     const Chunk ck = chunks[c];
-    adamw_partial_chunk<kBF16, kTmaThreads, kOpt>(ck, h_arr[ck.tensor], row_base, params, grads, m_arena, v_arena, a);
+    adamw_partial_chunk<kBF16, kTmaThreads, kOpt>(ck, h_arr[ck.tensor], row_base, params, grads, m_arena, v_arena, a,
+                                                  lowp);
   }
 }
 
@@ -895,6 +908,7 @@ struct adagc_ctx {
   int device = 0;
   int grid_wide = 1, grid_update = 1;  // norm and scale kernels: SMs x resident blocks; update: SMs x 2 or x 1
   bool update_bulk = false;            // update phase through the bulk-async (TMA) kernel
+  bool offsets_mult8 = true;           // every tensor offset is a multiple of 8 elements (bf16 arenas stay 16-byte aligned)
   bool keep_initial = false;           // ADAGC_EMA_KEEP_INITIAL
   bool global_adaptive = false;        // ADAGC_CLIP_GLOBAL_ADAPTIVE
   char* ws = nullptr;
@@ -956,7 +970,7 @@ bool prepare_update_kernels() {
          cudaFuncSetAttribute(adagc_update_kernel<kBF16, kOptLion>, cudaFuncAttributePreferredSharedMemoryCarveout,
                               cudaSharedmemCarveoutMaxL1) == cudaSuccess &&
          cudaFuncSetAttribute(adagc_update_tma_kernel<kBF16, kOptAdamW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              tma_smem_bytes(kBF16, kOptAdamW)) == cudaSuccess &&
+                              tma_smem_bytes(kBF16, kOptAdamW, true)) == cudaSuccess &&
          cudaFuncSetAttribute(adagc_update_tma_kernel<kBF16, kOptLion>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               tma_smem_bytes(kBF16, kOptLion)) == cudaSuccess &&
          cudaFuncSetAttribute(adagc_update_kernel<kBF16, kOptSgdM>, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -975,21 +989,22 @@ struct TableView {
 
 template <bool kBF16, int kOpt>
 void launch_update(adagc_ctx* ctx, const TableView& tv, float* p, const void* g, float* m, float* v,
-                   const AdamScalars& a, cudaStream_t s) {
+                   const AdamScalars& a, cudaStream_t s, uint16_t* lowp = nullptr) {
   const StatPtrs st = ctx->stats();
   if (ctx->update_bulk)
-    adagc_update_tma_kernel<kBF16, kOpt><<<tv.grid, kTmaThreads, tma_smem_bytes(kBF16, kOpt), s>>>(
-        p, g, m, v, tv.chunks, tv.begin, tv.mid, st.h, a, st.status);
+    adagc_update_tma_kernel<kBF16, kOpt>
+        <<<tv.grid, kTmaThreads, tma_smem_bytes(kBF16, kOpt, lowp != nullptr), s>>>(
+            p, g, m, v, tv.chunks, tv.begin, tv.mid, st.h, a, st.status, lowp);
   else
-    adagc_update_kernel<kBF16, kOpt><<<tv.grid, kThreads, 0, s>>>(p, g, m, v, tv.chunks, tv.begin, st.h, a);
+    adagc_update_kernel<kBF16, kOpt><<<tv.grid, kThreads, 0, s>>>(p, g, m, v, tv.chunks, tv.begin, st.h, a, lowp);
   ctx->launches++;
 }
 
 template <bool kBF16, int kOpt>
 void launch_update(adagc_ctx* ctx, float* p, const void* g, float* m, float* v, const AdamScalars& a,
-                   cudaStream_t s) {
+                   cudaStream_t s, uint16_t* lowp = nullptr) {
   const TableView tv = {ctx->d_chunks_upd(), ctx->d_begin_upd(), ctx->d_mid_upd(), ctx->grid_update};
-  launch_update<kBF16, kOpt>(ctx, tv, p, g, m, v, a, s);
+  launch_update<kBF16, kOpt>(ctx, tv, p, g, m, v, a, s, lowp);
 }
 
 void launch_norm(adagc_ctx* ctx, const TableView& tv, const void* d_grads, cudaStream_t s) {
@@ -1167,6 +1182,7 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
   ctx->arena_elems = extent;
   ctx->bf16 = desc->grad_dtype == ADAGC_BF16;
   ctx->lambda_abs = desc->lambda_abs;
+  for (int32_t i = 0; i < desc->n_tensors; ++i) ctx->offsets_mult8 = ctx->offsets_mult8 && desc->tensors[i].offset % 8 == 0;
   ctx->ws = static_cast<char*>(d_workspace);
   ctx->L = L;
 
@@ -1311,6 +1327,29 @@ int adagc_step(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, v
   else
     launch_update<false, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
                                     static_cast<float*>(d_v), a, s);
+  return finish_launches(ctx, s);
+}
+
+int adagc_step_emit_bf16(adagc_ctx* ctx, void* d_params, void* d_params_bf16, const void* d_grads, void* d_m,
+                         void* d_v, float* d_ema, int64_t step, double lr, double beta1, double beta2, double eps,
+                         double wd, double lambda_rel, double beta, int64_t warmup, void* cuda_stream) {
+  int rc = check_clip_args(ctx, d_ema, step, lambda_rel, beta, warmup);
+  if (rc != ADAGC_OK) return rc;
+  rc = check_adamw_args(d_params, d_grads, d_m, d_v, lr, beta1, beta2, eps, wd);
+  if (rc != ADAGC_OK) return rc;
+  if (!d_params_bf16) return ADAGC_E_INVALID_ARG;
+  if (!aligned16(d_params_bf16) || !ctx->offsets_mult8) return ADAGC_E_MISALIGNED;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  rc = enqueue_clip_phases(ctx, d_grads, d_ema, step, lambda_rel, beta, warmup, s);
+  if (rc != ADAGC_OK) return rc;
+  const AdamScalars a = make_adam_scalars(step, lr, beta1, beta2, eps, wd);
+  uint16_t* lowp = static_cast<uint16_t*>(d_params_bf16);
+  if (ctx->bf16)
+    launch_update<true, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
+                                   static_cast<float*>(d_v), a, s, lowp);
+  else
+    launch_update<false, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
+                                    static_cast<float*>(d_v), a, s, lowp);
   return finish_launches(ctx, s);
 }
 

@@ -101,7 +101,8 @@ def check_state(name: str, got: np.ndarray, ref: np.ndarray, rep: ParityReport, 
 
 
 def run_full(wl: workloads.Workload, n_steps: int, device="cuda", hyper_over: Optional[dict] = None,
-             lr_schedule=None, canary: bool = True, flags: int = 0, gamma0: Optional[float] = None) -> ParityReport:
+             lr_schedule=None, canary: bool = True, flags: int = 0, gamma0: Optional[float] = None,
+             emit_bf16: bool = False) -> ParityReport:
     """Every element of every tensor, fused AdaGC+AdamW step, GPU vs C oracle."""
     hp = hyper_of(wl, **(hyper_over or {}))
     offs = [t.offset for t in wl.tensors]
@@ -129,11 +130,16 @@ def run_full(wl: workloads.Workload, n_steps: int, device="cuda", hyper_over: Op
                                global_adaptive=bool(flags & binding.CLIP_GLOBAL_ADAPTIVE),
                                gamma0=None if not keep else np.full(wl.n_tensors, gamma0, np.float32))
     rep = ParityReport()
+    lowp = torch.full((wl.arena_elems,), 7.0, dtype=torch.bfloat16, device=device) if emit_bf16 else None
     for t in range(1, n_steps + 1):
         g = workloads.grads_for_step(wl, t, device)
         lr = hp["lr"] if lr_schedule is None else lr_schedule(t)
-        opt.step(theta, g, m, v, ema, t, lr, hp["beta1"], hp["beta2"], hp["eps"], hp["wd"],
-                 hp["lambda_rel"], hp["beta"], hp["warmup"])
+        if emit_bf16:
+            opt.step_emit_bf16(theta, lowp, g, m, v, ema, t, lr, hp["beta1"], hp["beta2"], hp["eps"], hp["wd"],
+                               hp["lambda_rel"], hp["beta"], hp["warmup"])
+        else:
+            opt.step(theta, g, m, v, ema, t, lr, hp["beta1"], hp["beta2"], hp["eps"], hp["wd"],
+                     hp["lambda_rel"], hp["beta"], hp["warmup"])
         r = ref.step(to_numpy_grads(g), lr=lr)
         st = opt.get_stats()
         check_decisions(st, opt.get_sumsq(), ema.cpu().numpy(), r, rep, t)
@@ -147,6 +153,21 @@ def run_full(wl: workloads.Workload, n_steps: int, device="cuda", hyper_over: Op
         check_state("theta", th[o:o + n], ref.theta[o:o + n], rep, t_.name)
         check_state("m", mm[o:o + n], ref.m[o:o + n], rep, t_.name)
         check_state("v", vv[o:o + n], ref.v[o:o + n], rep, t_.name)
+    if emit_bf16:
+        # the emitted working copy is the bf16 rounding of the fp32 master: exactly so for the GPU's own theta,
+        # and within one bf16 ulp of the rounding of the oracle's theta
+        got = to_numpy_grads(lowp)
+        for t_, o, n in zip(wl.tensors, offs, nums):
+            own = to_numpy_grads(theta[o:o + n].to(torch.bfloat16))
+            assert np.array_equal(got[o:o + n], own), f"bf16 copy of {t_.name} is not the rounding of theta"
+            # vs the oracle: one bf16 ulp for the rounding, plus the tolerance of the fp32 theta underneath
+            a = bf16_bits_to_f64(got[o:o + n])
+            b = ref.theta[o:o + n].astype(np.float64)
+            rms = float(np.linalg.norm(b)) / math.sqrt(max(b.size, 1))
+            bound = np.abs(b) * 2.0 ** -7 + RTOL * np.maximum(np.abs(b), rms)
+            assert (np.abs(a - b) <= bound).all(), f"bf16 parameters of {t_.name} differ from the oracle's theta"
+        if pad_mask is not None:
+            assert bool((lowp[pad_mask].float() == 7.0).all()), "bf16 copy: padding between tensors was written"
     if pad_mask is not None:
         for a in (theta, m, v):
             assert bool((a[pad_mask] == 777.0).all()), "guard bands between tensors were overwritten"

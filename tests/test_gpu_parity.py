@@ -177,6 +177,25 @@ def test_clip_only_small_layouts_all_elements(in_place):
         assert rep.clipped > 0
 
 
+@pytest.mark.parametrize("path", [binding.UPDATE_PATH_REGISTERS, binding.UPDATE_PATH_BULK], ids=["registers", "bulk"])
+def test_emit_bf16_parameters_all_elements(path):
+    """adagc_step_emit_bf16: fp32 master parameters plus the bf16 working copy from the same kernel."""
+    sizes = [1, 7, 8, 9, 255, 2049, 16384, 16385, 3 * 16384 + 5, 40 * 16384, 100003]
+    for dtype in ("bf16", "f32"):
+        rep = H.run_full(_ragged_workload(sizes, dtype), 6, flags=path, emit_bf16=True)
+        _report(f"emit bf16, {dtype} grads, path {path}", rep)
+    wl = workloads.build("llama2_7b", n_layer=2, d=256, ffn=688, vocab=1000)
+    _report(f"emit bf16 llama (small), path {path}", H.run_full(wl, 12, flags=path, emit_bf16=True))
+    # an fp32-gradient layout whose offsets are multiples of 4 but not of 8 cannot carry a bf16 arena
+    opt = binding.AdaGC([100, 60], [0, 100], torch.float32, 1.0, flags=path)
+    z = torch.zeros(160, device="cuda")
+    with pytest.raises(binding.AdagcError) as e:
+        opt.step_emit_bf16(z, torch.zeros(160, device="cuda", dtype=torch.bfloat16), z.clone(), z.clone(), z.clone(),
+                           torch.zeros(2, device="cuda"), 1, 1e-3, 0.9, 0.95, 1e-8, 0.1, 1.04, 0.99, 0)
+    assert e.value.status == -2
+    opt.close()
+
+
 def test_moe_layout_small_all_elements():
     """Mixture-of-experts tensor census ((7+3E)L+3 tensors, Section 4.3 "Memory"), reduced dimensions."""
     wl = workloads.build("moe_8x1b", n_layer=2, d=128, ffn=352, vocab=1000, kv_dim=32, n_experts=4)

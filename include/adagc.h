@@ -72,10 +72,15 @@ typedef enum {
  *                               d_ema hold the one gamma (entry 0 is the one read). */
 #define ADAGC_EMA_KEEP_INITIAL 4
 #define ADAGC_CLIP_GLOBAL_ADAPTIVE 8
+/* Sharded use (Section 4.3 "Communication": with a tensor split over several devices, the per-tensor norm
+ * needs one all-reduce of the partial sums of squares).  With this flag a tensor of the descriptor may have
+ * numel == 0 -- this rank holds no element of it -- so that every rank keeps the same tensor numbering and
+ * the same n_tensors-long vectors (gamma, sums of squares); the offset of an empty tensor is ignored. */
+#define ADAGC_ALLOW_EMPTY 16
 
 /* One parameter tensor. */
 typedef struct {
-  int64_t numel;    /* > 0; offset + numel <= 2^34 */
+  int64_t numel;    /* > 0 (0 allowed with ADAGC_ALLOW_EMPTY); offset + numel <= 2^34 */
   int64_t offset;   /* element offset into every arena; offset * sizeof(element) must be a
                        multiple of 16 bytes for every arena dtype (multiple of 8 elements with
                        bf16 gradients, of 4 with fp32 gradients) */
@@ -176,6 +181,49 @@ int adagc_step_sgdm(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d
  */
 int adagc_clip(adagc_ctx* ctx, const void* d_grads_in, void* d_grads_out, float* d_ema,
                int64_t step, double lambda_rel, double beta, int64_t warmup, void* cuda_stream);
+
+/*
+ * The step cut in two for models whose tensors are SHARDED over several GPUs (ZeRO-style flat shards,
+ * tensor parallelism).  Section 4.3 ("Communication"): a tensor's norm then needs one all-reduce of the
+ * partial sums of squares within the group that holds it; nothing else of the step crosses devices.
+ * Every rank creates its context over its LOCAL slices of the tensors (adagc_shard_plan computes them for
+ * flat equal shards; ADAGC_ALLOW_EMPTY lets a rank list tensors it holds nothing of) and runs, per step:
+ *
+ *   1. adagc_shard_sumsq        phase 1 on the local gradient slice; d_sumsq_out[i] = sum of squares of this
+ *                               rank's part of tensor i, float64, n_tensors entries, device memory;
+ *   2. the caller sums d_sumsq_out over the ranks (one all-reduce of 8 * n_tensors bytes, e.g. NCCL);
+ *   3. adagc_step_presummed /   phase 2 from the summed vector `d_sumsq` (decisions, gamma, statistics:
+ *      adagc_clip_presummed     identical on every rank, since every rank sees the same sums) and phase 3
+ *                               on the local slices.
+ *
+ * gamma (d_ema, n_tensors floats) is replicated: every rank holds and updates the full vector.  The other
+ * arguments are those of adagc_step / adagc_clip.  d_sumsq is read only and must not be the same buffer the
+ * next adagc_shard_sumsq writes before this call's kernels have run (same stream: always fine).
+ * With one rank the three calls compute exactly what adagc_step computes.
+ */
+int adagc_shard_sumsq(adagc_ctx* ctx, const void* d_grads, double* d_sumsq_out, void* cuda_stream);
+int adagc_step_presummed(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, void* d_v,
+                         float* d_ema, const double* d_sumsq, int64_t step, double lr, double beta1,
+                         double beta2, double eps, double wd, double lambda_rel, double beta, int64_t warmup,
+                         void* cuda_stream);
+int adagc_clip_presummed(adagc_ctx* ctx, const void* d_grads_in, void* d_grads_out, float* d_ema,
+                         const double* d_sumsq, int64_t step, double lambda_rel, double beta, int64_t warmup,
+                         void* cuda_stream);
+
+/*
+ * Flat equal shards: the arena [0, arena_elems) of `full` (arena_elems = max offset + numel) is cut into
+ * `world` consecutive ranges of shard_elems = ceil(arena_elems / world) rounded up to a multiple of 8
+ * elements; rank r owns [r * shard_elems, min((r + 1) * shard_elems, arena_elems)).  Writes, for every
+ * tensor i of `full`, this rank's slice into local[i] (n_tensors entries, host memory): numel = elements of
+ * tensor i inside the range (possibly 0), offset = where the slice starts, counted from the start of the
+ * range (so the rank's arenas are the sub-arrays of the full arenas that begin at *elem_begin), ndim = 0.
+ * *elem_begin / *elem_end receive the range; a rank whose range would start at or beyond arena_elems holds
+ * nothing and gets the empty range [0, 0); the three sharded entry points ignore the arena pointers of a
+ * context that holds no element (they may be NULL).  Host-only, no CUDA call.  Returns ADAGC_E_INVALID_ARG for
+ * world < 1 or rank outside [0, world), or the descriptor's own validation error.
+ */
+int adagc_shard_plan(const adagc_desc* full, int32_t rank, int32_t world, adagc_tensor* local,
+                     int64_t* elem_begin, int64_t* elem_end);
 
 /*
  * adagc_step fed from HOST memory: copies the gradient arena `h_grads` (arena_elems elements of the grad

@@ -16,7 +16,7 @@ ADAGC_F32, ADAGC_BF16 = 0, 1
 ADAGC_W_NONFINITE = 1
 ADAGC_E_TIMEOUT = 2
 UPDATE_PATH_AUTO, UPDATE_PATH_REGISTERS, UPDATE_PATH_BULK = 0, 1, 2
-EMA_KEEP_INITIAL, CLIP_GLOBAL_ADAPTIVE = 4, 8
+EMA_KEEP_INITIAL, CLIP_GLOBAL_ADAPTIVE, ALLOW_EMPTY = 4, 8, 16
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libadagc.so")
 _lib = None
@@ -70,6 +70,15 @@ def lib() -> C.CDLL:
     L.adagc_step_host.restype = C.c_int
     L.adagc_step_host.argtypes = [vp, vp, vp, vp, vp, f32p, vp, i64, dbl, dbl, dbl, dbl, dbl, dbl, dbl, i64,
                                   vp, vp, vp, vp]
+    L.adagc_shard_sumsq.restype = C.c_int
+    L.adagc_shard_sumsq.argtypes = [vp, vp, vp, vp]
+    L.adagc_step_presummed.restype = C.c_int
+    L.adagc_step_presummed.argtypes = [vp, vp, vp, vp, vp, f32p, vp, i64, dbl, dbl, dbl, dbl, dbl, dbl, dbl, i64, vp]
+    L.adagc_clip_presummed.restype = C.c_int
+    L.adagc_clip_presummed.argtypes = [vp, vp, vp, f32p, vp, i64, dbl, dbl, i64, vp]
+    L.adagc_shard_plan.restype = C.c_int
+    L.adagc_shard_plan.argtypes = [C.POINTER(adagc_desc), C.c_int32, C.c_int32, C.POINTER(adagc_tensor),
+                                   C.POINTER(i64), C.POINTER(i64)]
     L.adagc_get_stats.restype = C.c_int
     L.adagc_get_stats.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     L.adagc_get_sumsq.restype = C.c_int
@@ -129,6 +138,19 @@ def make_desc(numels: Sequence[int], offsets: Sequence[int], grad_dtype: int, la
     d.lambda_abs = float(lambda_abs)
     d.flags = int(flags)
     return d, arr
+
+
+def shard_plan(numels: Sequence[int], offsets: Sequence[int], grad_dtype: int, rank: int, world: int):
+    """adagc_shard_plan: this rank's slice of every tensor under flat equal shards.
+    Returns (local_numels, local_offsets, elem_begin, elem_end); host-only."""
+    d, keep = make_desc(numels, offsets, grad_dtype)
+    out = (adagc_tensor * max(len(numels), 1))()
+    b, e = C.c_int64(), C.c_int64()
+    rc = lib().adagc_shard_plan(C.byref(d), int(rank), int(world), out, C.byref(b), C.byref(e))
+    if rc != 0:
+        raise AdagcError(rc, "adagc_shard_plan")
+    n = len(numels)
+    return [int(out[i].numel) for i in range(n)], [int(out[i].offset) for i in range(n)], int(b.value), int(e.value)
 
 
 def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
@@ -227,6 +249,31 @@ class AdaGC:
                                    _stream_ptr(stream))
         if rc != 0:
             raise AdagcError(rc, "adagc_step_host")
+
+    def shard_sumsq(self, grads, sumsq_out, stream=None):
+        assert grads.dtype == self.grad_dtype and sumsq_out.dtype == torch.float64 and sumsq_out.is_cuda
+        assert sumsq_out.numel() >= self.n_tensors and sumsq_out.is_contiguous()
+        rc = lib().adagc_shard_sumsq(self._h, _ptr(grads), _ptr(sumsq_out), _stream_ptr(stream))
+        if rc != 0:
+            raise AdagcError(rc, "adagc_shard_sumsq")
+
+    def step_presummed(self, params, grads, m, v, ema, sumsq, step, lr, beta1, beta2, eps, wd, lambda_rel, beta,
+                       warmup, stream=None):
+        assert grads.dtype == self.grad_dtype and params.dtype == m.dtype == v.dtype == ema.dtype == torch.float32
+        assert sumsq.dtype == torch.float64 and sumsq.is_cuda and sumsq.numel() >= self.n_tensors
+        rc = lib().adagc_step_presummed(self._h, _ptr(params), _ptr(grads), _ptr(m), _ptr(v), _ptr(ema), _ptr(sumsq),
+                                        int(step), lr, beta1, beta2, eps, wd, lambda_rel, beta, int(warmup),
+                                        _stream_ptr(stream))
+        if rc != 0:
+            raise AdagcError(rc, "adagc_step_presummed")
+
+    def clip_presummed(self, grads_in, grads_out, ema, sumsq, step, lambda_rel, beta, warmup, stream=None):
+        assert grads_in.dtype == grads_out.dtype == self.grad_dtype and ema.dtype == torch.float32
+        assert sumsq.dtype == torch.float64 and sumsq.is_cuda and sumsq.numel() >= self.n_tensors
+        rc = lib().adagc_clip_presummed(self._h, _ptr(grads_in), _ptr(grads_out), _ptr(ema), _ptr(sumsq), int(step),
+                                        lambda_rel, beta, int(warmup), _stream_ptr(stream))
+        if rc != 0:
+            raise AdagcError(rc, "adagc_clip_presummed")
 
     def get_stats(self, stream=None):
         T = self.n_tensors

@@ -257,6 +257,22 @@ adagc_tensor_finalize_kernel(const double* __restrict__ partials, const TensorEn
   }
 }
 
+// Sharded use: the per-tensor sums of squares arrive already summed over the ranks that hold parts of each
+// tensor (Section 4.3 "Communication": one all-reduce of the partial sums), so phase 2 starts from them.
+// One thread per tensor.
+__global__ void __launch_bounds__(kFinalizeThreads)
+adagc_presummed_finalize_kernel(const double* __restrict__ sumsq_in, ClipScalars cs, int decide,
+                                float* __restrict__ ema, StatPtrs st) {
+  const int i = blockIdx.x * kFinalizeThreads + threadIdx.x;
+  if (i >= cs.n_tensors) return;
+  const double s = sumsq_in[i];
+  st.sumsq[i] = s;
+  if (decide) {
+    adagc_decide(i, s, cs, ema, st);
+    if (i == 0) *st.steps_done += 1ull;
+  }
+}
+
 // Warm-up branch of Algorithm 1: global norm (Eq. 2), one clip factor for every tensor, and
 // gamma_t,i = min{gamma_t-1,i, ||hat(g)_t,i||} with gamma_0,i = ||hat(g)_1,i||.  One block.
 __global__ void __launch_bounds__(kWarmupThreads)
@@ -830,7 +846,9 @@ int validate_desc(const adagc_desc* d, int64_t* n_chunks_out, int64_t* arena_ele
   if (d->param_dtype != ADAGC_F32 || d->state_dtype != ADAGC_F32) return ADAGC_E_DTYPE;
   if (d->grad_dtype != ADAGC_F32 && d->grad_dtype != ADAGC_BF16) return ADAGC_E_DTYPE;
   if (!(d->lambda_abs > 0.0) || !std::isfinite(d->lambda_abs)) return ADAGC_E_INVALID_ARG;
-  constexpr int kKnownFlags = ADAGC_UPDATE_PATH_MASK | ADAGC_EMA_KEEP_INITIAL | ADAGC_CLIP_GLOBAL_ADAPTIVE;
+  constexpr int kKnownFlags =
+      ADAGC_UPDATE_PATH_MASK | ADAGC_EMA_KEEP_INITIAL | ADAGC_CLIP_GLOBAL_ADAPTIVE | ADAGC_ALLOW_EMPTY;
+  const bool allow_empty = (d->flags & ADAGC_ALLOW_EMPTY) != 0;
   if ((d->flags & ~kKnownFlags) != 0 || (d->flags & ADAGC_UPDATE_PATH_MASK) == 3) return ADAGC_E_INVALID_ARG;
   const int64_t align = (d->grad_dtype == ADAGC_BF16) ? 8 : 4;
   int64_t n_chunks = 0, extent = 0;
@@ -838,6 +856,7 @@ int validate_desc(const adagc_desc* d, int64_t* n_chunks_out, int64_t* arena_ele
   spans.reserve(d->n_tensors);
   for (int32_t i = 0; i < d->n_tensors; ++i) {
     const adagc_tensor& t = d->tensors[i];
+    if (allow_empty && t.numel == 0) continue;  // this rank holds nothing of the tensor; its offset is ignored
     if (t.numel <= 0 || t.offset < 0 || t.ndim < 0 || t.ndim > 4) return ADAGC_E_INVALID_ARG;
     if (t.numel > (int64_t(1) << 34) || t.offset + t.numel > (int64_t(1) << 34)) return ADAGC_E_INVALID_ARG;
     if (t.ndim > 0) {
@@ -1043,12 +1062,15 @@ AdamScalars make_adam_scalars(int64_t step, double lr, double beta1, double beta
   return a;
 }
 
+// need_arenas = false: the context holds no element (a rank of a sharded model that owns nothing), so the arena
+// pointers are never dereferenced and may be anything, NULL included.
 int check_adamw_args(const void* d_params, const void* d_grads, const void* d_m, const void* d_v, double lr,
-                     double beta1, double beta2, double eps, double wd) {
-  if (!d_params || !d_grads || !d_m || !d_v) return ADAGC_E_INVALID_ARG;
+                     double beta1, double beta2, double eps, double wd, bool need_arenas = true) {
+  if (need_arenas && (!d_params || !d_grads || !d_m || !d_v)) return ADAGC_E_INVALID_ARG;
   if (!(beta1 >= 0.0 && beta1 < 1.0) || !(beta2 >= 0.0 && beta2 < 1.0)) return ADAGC_E_INVALID_ARG;
   if (!(eps >= 0.0) || !std::isfinite(eps) || !std::isfinite(lr) || !std::isfinite(wd)) return ADAGC_E_INVALID_ARG;
-  if (!aligned16(d_params) || !aligned16(d_grads) || !aligned16(d_m) || !aligned16(d_v)) return ADAGC_E_MISALIGNED;
+  if (need_arenas && (!aligned16(d_params) || !aligned16(d_grads) || !aligned16(d_m) || !aligned16(d_v)))
+    return ADAGC_E_MISALIGNED;
   return ADAGC_OK;
 }
 
@@ -1076,6 +1098,42 @@ int enqueue_clip_phases(adagc_ctx* ctx, const void* d_grads, float* d_ema, int64
   }
   if (ctx->timing) cudaEventRecord(ctx->ev[2], s);
   return ADAGC_OK;
+}
+
+// Phase 2 from per-tensor sums of squares the caller provides (already summed over the ranks of a sharded model).
+void enqueue_presummed_phase(adagc_ctx* ctx, const double* d_sumsq, float* d_ema, int64_t step, double lambda_rel,
+                             double beta, int64_t warmup, cudaStream_t s) {
+  if (ctx->timing) {
+    cudaEventRecord(ctx->ev[0], s);
+    cudaEventRecord(ctx->ev[1], s);  // no norm phase in this call
+  }
+  const ClipScalars cs = make_clip_scalars(ctx, step, lambda_rel, beta);
+  const bool in_warmup = step <= warmup;
+  const bool per_tensor = !in_warmup && !ctx->global_adaptive;
+  const int blocks = (ctx->T + kFinalizeThreads - 1) / kFinalizeThreads;
+  adagc_presummed_finalize_kernel<<<blocks, kFinalizeThreads, 0, s>>>(d_sumsq, cs, per_tensor ? 1 : 0, d_ema,
+                                                                     ctx->stats());
+  ctx->launches++;
+  if (ctx->global_adaptive) {
+    adagc_global_finalize_kernel<<<1, kWarmupThreads, 0, s>>>(cs, in_warmup ? 1 : 0, d_ema, ctx->stats());
+    ctx->launches++;
+  } else if (in_warmup) {
+    adagc_warmup_finalize_kernel<<<1, kWarmupThreads, 0, s>>>(cs, d_ema, ctx->stats());
+    ctx->launches++;
+  }
+  if (ctx->timing) cudaEventRecord(ctx->ev[2], s);
+}
+
+// Clip-only phase 3: hat(g) = h g in the gradient dtype.
+void launch_scale(adagc_ctx* ctx, const void* d_grads_in, void* d_grads_out, cudaStream_t s) {
+  const int in_place = d_grads_in == d_grads_out ? 1 : 0;
+  if (ctx->bf16)
+    adagc_scale_kernel<true><<<ctx->grid_wide, kThreads, 0, s>>>(d_grads_in, d_grads_out, ctx->d_chunks_wide(),
+                                                                ctx->d_begin_wide(), ctx->stats().h, in_place);
+  else
+    adagc_scale_kernel<false><<<ctx->grid_wide, kThreads, 0, s>>>(d_grads_in, d_grads_out, ctx->d_chunks_wide(),
+                                                                 ctx->d_begin_wide(), ctx->stats().h, in_place);
+  ctx->launches++;
 }
 
 // Norm, finalize and AdamW update of an AdaGC step (step > warmup), one group of tensors after the other.
@@ -1182,7 +1240,11 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
   ctx->arena_elems = extent;
   ctx->bf16 = desc->grad_dtype == ADAGC_BF16;
   ctx->lambda_abs = desc->lambda_abs;
-  for (int32_t i = 0; i < desc->n_tensors; ++i) ctx->offsets_mult8 = ctx->offsets_mult8 && desc->tensors[i].offset % 8 == 0;
+  bool any_empty = false;
+  for (int32_t i = 0; i < desc->n_tensors; ++i) {
+    if (desc->tensors[i].numel == 0) any_empty = true;
+    else ctx->offsets_mult8 = ctx->offsets_mult8 && desc->tensors[i].offset % 8 == 0;
+  }
   ctx->ws = static_cast<char*>(d_workspace);
   ctx->L = L;
 
@@ -1218,24 +1280,22 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
     balance_chunks(chunks, ctx->grid_wide, &table_wide, &begin_wide);
     balance_chunks(chunks, ctx->grid_update, &table_upd, &begin_upd, &mid_upd);
   }
+  auto upload = [&](size_t off, const void* src, size_t bytes) {
+    if (bytes == 0) return;  // a rank of a sharded model may hold no chunk at all
+    ok = ok && cudaMemcpyAsync(ctx->ws + off, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
+  };
   ok = ok && cudaMemsetAsync(ctx->ws, 0, L.total, s) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(ctx->ws + L.chunks_wide, table_wide.data(), sizeof(Chunk) * table_wide.size(),
-                             cudaMemcpyHostToDevice, s) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(ctx->ws + L.chunks_upd, table_upd.data(), sizeof(Chunk) * table_upd.size(),
-                             cudaMemcpyHostToDevice, s) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(ctx->ws + L.begin_wide, begin_wide.data(), sizeof(int32_t) * begin_wide.size(),
-                             cudaMemcpyHostToDevice, s) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(ctx->ws + L.begin_upd, begin_upd.data(), sizeof(int32_t) * begin_upd.size(),
-                             cudaMemcpyHostToDevice, s) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(ctx->ws + L.mid_upd, mid_upd.data(), sizeof(int32_t) * mid_upd.size(),
-                             cudaMemcpyHostToDevice, s) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(ctx->ws + L.tensors, tensors.data(), sizeof(TensorEntry) * tensors.size(),
-                             cudaMemcpyHostToDevice, s) == cudaSuccess;
+  upload(L.chunks_wide, table_wide.data(), sizeof(Chunk) * table_wide.size());
+  upload(L.chunks_upd, table_upd.data(), sizeof(Chunk) * table_upd.size());
+  upload(L.begin_wide, begin_wide.data(), sizeof(int32_t) * begin_wide.size());
+  upload(L.begin_upd, begin_upd.data(), sizeof(int32_t) * begin_upd.size());
+  upload(L.mid_upd, mid_upd.data(), sizeof(int32_t) * mid_upd.size());
+  upload(L.tensors, tensors.data(), sizeof(TensorEntry) * tensors.size());
   // groups of tensors (arena order) for the pipelined host step, each with its own balanced tables
   std::vector<Chunk> g_table_wide, g_table_upd;
   std::vector<int32_t> g_begin_wide(static_cast<size_t>(kMaxGroups) * (kGroupMaxGrid + 1), 0), g_begin_upd = g_begin_wide,
                        g_mid_upd = g_begin_wide, g_order(desc->n_tensors);
-  if (ok) {
+  if (ok && !any_empty) {  // (a shard that lists tensors it holds nothing of takes the unpipelined host step)
     const int64_t esz = ctx->bf16 ? 2 : 4;
     for (int32_t i = 0; i < desc->n_tensors; ++i) g_order[i] = i;
     std::sort(g_order.begin(), g_order.end(),
@@ -1279,9 +1339,6 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
       ctx->groups.push_back(gr);
     }
   }
-  auto upload = [&](size_t off, const void* src, size_t bytes) {
-    ok = ok && cudaMemcpyAsync(ctx->ws + off, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
-  };
   upload(L.g_chunks_wide, g_table_wide.data(), sizeof(Chunk) * g_table_wide.size());
   upload(L.g_chunks_upd, g_table_upd.data(), sizeof(Chunk) * g_table_upd.size());
   upload(L.g_begin_wide, g_begin_wide.data(), sizeof(int32_t) * g_begin_wide.size());
@@ -1412,15 +1469,89 @@ int adagc_clip(adagc_ctx* ctx, const void* d_grads_in, void* d_grads_out, float*
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   rc = enqueue_clip_phases(ctx, d_grads_in, d_ema, step, lambda_rel, beta, warmup, s);
   if (rc != ADAGC_OK) return rc;
-  const int in_place = d_grads_in == d_grads_out ? 1 : 0;
-  if (ctx->bf16)
-    adagc_scale_kernel<true><<<ctx->grid_wide, kThreads, 0, s>>>(d_grads_in, d_grads_out, ctx->d_chunks_wide(),
-                                                                ctx->d_begin_wide(), ctx->stats().h, in_place);
-  else
-    adagc_scale_kernel<false><<<ctx->grid_wide, kThreads, 0, s>>>(d_grads_in, d_grads_out, ctx->d_chunks_wide(),
-                                                                 ctx->d_begin_wide(), ctx->stats().h, in_place);
-  ctx->launches++;
+  launch_scale(ctx, d_grads_in, d_grads_out, s);
   return finish_launches(ctx, s);
+}
+
+int adagc_shard_sumsq(adagc_ctx* ctx, const void* d_grads, double* d_sumsq_out, void* cuda_stream) {
+  if (!ctx || !d_sumsq_out) return ADAGC_E_INVALID_ARG;
+  const bool holds = ctx->n_chunks > 0;  // a rank that owns nothing may pass any gradient pointer, NULL included
+  if (holds && !d_grads) return ADAGC_E_INVALID_ARG;
+  if ((holds && !aligned16(d_grads)) || (reinterpret_cast<uintptr_t>(d_sumsq_out) & 7u)) return ADAGC_E_MISALIGNED;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return ADAGC_E_CUDA;
+  if (dev != ctx->device) return ADAGC_E_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  const TableView wide = {ctx->d_chunks_wide(), ctx->d_begin_wide(), nullptr, ctx->grid_wide};
+  launch_norm(ctx, wide, d_grads, s);
+  // the same fixed-order per-tensor sum as the unsharded step, written to the caller's vector; no decision
+  StatPtrs st = ctx->stats();
+  st.sumsq = d_sumsq_out;
+  const int blocks = (ctx->T * 32 + kFinalizeThreads - 1) / kFinalizeThreads;
+  adagc_tensor_finalize_kernel<<<blocks, kFinalizeThreads, 0, s>>>(ctx->d_partials(), ctx->d_tensors(), ClipScalars{},
+                                                                  0, nullptr, st, nullptr, 0, ctx->T, 0);
+  ctx->launches++;
+  return cudaGetLastError() == cudaSuccess ? ADAGC_OK : ADAGC_E_CUDA;
+}
+
+int adagc_step_presummed(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, void* d_v, float* d_ema,
+                         const double* d_sumsq, int64_t step, double lr, double beta1, double beta2, double eps,
+                         double wd, double lambda_rel, double beta, int64_t warmup, void* cuda_stream) {
+  int rc = check_clip_args(ctx, d_ema, step, lambda_rel, beta, warmup);
+  if (rc != ADAGC_OK) return rc;
+  rc = check_adamw_args(d_params, d_grads, d_m, d_v, lr, beta1, beta2, eps, wd, ctx->n_chunks > 0);
+  if (rc != ADAGC_OK) return rc;
+  if (!d_sumsq) return ADAGC_E_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(d_sumsq) & 7u) return ADAGC_E_MISALIGNED;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  enqueue_presummed_phase(ctx, d_sumsq, d_ema, step, lambda_rel, beta, warmup, s);
+  const AdamScalars a = make_adam_scalars(step, lr, beta1, beta2, eps, wd);
+  if (ctx->bf16)
+    launch_update<true, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
+                                   static_cast<float*>(d_v), a, s);
+  else
+    launch_update<false, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
+                                    static_cast<float*>(d_v), a, s);
+  return finish_launches(ctx, s);
+}
+
+int adagc_clip_presummed(adagc_ctx* ctx, const void* d_grads_in, void* d_grads_out, float* d_ema,
+                         const double* d_sumsq, int64_t step, double lambda_rel, double beta, int64_t warmup,
+                         void* cuda_stream) {
+  int rc = check_clip_args(ctx, d_ema, step, lambda_rel, beta, warmup);
+  if (rc != ADAGC_OK) return rc;
+  const bool holds = ctx->n_chunks > 0;
+  if ((holds && (!d_grads_in || !d_grads_out)) || !d_sumsq) return ADAGC_E_INVALID_ARG;
+  if ((holds && (!aligned16(d_grads_in) || !aligned16(d_grads_out))) || (reinterpret_cast<uintptr_t>(d_sumsq) & 7u))
+    return ADAGC_E_MISALIGNED;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  enqueue_presummed_phase(ctx, d_sumsq, d_ema, step, lambda_rel, beta, warmup, s);
+  launch_scale(ctx, d_grads_in, d_grads_out, s);
+  return finish_launches(ctx, s);
+}
+
+int adagc_shard_plan(const adagc_desc* full, int32_t rank, int32_t world, adagc_tensor* local, int64_t* elem_begin,
+                     int64_t* elem_end) {
+  int64_t extent = 0;
+  const int rc = validate_desc(full, nullptr, &extent);
+  if (rc != ADAGC_OK) return rc;
+  if (!local || world < 1 || rank < 0 || rank >= world) return ADAGC_E_INVALID_ARG;
+  const int64_t shard = ((extent + world - 1) / world + 7) / 8 * 8;
+  int64_t b = std::min<int64_t>(extent, shard * rank), e = std::min<int64_t>(extent, shard * (rank + 1));
+  if (b == e) b = e = 0;  // a rank beyond the end of a small arena holds nothing: the empty range at the start
+  for (int32_t i = 0; i < full->n_tensors; ++i) {
+    const adagc_tensor& t = full->tensors[i];
+    const int64_t lo = std::max<int64_t>(t.offset, b), hi = std::min<int64_t>(t.offset + t.numel, e);
+    adagc_tensor out = {};
+    if (t.numel > 0 && hi > lo) {
+      out.numel = hi - lo;
+      out.offset = lo - b;
+    }
+    local[i] = out;
+  }
+  if (elem_begin) *elem_begin = b;
+  if (elem_end) *elem_end = e;
+  return ADAGC_OK;
 }
 
 int adagc_get_stats(adagc_ctx* ctx, float* h_norm, float* h_clipfactor, uint8_t* h_flag, uint64_t* h_clip_count,

@@ -389,3 +389,81 @@ def run_full_sgdm(wl: workloads.Workload, n_steps: int, device="cuda", flags: in
     assert opt.get_stats()["status"] == 0
     opt.close()
     return rep
+
+
+def run_full_sharded(wl: workloads.Workload, n_steps: int, world: int, device="cuda", mode: str = "adamw",
+                     hyper_over: Optional[dict] = None, flags: int = 0) -> ParityReport:
+    """The sharded step (adagc_shard_sumsq -> sum over ranks -> adagc_step_presummed / adagc_clip_presummed)
+    with `world` ranks emulated one after the other on one GPU, every element against the UNSHARDED C oracle.
+    Each rank has its own context over its slices (adagc_shard_plan), its own exchange buffer and its own
+    replica of gamma; the ranks' partial sums are added in rank order, which is what an all-reduce computes."""
+    from paper_2502_11034_b200 import sharded
+    hp = hyper_of(wl, **(hyper_over or {}))
+    offs = [t.offset for t in wl.tensors]
+    nums = [t.numel for t in wl.tensors]
+    ranks = [sharded.ShardedAdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], r, world, device=device,
+                                  flags=flags) for r in range(world)]
+    assert ranks[0].elem_begin == 0 and max(rk.elem_end for rk in ranks) == max(o + n for o, n in zip(offs, nums))
+    theta = workloads.init_params(wl, device)
+    theta0 = theta.cpu().numpy().copy()
+    pad = np.ones(wl.arena_elems, bool)
+    for o, n in zip(offs, nums):
+        pad[o:o + n] = False
+    pad_mask = torch.from_numpy(pad).to(device)
+    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    for a in (theta, m, v):
+        a[pad_mask] = 777.0
+    emas = [torch.full((wl.n_tensors,), float("nan"), dtype=torch.float32, device=device) for _ in ranks]
+    ref = c_oracle.ArenaOracle(offs, nums, theta0, lr=hp["lr"], beta1=hp["beta1"], beta2=hp["beta2"],
+                               eps=hp["eps"], wd=hp["wd"], lambda_rel=hp["lambda_rel"], beta=hp["beta"],
+                               lambda_abs=hp["lambda_abs"], warmup=hp["warmup"],
+                               global_adaptive=bool(flags & binding.CLIP_GLOBAL_ADAPTIVE))
+    gamma_ref = np.zeros(wl.n_tensors, np.float32)
+    rep = ParityReport()
+    for t in range(1, n_steps + 1):
+        g = workloads.grads_for_step(wl, t, device)
+        g_np = to_numpy_grads(g).copy()
+        out = g if mode == "clip_in_place" else (torch.full_like(g, 7.0) if mode == "clip" else None)
+        parts = [rk.local_sumsq(g[rk.elem_begin:rk.elem_end]).clone() for rk in ranks]
+        total = parts[0].clone()
+        for p in parts[1:]:
+            total += p                                       # stands in for the all-reduce over the ranks
+        for rk, ema in zip(ranks, emas):
+            b, e = rk.elem_begin, rk.elem_end
+            rk.sumsq.copy_(total)
+            if mode == "adamw":
+                rk.opt.step_presummed(theta[b:e], g[b:e], m[b:e], v[b:e], ema, rk.sumsq, t, hp["lr"], hp["beta1"],
+                                      hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"], hp["beta"], hp["warmup"])
+            else:
+                rk.opt.clip_presummed(g[b:e], out[b:e], ema, rk.sumsq, t, hp["lambda_rel"], hp["beta"], hp["warmup"])
+        if mode == "adamw":
+            r = ref.step(g_np)
+        else:
+            ssq = c_oracle.sumsq_tensors(g_np, offs, nums)
+            r = c_oracle.clip_decisions(ssq, gamma_ref, t, hp["lambda_rel"], hp["beta"], hp["lambda_abs"], hp["warmup"])
+        stats = [rk.opt.get_stats() for rk in ranks]
+        check_decisions(stats[0], total.cpu().numpy(), emas[0].cpu().numpy(), r, rep, t)
+        for st, ema in zip(stats[1:], emas[1:]):             # every rank took the same decisions, bit for bit
+            assert np.array_equal(st["flag"], stats[0]["flag"]) and np.array_equal(st["h"], stats[0]["h"])
+            assert torch.equal(ema, emas[0]) and np.array_equal(st["clip_count"], stats[0]["clip_count"])
+            assert st["steps_done"] == t and st["status"] == 0
+        if mode != "adamw":
+            got = to_numpy_grads(out)
+            for i, (o, n) in enumerate(zip(offs, nums)):
+                want = c_oracle.scale(np.ascontiguousarray(g_np[o:o + n]), float(r["h"][i]))
+                check_clipped_grads(got[o:o + n], want, f"step {t}, tensor {wl.tensors[i].name}")
+            if mode == "clip":
+                assert bool((out[pad_mask].float() == 7.0).all()), "padding between tensors was written"
+        rep.steps = t
+    if mode == "adamw":
+        th, mm, vv = theta.cpu().numpy(), m.cpu().numpy(), v.cpu().numpy()
+        for t_, o, n in zip(wl.tensors, offs, nums):
+            check_state("theta", th[o:o + n], ref.theta[o:o + n], rep, t_.name)
+            check_state("m", mm[o:o + n], ref.m[o:o + n], rep, t_.name)
+            check_state("v", vv[o:o + n], ref.v[o:o + n], rep, t_.name)
+        assert np.array_equal(stats[0]["clip_count"], ref.clip_count)
+        for a in (theta, m, v):
+            assert bool((a[pad_mask] == 777.0).all()), "guard bands between tensors were overwritten"
+    for rk in ranks:
+        rk.close()
+    return rep

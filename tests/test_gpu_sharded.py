@@ -1,0 +1,108 @@
+"""GPU parity of the sharded step: tensors cut over several ranks (flat equal shards), per-rank sums of
+squares, one sum over the ranks, then decisions and updates on every rank -- against the UNSHARDED oracle.
+
+Section 4.3 ("Communication") of the paper: a split tensor needs one all-reduce of partial sums of squares
+for its norm.  One GPU is available to these tests, so the ranks run one after the other on it, each through
+its own context, and their partial sums are added in rank order (the result an all-reduce delivers); no
+kernel waits on another.  Bar: as for the unsharded step (flags and counters bit-exact, norms / gamma / h /
+fp32 state 1e-5, bf16 clipped gradients one ulp); the float64 sums of squares agree to 1e-11."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2502_11034_b200 import binding, sharded, workloads
+
+import parity_harness as H
+
+pytestmark = pytest.mark.gpu
+
+
+def _ragged(sizes, dtype):
+    specs, total = workloads._layout([(f"t{i}", (n,)) for i, n in enumerate(sizes)])
+    hp = dict(workloads.PAPER_DEFAULTS, lambda_abs=0.05)
+    return workloads.Workload("ragged", 7, specs, dtype, hp, warmup=2, n_steps=8, arena_elems=total,
+                              grad_kind="student_t", grad_df=3, grad_scale=1e-3,
+                              extra={"spike_frac": 0.2, "spike_lo": 5.0, "spike_hi": 500.0})
+
+
+@pytest.mark.parametrize("world", [1, 2, 3, 8])
+def test_sharded_adamw_small_layouts_all_elements(world):
+    for name, over, hov in [("llama2_7b", dict(n_layer=2, d=256, ffn=688, vocab=1000), dict(lambda_abs=1e4)),
+                            ("many_small", dict(n_tensors=300, lo=1, hi=40000), dict(lambda_abs=1e4)),
+                            ("tiny", {}, dict(lambda_abs=0.5))]:
+        wl = workloads.build(name, **over)
+        rep = H.run_full_sharded(wl, 12, world, hyper_over=hov)
+        print(f"\n[parity] sharded x{world} {name}: {rep.line()}")
+        assert rep.clipped > 0
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_sharded_ragged_cuts_and_empty_ranks(dtype):
+    """Shard boundaries that fall inside tensors, on tensor starts, one element before / after chunk edges;
+    and more ranks than 8-element blocks, so that some ranks hold nothing at all."""
+    sizes = [1, 7, 8, 9, 255, 2049, 16384, 16385, 3 * 16384 + 5, 100003, 40 * 16384]
+    for world in (2, 5, 7):
+        rep = H.run_full_sharded(_ragged(sizes, dtype), 6, world)
+        print(f"\n[parity] sharded ragged {dtype} x{world}: {rep.line()}")
+    rep = H.run_full_sharded(_ragged([5, 3, 20], dtype), 5, 16)     # arena of 36 elements over 16 ranks
+    assert rep.steps == 5
+
+
+@pytest.mark.parametrize("mode", ["clip", "clip_in_place"])
+def test_sharded_clip_only_all_elements(mode):
+    for name, over, hov in [("llama32_1b", dict(n_layer=2, d=128, ffn=512, vocab=2000, kv_dim=32), dict(lambda_abs=1e4)),
+                            ("many_small", dict(n_tensors=300, lo=1, hi=40000), dict(lambda_abs=1e4))]:
+        wl = workloads.build(name, **over)
+        rep = H.run_full_sharded(wl, 13, 3, mode=mode, hyper_over=hov)
+        print(f"\n[parity] sharded {mode} {name}: {rep.line()}")
+        assert rep.clipped > 0
+
+
+def test_sharded_global_adaptive_variant():
+    wl = workloads.build("llama2_7b", n_layer=2, d=256, ffn=688, vocab=1000)
+    rep = H.run_full_sharded(wl, 10, 4, flags=binding.CLIP_GLOBAL_ADAPTIVE, hyper_over=dict(lambda_abs=1e4))
+    assert rep.steps == 10
+
+
+def test_one_rank_equals_the_unsharded_entry_bit_for_bit():
+    """With a single rank the three calls compute exactly what adagc_step computes."""
+    wl = workloads.build("gpt2_small", n_layer=2, d=96, vocab=1031, n_pos=64)
+    hp = H.hyper_of(wl, lambda_abs=1e4)
+    offs, nums = [t.offset for t in wl.tensors], [t.numel for t in wl.tensors]
+    res = []
+    for use_sharded in (False, True):
+        theta = workloads.init_params(wl, "cuda")
+        m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+        ema = torch.zeros(wl.n_tensors, device="cuda")
+        if use_sharded:
+            opt = sharded.ShardedAdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], 0, 1)
+            assert (opt.elem_begin, opt.elem_end) == (0, wl.arena_elems) and opt.local_numels == nums
+        else:
+            opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"])
+        for t in range(1, 9):
+            g = workloads.grads_for_step(wl, t, "cuda")
+            opt.step(theta, g, m, v, ema, t, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"],
+                     hp["lambda_rel"], hp["beta"], hp["warmup"])
+        st = (opt.opt if use_sharded else opt).get_stats()
+        res.append((theta.clone(), m.clone(), v.clone(), ema.clone(), st))
+        opt.close()
+    for a, b in zip(res[0][:4], res[1][:4]):
+        assert torch.equal(a, b)
+    assert np.array_equal(res[0][4]["clip_count"], res[1][4]["clip_count"]) and res[1][4]["steps_done"] == 8
+
+
+def test_presummed_argument_errors():
+    opt = binding.AdaGC([100, 60], [0, 104], torch.float32, 1.0, flags=binding.ALLOW_EMPTY)
+    z = torch.zeros(164, device="cuda")
+    ema = torch.zeros(2, device="cuda")
+    s = torch.zeros(2, dtype=torch.float64, device="cuda")
+    lib = binding.lib()
+    sp = binding._stream_ptr(None)
+    assert lib.adagc_shard_sumsq(opt._h, z.data_ptr(), None, sp) == -1
+    assert lib.adagc_shard_sumsq(opt._h, z.data_ptr() + 4, s.data_ptr(), sp) == -2
+    assert lib.adagc_step_presummed(opt._h, z.data_ptr(), z.data_ptr(), z.data_ptr(), z.data_ptr(), ema.data_ptr(), None,
+                                    1, 1e-3, 0.9, 0.95, 1e-8, 0.1, 1.04, 0.99, 0, sp) == -1
+    assert lib.adagc_clip_presummed(opt._h, z.data_ptr(), z.data_ptr(), ema.data_ptr(), s.data_ptr(), 0, 1.04, 0.99, 0,
+                                    sp) == -1
+    assert opt.launch_count() == 0
+    opt.close()

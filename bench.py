@@ -184,7 +184,13 @@ def time_oracle(wl, steps: int, warm: int):
     for _ in range(steps):
         ref.step(g)
     dt = time.perf_counter() - t0
-    info = {"kind": "oracle", "cores": c_oracle.num_threads(),
+    cpu_model = None
+    try:
+        with open("/proc/cpuinfo") as f:
+            cpu_model = next((ln.split(":", 1)[1].strip() for ln in f if ln.startswith("model name")), None)
+    except OSError:
+        pass
+    info = {"kind": "oracle", "cores": c_oracle.num_threads(), "cpu_model": cpu_model,
             "sample": f"{steps} step(s) of the C oracle over {len(picked)} tensors "
                       f"({picked[0].name}..{picked[-1].name}, {tot} params) of {wl.name}"}
     return tot * steps / dt, dt / steps, info
@@ -385,6 +391,89 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+def run_sharded(args, wl):
+    """--parallel sharded: the layout's arenas cut into N flat shards, one per rank; each step is
+    adagc_shard_sumsq -> all-reduce of n_tensors float64 (NCCL) -> adagc_step_presummed.  Total work is fixed as N
+    grows (strong scaling); with N = 1 it measures what the split of the step costs."""
+    from paper_2502_11034_b200 import binding, sharded, workloads
+    import torch.distributed as dist
+
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    hp = wl.hyper
+    offs, nums = [t.offset for t in wl.tensors], [t.numel for t in wl.tensors]
+    opt = sharded.ShardedAdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], rank, world, device=dev)
+    n_local = max(opt.local_elems, 8)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(workloads.BASE_SEED + rank)
+    theta = torch.empty(n_local, device=dev).normal_(0.0, 0.02, generator=gen)
+    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    g = torch.empty(n_local, device=dev).normal_(0.0, wl.grad_scale, generator=gen).to(wl.torch_grad_dtype)
+    ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device=dev)
+    args_h = (hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"], hp["beta"])
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if n_local * 14 <= (1 << 30) else None
+    t = 0
+
+    def one_step():
+        nonlocal t
+        t += 1
+        if flush is not None:
+            flush.fill_(t & 0xFF)
+        opt.step(theta, g, m, v, ema, t, *args_h, 1)
+
+    def sync_all():
+        torch.cuda.synchronize(dev)
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize(dev)
+
+    n_warm = max(args.warmup, 3)
+    for _ in range(n_warm):
+        one_step()
+    sync_all()
+    sampler = ClockSampler(local) if rank == 0 else None
+    if sampler:
+        sampler.start()
+    launches0 = opt.opt.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    e0.record()
+    for _ in range(args.steps):
+        one_step()
+    e1.record()
+    e1.synchronize()
+    seconds = e0.elapsed_time(e1) * 1e-3
+    sync_all()
+    clocks = sampler.stop() if sampler else None
+    seconds_max = max_over_ranks(seconds, dev)
+    st = opt.opt.get_stats()
+    assert st["status"] == 0 and st["steps_done"] == t
+    if rank == 0:
+        peak, peak_kind = measured_peak()
+        bpp = bytes_per_param(wl)
+        step_s = seconds_max / args.steps
+        line = {"metric": METRIC, "value": wl.n_params * args.steps / seconds_max, "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": n_warm, "ms_per_step": step_s * 1e3, "higher_is_better": True,
+                "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": dict(workload_config(wl), parallelism=f"flat shards x{world}, one all-reduce of "
+                                                                f"{wl.n_tensors} float64 per step"),
+                "clocks": clocks, "gpu_launches": int(opt.opt.launch_count() - launches0),
+                "roofline": {"bound": "hbm", "kernel": "whole sharded step", "unit": "GB/s", "peak": peak,
+                             "peak_source": f"of {peak_kind}",
+                             "achieved": bpp * wl.n_params / world / step_s / 1e9,
+                             "frac": bpp * wl.n_params / world / step_s / 1e9 / peak, "traffic": None}}
+        print(json.dumps(line), flush=True)
+    opt.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def pick_workload(args):
     from paper_2502_11034_b200 import workloads
     if args.workload:
@@ -405,10 +494,14 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default=None, help="tiny | gpt2_small | llama2_7b | many_small | llama32_1b | moe_8x1b")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--parallel", choices=["replicas", "sharded"], default="replicas",
+                    help="N > 1: independent replicas (default; the data-parallel case) or flat shards of one model")
     args = ap.parse_args()
     wl = pick_workload(args)
     if args.impl == "reference":
         run_reference(args, wl)
+    elif args.parallel == "sharded":
+        run_sharded(args, wl)
     else:
         run_ours(args, wl)
 

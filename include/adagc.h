@@ -253,6 +253,17 @@ int adagc_get_stats(adagc_ctx* ctx, float* h_norm, float* h_clipfactor, uint8_t*
  * Synchronises the stream. */
 int adagc_get_sumsq(adagc_ctx* ctx, double* h_sumsq, void* cuda_stream);
 
+/*
+ * "Thresholded initialization", variant 3 of the paper's EMA-initialization ablation (Section 5: gamma_t,i =
+ * min(||g_t,i||, 0.1)).  With cap > 0, every place where the default seeds gamma (step 1) or takes the running
+ * minimum (warm-up steps) sets gamma_t,i = min(||hat(g)_t,i||, cap) instead: the constant stands where
+ * gamma_t-1,i stands in Algorithm 1's warm-up line, so after warm-up gamma is the last warm-up step's clipped
+ * norm, capped.  With T_start = 0 the seed of step 1 is min(||g_1,i||, cap) and Eq. 3 applies to it at once.
+ * AdaGC steps after the first are unchanged.  cap = 0 (the default) switches the variant off.  Host-only; takes
+ * effect from the next step.  Returns ADAGC_E_INVALID_ARG for a negative or non-finite cap.
+ */
+int adagc_set_ema_cap(adagc_ctx* ctx, double cap);
+
 /* The update path this context uses: ADAGC_UPDATE_PATH_REGISTERS or ADAGC_UPDATE_PATH_BULK. */
 int adagc_update_path(const adagc_ctx* ctx);
 

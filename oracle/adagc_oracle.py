@@ -76,7 +76,7 @@ def l2_norm(g: np.ndarray) -> float:
 
 def clip_decisions(s: Sequence[float], gamma_prev: np.ndarray, step: int, hp: Hyper,
                    state_dtype=np.float32, keep_initial: bool = False,
-                   global_adaptive: bool = False) -> ClipResult:
+                   global_adaptive: bool = False, ema_cap: Optional[float] = None) -> ClipResult:
     """Clip factors, flags and the EMA update for one step, from per-tensor sums of squares.
 
     Warm-up branch: Eq. 2 and the min-seeding line of Algorithm 1.
@@ -88,12 +88,16 @@ def clip_decisions(s: Sequence[float], gamma_prev: np.ndarray, step: int, hp: Hy
                       the ablation) is used as gamma_{t-1} from the first step on;
       global_adaptive "Global AdaGC": one adaptive threshold for the whole model, i.e. this same algorithm
                       applied to the single tensor that all gradients form together; every tensor gets
-                      that one clip factor, flag and gamma.
+                      that one clip factor, flag and gamma;
+      ema_cap         "thresholded initialization" (variant 3 of the EMA-initialization ablation, cap 0.1 there):
+                      gamma_t,i = min(||hat(g)_t,i||, ema_cap) wherever the default seeds gamma or takes the
+                      running minimum; the constant stands where gamma_t-1,i stood, so no warm-up step
+                      remembers the one before it.
     """
     if global_adaptive:
         s_all = np.asarray(s, dtype=np.float64)
         one = clip_decisions([float(np.sum(s_all))], np.asarray(gamma_prev)[:1], step, hp, state_dtype,
-                             keep_initial, False)
+                             keep_initial, False, ema_cap)
         T = s_all.shape[0]
         n_i = np.sqrt(s_all)
         return ClipResult(n_i, np.full(T, one.h[0]), np.full(T, bool(one.flag[0])), one.h[0] * n_i,
@@ -123,11 +127,16 @@ def clip_decisions(s: Sequence[float], gamma_prev: np.ndarray, step: int, hp: Hy
             flag[i] = clip_all
             c[i] = h_t * n[i]                              # ||hat(g)_t,i||
             # gamma_t,i = min{gamma_t-1,i, ||hat(g)_t,i||},  gamma_0,i = ||hat(g)_1,i||
-            gam[i] = c[i] if seed else min(gam[i], c[i])
+            if ema_cap is not None and ema_cap > 0:
+                gam[i] = c[i] if c[i] < ema_cap else ema_cap
+            else:
+                gam[i] = c[i] if seed else min(gam[i], c[i])
     else:
         for i in range(T):
             if seed:                                       # T_start = 0: seed, then Eq. 3
                 gam[i] = float(np.asarray(n[i]).astype(state_dtype))
+                if ema_cap is not None and ema_cap > 0 and not gam[i] < ema_cap:
+                    gam[i] = ema_cap
             thr = hp.lambda_rel * gam[i]
             if thr > 0:
                 margin[i] = abs(n[i] - thr) / thr

@@ -114,15 +114,19 @@ void adagc_ref_clip_decisions(int32_t T, const double* s, float* gamma, int64_t 
                               clipped, margin, global_norm);
 }
 
-/* The same with the two ablation variants of the paper's Section 5 (bits of `variant`):
+/* The same with the ablation variants of the paper's Section 5 (bits of `variant`):
  *   1  keep the caller's gamma_0: no seeding at t = 1 ("constant initialization");
  *   2  "Global AdaGC": one adaptive threshold for the whole model = this algorithm on the single tensor
- *      that all gradients form together; every tensor gets that clip factor, flag and gamma. */
-void adagc_ref_clip_decisions_ex(int32_t T, const double* s, float* gamma, int64_t step,
-                                 double lambda_rel, double beta, double lambda_abs, int64_t warmup,
-                                 int variant, double* norm, double* h, uint8_t* flag, double* clipped,
-                                 double* margin, double* global_norm) {
+ *      that all gradients form together; every tensor gets that clip factor, flag and gamma;
+ * and, with gamma_cap > 0, "thresholded initialization" (EMA Initialization Strategy, variant 3): wherever the
+ * default seeds gamma or takes the running minimum, gamma_t,i = min(||hat(g)_t,i||, gamma_cap) instead -- the
+ * constant takes the place of gamma_t-1,i, so nothing is carried from one warm-up step to the next. */
+void adagc_ref_clip_decisions_cap(int32_t T, const double* s, float* gamma, int64_t step,
+                                  double lambda_rel, double beta, double lambda_abs, int64_t warmup,
+                                  int variant, double gamma_cap, double* norm, double* h, uint8_t* flag,
+                                  double* clipped, double* margin, double* global_norm) {
   const int seed = (step == 1) && !(variant & 1);
+  const int capped = gamma_cap > 0.0;
   long double tot = 0.0L;
   for (int32_t i = 0; i < T; ++i) {
     norm[i] = sqrt(s[i]);
@@ -134,8 +138,8 @@ void adagc_ref_clip_decisions_ex(int32_t T, const double* s, float* gamma, int64
     double s1 = (double)tot, n1, h1, c1, m1, G1;
     uint8_t f1;
     float g1 = gamma[0];
-    adagc_ref_clip_decisions_ex(1, &s1, &g1, step, lambda_rel, beta, lambda_abs, warmup, variant & 1, &n1, &h1,
-                                &f1, &c1, &m1, &G1);
+    adagc_ref_clip_decisions_cap(1, &s1, &g1, step, lambda_rel, beta, lambda_abs, warmup, variant & 1, gamma_cap,
+                                 &n1, &h1, &f1, &c1, &m1, &G1);
     for (int32_t i = 0; i < T; ++i) {
       h[i] = h1;
       flag[i] = f1;
@@ -154,12 +158,15 @@ void adagc_ref_clip_decisions_ex(int32_t T, const double* s, float* gamma, int64
       clipped[i] = h_t * norm[i]; /* ||hat(g)_t,i|| */
       margin[i] = lambda_abs > 0 ? fabs(G - lambda_abs) / lambda_abs : INFINITY;
       double gprev = (double)gamma[i];
-      double gnew = seed ? clipped[i] : (clipped[i] < gprev ? clipped[i] : gprev);
+      double gnew;
+      if (capped) gnew = clipped[i] < gamma_cap ? clipped[i] : gamma_cap;
+      else gnew = seed ? clipped[i] : (clipped[i] < gprev ? clipped[i] : gprev);
       gamma[i] = (float)gnew;
     }
   } else {
     for (int32_t i = 0; i < T; ++i) {
       double gprev = seed ? (double)(float)norm[i] : (double)gamma[i];
+      if (seed && capped && !(gprev < gamma_cap)) gprev = gamma_cap;
       const double thr = lambda_rel * gprev;
       margin[i] = thr > 0 ? fabs(norm[i] - thr) / thr : INFINITY;
       if (norm[i] > thr) {
@@ -174,6 +181,14 @@ void adagc_ref_clip_decisions_ex(int32_t T, const double* s, float* gamma, int64
       gamma[i] = (float)(beta * gprev + (1.0 - beta) * clipped[i]);
     }
   }
+}
+
+void adagc_ref_clip_decisions_ex(int32_t T, const double* s, float* gamma, int64_t step,
+                                 double lambda_rel, double beta, double lambda_abs, int64_t warmup,
+                                 int variant, double* norm, double* h, uint8_t* flag, double* clipped,
+                                 double* margin, double* global_norm) {
+  adagc_ref_clip_decisions_cap(T, s, gamma, step, lambda_rel, beta, lambda_abs, warmup, variant, 0.0, norm, h,
+                               flag, clipped, margin, global_norm);
 }
 
 /* The four AdamW lines of Algorithm 1 on hat(g) = h * g for n elements, in place. */

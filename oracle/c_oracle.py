@@ -50,6 +50,10 @@ def lib():
         L.adagc_ref_clip_decisions_ex.argtypes = [C.c_int32, _f64p, _f32p, C.c_int64, C.c_double, C.c_double,
                                                   C.c_double, C.c_int64, C.c_int, _f64p, _f64p, _u8p, _f64p, _f64p,
                                                   _f64p]
+        L.adagc_ref_clip_decisions_cap.restype = None
+        L.adagc_ref_clip_decisions_cap.argtypes = [C.c_int32, _f64p, _f32p, C.c_int64, C.c_double, C.c_double,
+                                                   C.c_double, C.c_int64, C.c_int, C.c_double, _f64p, _f64p, _u8p,
+                                                   _f64p, _f64p, _f64p]
         L.adagc_ref_adamw.restype = None
         L.adagc_ref_adamw.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int64,
                                       C.c_double, C.c_int64] + [C.c_double] * 5
@@ -96,8 +100,10 @@ def sumsq_tensors(arena: np.ndarray, offsets: Sequence[int], numels: Sequence[in
 
 
 def clip_decisions(s: np.ndarray, gamma: np.ndarray, step: int, lambda_rel: float, beta: float,
-                   lambda_abs: float, warmup: int, keep_initial: bool = False, global_adaptive: bool = False):
-    """Returns dict(norm, h, flag, clipped, margin, global_norm); `gamma` (fp32) is updated in place."""
+                   lambda_abs: float, warmup: int, keep_initial: bool = False, global_adaptive: bool = False,
+                   ema_cap: float = 0.0):
+    """Returns dict(norm, h, flag, clipped, margin, global_norm); `gamma` (fp32) is updated in place.
+    ema_cap > 0 selects the "thresholded initialization" variant (gamma = min(clipped norm, ema_cap) in warm-up)."""
     s = np.ascontiguousarray(s, dtype=np.float64)
     T = len(s)
     assert gamma.dtype == np.float32 and gamma.flags["C_CONTIGUOUS"] and len(gamma) == T
@@ -105,8 +111,8 @@ def clip_decisions(s: np.ndarray, gamma: np.ndarray, step: int, lambda_rel: floa
     flag = np.empty(T, np.uint8)
     G = np.empty(1, np.float64)
     variant = (1 if keep_initial else 0) | (2 if global_adaptive else 0)
-    lib().adagc_ref_clip_decisions_ex(T, s, gamma, step, lambda_rel, beta, lambda_abs, warmup, variant,
-                                      norm, h, flag, clipped, margin, G)
+    lib().adagc_ref_clip_decisions_cap(T, s, gamma, step, lambda_rel, beta, lambda_abs, warmup, variant,
+                                       float(ema_cap), norm, h, flag, clipped, margin, G)
     return dict(norm=norm, h=h, flag=flag.astype(bool), clipped=clipped, margin=margin,
                 global_norm=float(G[0]), gamma=gamma)
 
@@ -163,8 +169,8 @@ class ArenaOracle:
     def __init__(self, offsets: Sequence[int], numels: Sequence[int], theta0: np.ndarray, *,
                  lr: float, beta1: float, beta2: float, eps: float, wd: float, lambda_rel: float,
                  beta: float, lambda_abs: float, warmup: int, keep_initial: bool = False,
-                 global_adaptive: bool = False, gamma0: Optional[np.ndarray] = None):
-        self.keep_initial, self.global_adaptive = keep_initial, global_adaptive
+                 global_adaptive: bool = False, gamma0: Optional[np.ndarray] = None, ema_cap: float = 0.0):
+        self.keep_initial, self.global_adaptive, self.ema_cap = keep_initial, global_adaptive, float(ema_cap)
         self.off = np.ascontiguousarray(offsets, dtype=np.int64)
         self.numel = np.ascontiguousarray(numels, dtype=np.int64)
         self.T = len(self.off)
@@ -179,7 +185,7 @@ class ArenaOracle:
         self._s = np.empty(self.T, np.float64)
 
     def step(self, grads: np.ndarray, lr: Optional[float] = None):
-        if self.keep_initial or self.global_adaptive:
+        if self.keep_initial or self.global_adaptive or self.ema_cap > 0:
             return self._step_variant(grads, lr)
         self.t += 1
         p, bf = _grad_ptr(grads)
@@ -211,7 +217,8 @@ class ArenaOracle:
         self.t += 1
         s = sumsq_tensors(grads, self.off, self.numel)
         r = clip_decisions(s, self.gamma, self.t, self.hp["lambda_rel"], self.hp["beta"],
-                           self.hp["lambda_abs"], self.hp["warmup"], self.keep_initial, self.global_adaptive)
+                           self.hp["lambda_abs"], self.hp["warmup"], self.keep_initial, self.global_adaptive,
+                           self.ema_cap)
         self.clip_count += r["flag"].astype(np.uint64)
         r["gamma"] = self.gamma.copy()
         return r

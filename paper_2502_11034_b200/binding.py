@@ -83,6 +83,8 @@ def lib() -> C.CDLL:
     L.adagc_get_stats.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     L.adagc_get_sumsq.restype = C.c_int
     L.adagc_get_sumsq.argtypes = [vp, vp, vp]
+    L.adagc_set_ema_cap.restype = C.c_int
+    L.adagc_set_ema_cap.argtypes = [vp, dbl]
     L.adagc_update_path.restype = C.c_int
     L.adagc_update_path.argtypes = [vp]
     L.adagc_arena_elems.restype = i64
@@ -293,6 +295,11 @@ class AdaGC:
         if rc != 0:
             raise AdagcError(rc, "adagc_get_sumsq")
         return out
+
+    def set_ema_cap(self, cap: float):
+        rc = lib().adagc_set_ema_cap(self._h, float(cap))
+        if rc != 0:
+            raise AdagcError(rc, "adagc_set_ema_cap")
 
     def debug_wait_timeout(self, limit_ms: float, stream=None):
         rc = lib().adagc_debug_wait_timeout(self._h, float(limit_ms), _stream_ptr(stream))

@@ -78,6 +78,7 @@ struct ClipScalars {
   int64_t step;
   int32_t n_tensors;
   int32_t seed;  // 1: gamma is seeded at this step (t = 1, unless the descriptor keeps the caller's gamma_0)
+  double ema_cap;  // > 0: "thresholded initialization" -- seeding and warm-up set gamma = min(clipped norm, ema_cap)
 };
 
 struct AdamScalars {
@@ -218,7 +219,8 @@ __device__ __forceinline__ void adagc_decide(int i, double s, const ClipScalars&
                                              float* __restrict__ ema, const StatPtrs& st) {
   const double n = sqrt(s);  // ||g_t,i||
   // gamma is fp32 state; with T_start = 0 the first step seeds it with this step's norm
-  const double g_prev = cs.seed ? (double)(float)n : (double)ema[i];
+  double g_prev = cs.seed ? (double)(float)n : (double)ema[i];
+  if (cs.seed && cs.ema_cap > 0.0 && !(g_prev < cs.ema_cap)) g_prev = cs.ema_cap;
   const double thr = __dmul_rn(cs.lambda_rel, g_prev);
   const bool clip = n > thr;  // strict: equality is not a clip
   const double h = clip ? __ddiv_rn(thr, n) : 1.0;
@@ -301,7 +303,9 @@ adagc_warmup_finalize_kernel(ClipScalars cs, float* __restrict__ ema, StatPtrs s
     const double n = sqrt(s);
     const double c = __dmul_rn(h, n);  // ||hat(g)_t,i||
     double g_new = c;
-    if (!cs.seed) {
+    if (cs.ema_cap > 0.0) {  // the constant stands where gamma_t-1,i stands in the default
+      g_new = (c < cs.ema_cap) ? c : cs.ema_cap;
+    } else if (!cs.seed) {
       const double g_prev = (double)ema[i];
       g_new = (c < g_prev) ? c : g_prev;
     }
@@ -343,9 +347,11 @@ adagc_global_finalize_kernel(ClipScalars cs, int in_warmup, float* __restrict__ 
     clip = G > cs.lambda_abs;
     h = clip ? __ddiv_rn(cs.lambda_abs, G) : 1.0;
     const double c = __dmul_rn(h, G);
-    g_new = cs.seed ? c : ((c < g_in) ? c : g_in);
+    if (cs.ema_cap > 0.0) g_new = (c < cs.ema_cap) ? c : cs.ema_cap;
+    else g_new = cs.seed ? c : ((c < g_in) ? c : g_in);
   } else {
-    const double g_prev = cs.seed ? (double)(float)G : g_in;
+    double g_prev = cs.seed ? (double)(float)G : g_in;
+    if (cs.seed && cs.ema_cap > 0.0 && !(g_prev < cs.ema_cap)) g_prev = cs.ema_cap;
     const double thr = __dmul_rn(cs.lambda_rel, g_prev);
     clip = G > thr;
     h = clip ? __ddiv_rn(thr, G) : 1.0;
@@ -729,11 +735,22 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
   }
   if (!healthy) return;
 
+  // partial chunks: table entry and clip factor are fetched one chunk ahead, so that a warp moving from one small
+  // chunk to the next never waits on two dependent loads with nothing else in flight
+  if (mid >= end) return;
   int row_base = 0;
+  Chunk ck = chunks[mid];
+  float h = h_arr[ck.tensor];
   for (int c = mid; c < end; ++c) {
-    const Chunk ck = chunks[c];
-    adamw_partial_chunk<kBF16, kTmaThreads, kOpt>(ck, h_arr[ck.tensor], row_base, params, grads, m_arena, v_arena, a,
-                                                  lowp);
+    Chunk ck_next = ck;
+    float h_next = h;
+    if (c + 1 < end) {
+      ck_next = chunks[c + 1];
+      h_next = h_arr[ck_next.tensor];
+    }
+    adamw_partial_chunk<kBF16, kTmaThreads, kOpt>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp);
+    ck = ck_next;
+    h = h_next;
   }
 }
 
@@ -930,6 +947,7 @@ struct adagc_ctx {
   bool offsets_mult8 = true;           // every tensor offset is a multiple of 8 elements (bf16 arenas stay 16-byte aligned)
   bool keep_initial = false;           // ADAGC_EMA_KEEP_INITIAL
   bool global_adaptive = false;        // ADAGC_CLIP_GLOBAL_ADAPTIVE
+  double ema_cap = 0.0;                // adagc_set_ema_cap: > 0 selects thresholded initialization
   char* ws = nullptr;
   Layout L{};
   uint64_t launches = 0;
@@ -1043,6 +1061,7 @@ ClipScalars make_clip_scalars(const adagc_ctx* ctx, int64_t step, double lambda_
   cs.step = step;
   cs.n_tensors = ctx->T;
   cs.seed = (step == 1 && !ctx->keep_initial) ? 1 : 0;
+  cs.ema_cap = ctx->ema_cap;
   return cs;
 }
 
@@ -1633,6 +1652,12 @@ int adagc_debug_wait_timeout(adagc_ctx* ctx, double limit_ms, void* cuda_stream)
       static_cast<uint64_t>(limit_ms * 1e6), ctx->stats().status);
   ctx->launches++;
   return cudaGetLastError() == cudaSuccess ? ADAGC_OK : ADAGC_E_CUDA;
+}
+
+int adagc_set_ema_cap(adagc_ctx* ctx, double cap) {
+  if (!ctx || !(cap >= 0.0) || !std::isfinite(cap)) return ADAGC_E_INVALID_ARG;
+  ctx->ema_cap = cap;
+  return ADAGC_OK;
 }
 
 int adagc_update_path(const adagc_ctx* ctx) {

@@ -102,12 +102,14 @@ def check_state(name: str, got: np.ndarray, ref: np.ndarray, rep: ParityReport, 
 
 def run_full(wl: workloads.Workload, n_steps: int, device="cuda", hyper_over: Optional[dict] = None,
              lr_schedule=None, canary: bool = True, flags: int = 0, gamma0: Optional[float] = None,
-             emit_bf16: bool = False) -> ParityReport:
+             emit_bf16: bool = False, ema_cap: float = 0.0) -> ParityReport:
     """Every element of every tensor, fused AdaGC+AdamW step, GPU vs C oracle."""
     hp = hyper_of(wl, **(hyper_over or {}))
     offs = [t.offset for t in wl.tensors]
     nums = [t.numel for t in wl.tensors]
     opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=device, flags=flags)
+    if ema_cap > 0:
+        opt.set_ema_cap(ema_cap)
     theta = workloads.init_params(wl, device)
     theta0 = theta.cpu().numpy().copy()
     pad_mask = None
@@ -128,7 +130,8 @@ def run_full(wl: workloads.Workload, n_steps: int, device="cuda", hyper_over: Op
                                eps=hp["eps"], wd=hp["wd"], lambda_rel=hp["lambda_rel"], beta=hp["beta"],
                                lambda_abs=hp["lambda_abs"], warmup=hp["warmup"], keep_initial=keep,
                                global_adaptive=bool(flags & binding.CLIP_GLOBAL_ADAPTIVE),
-                               gamma0=None if not keep else np.full(wl.n_tensors, gamma0, np.float32))
+                               gamma0=None if not keep else np.full(wl.n_tensors, gamma0, np.float32),
+                               ema_cap=ema_cap)
     rep = ParityReport()
     lowp = torch.full((wl.arena_elems,), 7.0, dtype=torch.bfloat16, device=device) if emit_bf16 else None
     for t in range(1, n_steps + 1):

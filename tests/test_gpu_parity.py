@@ -217,6 +217,23 @@ def test_ablation_variants_all_elements(variant):
     assert rep.steps == 16
 
 
+def test_thresholded_initialization_all_elements():
+    """Section 5, EMA-initialization variant 3: gamma = min(clipped norm, cap) at seeding and in warm-up."""
+    wl = workloads.build("llama2_7b", n_layer=2, d=256, ffn=688, vocab=1000)
+    for warmup, cap, flags in ((4, 0.01, 0), (0, 0.005, 0), (3, 0.02, binding.CLIP_GLOBAL_ADAPTIVE)):
+        rep = H.run_full(wl, 14, flags=flags, ema_cap=cap, hyper_over=dict(warmup=warmup, lambda_abs=1e4))
+        _report(f"thresholded init warmup={warmup} cap={cap} flags={flags}", rep)
+        assert rep.clipped > 0
+    wl = workloads.build("many_small", n_tensors=300, lo=1, hi=40000)
+    rep = H.run_full(wl, 12, ema_cap=0.1, hyper_over=dict(lambda_abs=1e4))          # the paper's cap
+    _report("thresholded init many_small cap=0.1", rep)
+    opt = binding.AdaGC([8], [0], torch.float32, 1.0)
+    for bad in (-1.0, float("nan"), float("inf")):
+        with pytest.raises(binding.AdagcError):
+            opt.set_ema_cap(bad)
+    opt.close()
+
+
 def _ragged_workload(sizes, dtype):
     specs, total = workloads._layout([(f"t{i}", (n,)) for i, n in enumerate(sizes)])
     hp = dict(workloads.PAPER_DEFAULTS, lambda_abs=0.05)

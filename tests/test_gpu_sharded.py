@@ -106,3 +106,19 @@ def test_presummed_argument_errors():
                                     sp) == -1
     assert opt.launch_count() == 0
     opt.close()
+
+
+def test_bench_sharded_mode_prints_one_json_line():
+    """`bench.py --parallel sharded` at N = 1: the split step over the whole layout, one JSON line."""
+    import json
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--parallel", "sharded", "--workload",
+                          "gpt2_small", "--steps", "3"], capture_output=True, text=True, timeout=600)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["scaling"] == "strong" and line["n_gpus"] == 1 and line["value"] > 0
+    assert line["gpu_launches"] == 3 * 4          # per step: norm, per-tensor sum, decision, update
+    assert 0.3 < line["roofline"]["frac"] < 1.2

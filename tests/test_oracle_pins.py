@@ -705,6 +705,70 @@ def test_keep_initial_uses_the_callers_gamma_from_the_first_step(impl_name):
     np.testing.assert_array_equal(a["gamma"], b["gamma"])
 
 
+@pytest.mark.parametrize("impl_name", ["numpy", "c"])
+def test_thresholded_initialization_hand_values_and_special_cases(impl_name):
+    """Thresholded initialization of the ablation (variant 3, gamma_t,i = min(||g_t,i||, cap), cap 0.1 there):
+    the constant takes the place of gamma_t-1,i in the warm-up line, so the value after warm-up is
+    min(last warm-up clipped norm, cap) and earlier warm-up steps leave no trace."""
+    hp = npo.Hyper(warmup=3, lambda_abs=100.0, lambda_rel=2.0, beta=0.5)         # no warm-up clipping: hat(g) = g
+    gam = np.array([np.nan, np.nan], np.float32)                                  # incoming content is irrelevant
+    seq = [([25.0, 144.0], [5.0, 6.0]),       # norms 5, 12; cap 6 -> 5, 6
+           ([49.0, 9.0], [6.0, 3.0]),         # norms 7, 3 -> 6, 3: NOT min with the previous 5 (no running minimum)
+           ([1.0, 100.0], [1.0, 6.0])]        # norms 1, 10 -> 1, 6
+    for t, (s, want) in enumerate(seq, start=1):
+        r = _decide(impl_name, s, gam, t, hp, ema_cap=6.0)
+        gam = r["gamma"]
+        assert list(gam) == want and not np.asarray(r["flag"]).any()
+    # first AdaGC step uses what the last warm-up step left: thresholds 2*1 and 2*6
+    r = _decide(impl_name, [16.0, 100.0], gam, 4, hp, ema_cap=6.0)
+    np.testing.assert_array_equal(np.asarray(r["flag"]), [True, False])            # 4 > 2 ; 10 <= 12
+    np.testing.assert_array_equal(r["gamma"], np.array([0.5 * 1 + 0.5 * 2, 0.5 * 6 + 0.5 * 10], np.float32))
+    # warm-up clipping active: the capped quantity is the CLIPPED norm h_t ||g_t,i|| (Algorithm 1 writes the hat)
+    hpc = npo.Hyper(warmup=3, lambda_abs=6.5, lambda_rel=2.0, beta=0.5)           # G = 13 -> h = 0.5
+    r = _decide(impl_name, [25.0, 144.0], np.zeros(2, np.float32), 1, hpc, ema_cap=4.0)
+    assert list(r["gamma"]) == [2.5, 4.0] and list(np.asarray(r["h"])) == [0.5, 0.5]
+    # T_start = 0: the seed of step 1 is capped, then Eq. 3 applies to it
+    hp0 = npo.Hyper(warmup=0, lambda_rel=2.0, beta=0.5)
+    r = _decide(impl_name, [9.0, 16.0], np.zeros(2, np.float32), 1, hp0, ema_cap=1.5)
+    np.testing.assert_array_equal(np.asarray(r["flag"]), [False, True])            # 3 <= 2*1.5 ; 4 > 2*1.5
+    np.testing.assert_array_equal(r["gamma"], np.array([0.5 * 1.5 + 0.5 * 3, 0.5 * 1.5 + 0.5 * 3], np.float32))
+    # special cases that reduce to the default: one warm-up step with a cap nothing reaches (the seed IS the clipped
+    # norm), and any AdaGC step after the first (the variant only touches seeding and warm-up)
+    rng = np.random.RandomState(5)
+    s = (rng.standard_t(3, size=50) ** 2 + 1e-3).tolist()
+    hp1 = npo.Hyper(warmup=1, lambda_abs=0.7)
+    a = _decide(impl_name, s, np.zeros(50, np.float32), 1, hp1, ema_cap=1e30)
+    b = _decide(impl_name, s, np.zeros(50, np.float32), 1, hp1)
+    np.testing.assert_array_equal(a["gamma"], b["gamma"])
+    g0 = np.abs(rng.normal(size=50)).astype(np.float32)
+    a = _decide(impl_name, s, g0.copy(), 9, hp1, ema_cap=0.1)
+    b = _decide(impl_name, s, g0.copy(), 9, hp1)
+    np.testing.assert_array_equal(a["gamma"], b["gamma"])
+    np.testing.assert_array_equal(np.asarray(a["flag"]), np.asarray(b["flag"]))
+
+
+def test_thresholded_initialization_brute_force_and_oracles_agree():
+    """gamma after warm-up = min(h_T ||g_T,i||, cap) for the LAST warm-up step T (brute force over a random run),
+    never above the cap; numpy and C oracles agree bit for bit on gamma and flags."""
+    rng = np.random.RandomState(77)
+    T, W, cap = 40, 6, 0.1
+    hp = npo.Hyper(warmup=W, lambda_abs=1.0, lambda_rel=1.04, beta=0.99)
+    gn, gc = np.zeros(T, np.float32), np.zeros(T, np.float32)
+    for t in range(1, W + 5):
+        s = (np.abs(rng.standard_t(2, size=T)) * 0.05) ** 2
+        rn = _decide("numpy", s.tolist(), gn, t, hp, ema_cap=cap)
+        rc = _decide("c", s.tolist(), gc, t, hp, ema_cap=cap)
+        gn, gc = rn["gamma"], rc["gamma"]
+        np.testing.assert_array_equal(gn, gc)
+        np.testing.assert_array_equal(np.asarray(rn["flag"]), np.asarray(rc["flag"]))
+        if t <= W:
+            G = math.sqrt(float(np.sum(s)))
+            h = min(1.0 / G, 1.0)
+            want = np.minimum(h * np.sqrt(s), cap).astype(np.float32)
+            np.testing.assert_array_equal(gn, want)
+            assert (gn <= np.float32(cap)).all()
+
+
 # ----------------------------------------------------------------------------- SGD with momentum on the clipped gradient
 @pytest.mark.parametrize("impl_name", ["numpy", "c"])
 def test_sgdm_matches_library_sgd(impl_name):

@@ -139,6 +139,28 @@ int adagc_step(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, v
                double wd, double lambda_rel, double beta, int64_t warmup, void* cuda_stream);
 
 /*
+ * adagc_step for CUDA graphs: the enqueued work is identical for every step, so a graph captured once can be
+ * replayed for the whole run.  What adagc_step takes from its `step` argument is kept on the device instead:
+ *   - t = (steps this context has executed so far) + 1, read from the context's device-side counter (the one
+ *     adagc_get_stats reports as steps_done; every step-type entry point advances it).  The warm-up switch
+ *     (t <= warmup), the seeding of gamma at t = 1 and the bias corrections 1 - beta^t follow from it on the
+ *     device, in float64 as on the host.  After a restart set the counter with adagc_set_step_counter.
+ *   - eta_t: if d_lr is not NULL it points to one fp32 value in DEVICE memory that is read at every execution
+ *     (update it between replays to follow a schedule); if NULL the value `lr` is used.
+ * The other arguments are those of adagc_step.  Five launches per step (prologue, norm, per-tensor
+ * finalize, warm-up finalize -- which returns at once outside warm-up -- and update) instead of three.
+ * Results agree with adagc_step's to the last bit whenever the device and host evaluations of beta^t round
+ * to the same fp32 coefficients, and within the library's tolerance (1e-5) always.
+ */
+int adagc_step_capturable(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, void* d_v,
+                          float* d_ema, const float* d_lr, double lr, double beta1, double beta2, double eps,
+                          double wd, double lambda_rel, double beta, int64_t warmup, void* cuda_stream);
+
+/* Sets the device-side step counter (steps executed so far) -- for adagc_step_capturable after a restart from
+ * saved state at step t0: pass t0 - 1.  Enqueues one tiny kernel. */
+int adagc_set_step_counter(adagc_ctx* ctx, uint64_t steps_done, void* cuda_stream);
+
+/*
  * adagc_step that also emits the model's working copy of the parameters: mixed-precision training keeps fp32
  * master parameters in the optimizer and runs the model on a bf16 copy (the paper's runs use bfloat16
  * precision).  Besides everything adagc_step does, d_params_bf16[j] = bf16(theta_t[j]) (round to nearest even)

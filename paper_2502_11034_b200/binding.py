@@ -59,6 +59,10 @@ def lib() -> C.CDLL:
     L.adagc_destroy.argtypes = [vp]
     L.adagc_step.restype = C.c_int
     L.adagc_step.argtypes = [vp, vp, vp, vp, vp, f32p, i64, dbl, dbl, dbl, dbl, dbl, dbl, dbl, i64, vp]
+    L.adagc_step_capturable.restype = C.c_int
+    L.adagc_step_capturable.argtypes = [vp, vp, vp, vp, vp, f32p, vp, dbl, dbl, dbl, dbl, dbl, dbl, dbl, i64, vp]
+    L.adagc_set_step_counter.restype = C.c_int
+    L.adagc_set_step_counter.argtypes = [vp, C.c_uint64, vp]
     L.adagc_step_emit_bf16.restype = C.c_int
     L.adagc_step_emit_bf16.argtypes = [vp, vp, vp, vp, vp, vp, f32p, i64, dbl, dbl, dbl, dbl, dbl, dbl, dbl, i64, vp]
     L.adagc_step_lion.restype = C.c_int
@@ -210,6 +214,23 @@ class AdaGC:
                               lr, beta1, beta2, eps, wd, lambda_rel, beta, int(warmup), _stream_ptr(stream))
         if rc != 0:
             raise AdagcError(rc, "adagc_step")
+
+    def step_capturable(self, params, grads, m, v, ema, lr, beta1, beta2, eps, wd, lambda_rel, beta, warmup,
+                        lr_dev: Optional[torch.Tensor] = None, stream=None):
+        """adagc_step_capturable: the step number lives on the device; `lr_dev` (one fp32 on the device), if given,
+        is read at every execution instead of `lr`."""
+        assert grads.dtype == self.grad_dtype and params.dtype == m.dtype == v.dtype == ema.dtype == torch.float32
+        assert lr_dev is None or (lr_dev.dtype == torch.float32 and lr_dev.is_cuda)
+        rc = lib().adagc_step_capturable(self._h, _ptr(params), _ptr(grads), _ptr(m), _ptr(v), _ptr(ema),
+                                         _ptr(lr_dev), lr, beta1, beta2, eps, wd, lambda_rel, beta, int(warmup),
+                                         _stream_ptr(stream))
+        if rc != 0:
+            raise AdagcError(rc, "adagc_step_capturable")
+
+    def set_step_counter(self, steps_done: int, stream=None):
+        rc = lib().adagc_set_step_counter(self._h, int(steps_done), _stream_ptr(stream))
+        if rc != 0:
+            raise AdagcError(rc, "adagc_set_step_counter")
 
     def step_emit_bf16(self, params, params_bf16, grads, m, v, ema, step, lr, beta1, beta2, eps, wd, lambda_rel, beta,
                        warmup, stream=None):

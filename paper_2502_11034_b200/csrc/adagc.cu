@@ -89,6 +89,21 @@ struct AdamScalars {
   float eps;
 };
 
+// Scalars of one step kept in device memory: written by adagc_step_prologue_kernel from the device-side step
+// counter, read by the phases of a capturable step (the launches then carry nothing that changes from step to step).
+struct DeviceStep {
+  ClipScalars cs;
+  AdamScalars a;
+  int32_t in_warmup;  // t <= T_start
+  int32_t pad;
+};
+
+struct StepHyper {  // what the host hands to the prologue kernel
+  double lr, beta1, beta2, eps, wd, lambda_rel, beta, lambda_abs, ema_cap;
+  int64_t warmup;
+  int32_t n_tensors, keep_initial;
+};
+
 // ------------------------------------------------------------------------------------------------
 // small device helpers
 // ------------------------------------------------------------------------------------------------
@@ -239,7 +254,12 @@ __device__ __forceinline__ void adagc_decide(int i, double s, const ClipScalars&
 __global__ void __launch_bounds__(kFinalizeThreads)
 adagc_tensor_finalize_kernel(const double* __restrict__ partials, const TensorEntry* __restrict__ tensors,
                              ClipScalars cs, int decide, float* __restrict__ ema, StatPtrs st,
-                             const int32_t* __restrict__ order, int first, int count, int bump_steps) {
+                             const int32_t* __restrict__ order, int first, int count, int bump_steps,
+                             const DeviceStep* __restrict__ ds = nullptr) {
+  if (ds) {  // capturable step: scalars and the warm-up switch come from device memory
+    cs = ds->cs;
+    decide = decide && !ds->in_warmup;
+  }
   // the warps of this launch take `count` tensors: order[first..first+count) if an order is given
   // (a group of the pipelined host step), else the tensors first..first+count-1
   const int k = (blockIdx.x * kFinalizeThreads + threadIdx.x) >> 5;
@@ -275,10 +295,50 @@ adagc_presummed_finalize_kernel(const double* __restrict__ sumsq_in, ClipScalars
   }
 }
 
+// adagc_set_step_counter: the value travels as a kernel argument, so no host buffer has to outlive the call.
+__global__ void adagc_set_counter_kernel(unsigned long long* __restrict__ dst, unsigned long long value) { *dst = value; }
+
+// Capturable step, first launch: derive this step's scalars on the device.  t = steps executed so far + 1, eta_t
+// from device memory if the caller keeps it there; the bias corrections 1 - beta^t are formed in float64 like the
+// host does for adagc_step and rounded once to the kernels' fp32.
+__global__ void adagc_step_prologue_kernel(const unsigned long long* __restrict__ steps_done,
+                                           const float* __restrict__ d_lr, StepHyper hh, DeviceStep* __restrict__ out) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  const long long t = static_cast<long long>(*steps_done) + 1;
+  const double lr = d_lr ? (double)*d_lr : hh.lr;
+  DeviceStep ds;
+  ds.cs.lambda_rel = hh.lambda_rel;
+  ds.cs.beta = hh.beta;
+  ds.cs.one_minus_beta = 1.0 - hh.beta;
+  ds.cs.lambda_abs = hh.lambda_abs;
+  ds.cs.step = t;
+  ds.cs.n_tensors = hh.n_tensors;
+  ds.cs.seed = (t == 1 && !hh.keep_initial) ? 1 : 0;
+  ds.cs.ema_cap = hh.ema_cap;
+  const double bc1 = 1.0 - pow(hh.beta1, (double)t);
+  const double bc2 = 1.0 - pow(hh.beta2, (double)t);
+  ds.a.beta1 = (float)hh.beta1;
+  ds.a.one_minus_beta1 = (float)(1.0 - hh.beta1);
+  ds.a.beta2 = (float)hh.beta2;
+  ds.a.one_minus_beta2 = (float)(1.0 - hh.beta2);
+  ds.a.inv_bc2 = (float)(1.0 / bc2);
+  ds.a.step_size = (float)(lr / bc1);
+  ds.a.decay = (float)(1.0 - lr * hh.wd);
+  ds.a.eps = (float)hh.eps;
+  ds.in_warmup = t <= hh.warmup ? 1 : 0;
+  ds.pad = 0;
+  *out = ds;
+}
+
 // Warm-up branch of Algorithm 1: global norm (Eq. 2), one clip factor for every tensor, and
 // gamma_t,i = min{gamma_t-1,i, ||hat(g)_t,i||} with gamma_0,i = ||hat(g)_1,i||.  One block.
 __global__ void __launch_bounds__(kWarmupThreads)
-adagc_warmup_finalize_kernel(ClipScalars cs, float* __restrict__ ema, StatPtrs st) {
+adagc_warmup_finalize_kernel(ClipScalars cs, float* __restrict__ ema, StatPtrs st,
+                             const DeviceStep* __restrict__ ds = nullptr) {
+  if (ds) {  // capturable step: always launched, does nothing outside warm-up
+    if (!ds->in_warmup) return;
+    cs = ds->cs;
+  }
   __shared__ double warp_part[kWarmupThreads / 32];
   __shared__ double total_s;
   const int tid = threadIdx.x;
@@ -322,7 +382,12 @@ adagc_warmup_finalize_kernel(ClipScalars cs, float* __restrict__ ema, StatPtrs s
 // model, i.e. Algorithm 1 applied to the single tensor that all gradients form together.  One block;
 // every tensor receives the same clip factor, flag and gamma.  `in_warmup` selects Eq. 2 or Eq. 3.
 __global__ void __launch_bounds__(kWarmupThreads)
-adagc_global_finalize_kernel(ClipScalars cs, int in_warmup, float* __restrict__ ema, StatPtrs st) {
+adagc_global_finalize_kernel(ClipScalars cs, int in_warmup, float* __restrict__ ema, StatPtrs st,
+                             const DeviceStep* __restrict__ ds = nullptr) {
+  if (ds) {
+    cs = ds->cs;
+    in_warmup = ds->in_warmup;
+  }
   __shared__ double warp_part[kWarmupThreads / 32];
   __shared__ double total_s;
   const int tid = threadIdx.x;
@@ -496,7 +561,8 @@ __global__ void __launch_bounds__(kThreads)
 adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, float* __restrict__ m_arena,
                     float* __restrict__ v_arena, const Chunk* __restrict__ chunks,
                     const int32_t* __restrict__ block_begin, const float* __restrict__ h_arr, AdamScalars a,
-                    uint16_t* __restrict__ lowp) {
+                    uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a) {
+  if (d_a) a = *d_a;  // capturable step: coefficients from device memory
   const int tid = threadIdx.x;
   int c = block_begin[blockIdx.x];
   const int n_chunks = block_begin[blockIdx.x + 1];  // end of this block's entries
@@ -617,7 +683,8 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
                         float* __restrict__ v_arena, const Chunk* __restrict__ chunks,
                         const int32_t* __restrict__ block_begin, const int32_t* __restrict__ block_mid,
                         const float* __restrict__ h_arr, AdamScalars a, int* __restrict__ status,
-                        uint16_t* __restrict__ lowp) {
+                        uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a) {
+  if (d_a) a = *d_a;  // capturable step: coefficients from device memory
   extern __shared__ __align__(128) unsigned char tile_smem[];
   constexpr int kGBytes = kBF16 ? 2 : 4;
   constexpr int kStateBytes = kOpt == kOptAdamW ? 12 : 8;  // theta, m (and v) per element; g follows them
@@ -827,7 +894,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {  // byte offsets of the workspace sections
   size_t chunks_wide, chunks_upd, begin_wide, begin_upd, mid_upd, g_chunks_wide, g_chunks_upd, g_begin_wide,
-      g_begin_upd, g_mid_upd, g_order, tensors, partials, sumsq, norm, h, clip_count, scalars, flag,
+      g_begin_upd, g_mid_upd, g_order, tensors, partials, sumsq, norm, h, clip_count, scalars, dev_step, flag,
       total;
 };
 
@@ -853,6 +920,7 @@ Layout make_layout(int64_t n_chunks, int64_t T) {
   L.h = o;          o = align_up(o + sizeof(float) * T, 256);
   L.clip_count = o; o = align_up(o + sizeof(uint64_t) * T, 256);
   L.scalars = o;    o = align_up(o + 256, 256);  // steps_done (u64) at +0, status (i32) at +8
+  L.dev_step = o;   o = align_up(o + sizeof(DeviceStep), 256);
   L.flag = o;       o = align_up(o + T, 256);
   L.total = o;
   return L;
@@ -1026,22 +1094,22 @@ struct TableView {
 
 template <bool kBF16, int kOpt>
 void launch_update(adagc_ctx* ctx, const TableView& tv, float* p, const void* g, float* m, float* v,
-                   const AdamScalars& a, cudaStream_t s, uint16_t* lowp = nullptr) {
+                   const AdamScalars& a, cudaStream_t s, uint16_t* lowp = nullptr, const AdamScalars* d_a = nullptr) {
   const StatPtrs st = ctx->stats();
   if (ctx->update_bulk)
     adagc_update_tma_kernel<kBF16, kOpt>
         <<<tv.grid, kTmaThreads, tma_smem_bytes(kBF16, kOpt, lowp != nullptr), s>>>(
-            p, g, m, v, tv.chunks, tv.begin, tv.mid, st.h, a, st.status, lowp);
+            p, g, m, v, tv.chunks, tv.begin, tv.mid, st.h, a, st.status, lowp, d_a);
   else
-    adagc_update_kernel<kBF16, kOpt><<<tv.grid, kThreads, 0, s>>>(p, g, m, v, tv.chunks, tv.begin, st.h, a, lowp);
+    adagc_update_kernel<kBF16, kOpt><<<tv.grid, kThreads, 0, s>>>(p, g, m, v, tv.chunks, tv.begin, st.h, a, lowp, d_a);
   ctx->launches++;
 }
 
 template <bool kBF16, int kOpt>
 void launch_update(adagc_ctx* ctx, float* p, const void* g, float* m, float* v, const AdamScalars& a,
-                   cudaStream_t s, uint16_t* lowp = nullptr) {
+                   cudaStream_t s, uint16_t* lowp = nullptr, const AdamScalars* d_a = nullptr) {
   const TableView tv = {ctx->d_chunks_upd(), ctx->d_begin_upd(), ctx->d_mid_upd(), ctx->grid_update};
-  launch_update<kBF16, kOpt>(ctx, tv, p, g, m, v, a, s, lowp);
+  launch_update<kBF16, kOpt>(ctx, tv, p, g, m, v, a, s, lowp, d_a);
 }
 
 void launch_norm(adagc_ctx* ctx, const TableView& tv, const void* d_grads, cudaStream_t s) {
@@ -1490,6 +1558,53 @@ int adagc_clip(adagc_ctx* ctx, const void* d_grads_in, void* d_grads_out, float*
   if (rc != ADAGC_OK) return rc;
   launch_scale(ctx, d_grads_in, d_grads_out, s);
   return finish_launches(ctx, s);
+}
+
+int adagc_step_capturable(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, void* d_v, float* d_ema,
+                          const float* d_lr, double lr, double beta1, double beta2, double eps, double wd,
+                          double lambda_rel, double beta, int64_t warmup, void* cuda_stream) {
+  int rc = check_clip_args(ctx, d_ema, 1, lambda_rel, beta, warmup);
+  if (rc != ADAGC_OK) return rc;
+  rc = check_adamw_args(d_params, d_grads, d_m, d_v, lr, beta1, beta2, eps, wd);
+  if (rc != ADAGC_OK) return rc;
+  if (d_lr && (reinterpret_cast<uintptr_t>(d_lr) & 3u)) return ADAGC_E_MISALIGNED;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  DeviceStep* ds = reinterpret_cast<DeviceStep*>(ctx->ws + ctx->L.dev_step);
+  StepHyper hh;
+  hh.lr = lr; hh.beta1 = beta1; hh.beta2 = beta2; hh.eps = eps; hh.wd = wd;
+  hh.lambda_rel = lambda_rel; hh.beta = beta; hh.lambda_abs = ctx->lambda_abs; hh.ema_cap = ctx->ema_cap;
+  hh.warmup = warmup; hh.n_tensors = ctx->T; hh.keep_initial = ctx->keep_initial ? 1 : 0;
+  const StatPtrs st = ctx->stats();
+  // the same launches every step: what differs between steps is read from device memory
+  adagc_step_prologue_kernel<<<1, 32, 0, s>>>(st.steps_done, d_lr, hh, ds);
+  ctx->launches++;
+  const TableView wide = {ctx->d_chunks_wide(), ctx->d_begin_wide(), nullptr, ctx->grid_wide};
+  launch_norm(ctx, wide, d_grads, s);
+  const int blocks = (ctx->T * 32 + kFinalizeThreads - 1) / kFinalizeThreads;
+  adagc_tensor_finalize_kernel<<<blocks, kFinalizeThreads, 0, s>>>(ctx->d_partials(), ctx->d_tensors(), ClipScalars{},
+                                                                  ctx->global_adaptive ? 0 : 1, d_ema, st, nullptr, 0,
+                                                                  ctx->T, 1, ds);
+  ctx->launches++;
+  if (ctx->global_adaptive)
+    adagc_global_finalize_kernel<<<1, kWarmupThreads, 0, s>>>(ClipScalars{}, 0, d_ema, st, ds);
+  else
+    adagc_warmup_finalize_kernel<<<1, kWarmupThreads, 0, s>>>(ClipScalars{}, d_ema, st, ds);
+  ctx->launches++;
+  if (ctx->bf16)
+    launch_update<true, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
+                                   static_cast<float*>(d_v), AdamScalars{}, s, nullptr, &ds->a);
+  else
+    launch_update<false, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
+                                    static_cast<float*>(d_v), AdamScalars{}, s, nullptr, &ds->a);
+  return cudaGetLastError() == cudaSuccess ? ADAGC_OK : ADAGC_E_CUDA;
+}
+
+int adagc_set_step_counter(adagc_ctx* ctx, uint64_t steps_done, void* cuda_stream) {
+  if (!ctx) return ADAGC_E_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  adagc_set_counter_kernel<<<1, 1, 0, s>>>(ctx->stats().steps_done, static_cast<unsigned long long>(steps_done));
+  ctx->launches++;
+  return cudaGetLastError() == cudaSuccess ? ADAGC_OK : ADAGC_E_CUDA;
 }
 
 int adagc_shard_sumsq(adagc_ctx* ctx, const void* d_grads, double* d_sumsq_out, void* cuda_stream) {

@@ -102,7 +102,7 @@ def check_state(name: str, got: np.ndarray, ref: np.ndarray, rep: ParityReport, 
 
 def run_full(wl: workloads.Workload, n_steps: int, device="cuda", hyper_over: Optional[dict] = None,
              lr_schedule=None, canary: bool = True, flags: int = 0, gamma0: Optional[float] = None,
-             emit_bf16: bool = False, ema_cap: float = 0.0) -> ParityReport:
+             emit_bf16: bool = False, ema_cap: float = 0.0, capturable: str = "") -> ParityReport:
     """Every element of every tensor, fused AdaGC+AdamW step, GPU vs C oracle."""
     hp = hyper_of(wl, **(hyper_over or {}))
     offs = [t.offset for t in wl.tensors]
@@ -134,10 +134,31 @@ def run_full(wl: workloads.Workload, n_steps: int, device="cuda", hyper_over: Op
                                ema_cap=ema_cap)
     rep = ParityReport()
     lowp = torch.full((wl.arena_elems,), 7.0, dtype=torch.bfloat16, device=device) if emit_bf16 else None
+    # capturable = "eager": adagc_step_capturable called every step; "graph": captured ONCE into a CUDA graph before
+    # the first step and replayed for every step (gradients and eta_t are refreshed in place between replays)
+    graph = g_static = lr_dev = None
+    if capturable:
+        lr_dev = torch.zeros(1, dtype=torch.float32, device=device)
+        g_static = torch.zeros(wl.arena_elems, dtype=wl.torch_grad_dtype, device=device)
+        cap_args = (theta, g_static, m, v, ema, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"],
+                    hp["beta"], hp["warmup"], lr_dev)
+        if capturable == "graph":
+            graph = torch.cuda.CUDAGraph()
+            torch.cuda.synchronize()
+            with torch.cuda.graph(graph):
+                opt.step_capturable(*cap_args)
+            assert opt.get_stats()["steps_done"] == 0, "capturing must not execute a step"
     for t in range(1, n_steps + 1):
         g = workloads.grads_for_step(wl, t, device)
         lr = hp["lr"] if lr_schedule is None else lr_schedule(t)
-        if emit_bf16:
+        if capturable:
+            g_static.copy_(g)
+            lr_dev.fill_(lr)
+            if graph is not None:
+                graph.replay()
+            else:
+                opt.step_capturable(*cap_args)
+        elif emit_bf16:
             opt.step_emit_bf16(theta, lowp, g, m, v, ema, t, lr, hp["beta1"], hp["beta2"], hp["eps"], hp["wd"],
                                hp["lambda_rel"], hp["beta"], hp["warmup"])
         else:

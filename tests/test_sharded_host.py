@@ -93,6 +93,13 @@ def test_empty_tensors_need_the_flag():
     assert chunks([100], [0], flags=32) == -1                                      # unknown flag
 
 
+def _free_port() -> int:
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
 def _worker(rank, world, port, out):
     sys.path.insert(0, ROOT)
     from oracle import c_oracle
@@ -126,7 +133,7 @@ def _worker(rank, world, port, out):
 def test_two_gloo_ranks_sum_their_shards_to_the_unsharded_norms():
     ctx = mp.get_context("spawn")
     q = ctx.Queue()
-    port = 31500 + os.getpid() % 2000
+    port = _free_port()
     procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
     for p in procs:
         p.start()

@@ -61,7 +61,10 @@ __host__ __device__ __forceinline__ int64_t chunk_start(const Chunk& c) { return
 // [block_begin[b], block_begin[b+1]) of its kernel's table.  The assignment balances elements (plus a
 // fixed cost per chunk) over the blocks; with equal chunks it is plain round-robin.
 constexpr int kMaxGrid = 8192;          // entries reserved for each block_begin array
+// per-chunk cost added to the element count; measured on the layout of 20 000 small tensors: the norm / scale grid
+// (two block barriers and a table fetch per chunk) balances best with a larger constant than the update grid
 constexpr int kChunkFixedCost = 1024;
+constexpr int kChunkFixedCostWide = 8192;
 // adagc_step_host in steady state: the tensors are cut (in arena order) into at most kMaxGroups groups; each
 // group's gradients are copied on a second stream while the previous groups run norm/finalize/update.
 constexpr int kMaxGroups = 64;
@@ -268,7 +271,18 @@ adagc_tensor_finalize_kernel(const double* __restrict__ partials, const TensorEn
   const int w = order ? order[first + k] : first + k;
   const TensorEntry te = tensors[w];
   double acc = 0.0;
-  for (int j = lane; j < te.n_chunks; j += 32) acc += partials[te.first_chunk + j];
+  // the additions stay in index order; unrolling only lets the loads of the next terms start early (the embedding
+  // of a large model has thousands of partials, and one warp walks them)
+  const double* __restrict__ tp = partials + te.first_chunk;
+  int j = lane;
+  for (; j + 15 * 32 < te.n_chunks; j += 16 * 32) {
+    double t[16];
+#pragma unroll
+    for (int u = 0; u < 16; ++u) t[u] = __ldcg(tp + j + u * 32);
+#pragma unroll
+    for (int u = 0; u < 16; ++u) acc += t[u];
+  }
+  for (; j < te.n_chunks; j += 32) acc += __ldcg(tp + j);
   acc = warp_sum(acc);
   if (lane == 0) {
     st.sumsq[w] = acc;
@@ -974,6 +988,7 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 // (kChunkElems elements), [block_mid[b], block_begin[b+1]) are partial.
 void balance_chunks(const std::vector<Chunk>& chunks, int grid, std::vector<Chunk>* table,
                     std::vector<int32_t>* block_begin, std::vector<int32_t>* block_mid = nullptr) {
+  const int fixed_cost = block_mid ? kChunkFixedCost : kChunkFixedCostWide;  // update tables carry block_mid
   using Load = std::pair<int64_t, int>;  // (work assigned, block)
   std::priority_queue<Load, std::vector<Load>, std::greater<Load>> heap;
   for (int b = 0; b < grid; ++b) heap.emplace(0, b);
@@ -984,7 +999,7 @@ void balance_chunks(const std::vector<Chunk>& chunks, int grid, std::vector<Chun
     heap.pop();
     owner[i] = top.second;
     count[top.second] += 1;
-    heap.emplace(top.first + chunks[i].count + kChunkFixedCost, top.second);
+    heap.emplace(top.first + chunks[i].count + fixed_cost, top.second);
   }
   block_begin->assign(grid + 1, 0);
   for (int b = 0; b < grid; ++b) (*block_begin)[b + 1] = (*block_begin)[b] + count[b];

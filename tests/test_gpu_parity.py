@@ -87,6 +87,26 @@ def test_llama2_7b_sampled():
     assert 8 <= rep.clipped < 291
 
 
+def test_one_tensor_beyond_2_to_32_elements():
+    """Maximum sizes: a single tensor of 2^32 + 12345 elements (262 145 chunks, element indices that do not fit
+    32 bits) followed by a small tensor whose offset lies beyond 2^32.  All norms and decisions against the
+    oracle (it streams the whole gradient), state on sampled elements including both ends and the last chunk."""
+    n_big = 2 ** 32 + 12345
+    specs, total = workloads._layout([("big", (n_big,)), ("small", (1000,))])
+    free, _ = torch.cuda.mem_get_info()
+    need = total * 14 + (6 << 30)
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GiB of device memory, {free >> 30} GiB free")
+    hp = dict(workloads.PAPER_DEFAULTS, lambda_abs=1e4)
+    wl = workloads.Workload("one_huge_tensor", 8, specs, "bf16", hp, warmup=1, n_steps=3, arena_elems=total,
+                            grad_kind="normal", grad_scale=1e-4,
+                            extra={"spike_step": 3, "spike_tensor": 1, "spike_factor": 40.0})
+    assert specs[1].offset > 2 ** 32
+    rep = H.run_sampled(wl, 3, mode="adamw", k=4096)
+    _report("one tensor of 2^32 + 12345 elements", rep)
+    assert rep.decisions == 6 and rep.clipped >= 1
+
+
 def test_hand_worked_example_on_the_gpu():
     """The 2-tensor worked example (tests/golden/worked_example.json): every norm, clip factor, flag and gamma
     of the table is exactly representable, so the CUDA path must reproduce the table exactly."""

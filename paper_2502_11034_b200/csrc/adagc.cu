@@ -135,6 +135,29 @@ __device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p);
 __device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
 __device__ __forceinline__ void st_stream(uint4* p, uint4 v) { __stcs(p, v); }
 
+// L2 eviction-priority policies (createpolicy) and loads that carry one.  The norm kernel marks the gradient lines
+// it reads evict_last, the bulk-async update kernel marks everything it moves evict_first.  Measured on B200 with
+// all three hints together: 29.12 -> 28.73 ms on the 7B-shaped layout, 5.36 -> 5.30 ms on the 1B-shaped one,
+// 1.065 -> 1.039 ms on the layout of 20 000 small tensors, no change on the GPT-2-small-shaped one; any subset of
+// the hints alone measured slower than none.
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint4 ld_nc_l2_hint(const uint4* ptr, uint64_t policy) {
+  uint4 v;
+  asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(ptr), "l"(policy));
+  return v;
+}
+
 __device__ __forceinline__ double sq_acc(double acc, float x) {
   const double d = (double)x;
   return fma(d, d, acc);
@@ -147,19 +170,21 @@ __device__ __forceinline__ double sq_acc(double acc, float x) {
 // threads: fixed element -> thread mapping, float64 per-thread accumulators, fixed shuffle tree, then a
 // fixed-order sum of the warp totals.  The result is valid in thread 0.  Ends with a barrier, so
 // `warp_part` can be reused at once.
-template <bool kBF16>
+// kKeepInL2: load with the evict_last policy (the step's norm phase, whose gradient is read again by the update).
+template <bool kBF16, bool kKeepInL2 = false>
 __device__ __forceinline__ double block_chunk_sumsq(const uint4* __restrict__ vec, int count, double* warp_part) {
   constexpr int kEPV = kBF16 ? 8 : 4;  // elements per 16-byte vector
   constexpr int kUnroll = 8;           // independent 16-byte loads in flight per thread
   const int tid = threadIdx.x;
   const int nvec = count / kEPV;
   double acc0 = 0.0, acc1 = 0.0;
+  const uint64_t keep = kKeepInL2 ? l2_policy_evict_last() : 0ull;
   for (int base = 0; base < nvec; base += kThreads * kUnroll) {
     uint4 q[kUnroll];
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
       const int i = base + u * kThreads + tid;
-      q[u] = (i < nvec) ? __ldg(vec + i) : make_uint4(0u, 0u, 0u, 0u);
+      q[u] = (i < nvec) ? (kKeepInL2 ? ld_nc_l2_hint(vec + i, keep) : __ldg(vec + i)) : make_uint4(0u, 0u, 0u, 0u);
     }
 #pragma unroll
     for (int u = 0; u < kUnroll; ++u) {
@@ -214,7 +239,7 @@ adagc_norm_kernel(const void* __restrict__ grads, const Chunk* __restrict__ chun
     const Chunk ck = chunks[c];
     const uint4* vec =
         reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + chunk_start(ck) * (kBF16 ? 2 : 4));
-    const double s = block_chunk_sumsq<kBF16>(vec, ck.count, warp_part);
+    const double s = block_chunk_sumsq<kBF16, true>(vec, ck.count, warp_part);
     if (threadIdx.x == 0) partials[ck.partial] = s;
   }
 }
@@ -671,15 +696,17 @@ __global__ void adagc_debug_wait_kernel(uint64_t limit_ns, int* __restrict__ sta
   const bool arrived = mbar_wait_bounded(&bar, 0, limit_ns);
   if (!__syncthreads_and(arrived ? 1 : 0) && threadIdx.x == 0) atomicOr(status, ADAGC_E_TIMEOUT);
 }
-__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(smem_dst)),
-               "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
+__device__ __forceinline__ void bulk_load_hint(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar,
+                                               uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+      : "memory");
 }
-__device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, uint32_t bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(smem_src)),
-               "r"(bytes)
+__device__ __forceinline__ void bulk_store_hint(void* gdst, const void* smem_src, uint32_t bytes, uint64_t policy) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::"l"(gdst),
+               "r"(smem_u32(smem_src)), "r"(bytes), "l"(policy)
                : "memory");
 }
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
@@ -718,15 +745,17 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
   }
   __syncthreads();
 
+  const uint64_t stream_policy = l2_policy_evict_first();  // every byte this kernel moves is used once
   // thread 0 only: start the four loads of one tile (tile `sub` of the chunk that starts at element e0)
   auto issue_tile = [&](int64_t e0, int sub, int s) {
     const int64_t e = e0 + static_cast<int64_t>(sub) * kTile;
     unsigned char* b = tile_smem + static_cast<size_t>(s) * stage_stride;
     mbar_arrive_expect_tx(&full_bar[s], kStageBytes);
-    bulk_load(b, params + e, kTile * 4, &full_bar[s]);
-    bulk_load(b + kTile * 4, m_arena + e, kTile * 4, &full_bar[s]);
-    if (kOpt == kOptAdamW) bulk_load(b + kTile * 8, v_arena + e, kTile * 4, &full_bar[s]);
-    bulk_load(b + kTile * kStateBytes, static_cast<const char*>(grads) + e * kGBytes, kTile * kGBytes, &full_bar[s]);
+    bulk_load_hint(b, params + e, kTile * 4, &full_bar[s], stream_policy);
+    bulk_load_hint(b + kTile * 4, m_arena + e, kTile * 4, &full_bar[s], stream_policy);
+    if (kOpt == kOptAdamW) bulk_load_hint(b + kTile * 8, v_arena + e, kTile * 4, &full_bar[s], stream_policy);
+    bulk_load_hint(b + kTile * kStateBytes, static_cast<const char*>(grads) + e * kGBytes, kTile * kGBytes, &full_bar[s],
+                   stream_policy);
   };
 
   bool healthy = true;
@@ -786,10 +815,10 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
       }
       if (tid == 0) {
         const int64_t e = chunk_start(ck) + static_cast<int64_t>(sub) * kTile;
-        bulk_store(params + e, b, kTile * 4);
-        bulk_store(m_arena + e, b + kTile * 4, kTile * 4);
-        if (kOpt == kOptAdamW) bulk_store(v_arena + e, b + kTile * 8, kTile * 4);
-        if (lowp) bulk_store(lowp + e, b + kStageBytes, kTile * 2);
+        bulk_store_hint(params + e, b, kTile * 4, stream_policy);
+        bulk_store_hint(m_arena + e, b + kTile * 4, kTile * 4, stream_policy);
+        if (kOpt == kOptAdamW) bulk_store_hint(v_arena + e, b + kTile * 8, kTile * 4, stream_policy);
+        if (lowp) bulk_store_hint(lowp + e, b + kStageBytes, kTile * 2, stream_policy);
         bulk_commit();
       }
       if (last_of_chunk) {

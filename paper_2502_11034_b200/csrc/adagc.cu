@@ -130,13 +130,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
 }
 
-__device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
 __device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
 __device__ __forceinline__ void st_stream(uint4* p, uint4 v) { __stcs(p, v); }
 
 // L2 eviction-priority policies (createpolicy) and loads that carry one.  The norm kernel marks the gradient lines
-// it reads evict_last, the bulk-async update kernel marks everything it moves evict_first.  Measured on B200 with
+// it reads evict_last; the bulk-async update kernel marks everything it moves evict_first, and the register paths
+// (partial chunks, the register-streaming update kernel, the clip-only scale kernel) make their one read of the
+// gradient an evict_first load, which hands those lines back.  Measured on B200 with
 // all three hints together: 29.12 -> 28.73 ms on the 7B-shaped layout, 5.36 -> 5.30 ms on the 1B-shaped one,
 // 1.065 -> 1.039 ms on the layout of 20 000 small tensors, no change on the GPT-2-small-shaped one; any subset of
 // the hints alone measured slower than none.
@@ -155,6 +156,15 @@ __device__ __forceinline__ uint4 ld_nc_l2_hint(const uint4* ptr, uint64_t policy
   asm volatile("ld.global.nc.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                : "l"(ptr), "l"(policy));
+  return v;
+}
+
+__device__ __forceinline__ uint4 ld_l2_hint(const uint4* ptr, uint64_t policy) {  // coherent variant (in-place users)
+  uint4 v;
+  asm volatile("ld.global.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(ptr), "l"(policy)
+               : "memory");
   return v;
 }
 
@@ -523,12 +533,16 @@ __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gba
                                              const AdamScalars& a, uint4* __restrict__ lowp8 = nullptr) {
   float g[8];
   if (kBF16) {
-    const uint4 q = ld_stream(reinterpret_cast<const uint4*>(gbase) + i);
+    // the norm kernel left these lines marked evict_last; this last read of them hands them back
+    const uint4 q = ld_nc_l2_hint(reinterpret_cast<const uint4*>(gbase) + i, l2_policy_evict_first());
     g[0] = bf16_lo(q.x); g[1] = bf16_hi(q.x); g[2] = bf16_lo(q.y); g[3] = bf16_hi(q.y);
     g[4] = bf16_lo(q.z); g[5] = bf16_hi(q.z); g[6] = bf16_lo(q.w); g[7] = bf16_hi(q.w);
   } else {
-    const float4 ga = ld_stream(reinterpret_cast<const float4*>(gbase) + 2 * i);
-    const float4 gb = ld_stream(reinterpret_cast<const float4*>(gbase) + 2 * i + 1);
+    const uint64_t done = l2_policy_evict_first();
+    const uint4 qa = ld_nc_l2_hint(reinterpret_cast<const uint4*>(gbase) + 2 * i, done);
+    const uint4 qb = ld_nc_l2_hint(reinterpret_cast<const uint4*>(gbase) + 2 * i + 1, done);
+    const float4 ga = make_float4(__uint_as_float(qa.x), __uint_as_float(qa.y), __uint_as_float(qa.z), __uint_as_float(qa.w));
+    const float4 gb = make_float4(__uint_as_float(qb.x), __uint_as_float(qb.y), __uint_as_float(qb.z), __uint_as_float(qb.w));
     g[0] = ga.x; g[1] = ga.y; g[2] = ga.z; g[3] = ga.w;
     g[4] = gb.x; g[5] = gb.y; g[6] = gb.z; g[7] = gb.w;
   }
@@ -893,6 +907,7 @@ adagc_scale_kernel(const void* __restrict__ gin, void* __restrict__ gout, const 
   constexpr int kBatch = ADAGC_SCALE_BATCH;  // 16-byte loads in flight per thread
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   int row_base = 0;  // rows (32 vectors) dealt so far: successive chunks continue one round-robin over the warps
+  const uint64_t done = l2_policy_evict_first();
   const int c_end = block_begin[blockIdx.x + 1];
   for (int c = block_begin[blockIdx.x]; c < c_end; ++c) {
     const Chunk ck = chunks[c];
@@ -908,7 +923,7 @@ adagc_scale_kernel(const void* __restrict__ gin, void* __restrict__ gout, const 
 #pragma unroll
       for (int u = 0; u < kBatch; ++u) {
         const int i = ((r0 + u * kWarps) << 5) + lane;
-        if (i < nvec) q[u] = ld_stream(src + i);
+        if (i < nvec) q[u] = ld_l2_hint(src + i, done);  // last read of lines the norm kernel marked evict_last
       }
 #pragma unroll
       for (int u = 0; u < kBatch; ++u) {

@@ -42,10 +42,10 @@ UNIT = "params/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
-# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the update kernel: 25.54 B/param measured on
-# the GPT-2-small-shaped layout (committed ncu summary of that capture: 3178.5 MB for 124 439 808
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the update kernel: 25.53 B/param measured on
+# the GPT-2-small-shaped layout (committed ncu summary of that capture: 3177.4 MB for 124 439 808
 # params), scaled by the parameter count because the traffic of this streaming kernel grows in proportion.
-TRAFFIC_BYTES_PER_PARAM = {"bf16": 3178.501e6 / 124439808}
+TRAFFIC_BYTES_PER_PARAM = {"bf16": 3177.385e6 / 124439808}
 
 
 # ------------------------------------------------------------------------------------ helpers

@@ -77,6 +77,14 @@ typedef enum {
  * numel == 0 -- this rank holds no element of it -- so that every rank keeps the same tensor numbering and
  * the same n_tensors-long vectors (gamma, sums of squares); the offset of an empty tensor is ignored. */
 #define ADAGC_ALLOW_EMPTY 16
+/* Small layouts: adagc_step runs as ONE kernel (norm, decisions and AdamW separated by grid-wide barriers inside a
+ * cooperative launch) instead of three.  Worth it only where the three dependent launches cost more than the data
+ * movement (a few MB of arenas); accepted for layouts of at most 4096 chunks of 16384 elements (adagc_create
+ * returns ADAGC_E_INVALID_ARG beyond that, with ADAGC_CLIP_GLOBAL_ADAPTIVE, or on a device without cooperative
+ * launch).  Only adagc_step takes the fused route; every other entry point of the context is unchanged.  The
+ * barriers wait with a time limit; if one gives up, ADAGC_E_TIMEOUT is set in the status word and the context must
+ * be created anew. */
+#define ADAGC_FUSED_SMALL 32
 
 /* One parameter tensor. */
 typedef struct {

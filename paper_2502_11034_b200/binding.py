@@ -16,7 +16,7 @@ ADAGC_F32, ADAGC_BF16 = 0, 1
 ADAGC_W_NONFINITE = 1
 ADAGC_E_TIMEOUT = 2
 UPDATE_PATH_AUTO, UPDATE_PATH_REGISTERS, UPDATE_PATH_BULK = 0, 1, 2
-EMA_KEEP_INITIAL, CLIP_GLOBAL_ADAPTIVE, ALLOW_EMPTY = 4, 8, 16
+EMA_KEEP_INITIAL, CLIP_GLOBAL_ADAPTIVE, ALLOW_EMPTY, FUSED_SMALL = 4, 8, 16, 32
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libadagc.so")
 _lib = None

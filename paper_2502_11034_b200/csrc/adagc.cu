@@ -65,6 +65,7 @@ constexpr int kMaxGrid = 8192;          // entries reserved for each block_begin
 // (two block barriers and a table fetch per chunk) balances best with a larger constant than the update grid
 constexpr int kChunkFixedCost = 1024;
 constexpr int kChunkFixedCostWide = 8192;
+constexpr int64_t kFusedMaxChunks = 4096;  // largest layout (64 Mi elements) the one-kernel step accepts
 // adagc_step_host in steady state: the tensors are cut (in arena order) into at most kMaxGroups groups; each
 // group's gradients are copied on a second stream while the previous groups run norm/finalize/update.
 constexpr int kMaxGroups = 64;
@@ -287,6 +288,24 @@ __device__ __forceinline__ void adagc_decide(int i, double s, const ClipScalars&
   if (!isfinite(s)) atomicOr(st.status, ADAGC_W_NONFINITE);
 }
 
+// Fixed-order sum of one tensor's chunk partials by one warp (identical in every lane on return).
+__device__ __forceinline__ double tensor_partial_sum(const double* __restrict__ partials, const TensorEntry te, int lane) {
+  double acc = 0.0;
+  // the additions stay in index order; batching only lets the loads of the next terms start early (the embedding
+  // of a large model has thousands of partials, and one warp walks them)
+  const double* __restrict__ tp = partials + te.first_chunk;
+  int j = lane;
+  for (; j + 15 * 32 < te.n_chunks; j += 16 * 32) {
+    double t[16];
+#pragma unroll
+    for (int u = 0; u < 16; ++u) t[u] = __ldcg(tp + j + u * 32);
+#pragma unroll
+    for (int u = 0; u < 16; ++u) acc += t[u];
+  }
+  for (; j < te.n_chunks; j += 32) acc += __ldcg(tp + j);
+  return warp_sum(acc);
+}
+
 // One warp per tensor: fixed-order sum of the tensor's chunk partials; in the AdaGC branch the
 // same warp takes the decision.
 __global__ void __launch_bounds__(kFinalizeThreads)
@@ -304,21 +323,7 @@ adagc_tensor_finalize_kernel(const double* __restrict__ partials, const TensorEn
   const int lane = threadIdx.x & 31;
   if (k >= count) return;
   const int w = order ? order[first + k] : first + k;
-  const TensorEntry te = tensors[w];
-  double acc = 0.0;
-  // the additions stay in index order; unrolling only lets the loads of the next terms start early (the embedding
-  // of a large model has thousands of partials, and one warp walks them)
-  const double* __restrict__ tp = partials + te.first_chunk;
-  int j = lane;
-  for (; j + 15 * 32 < te.n_chunks; j += 16 * 32) {
-    double t[16];
-#pragma unroll
-    for (int u = 0; u < 16; ++u) t[u] = __ldcg(tp + j + u * 32);
-#pragma unroll
-    for (int u = 0; u < 16; ++u) acc += t[u];
-  }
-  for (; j < te.n_chunks; j += 32) acc += __ldcg(tp + j);
-  acc = warp_sum(acc);
+  const double acc = tensor_partial_sum(partials, tensors[w], lane);
   if (lane == 0) {
     st.sumsq[w] = acc;
     if (decide) {
@@ -381,28 +386,25 @@ __global__ void adagc_step_prologue_kernel(const unsigned long long* __restrict_
 
 // Warm-up branch of Algorithm 1: global norm (Eq. 2), one clip factor for every tensor, and
 // gamma_t,i = min{gamma_t-1,i, ||hat(g)_t,i||} with gamma_0,i = ||hat(g)_1,i||.  One block.
-__global__ void __launch_bounds__(kWarmupThreads)
-adagc_warmup_finalize_kernel(ClipScalars cs, float* __restrict__ ema, StatPtrs st,
-                             const DeviceStep* __restrict__ ds = nullptr) {
-  if (ds) {  // capturable step: always launched, does nothing outside warm-up
-    if (!ds->in_warmup) return;
-    cs = ds->cs;
-  }
-  __shared__ double warp_part[kWarmupThreads / 32];
-  __shared__ double total_s;
+// Body for one block of kBlock threads (warp_part: kBlock / 32 doubles of shared memory, total_s: one).
+template <int kBlock>
+__device__ __forceinline__ void warmup_finalize_block(const ClipScalars& cs, float* __restrict__ ema, const StatPtrs& st,
+                                                      double* warp_part, double* total_s_ptr) {
   const int tid = threadIdx.x;
   double acc = 0.0;
-  for (int i = tid; i < cs.n_tensors; i += kWarmupThreads) acc += st.sumsq[i];
+  for (int i = tid; i < cs.n_tensors; i += kBlock) acc += st.sumsq[i];
   acc = warp_sum(acc);
   if ((tid & 31) == 0) warp_part[tid >> 5] = acc;
   __syncthreads();
   if (tid == 0) {
     double s = warp_part[0];
-    for (int k = 1; k < kWarmupThreads / 32; ++k) s += warp_part[k];
-    total_s = s;
+    for (int k = 1; k < kBlock / 32; ++k) s += warp_part[k];
+    *total_s_ptr = s;
     *st.steps_done += 1ull;
   }
   __syncthreads();
+  const double total_s = *total_s_ptr;
+  constexpr int kWarmupThreads = kBlock;  // stride of the per-tensor loop below
   const double G = sqrt(total_s);  // ||g_t||
   const bool clip_all = G > cs.lambda_abs;
   const double h = clip_all ? __ddiv_rn(cs.lambda_abs, G) : 1.0;  // min{lambda_abs / ||g_t||, 1}
@@ -425,6 +427,18 @@ adagc_warmup_finalize_kernel(ClipScalars cs, float* __restrict__ ema, StatPtrs s
     if (clip_all) st.clip_count[i] += 1ull;
     if (!isfinite(s)) atomicOr(st.status, ADAGC_W_NONFINITE);
   }
+}
+
+__global__ void __launch_bounds__(kWarmupThreads)
+adagc_warmup_finalize_kernel(ClipScalars cs, float* __restrict__ ema, StatPtrs st,
+                             const DeviceStep* __restrict__ ds = nullptr) {
+  if (ds) {  // capturable step: always launched, does nothing outside warm-up
+    if (!ds->in_warmup) return;
+    cs = ds->cs;
+  }
+  __shared__ double warp_part[kWarmupThreads / 32];
+  __shared__ double total_s;
+  warmup_finalize_block<kWarmupThreads>(cs, ema, st, warp_part, &total_s);
 }
 
 // "Global AdaGC" (the adaptivity / locality ablation of Section 5): one adaptive threshold for the whole
@@ -946,6 +960,100 @@ adagc_scale_kernel(const void* __restrict__ gin, void* __restrict__ gout, const 
 }
 
 // ------------------------------------------------------------------------------------------------
+// Small layouts: the whole step in ONE kernel.  When the arenas are a few MB, the three dependent launches of a
+// step cost more than the data movement; here every block computes the partial sums of its chunks, the grid
+// meets at a barrier, the decisions are taken (one warp per tensor; warm-up: block 0 after one more barrier), the
+// grid meets again and every block updates its chunks.  The kernel is launched cooperatively, so all blocks are
+// resident and the barriers cannot deadlock; each wait is bounded all the same.
+// ------------------------------------------------------------------------------------------------
+// Barrier number `index` (counted over all launches of this context) of a grid of gridDim.x blocks on a counter that
+// only ever grows.  Returns false if the other blocks did not arrive within the time limit.
+__device__ __forceinline__ bool grid_barrier_bounded(unsigned long long* counter, unsigned long long index) {
+  __shared__ int arrived_flag;
+  __syncthreads();  // this block's work before the barrier is complete ...
+  if (threadIdx.x == 0) {
+    __threadfence();  // ... and visible to the other blocks before the arrival is
+    atomicAdd(counter, 1ull);
+    const unsigned long long target = (index + 1ull) * gridDim.x;
+    const uint64_t t0 = global_timer_ns();
+    int ok = 1;
+    for (uint32_t spins = 1; *reinterpret_cast<volatile unsigned long long*>(counter) < target; ++spins) {
+      if ((spins & 63u) == 0 && global_timer_ns() - t0 > kWaitLimitNs) {
+        ok = 0;
+        break;
+      }
+    }
+    __threadfence();
+    arrived_flag = ok;
+  }
+  __syncthreads();
+  return arrived_flag != 0;
+}
+
+template <bool kBF16>
+__global__ void __launch_bounds__(kThreads)
+adagc_fused_small_kernel(float* __restrict__ params, const void* __restrict__ grads, float* __restrict__ m_arena,
+                         float* __restrict__ v_arena, float* ema, const Chunk* __restrict__ chunks,
+                         const int32_t* __restrict__ block_begin, const TensorEntry* __restrict__ tensors,
+                         double* partials, ClipScalars cs, int in_warmup, AdamScalars a, StatPtrs st,
+                         unsigned long long* barrier_counter, unsigned long long barrier_index) {
+  __shared__ double warp_part[kThreads / 32];
+  __shared__ double total_s;
+  const int c_begin = block_begin[blockIdx.x], c_end = block_begin[blockIdx.x + 1];
+  // phase 1: sums of squares of this block's chunks
+  for (int c = c_begin; c < c_end; ++c) {
+    const Chunk ck = chunks[c];
+    const uint4* vec =
+        reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + chunk_start(ck) * (kBF16 ? 2 : 4));
+    const double s = block_chunk_sumsq<kBF16>(vec, ck.count, warp_part);
+    if (threadIdx.x == 0) partials[ck.partial] = s;
+  }
+  bool ok = grid_barrier_bounded(barrier_counter, barrier_index);
+  // phase 2: one warp per tensor over the whole grid; outside warm-up that warp also decides
+  if (ok) {
+    const int warps = gridDim.x * (kThreads / 32);
+    const int lane = threadIdx.x & 31;
+    for (int w = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5); w < cs.n_tensors; w += warps) {
+      const double acc = tensor_partial_sum(partials, tensors[w], lane);
+      if (lane == 0) {
+        st.sumsq[w] = acc;
+        if (!in_warmup) {
+          adagc_decide(w, acc, cs, ema, st);
+          if (w == 0) *st.steps_done += 1ull;
+        }
+      }
+    }
+    if (in_warmup) {  // the global norm needs every tensor's sum first
+      ok = grid_barrier_bounded(barrier_counter, barrier_index + 1);
+      if (ok && blockIdx.x == 0) warmup_finalize_block<kThreads>(cs, ema, st, warp_part, &total_s);
+    }
+  }
+  if (ok) ok = grid_barrier_bounded(barrier_counter, barrier_index + (in_warmup ? 2 : 1));
+  if (!ok) {
+    if (threadIdx.x == 0) atomicOr(st.status, ADAGC_E_TIMEOUT);
+    return;
+  }
+  // phase 3: AdamW on this block's chunks; the clip factors were written by other blocks of this launch
+  int row_base = 0;
+  for (int c = c_begin; c < c_end; ++c) {
+    const Chunk ck = chunks[c];
+    const float h = __ldcg(st.h + ck.tensor);
+    if (ck.count == kChunkElems) {
+      const int64_t start = chunk_start(ck);
+      float4* __restrict__ p4 = reinterpret_cast<float4*>(params + start);
+      float4* __restrict__ m4 = reinterpret_cast<float4*>(m_arena + start);
+      float4* __restrict__ v4 = reinterpret_cast<float4*>(v_arena + start);
+      const char* __restrict__ gbase = static_cast<const char*>(grads) + start * (kBF16 ? 2 : 4);
+#pragma unroll 2
+      for (int k = 0; k < kChunkElems / 8 / kThreads; ++k)
+        adamw_group8<kBF16, kOptAdamW>(k * kThreads + threadIdx.x, gbase, p4, m4, v4, h, a);
+    } else {
+      adamw_partial_chunk<kBF16, kThreads, kOptAdamW>(ck, h, row_base, params, grads, m_arena, v_arena, a);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -990,7 +1098,9 @@ int validate_desc(const adagc_desc* d, int64_t* n_chunks_out, int64_t* arena_ele
   if (d->grad_dtype != ADAGC_F32 && d->grad_dtype != ADAGC_BF16) return ADAGC_E_DTYPE;
   if (!(d->lambda_abs > 0.0) || !std::isfinite(d->lambda_abs)) return ADAGC_E_INVALID_ARG;
   constexpr int kKnownFlags =
-      ADAGC_UPDATE_PATH_MASK | ADAGC_EMA_KEEP_INITIAL | ADAGC_CLIP_GLOBAL_ADAPTIVE | ADAGC_ALLOW_EMPTY;
+      ADAGC_UPDATE_PATH_MASK | ADAGC_EMA_KEEP_INITIAL | ADAGC_CLIP_GLOBAL_ADAPTIVE | ADAGC_ALLOW_EMPTY |
+      ADAGC_FUSED_SMALL;
+  if ((d->flags & ADAGC_FUSED_SMALL) && (d->flags & ADAGC_CLIP_GLOBAL_ADAPTIVE)) return ADAGC_E_INVALID_ARG;
   const bool allow_empty = (d->flags & ADAGC_ALLOW_EMPTY) != 0;
   if ((d->flags & ~kKnownFlags) != 0 || (d->flags & ADAGC_UPDATE_PATH_MASK) == 3) return ADAGC_E_INVALID_ARG;
   const int64_t align = (d->grad_dtype == ADAGC_BF16) ? 8 : 4;
@@ -1075,6 +1185,8 @@ struct adagc_ctx {
   bool keep_initial = false;           // ADAGC_EMA_KEEP_INITIAL
   bool global_adaptive = false;        // ADAGC_CLIP_GLOBAL_ADAPTIVE
   double ema_cap = 0.0;                // adagc_set_ema_cap: > 0 selects thresholded initialization
+  bool fused_small = false;            // ADAGC_FUSED_SMALL: adagc_step runs as one cooperative kernel
+  unsigned long long barriers_done = 0;  // grid barriers executed by earlier fused launches of this context
   char* ws = nullptr;
   Layout L{};
   uint64_t launches = 0;
@@ -1314,6 +1426,45 @@ int enqueue_grouped_adamw(adagc_ctx* ctx, void* d_params, const void* d_grads, v
   return ADAGC_OK;
 }
 
+int finish_launches(adagc_ctx* ctx, cudaStream_t s) {
+  if (ctx->timing) {
+    cudaEventRecord(ctx->ev[3], s);
+    ctx->timing_valid = true;
+  }
+  return cudaGetLastError() == cudaSuccess ? ADAGC_OK : ADAGC_E_CUDA;
+}
+
+// adagc_step of a context created with ADAGC_FUSED_SMALL: one cooperative launch.
+int launch_fused_small(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, void* d_v, float* d_ema,
+                       ClipScalars cs, bool in_warmup, AdamScalars a, cudaStream_t s) {
+  if (ctx->timing) {
+    cudaEventRecord(ctx->ev[0], s);
+    cudaEventRecord(ctx->ev[1], s);
+    cudaEventRecord(ctx->ev[2], s);  // the phases are not separable here: the whole kernel is reported as the third
+  }
+  float* p = static_cast<float*>(d_params);
+  float* m = static_cast<float*>(d_m);
+  float* v = static_cast<float*>(d_v);
+  const Chunk* chunks = ctx->d_chunks_upd();
+  const int32_t* begin = ctx->d_begin_upd();
+  const TensorEntry* tensors = ctx->d_tensors();
+  double* partials = ctx->d_partials();
+  int warm = in_warmup ? 1 : 0;
+  StatPtrs st = ctx->stats();
+  unsigned long long* counter = reinterpret_cast<unsigned long long*>(ctx->ws + ctx->L.scalars + 16);
+  unsigned long long index = ctx->barriers_done;
+  void* args[] = {&p, &d_grads, &m, &v, &d_ema, &chunks, &begin, &tensors, &partials, &cs, &warm, &a, &st, &counter, &index};
+  const void* fn = ctx->bf16 ? reinterpret_cast<const void*>(adagc_fused_small_kernel<true>)
+                             : reinterpret_cast<const void*>(adagc_fused_small_kernel<false>);
+  if (cudaLaunchCooperativeKernel(fn, dim3(ctx->grid_update), dim3(kThreads), args, 0, s) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return ADAGC_E_CUDA;
+  }
+  ctx->barriers_done += in_warmup ? 3 : 2;
+  ctx->launches++;
+  return finish_launches(ctx, s);
+}
+
 void release_ctx(adagc_ctx* ctx) {
   for (int k = 0; k < 4; ++k)
     if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
@@ -1324,13 +1475,6 @@ void release_ctx(adagc_ctx* ctx) {
   delete ctx;
 }
 
-int finish_launches(adagc_ctx* ctx, cudaStream_t s) {
-  if (ctx->timing) {
-    cudaEventRecord(ctx->ev[3], s);
-    ctx->timing_valid = true;
-  }
-  return cudaGetLastError() == cudaSuccess ? ADAGC_OK : ADAGC_E_CUDA;
-}
 
 }  // namespace
 
@@ -1419,6 +1563,20 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
       ctx->grid_update = static_cast<int>(std::max<int64_t>(
           1, std::min<int64_t>({n_chunks, sms * (ctx->update_bulk ? 1 : kUpdateBlocksPerSM), kMaxGrid})));
     }
+  }
+  if (ok && (desc->flags & ADAGC_FUSED_SMALL)) {
+    // the one-kernel step needs every block resident at once (cooperative launch) and is meant for small layouts
+    int coop = 0, occ_f = 0;
+    ok = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, ctx->device) == cudaSuccess &&
+         (ctx->bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_f, adagc_fused_small_kernel<true>, kThreads, 0)
+                    : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_f, adagc_fused_small_kernel<false>, kThreads, 0)) ==
+             cudaSuccess;
+    if (ok && (!coop || n_chunks > kFusedMaxChunks ||
+               ctx->grid_update > static_cast<int64_t>(prop.multiProcessorCount) * occ_f)) {
+      release_ctx(ctx);
+      return ADAGC_E_INVALID_ARG;
+    }
+    ctx->fused_small = ok;
   }
   std::vector<Chunk> table_wide, table_upd;
   std::vector<int32_t> begin_wide, begin_upd, mid_upd;
@@ -1521,6 +1679,9 @@ int adagc_step(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, v
   rc = check_adamw_args(d_params, d_grads, d_m, d_v, lr, beta1, beta2, eps, wd);
   if (rc != ADAGC_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (ctx->fused_small)
+    return launch_fused_small(ctx, d_params, d_grads, d_m, d_v, d_ema, make_clip_scalars(ctx, step, lambda_rel, beta),
+                              step <= warmup, make_adam_scalars(step, lr, beta1, beta2, eps, wd), s);
   rc = enqueue_clip_phases(ctx, d_grads, d_ema, step, lambda_rel, beta, warmup, s);
   if (rc != ADAGC_OK) return rc;
   const AdamScalars a = make_adam_scalars(step, lr, beta1, beta2, eps, wd);

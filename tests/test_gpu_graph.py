@@ -113,3 +113,72 @@ def test_graph_replay_cuts_the_launch_cost_of_a_small_layout():
     assert us_graph < 1.5 * us_eager
     assert opt.get_stats()["status"] == 0
     opt.close()
+
+
+# ------------------------------------------------------------------ the one-kernel step for small layouts
+def _ragged(sizes, dtype):
+    specs, total = workloads._layout([(f"t{i}", (n,)) for i, n in enumerate(sizes)])
+    hp = dict(workloads.PAPER_DEFAULTS, lambda_abs=0.05)
+    return workloads.Workload("ragged", 7, specs, dtype, hp, warmup=2, n_steps=8, arena_elems=total,
+                              grad_kind="student_t", grad_df=3, grad_scale=1e-3,
+                              extra={"spike_frac": 0.2, "spike_lo": 5.0, "spike_hi": 500.0})
+
+
+def test_fused_small_step_matches_the_oracle():
+    """ADAGC_FUSED_SMALL: norm, decisions and AdamW in one cooperative kernel with grid barriers in between."""
+    F = binding.FUSED_SMALL
+    wl = workloads.build("tiny")
+    rep = H.run_full(wl, wl.n_steps, flags=F)
+    print(f"\n[parity] fused tiny: {rep.line()}")
+    assert rep.clipped > 0
+    H.run_full(wl, wl.n_steps, flags=F, hyper_over=dict(lambda_abs=0.5))                 # warm-up that clips
+    H.run_full(wl, 8, flags=F, hyper_over=dict(warmup=0))
+    sizes = [1, 7, 8, 9, 255, 2049, 16384, 16385, 3 * 16384 + 5, 100003, 40 * 16384]
+    for dtype in ("f32", "bf16"):
+        for path in (0, binding.UPDATE_PATH_REGISTERS):                                  # grids of one and two blocks per SM
+            rep = H.run_full(_ragged(sizes, dtype), 8, flags=F | path)
+            print(f"[parity] fused ragged {dtype} path {path}: {rep.line()}")
+    wl = workloads.build("many_small", n_tensors=300, lo=1, hi=40000)
+    rep = H.run_full(wl, 12, flags=F, hyper_over=dict(lambda_abs=1e4), ema_cap=0.1)
+    assert 0 < rep.clipped < rep.decisions
+    wl = workloads.build("llama2_7b", n_layer=2, d=256, ffn=688, vocab=1000)
+    rep = H.run_full(wl, 14, flags=F | binding.EMA_KEEP_INITIAL, gamma0=0.02, hyper_over=dict(warmup=0, lambda_abs=1e4))
+    assert rep.steps == 14
+
+
+def test_fused_small_limits_and_timing():
+    """Too large a layout is refused at create; on the tiny layout the one-kernel step is timed against the
+    three-launch step (printed for the record) and must not be slower."""
+    with pytest.raises(binding.AdagcError) as e:
+        binding.AdaGC([4097 * 16384], [0], torch.float32, 1.0, flags=binding.FUSED_SMALL)
+    assert e.value.status == -1
+    with pytest.raises(binding.AdagcError):
+        binding.AdaGC([1000], [0], torch.float32, 1.0, flags=binding.FUSED_SMALL | binding.CLIP_GLOBAL_ADAPTIVE)
+    wl = workloads.build("tiny")
+    hp = H.hyper_of(wl)
+    offs, nums = [t.offset for t in wl.tensors], [t.numel for t in wl.tensors]
+    a = (hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"], hp["beta"], hp["warmup"])
+    res = {}
+    for name, flags in (("three launches", 0), ("one kernel", binding.FUSED_SMALL)):
+        opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], flags=flags)
+        theta = workloads.init_params(wl, "cuda")
+        m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+        ema = torch.zeros(wl.n_tensors, device="cuda")
+        g = workloads.grads_for_step(wl, 1, "cuda")
+        t = 0
+        for _ in range(30):
+            t += 1
+            opt.step(theta, g, m, v, ema, t, *a)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(300):
+            t += 1
+            opt.step(theta, g, m, v, ema, t, *a)
+        torch.cuda.synchronize()
+        res[name] = (time.perf_counter() - t0) / 300 * 1e6
+        st = opt.get_stats()
+        assert st["status"] == 0 and st["steps_done"] == t
+        assert opt.launch_count() == (3 * t + hp["warmup"] if flags == 0 else t)   # each warm-up step: one kernel more
+        opt.close()
+    print(f"\n[timing] tiny layout, us per step: {res}")
+    assert res["one kernel"] < 1.1 * res["three launches"]

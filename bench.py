@@ -2,6 +2,7 @@
 """Benchmark of the fused AdaGC + AdamW step (Algorithm 1 of arXiv 2502.11034) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+                    [--parallel replicas|sharded]
 
 A step is one pass of the whole path (norm -> clip decision / gamma update -> AdamW on the clipped
 gradient) over every tensor of a synthetic, seeded layout; the default layout is shaped like

@@ -7,4 +7,4 @@ fails loudly if it has not been built (there is no CPU fallback).
 """
 from . import workloads  # noqa: F401
 
-__all__ = ["workloads", "binding", "build"]
+__all__ = ["workloads", "binding", "sharded", "build"]

@@ -493,7 +493,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", default=None, help="tiny | gpt2_small | llama2_7b | many_small | llama32_1b | moe_8x1b")
+    ap.add_argument("--workload", default=None, help="tiny | gpt2_small | llama2_7b | many_small | llama32_1b | moe_8x1b | moe_ernie")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--parallel", choices=["replicas", "sharded"], default="replicas",
                     help="N > 1: independent replicas (default; the data-parallel case) or flat shards of one model")

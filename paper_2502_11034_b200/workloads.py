@@ -179,7 +179,32 @@ def moe_8x1b(n_layer: int = 24, d: int = 2048, ffn: int = 5632, vocab: int = 320
                     notes="Mixtral-8x1B-shaped MoE: (7+3E)L+3 tensors, experts get heavy-tailed gradients")
 
 
-_BUILDERS = {"tiny": tiny_mlp, "moe_8x1b": moe_8x1b, "gpt2_small": gpt2_small, "llama2_7b": llama2_7b,
+def moe_ernie(n_layer: int = 25, d: int = 2560, ffn: int = 1024, vocab: int = 32000, kv_dim: int = 512,
+              n_experts: int = 48, n_shared: int = 1) -> Workload:
+    """Fine-grained mixture-of-experts layout shaped like the paper's ERNIE 10B-A1.4B run (hyper-parameter
+    table: 25 layers, hidden 2560, expert FFN 1024, 20 heads, 4 key-value heads of 128, one shared and 48
+    routed experts).  Tensor census exactly as Section 4.3 "Memory" counts it: per layer four attention
+    matrices, three matrices for each of the 1 + E experts and two norm vectors, plus embedding, final norm
+    and LM head: (9 + 3E) L + 3 = 3828 tensors.  The vocabulary size is not given in the paper; 32000 is
+    assumed (it only sets the size of two tensors)."""
+    shapes: List[Tuple[str, Tuple[int, ...]]] = [("embed", (vocab, d))]
+    for l in range(n_layer):
+        p = f"l{l}."
+        shapes += [(p + "attn_norm", (d,)), (p + "q_proj", (d, d)), (p + "k_proj", (kv_dim, d)),
+                   (p + "v_proj", (kv_dim, d)), (p + "o_proj", (d, d)), (p + "ffn_norm", (d,))]
+        for e in range(n_shared + n_experts):
+            tag = f"s{e}" if e < n_shared else f"e{e - n_shared}"
+            shapes += [(p + tag + ".gate_proj", (ffn, d)), (p + tag + ".up_proj", (ffn, d)),
+                       (p + tag + ".down_proj", (d, ffn))]
+    shapes += [("final_norm", (d,)), ("lm_head", (vocab, d))]
+    specs, total = _layout(shapes)
+    return Workload("moe_ernie", 7, specs, "bf16", dict(PAPER_DEFAULTS), warmup=5, n_steps=20, arena_elems=total,
+                    grad_kind="student_t", grad_df=3, grad_scale=1e-4,
+                    extra={"spike_frac": 0.01, "spike_lo": 10.0, "spike_hi": 1000.0},
+                    notes="ERNIE-10B-A1.4B-shaped MoE: (9+3E)L+3 tensors, 2.6 M-element expert matrices")
+
+
+_BUILDERS = {"tiny": tiny_mlp, "moe_8x1b": moe_8x1b, "moe_ernie": moe_ernie, "gpt2_small": gpt2_small, "llama2_7b": llama2_7b,
              "many_small": many_small, "llama32_1b": llama32_1b}
 
 

@@ -225,6 +225,15 @@ def test_moe_layout_small_all_elements():
     assert 0 < rep.clipped < rep.decisions
 
 
+def test_ernie_moe_layout_small_all_elements():
+    """The fine-grained MoE census the paper prints ((9+3E)L+3 tensors, Section 4.3 "Memory"), reduced dimensions."""
+    wl = workloads.build("moe_ernie", n_layer=2, d=160, ffn=64, vocab=1000, kv_dim=32, n_experts=6)
+    assert wl.n_tensors == (9 + 3 * 6) * 2 + 3
+    rep = H.run_full(wl, 20, hyper_over=dict(lambda_abs=1e4))
+    _report("ernie moe (small)", rep)
+    assert 0 < rep.clipped < rep.decisions
+
+
 @pytest.mark.parametrize("variant", ["keep_initial", "global_adaptive", "both"])
 def test_ablation_variants_all_elements(variant):
     """Section 5 variants: caller-given gamma_0 (no seeding at t = 1) and Global AdaGC (one adaptive threshold)."""

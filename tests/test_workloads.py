@@ -21,7 +21,9 @@ def test_layout_census():
     moe = W.build("moe_8x1b")
     assert moe.n_tensors == (7 + 3 * 8) * 24 + 3 == 747 and 6.5e9 < moe.n_params < 7.5e9
     assert moe.hyper["beta2"] == 0.999
-    for wl in (tiny, g2, l7, l1, ms, moe):
+    ernie = W.build("moe_ernie")                     # the census the paper itself prints: (9 + 3E) L + 3 with E = 48, L = 25
+    assert ernie.n_tensors == (9 + 3 * 48) * 25 + 3 == 3828 and 9.5e9 < ernie.n_params < 10.5e9
+    for wl in (tiny, g2, l7, l1, ms, moe, ernie):
         offs = np.array([t.offset for t in wl.tensors])
         nums = np.array([t.numel for t in wl.tensors])
         assert (offs % W.ALIGN_ELEMS == 0).all()

@@ -99,7 +99,7 @@ typedef struct {
 
 /* The model: a list of tensors plus the dtypes of the arenas. */
 typedef struct {
-  int32_t n_tensors;           /* >= 1 */
+  int32_t n_tensors;           /* 1 .. 2^24 */
   int32_t param_dtype;         /* ADAGC_F32 */
   int32_t grad_dtype;          /* ADAGC_F32 or ADAGC_BF16 */
   int32_t state_dtype;         /* ADAGC_F32 (m and v) */

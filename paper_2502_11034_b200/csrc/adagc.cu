@@ -1093,7 +1093,7 @@ Layout make_layout(int64_t n_chunks, int64_t T) {
 }
 
 int validate_desc(const adagc_desc* d, int64_t* n_chunks_out, int64_t* arena_elems_out) {
-  if (!d || !d->tensors || d->n_tensors < 1) return ADAGC_E_INVALID_ARG;
+  if (!d || !d->tensors || d->n_tensors < 1 || d->n_tensors > (1 << 24)) return ADAGC_E_INVALID_ARG;
   if (d->param_dtype != ADAGC_F32 || d->state_dtype != ADAGC_F32) return ADAGC_E_DTYPE;
   if (d->grad_dtype != ADAGC_F32 && d->grad_dtype != ADAGC_BF16) return ADAGC_E_DTYPE;
   if (!(d->lambda_abs > 0.0) || !std::isfinite(d->lambda_abs)) return ADAGC_E_INVALID_ARG;

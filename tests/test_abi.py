@@ -58,6 +58,9 @@ def test_descriptor_validation_codes():
     assert chunks([100], [0], dt=2)[0] == -5
     assert chunks([100], [0], param_dtype=binding.ADAGC_BF16)[0] == -5
     assert chunks([100], [0], flags=binding.UPDATE_PATH_BULK)[0] == 1
+    d, keep = binding.make_desc([8], [0], binding.ADAGC_F32)
+    d.n_tensors = (1 << 24) + 1                                          # more tensors than the descriptor may list
+    assert int(lib.adagc_num_chunks(C.byref(d))) == -1
     assert chunks([100], [0], flags=3)[0] == -1 and chunks([100], [0], flags=64)[0] == -1   # unknown flags
     assert chunks([100], [0], flags=binding.EMA_KEEP_INITIAL | binding.CLIP_GLOBAL_ADAPTIVE | 2)[0] == 1
     assert lib.adagc_workspace_bytes(None) == 0

@@ -351,6 +351,24 @@ def run_ours(args, wl):
                                             "frac": (bpp + 2) * wl.n_params / (emit_ms[2] * 1e-3) / 1e9 / peak}
         del lowp
 
+    # small layouts: the one-kernel step (ADAGC_FUSED_SMALL), wall clock over back-to-back steps like a training loop
+    if opt.n_chunks <= 4096:
+        fused = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=dev, flags=binding.FUSED_SMALL)
+        ema_f = torch.zeros_like(ema)
+        for name, o, e_ in (("three_launch_step_us_back_to_back", opt, ema), ("fused_small_step_us_back_to_back", fused, ema_f)):
+            tt = 100
+            for _ in range(20):
+                tt += 1
+                o.step(theta, g, m, v, e_, tt, *args_h, T_START)
+            torch.cuda.synchronize(dev)
+            w0 = time.perf_counter()
+            for _ in range(200):
+                tt += 1
+                o.step(theta, g, m, v, e_, tt, *args_h, T_START)
+            torch.cuda.synchronize(dev)
+            extra[name] = (time.perf_counter() - w0) / 200 * 1e6
+        fused.close()
+
     # ---- end to end through the host-buffer entry point
     e2e_steps = max(1, min(args.steps, 5))
     g_host = torch.empty(wl.arena_elems, dtype=wl.torch_grad_dtype).pin_memory()

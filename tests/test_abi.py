@@ -104,3 +104,41 @@ def test_binding_and_oracle_do_not_import_each_other():
         if fn.endswith((".py", ".c")):
             text = open(os.path.join(ROOT, "oracle", fn)).read()
             assert "paper_2502_11034_b200" not in text and "adagc.h" not in text
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/adagc.h must compile as C99 on its own (the boundary is a C ABI), and a C program that calls the
+    host-only entry points links against the library and gets the documented answers."""
+    import subprocess
+    src = tmp_path / "use_adagc.c"
+    src.write_text(r'''
+#include "adagc.h"
+#include <stdio.h>
+int main(void) {
+  adagc_tensor t[2] = {{0}};
+  adagc_desc d = {0};
+  adagc_tensor local[2];
+  int64_t b = -1, e = -1;
+  t[0].numel = 20000; t[0].offset = 0;
+  t[1].numel = 100;   t[1].offset = 20000;
+  d.n_tensors = 2; d.param_dtype = ADAGC_F32; d.grad_dtype = ADAGC_BF16; d.state_dtype = ADAGC_F32;
+  d.tensors = t; d.lambda_abs = 1.0;
+  if (adagc_num_chunks(&d) != 3) return 1;
+  if (adagc_workspace_bytes(&d) == 0) return 2;
+  if (adagc_shard_plan(&d, 1, 2, local, &b, &e) != ADAGC_OK) return 3;
+  if (b != 10056 || e != 20100 || local[0].numel != 20000 - 10056 || local[1].numel != 100) return 4;
+  d.lambda_abs = -1.0;
+  if (adagc_num_chunks(&d) != ADAGC_E_INVALID_ARG) return 5;
+  printf("%s\n", adagc_strerror(ADAGC_E_OVERLAP));
+  return 0;
+}
+''')
+    inc = os.path.join(ROOT, "include")
+    libdir = os.path.join(ROOT, "paper_2502_11034_b200")
+    binding.lib()                                           # the library exists (built by the build step)
+    exe = tmp_path / "use_adagc"
+    subprocess.run(["gcc", "-std=c99", "-pedantic", "-Wall", "-Werror", "-I", inc, str(src), "-o", str(exe),
+                    "-L", libdir, "-ladagc", f"-Wl,-rpath,{libdir}"], check=True)
+    out = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert out.returncode == 0, f"C program failed at check {out.returncode}"
+    assert out.stdout.strip() == "tensors overlap"

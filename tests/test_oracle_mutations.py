@@ -86,3 +86,58 @@ def test_every_planted_mistake_is_caught(name):
         except Exception as e:                            # a mistake may also crash a pin; that counts
             caught.append(f"{pin.__name__} ({type(e).__name__})")
     assert caught, f"no pin notices: {name}"
+
+
+# ---------------------------------------------------------------- the optimizer variants and the Section 5 ablations
+VARIANT_MUTATIONS = {
+    "Lion: momentum interpolation with beta2": ("a, b = beta1 * mm, (1.0 - beta1) * gh", "a, b = beta2 * mm, (1.0 - beta2) * gh"),
+    "Lion: sign of the step flipped": ("th1 = th - lr * (np.sign(c) + wd * th)", "th1 = th + lr * (np.sign(c) + wd * th)"),
+    "Lion: stored momentum uses beta1": ("m1 = beta2 * mm + (1.0 - beta2) * gh", "m1 = beta1 * mm + (1.0 - beta1) * gh"),
+    "Lion: unclipped gradient": ("gh = float(h) * np.asarray(g, dtype=np.float64)\n    a, b", "gh = np.asarray(g, dtype=np.float64)\n    a, b"),
+    "SGD: decay with the wrong sign": ("+ wd * th\n    m1 = momentum", "- wd * th\n    m1 = momentum"),
+    "SGD: dampened momentum": ("m1 = momentum * np.asarray(m, dtype=np.float64) + d", "m1 = momentum * np.asarray(m, dtype=np.float64) + (1.0 - momentum) * d"),
+    "thresholded init keeps the larger value": ("gam[i] = c[i] if c[i] < ema_cap else ema_cap", "gam[i] = c[i] if c[i] > ema_cap else ema_cap"),
+    "thresholded init keeps a running minimum": ("gam[i] = c[i] if c[i] < ema_cap else ema_cap", "gam[i] = min(gam[i], c[i], ema_cap)"),
+    "thresholded init not applied to the seed of T_start = 0": ("if ema_cap is not None and ema_cap > 0 and not gam[i] < ema_cap:", "if False:"),
+    "constant init is overwritten at t = 1": ("seed = step == 1 and not keep_initial", "seed = step == 1"),
+    "Global AdaGC uses the largest tensor only": ("one = clip_decisions([float(np.sum(s_all))]", "one = clip_decisions([float(np.max(s_all))]"),
+    "Global AdaGC keeps per-tensor gamma": ("np.full(T, one.gamma[0], dtype=state_dtype), one.global_norm", "np.asarray(gamma_prev, dtype=state_dtype), one.global_norm"),
+}
+
+VARIANT_PINS = [(pins.test_lion_closed_forms, ("numpy",)), (pins.test_lion_brute_force_and_oracles_agree, ()),
+                (pins.test_sgdm_matches_library_sgd, ("numpy",)),
+                (pins.test_thresholded_initialization_hand_values_and_special_cases, ("numpy",)),
+                (pins.test_thresholded_initialization_brute_force_and_oracles_agree, ()),
+                (pins.test_keep_initial_uses_the_callers_gamma_from_the_first_step, ("numpy",)),
+                (pins.test_global_adaptive_is_the_algorithm_on_the_concatenated_gradient, ("numpy",))]
+
+
+def _mutant_module(old, new):
+    text = open(SRC).read()
+    assert text.count(old) == 1, f"mutation anchor {old!r} must occur exactly once in the oracle"
+    mod = types.ModuleType("adagc_oracle_variant_mutant")
+    mod.__file__ = SRC
+    sys.modules[mod.__name__] = mod
+    exec(compile(text.replace(old, new), SRC, "exec"), mod.__dict__)
+    return mod
+
+
+@pytest.mark.parametrize("name", sorted(VARIANT_MUTATIONS))
+def test_every_planted_mistake_in_a_variant_is_caught(name, monkeypatch):
+    """The same game for Lion, momentum SGD and the ablation variants: the pins call the numpy oracle through the
+    name `npo` of their module, which is pointed at a mutated copy for the duration of the test."""
+    monkeypatch.setattr(pins, "npo", _mutant_module(*VARIANT_MUTATIONS[name]))
+    caught = []
+    for pin, args in VARIANT_PINS:
+        try:
+            pin(*args)
+        except AssertionError:
+            caught.append(pin.__name__)
+        except Exception as e:
+            caught.append(f"{pin.__name__} ({type(e).__name__})")
+    assert caught, f"no pin notices: {name}"
+
+
+def test_unmutated_variant_pins_pass():
+    for pin, args in VARIANT_PINS:
+        pin(*args)

@@ -283,6 +283,24 @@ def test_ragged_tails_and_chunk_edges(dtype, path):
     assert rep.clipped > 0
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_random_layouts(seed):
+    """Seeded random layouts: tensor count, sizes (log-uniform, so tails, single chunks and multi-chunk tensors
+    mix), gradient dtype, update kernel, warm-up length, thresholds and entry point all drawn at random."""
+    rng = np.random.RandomState(1000 + seed)
+    n_t = int(rng.randint(1, 60))
+    sizes = np.unique(np.round(np.exp(rng.uniform(0.0, np.log(300000.0), size=n_t))).astype(np.int64)).tolist()
+    rng.shuffle(sizes)
+    dtype = ["f32", "bf16"][int(rng.randint(2))]
+    flags = [0, binding.UPDATE_PATH_REGISTERS, binding.UPDATE_PATH_BULK, binding.FUSED_SMALL][int(rng.randint(4))]
+    over = dict(warmup=int(rng.randint(0, 4)), lambda_abs=float(np.exp(rng.uniform(np.log(1e-3), np.log(1e2)))),
+                lambda_rel=float(rng.uniform(1.0, 1.3)), beta=float(rng.uniform(0.5, 0.999)))
+    wl = _ragged_workload(sizes, dtype)
+    how = ["", "", "eager", "graph"][int(rng.randint(4))] if flags != binding.FUSED_SMALL else ""
+    rep = H.run_full(wl, 7, flags=flags, hyper_over=over, capturable=how)
+    _report(f"random layout {seed}: T={len(sizes)} {dtype} flags={flags} {over} capturable={how!r}", rep)
+
+
 def test_single_tensor_and_warmup_zero():
     """T = 1 (the 'global adaptive' view) and T_start = 0 (gamma seeded from the first norm)."""
     wl = _ragged_workload([50000], "bf16")

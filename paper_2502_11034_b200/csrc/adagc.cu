@@ -269,23 +269,39 @@ struct StatPtrs {
 };
 
 // AdaGC branch of Algorithm 1 for one tensor (Eq. 3 and the gamma update).
-__device__ __forceinline__ void adagc_decide(int i, double s, const ClipScalars& cs,
-                                             float* __restrict__ ema, const StatPtrs& st) {
-  const double n = sqrt(s);  // ||g_t,i||
+struct Decision {
+  double n, h, g_new;  // norm, clip factor, gamma after the step
+  bool clip;
+};
+
+// The arithmetic of the decision alone (no memory touched): the same inputs give the same bits wherever it runs.
+__device__ __forceinline__ Decision adagc_decision(double s, float gamma_stored, const ClipScalars& cs) {
+  Decision d;
+  d.n = sqrt(s);  // ||g_t,i||
   // gamma is fp32 state; with T_start = 0 the first step seeds it with this step's norm
-  double g_prev = cs.seed ? (double)(float)n : (double)ema[i];
+  double g_prev = cs.seed ? (double)(float)d.n : (double)gamma_stored;
   if (cs.seed && cs.ema_cap > 0.0 && !(g_prev < cs.ema_cap)) g_prev = cs.ema_cap;
   const double thr = __dmul_rn(cs.lambda_rel, g_prev);
-  const bool clip = n > thr;  // strict: equality is not a clip
-  const double h = clip ? __ddiv_rn(thr, n) : 1.0;
-  const double c = clip ? thr : n;  // clipped norm: exactly lambda_rel * gamma when active
-  const double g_new = __dadd_rn(__dmul_rn(cs.beta, g_prev), __dmul_rn(cs.one_minus_beta, c));
-  ema[i] = (float)g_new;
-  st.norm[i] = (float)n;
-  st.h[i] = (float)h;
-  st.flag[i] = clip ? 1 : 0;
-  if (clip) st.clip_count[i] += 1ull;
+  d.clip = d.n > thr;  // strict: equality is not a clip
+  d.h = d.clip ? __ddiv_rn(thr, d.n) : 1.0;
+  const double c = d.clip ? thr : d.n;  // clipped norm: exactly lambda_rel * gamma when active
+  d.g_new = __dadd_rn(__dmul_rn(cs.beta, g_prev), __dmul_rn(cs.one_minus_beta, c));
+  return d;
+}
+
+__device__ __forceinline__ void adagc_commit(int i, double s, const Decision& d, float* __restrict__ ema,
+                                             const StatPtrs& st) {
+  ema[i] = (float)d.g_new;
+  st.norm[i] = (float)d.n;
+  st.h[i] = (float)d.h;
+  st.flag[i] = d.clip ? 1 : 0;
+  if (d.clip) st.clip_count[i] += 1ull;
   if (!isfinite(s)) atomicOr(st.status, ADAGC_W_NONFINITE);
+}
+
+__device__ __forceinline__ void adagc_decide(int i, double s, const ClipScalars& cs,
+                                             float* __restrict__ ema, const StatPtrs& st) {
+  adagc_commit(i, s, adagc_decision(s, ema[i], cs), ema, st);
 }
 
 // Fixed-order sum of one tensor's chunk partials by one warp (identical in every lane on return).
@@ -996,44 +1012,93 @@ adagc_fused_small_kernel(float* __restrict__ params, const void* __restrict__ gr
                          float* __restrict__ v_arena, float* ema, const Chunk* __restrict__ chunks,
                          const int32_t* __restrict__ block_begin, const TensorEntry* __restrict__ tensors,
                          double* partials, ClipScalars cs, int in_warmup, AdamScalars a, StatPtrs st,
-                         unsigned long long* barrier_counter, unsigned long long barrier_index) {
+                         unsigned long long* barrier_counter, unsigned long long barrier_index, float* gamma_prev) {
   __shared__ double warp_part[kThreads / 32];
   __shared__ double total_s;
+  __shared__ float h_shared;
   const int c_begin = block_begin[blockIdx.x], c_end = block_begin[blockIdx.x + 1];
-  // phase 1: sums of squares of this block's chunks
+  // phase 1: sums of squares of this block's chunks; the block that holds a tensor's first chunk also sets aside
+  // the gamma the step starts from, so that after the barrier any block can take that tensor's decision
   for (int c = c_begin; c < c_end; ++c) {
     const Chunk ck = chunks[c];
     const uint4* vec =
         reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + chunk_start(ck) * (kBF16 ? 2 : 4));
     const double s = block_chunk_sumsq<kBF16>(vec, ck.count, warp_part);
-    if (threadIdx.x == 0) partials[ck.partial] = s;
+    if (threadIdx.x == 0) {
+      partials[ck.partial] = s;
+      if (!in_warmup && ck.partial == tensors[ck.tensor].first_chunk) gamma_prev[ck.tensor] = ema[ck.tensor];
+    }
   }
   bool ok = grid_barrier_bounded(barrier_counter, barrier_index);
-  // phase 2: one warp per tensor over the whole grid; outside warm-up that warp also decides
+  if (ok && !in_warmup) {
+    // AdaGC step: no second barrier.  Every block takes the decision of the tensors its chunks belong to (same
+    // partials, same order, same gamma: same bits in every block); only the block that holds a tensor's first chunk
+    // writes gamma and the statistics.  Tensors without any chunk are handled by a grid-wide loop.
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int warps = gridDim.x * (kThreads / 32);
+    for (int w = blockIdx.x * (kThreads / 32) + warp; w < cs.n_tensors; w += warps) {
+      if (tensors[w].n_chunks != 0 || lane != 0) continue;
+      st.sumsq[w] = 0.0;
+      adagc_decide(w, 0.0, cs, ema, st);
+      if (w == 0) *st.steps_done += 1ull;
+    }
+    int cur = -1, row_base = 0;
+    float h = 1.0f;
+    Decision d = {};
+    double s_cur = 0.0;
+    int first_chunk = -1;
+    for (int c = c_begin; c < c_end; ++c) {
+      const Chunk ck = chunks[c];
+      if (ck.tensor != cur) {  // uniform over the block
+        cur = ck.tensor;
+        __syncthreads();  // everyone has read h_shared of the previous tensor
+        if (warp == 0) {
+          const TensorEntry te = tensors[cur];
+          s_cur = tensor_partial_sum(partials, te, lane);
+          first_chunk = te.first_chunk;
+          d = adagc_decision(s_cur, __ldcg(gamma_prev + cur), cs);
+          if (lane == 0) h_shared = (float)d.h;
+        }
+        __syncthreads();
+        h = h_shared;
+      }
+      if (threadIdx.x == 0 && ck.partial == first_chunk) {  // this block owns the tensor's record
+        st.sumsq[cur] = s_cur;
+        adagc_commit(cur, s_cur, d, ema, st);
+        if (cur == 0) *st.steps_done += 1ull;
+      }
+      if (ck.count == kChunkElems) {
+        const int64_t start = chunk_start(ck);
+        float4* __restrict__ p4 = reinterpret_cast<float4*>(params + start);
+        float4* __restrict__ m4 = reinterpret_cast<float4*>(m_arena + start);
+        float4* __restrict__ v4 = reinterpret_cast<float4*>(v_arena + start);
+        const char* __restrict__ gbase = static_cast<const char*>(grads) + start * (kBF16 ? 2 : 4);
+#pragma unroll 2
+        for (int k = 0; k < kChunkElems / 8 / kThreads; ++k)
+          adamw_group8<kBF16, kOptAdamW>(k * kThreads + threadIdx.x, gbase, p4, m4, v4, h, a);
+      } else {
+        adamw_partial_chunk<kBF16, kThreads, kOptAdamW>(ck, h, row_base, params, grads, m_arena, v_arena, a);
+      }
+    }
+    return;
+  }
+  // warm-up step: the global norm couples all tensors, so the decisions wait for every tensor's sum
   if (ok) {
     const int warps = gridDim.x * (kThreads / 32);
     const int lane = threadIdx.x & 31;
     for (int w = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5); w < cs.n_tensors; w += warps) {
       const double acc = tensor_partial_sum(partials, tensors[w], lane);
-      if (lane == 0) {
-        st.sumsq[w] = acc;
-        if (!in_warmup) {
-          adagc_decide(w, acc, cs, ema, st);
-          if (w == 0) *st.steps_done += 1ull;
-        }
-      }
+      if (lane == 0) st.sumsq[w] = acc;
     }
-    if (in_warmup) {  // the global norm needs every tensor's sum first
-      ok = grid_barrier_bounded(barrier_counter, barrier_index + 1);
-      if (ok && blockIdx.x == 0) warmup_finalize_block<kThreads>(cs, ema, st, warp_part, &total_s);
-    }
+    ok = grid_barrier_bounded(barrier_counter, barrier_index + 1);
+    if (ok && blockIdx.x == 0) warmup_finalize_block<kThreads>(cs, ema, st, warp_part, &total_s);
   }
-  if (ok) ok = grid_barrier_bounded(barrier_counter, barrier_index + (in_warmup ? 2 : 1));
+  if (ok) ok = grid_barrier_bounded(barrier_counter, barrier_index + 2);
   if (!ok) {
     if (threadIdx.x == 0) atomicOr(st.status, ADAGC_E_TIMEOUT);
     return;
   }
-  // phase 3: AdamW on this block's chunks; the clip factors were written by other blocks of this launch
+  // AdamW on this block's chunks; the clip factor was written by block 0 of this launch
   int row_base = 0;
   for (int c = c_begin; c < c_end; ++c) {
     const Chunk ck = chunks[c];
@@ -1060,7 +1125,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {  // byte offsets of the workspace sections
   size_t chunks_wide, chunks_upd, begin_wide, begin_upd, mid_upd, g_chunks_wide, g_chunks_upd, g_begin_wide,
-      g_begin_upd, g_mid_upd, g_order, tensors, partials, sumsq, norm, h, clip_count, scalars, dev_step, flag,
+      g_begin_upd, g_mid_upd, g_order, tensors, partials, sumsq, norm, h, clip_count, scalars, dev_step, gamma_prev, flag,
       total;
 };
 
@@ -1087,6 +1152,7 @@ Layout make_layout(int64_t n_chunks, int64_t T) {
   L.clip_count = o; o = align_up(o + sizeof(uint64_t) * T, 256);
   L.scalars = o;    o = align_up(o + 256, 256);  // steps_done (u64) at +0, status (i32) at +8
   L.dev_step = o;   o = align_up(o + sizeof(DeviceStep), 256);
+  L.gamma_prev = o; o = align_up(o + sizeof(float) * T, 256);  // one-kernel step: gamma as it was before the step
   L.flag = o;       o = align_up(o + T, 256);
   L.total = o;
   return L;
@@ -1453,14 +1519,16 @@ int launch_fused_small(adagc_ctx* ctx, void* d_params, const void* d_grads, void
   StatPtrs st = ctx->stats();
   unsigned long long* counter = reinterpret_cast<unsigned long long*>(ctx->ws + ctx->L.scalars + 16);
   unsigned long long index = ctx->barriers_done;
-  void* args[] = {&p, &d_grads, &m, &v, &d_ema, &chunks, &begin, &tensors, &partials, &cs, &warm, &a, &st, &counter, &index};
+  float* gamma_prev = reinterpret_cast<float*>(ctx->ws + ctx->L.gamma_prev);
+  void* args[] = {&p,        &d_grads, &m,    &v, &d_ema, &chunks,  &begin, &tensors,
+                  &partials, &cs,      &warm, &a, &st,    &counter, &index, &gamma_prev};
   const void* fn = ctx->bf16 ? reinterpret_cast<const void*>(adagc_fused_small_kernel<true>)
                              : reinterpret_cast<const void*>(adagc_fused_small_kernel<false>);
   if (cudaLaunchCooperativeKernel(fn, dim3(ctx->grid_update), dim3(kThreads), args, 0, s) != cudaSuccess) {
     (void)cudaGetLastError();
     return ADAGC_E_CUDA;
   }
-  ctx->barriers_done += in_warmup ? 3 : 2;
+  ctx->barriers_done += in_warmup ? 3 : 1;
   ctx->launches++;
   return finish_launches(ctx, s);
 }

@@ -182,3 +182,31 @@ def test_fused_small_limits_and_timing():
         opt.close()
     print(f"\n[timing] tiny layout, us per step: {res}")
     assert res["one kernel"] < 1.1 * res["three launches"]
+
+
+def test_fused_small_with_tensors_the_rank_holds_nothing_of():
+    """ADAGC_ALLOW_EMPTY tensors (no chunk at all) still get their statistics and their gamma decay in the one-kernel
+    step; the result is bit-identical to the three-launch step on the same descriptor."""
+    nums, offs = [100, 0, 5000, 0, 40000], [0, 0, 104, 0, 5104]
+    total = 5104 + 40000
+    a = (1e-3, 0.9, 0.95, 1e-8, 0.1, 1.04, 0.9, 2)
+    res = []
+    for flags in (binding.ALLOW_EMPTY, binding.ALLOW_EMPTY | binding.FUSED_SMALL):
+        opt = binding.AdaGC(nums, offs, torch.float32, 0.01, flags=flags)
+        gen = torch.Generator(device="cuda").manual_seed(5)
+        theta = torch.randn(total, device="cuda", generator=gen) * 0.02
+        m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+        ema = torch.full((5,), float("nan"), device="cuda")
+        for t in range(1, 8):
+            g = torch.randn(total, device="cuda", generator=gen) * (1e-3 if t != 5 else 0.1)
+            opt.step(theta, g, m, v, ema, t, *a)
+        st = opt.get_stats()
+        res.append((theta.clone(), m.clone(), v.clone(), ema.clone(), st))
+        opt.close()
+    for x, y in zip(res[0][:4], res[1][:4]):
+        assert torch.equal(x, y)
+    for k in ("norm", "h", "flag", "clip_count"):
+        assert np.array_equal(res[0][4][k], res[1][4][k])
+    assert res[1][4]["steps_done"] == 7 and res[1][4]["status"] == 0
+    assert res[1][4]["norm"][1] == 0.0 and float(res[1][3][1]) == 0.0          # empty tensor: norm 0, gamma decayed from 0
+    assert res[0][4]["clip_count"].sum() > 0

@@ -1,7 +1,7 @@
 """Run a few fused AdaGC + AdamW steps (or clip-only steps) on a named synthetic layout.
 
     python -m paper_2502_11034_b200.run_steps --workload gpt2_small --steps 4 [--mode step|clip|lion|sgdm] [--n-layer N]
-        [--update-path auto|registers|bulk]
+        [--update-path auto|registers|bulk] [--fused-small]
 
 A minimal driver of the C ABI (adagc_create / adagc_step / adagc_clip / adagc_get_stats): useful as
 an example and as a small, short-running target for profilers.  Prints the per-phase device times.
@@ -24,6 +24,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=1, help="T_start: steps of global-norm clipping")
     ap.add_argument("--update-path", choices=["auto", "registers", "bulk"], default="auto",
                     help="kernel of the update phase (adagc_desc.flags)")
+    ap.add_argument("--fused-small", action="store_true",
+                    help="ADAGC_FUSED_SMALL: adagc_step as one cooperative kernel (small layouts, --mode step)")
     args = ap.parse_args()
     over = {} if args.n_layer is None else {"n_layer": args.n_layer}
     wl = workloads.build(args.workload, **over)
@@ -33,6 +35,8 @@ def main():
     offs, nums = [t.offset for t in wl.tensors], [t.numel for t in wl.tensors]
     flags = {"auto": binding.UPDATE_PATH_AUTO, "registers": binding.UPDATE_PATH_REGISTERS,
              "bulk": binding.UPDATE_PATH_BULK}[args.update_path]
+    if args.fused_small:
+        flags |= binding.FUSED_SMALL
     opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=dev, flags=flags)
     theta = workloads.init_params(wl, dev)
     m, v = torch.zeros_like(theta), torch.zeros_like(theta)

@@ -105,7 +105,7 @@ typedef struct {
   int32_t state_dtype;         /* ADAGC_F32 (m and v) */
   const adagc_tensor* tensors; /* host array, copied by adagc_create */
   double lambda_abs;           /* warm-up global-norm threshold of Eq. 2, > 0 (paper: 1.0) */
-  int32_t flags;               /* 0, or one ADAGC_UPDATE_PATH_* value, optionally OR-ed with the variant flags */
+  int32_t flags;               /* 0, or one ADAGC_UPDATE_PATH_* value, optionally OR-ed with the other ADAGC_* flags above */
   int32_t reserved;            /* set to 0 */
 } adagc_desc;
 
@@ -120,8 +120,8 @@ int64_t adagc_num_chunks(const adagc_desc* desc);
 /* Validate the descriptor, build the chunk table and upload it into `d_workspace`
  * (device memory, 256-byte aligned, at least adagc_workspace_bytes(desc) bytes, owned by the
  * caller and kept alive until adagc_destroy).  Synchronises `cuda_stream` once.
- * The CUDA device current at this call is the one the context is bound to: adagc_step, adagc_clip and
- * adagc_step_lion return ADAGC_E_INVALID_ARG when another device is current.  A context is not
+ * The CUDA device current at this call is the one the context is bound to: the step and clip entry
+ * points return ADAGC_E_INVALID_ARG when another device is current.  A context is not
  * thread-safe: one caller at a time. */
 int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_bytes,
                  void* cuda_stream, adagc_ctx** out);

@@ -1006,35 +1006,66 @@ __device__ __forceinline__ bool grid_barrier_bounded(unsigned long long* counter
   return arrived_flag != 0;
 }
 
+// Work unit of the one-kernel step: a slice of kSlice elements of a chunk, so that a layout of a few dozen chunks
+// still spreads over every SM.  Unit u = 4 * (table position of the chunk) + (slice in the chunk); block b takes the
+// units b, b + gridDim.x, ...  Each slice has its own partial sum (slot 4 * chunk + slice; slots of slices a short
+// chunk does not have stay zero), and a tensor's sum of squares is the fixed-order sum of its slots.
+constexpr int kSlice = 4096;
+constexpr int kSlicesPerChunk = kChunkElems / kSlice;
+
 template <bool kBF16>
 __global__ void __launch_bounds__(kThreads)
 adagc_fused_small_kernel(float* __restrict__ params, const void* __restrict__ grads, float* __restrict__ m_arena,
-                         float* __restrict__ v_arena, float* ema, const Chunk* __restrict__ chunks,
-                         const int32_t* __restrict__ block_begin, const TensorEntry* __restrict__ tensors,
-                         double* partials, ClipScalars cs, int in_warmup, AdamScalars a, StatPtrs st,
-                         unsigned long long* barrier_counter, unsigned long long barrier_index, float* gamma_prev) {
+                         float* __restrict__ v_arena, float* ema, const Chunk* __restrict__ chunks, int n_chunks,
+                         const TensorEntry* __restrict__ tensors, double* slice_partials, ClipScalars cs, int in_warmup,
+                         AdamScalars a, StatPtrs st, unsigned long long* barrier_counter,
+                         unsigned long long barrier_index, float* gamma_prev) {
   __shared__ double warp_part[kThreads / 32];
   __shared__ double total_s;
   __shared__ float h_shared;
-  const int c_begin = block_begin[blockIdx.x], c_end = block_begin[blockIdx.x + 1];
-  // phase 1: sums of squares of this block's chunks; the block that holds a tensor's first chunk also sets aside
-  // the gamma the step starts from, so that after the barrier any block can take that tensor's decision
-  for (int c = c_begin; c < c_end; ++c) {
-    const Chunk ck = chunks[c];
-    const uint4* vec =
-        reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + chunk_start(ck) * (kBF16 ? 2 : 4));
-    const double s = block_chunk_sumsq<kBF16>(vec, ck.count, warp_part);
+  const int n_units = n_chunks * kSlicesPerChunk;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  auto slices_of = [](const TensorEntry te) {
+    TensorEntry x;
+    x.first_chunk = te.first_chunk * kSlicesPerChunk;
+    x.n_chunks = te.n_chunks * kSlicesPerChunk;
+    return x;
+  };
+  // phase 1: sums of squares of this block's slices; the block that holds a tensor's very first slice also sets
+  // aside the gamma the step starts from, so that after the barrier any block can take that tensor's decision
+  for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+    const Chunk ck = chunks[u / kSlicesPerChunk];
+    const int k = u % kSlicesPerChunk, begin = k * kSlice;
+    if (begin >= ck.count) continue;  // uniform over the block
+    const int count = min(kSlice, ck.count - begin);
+    const uint4* vec = reinterpret_cast<const uint4*>(static_cast<const char*>(grads) +
+                                                      (chunk_start(ck) + begin) * (kBF16 ? 2 : 4));
+    const double s = block_chunk_sumsq<kBF16>(vec, count, warp_part);
     if (threadIdx.x == 0) {
-      partials[ck.partial] = s;
-      if (!in_warmup && ck.partial == tensors[ck.tensor].first_chunk) gamma_prev[ck.tensor] = ema[ck.tensor];
+      slice_partials[ck.partial * kSlicesPerChunk + k] = s;
+      if (!in_warmup && k == 0 && ck.partial == tensors[ck.tensor].first_chunk) gamma_prev[ck.tensor] = ema[ck.tensor];
     }
   }
   bool ok = grid_barrier_bounded(barrier_counter, barrier_index);
-  if (ok && !in_warmup) {
-    // AdaGC step: no second barrier.  Every block takes the decision of the tensors its chunks belong to (same
-    // partials, same order, same gamma: same bits in every block); only the block that holds a tensor's first chunk
-    // writes gamma and the statistics.  Tensors without any chunk are handled by a grid-wide loop.
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (ok && in_warmup) {
+    // warm-up step: the global norm couples all tensors, so the decisions wait for every tensor's sum
+    const int warps = gridDim.x * (kThreads / 32);
+    for (int w = blockIdx.x * (kThreads / 32) + warp; w < cs.n_tensors; w += warps) {
+      const double acc = tensor_partial_sum(slice_partials, slices_of(tensors[w]), lane);
+      if (lane == 0) st.sumsq[w] = acc;
+    }
+    ok = grid_barrier_bounded(barrier_counter, barrier_index + 1);
+    if (ok && blockIdx.x == 0) warmup_finalize_block<kThreads>(cs, ema, st, warp_part, &total_s);
+    if (ok) ok = grid_barrier_bounded(barrier_counter, barrier_index + 2);
+  }
+  if (!ok) {
+    if (threadIdx.x == 0) atomicOr(st.status, ADAGC_E_TIMEOUT);
+    return;
+  }
+  if (!in_warmup) {
+    // AdaGC step: no further barrier.  Every block takes the decision of the tensors its slices belong to (same
+    // partials, same order, same gamma: same bits in every block); only the block that holds a tensor's very first
+    // slice writes gamma and the statistics.  Tensors without any chunk are handled by a grid-wide loop.
     const int warps = gridDim.x * (kThreads / 32);
     for (int w = blockIdx.x * (kThreads / 32) + warp; w < cs.n_tensors; w += warps) {
       if (tensors[w].n_chunks != 0 || lane != 0) continue;
@@ -1042,19 +1073,24 @@ adagc_fused_small_kernel(float* __restrict__ params, const void* __restrict__ gr
       adagc_decide(w, 0.0, cs, ema, st);
       if (w == 0) *st.steps_done += 1ull;
     }
-    int cur = -1, row_base = 0;
-    float h = 1.0f;
-    Decision d = {};
-    double s_cur = 0.0;
-    int first_chunk = -1;
-    for (int c = c_begin; c < c_end; ++c) {
-      const Chunk ck = chunks[c];
-      if (ck.tensor != cur) {  // uniform over the block
-        cur = ck.tensor;
+  }
+  int cur = -1, row_base = 0, first_chunk = -1;
+  float h = 1.0f;
+  Decision d = {};
+  double s_cur = 0.0;
+  for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+    const Chunk ck = chunks[u / kSlicesPerChunk];
+    const int k = u % kSlicesPerChunk, begin = k * kSlice;
+    if (begin >= ck.count) continue;
+    if (ck.tensor != cur) {  // uniform over the block
+      cur = ck.tensor;
+      if (in_warmup) {
+        h = __ldcg(st.h + cur);  // written by block 0 of this launch
+      } else {
         __syncthreads();  // everyone has read h_shared of the previous tensor
         if (warp == 0) {
           const TensorEntry te = tensors[cur];
-          s_cur = tensor_partial_sum(partials, te, lane);
+          s_cur = tensor_partial_sum(slice_partials, slices_of(te), lane);
           first_chunk = te.first_chunk;
           d = adagc_decision(s_cur, __ldcg(gamma_prev + cur), cs);
           if (lane == 0) h_shared = (float)d.h;
@@ -1062,59 +1098,16 @@ adagc_fused_small_kernel(float* __restrict__ params, const void* __restrict__ gr
         __syncthreads();
         h = h_shared;
       }
-      if (threadIdx.x == 0 && ck.partial == first_chunk) {  // this block owns the tensor's record
-        st.sumsq[cur] = s_cur;
-        adagc_commit(cur, s_cur, d, ema, st);
-        if (cur == 0) *st.steps_done += 1ull;
-      }
-      if (ck.count == kChunkElems) {
-        const int64_t start = chunk_start(ck);
-        float4* __restrict__ p4 = reinterpret_cast<float4*>(params + start);
-        float4* __restrict__ m4 = reinterpret_cast<float4*>(m_arena + start);
-        float4* __restrict__ v4 = reinterpret_cast<float4*>(v_arena + start);
-        const char* __restrict__ gbase = static_cast<const char*>(grads) + start * (kBF16 ? 2 : 4);
-#pragma unroll 2
-        for (int k = 0; k < kChunkElems / 8 / kThreads; ++k)
-          adamw_group8<kBF16, kOptAdamW>(k * kThreads + threadIdx.x, gbase, p4, m4, v4, h, a);
-      } else {
-        adamw_partial_chunk<kBF16, kThreads, kOptAdamW>(ck, h, row_base, params, grads, m_arena, v_arena, a);
-      }
     }
-    return;
-  }
-  // warm-up step: the global norm couples all tensors, so the decisions wait for every tensor's sum
-  if (ok) {
-    const int warps = gridDim.x * (kThreads / 32);
-    const int lane = threadIdx.x & 31;
-    for (int w = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5); w < cs.n_tensors; w += warps) {
-      const double acc = tensor_partial_sum(partials, tensors[w], lane);
-      if (lane == 0) st.sumsq[w] = acc;
+    if (!in_warmup && threadIdx.x == 0 && k == 0 && ck.partial == first_chunk) {  // this block owns the tensor's record
+      st.sumsq[cur] = s_cur;
+      adagc_commit(cur, s_cur, d, ema, st);
+      if (cur == 0) *st.steps_done += 1ull;
     }
-    ok = grid_barrier_bounded(barrier_counter, barrier_index + 1);
-    if (ok && blockIdx.x == 0) warmup_finalize_block<kThreads>(cs, ema, st, warp_part, &total_s);
-  }
-  if (ok) ok = grid_barrier_bounded(barrier_counter, barrier_index + 2);
-  if (!ok) {
-    if (threadIdx.x == 0) atomicOr(st.status, ADAGC_E_TIMEOUT);
-    return;
-  }
-  // AdamW on this block's chunks; the clip factor was written by block 0 of this launch
-  int row_base = 0;
-  for (int c = c_begin; c < c_end; ++c) {
-    const Chunk ck = chunks[c];
-    const float h = __ldcg(st.h + ck.tensor);
-    if (ck.count == kChunkElems) {
-      const int64_t start = chunk_start(ck);
-      float4* __restrict__ p4 = reinterpret_cast<float4*>(params + start);
-      float4* __restrict__ m4 = reinterpret_cast<float4*>(m_arena + start);
-      float4* __restrict__ v4 = reinterpret_cast<float4*>(v_arena + start);
-      const char* __restrict__ gbase = static_cast<const char*>(grads) + start * (kBF16 ? 2 : 4);
-#pragma unroll 2
-      for (int k = 0; k < kChunkElems / 8 / kThreads; ++k)
-        adamw_group8<kBF16, kOptAdamW>(k * kThreads + threadIdx.x, gbase, p4, m4, v4, h, a);
-    } else {
-      adamw_partial_chunk<kBF16, kThreads, kOptAdamW>(ck, h, row_base, params, grads, m_arena, v_arena, a);
-    }
+    Chunk sub = ck;
+    sub.start4 = ck.start4 + static_cast<uint32_t>(begin / 4);
+    sub.count = min(kSlice, ck.count - begin);
+    adamw_partial_chunk<kBF16, kThreads, kOptAdamW>(sub, h, row_base, params, grads, m_arena, v_arena, a);
   }
 }
 
@@ -1125,11 +1118,11 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {  // byte offsets of the workspace sections
   size_t chunks_wide, chunks_upd, begin_wide, begin_upd, mid_upd, g_chunks_wide, g_chunks_upd, g_begin_wide,
-      g_begin_upd, g_mid_upd, g_order, tensors, partials, sumsq, norm, h, clip_count, scalars, dev_step, gamma_prev, flag,
+      g_begin_upd, g_mid_upd, g_order, tensors, partials, sumsq, norm, h, clip_count, scalars, dev_step, gamma_prev, slice_partials, flag,
       total;
 };
 
-Layout make_layout(int64_t n_chunks, int64_t T) {
+Layout make_layout(int64_t n_chunks, int64_t T, bool fused_small = false) {
   Layout L;
   size_t o = 0;
   L.chunks_wide = o; o = align_up(o + sizeof(Chunk) * n_chunks, 256);  // order of the norm / scale grid
@@ -1153,6 +1146,8 @@ Layout make_layout(int64_t n_chunks, int64_t T) {
   L.scalars = o;    o = align_up(o + 256, 256);  // steps_done (u64) at +0, status (i32) at +8
   L.dev_step = o;   o = align_up(o + sizeof(DeviceStep), 256);
   L.gamma_prev = o; o = align_up(o + sizeof(float) * T, 256);  // one-kernel step: gamma as it was before the step
+  L.slice_partials = o;  // one-kernel step: one partial per slice of a chunk
+  if (fused_small) o = align_up(o + sizeof(double) * n_chunks * 4, 256);
   L.flag = o;       o = align_up(o + T, 256);
   L.total = o;
   return L;
@@ -1252,6 +1247,7 @@ struct adagc_ctx {
   bool global_adaptive = false;        // ADAGC_CLIP_GLOBAL_ADAPTIVE
   double ema_cap = 0.0;                // adagc_set_ema_cap: > 0 selects thresholded initialization
   bool fused_small = false;            // ADAGC_FUSED_SMALL: adagc_step runs as one cooperative kernel
+  int grid_fused = 1;                  // its grid: every block resident at once
   unsigned long long barriers_done = 0;  // grid barriers executed by earlier fused launches of this context
   char* ws = nullptr;
   Layout L{};
@@ -1512,19 +1508,19 @@ int launch_fused_small(adagc_ctx* ctx, void* d_params, const void* d_grads, void
   float* m = static_cast<float*>(d_m);
   float* v = static_cast<float*>(d_v);
   const Chunk* chunks = ctx->d_chunks_upd();
-  const int32_t* begin = ctx->d_begin_upd();
+  int n_chunks = ctx->n_chunks;
   const TensorEntry* tensors = ctx->d_tensors();
-  double* partials = ctx->d_partials();
+  double* partials = reinterpret_cast<double*>(ctx->ws + ctx->L.slice_partials);
   int warm = in_warmup ? 1 : 0;
   StatPtrs st = ctx->stats();
   unsigned long long* counter = reinterpret_cast<unsigned long long*>(ctx->ws + ctx->L.scalars + 16);
   unsigned long long index = ctx->barriers_done;
   float* gamma_prev = reinterpret_cast<float*>(ctx->ws + ctx->L.gamma_prev);
-  void* args[] = {&p,        &d_grads, &m,    &v, &d_ema, &chunks,  &begin, &tensors,
+  void* args[] = {&p,        &d_grads, &m,    &v, &d_ema, &chunks,  &n_chunks, &tensors,
                   &partials, &cs,      &warm, &a, &st,    &counter, &index, &gamma_prev};
   const void* fn = ctx->bf16 ? reinterpret_cast<const void*>(adagc_fused_small_kernel<true>)
                              : reinterpret_cast<const void*>(adagc_fused_small_kernel<false>);
-  if (cudaLaunchCooperativeKernel(fn, dim3(ctx->grid_update), dim3(kThreads), args, 0, s) != cudaSuccess) {
+  if (cudaLaunchCooperativeKernel(fn, dim3(ctx->grid_fused), dim3(kThreads), args, 0, s) != cudaSuccess) {
     (void)cudaGetLastError();
     return ADAGC_E_CUDA;
   }
@@ -1551,7 +1547,7 @@ extern "C" {
 size_t adagc_workspace_bytes(const adagc_desc* desc) {
   int64_t n_chunks = 0;
   if (validate_desc(desc, &n_chunks, nullptr) != ADAGC_OK) return 0;
-  return make_layout(n_chunks, desc->n_tensors).total;
+  return make_layout(n_chunks, desc->n_tensors, (desc->flags & ADAGC_FUSED_SMALL) != 0).total;
 }
 
 int64_t adagc_num_chunks(const adagc_desc* desc) {
@@ -1567,7 +1563,7 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
   int64_t n_chunks = 0, extent = 0;
   const int rc = validate_desc(desc, &n_chunks, &extent);
   if (rc != ADAGC_OK) return rc;
-  const Layout L = make_layout(n_chunks, desc->n_tensors);
+  const Layout L = make_layout(n_chunks, desc->n_tensors, (desc->flags & ADAGC_FUSED_SMALL) != 0);
   if (!d_workspace || workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(d_workspace) & 255u))
     return ADAGC_E_WORKSPACE;
 
@@ -1639,12 +1635,13 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
          (ctx->bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_f, adagc_fused_small_kernel<true>, kThreads, 0)
                     : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_f, adagc_fused_small_kernel<false>, kThreads, 0)) ==
              cudaSuccess;
-    if (ok && (!coop || n_chunks > kFusedMaxChunks ||
-               ctx->grid_update > static_cast<int64_t>(prop.multiProcessorCount) * occ_f)) {
+    if (ok && (!coop || n_chunks > kFusedMaxChunks || occ_f < 1)) {
       release_ctx(ctx);
       return ADAGC_E_INVALID_ARG;
     }
     ctx->fused_small = ok;
+    ctx->grid_fused = static_cast<int>(std::max<int64_t>(
+        1, std::min<int64_t>(n_chunks * 4, static_cast<int64_t>(prop.multiProcessorCount) * std::min(occ_f, 2))));
   }
   std::vector<Chunk> table_wide, table_upd;
   std::vector<int32_t> begin_wide, begin_upd, mid_upd;

@@ -25,7 +25,12 @@ Readings taken where the paper is silent or ambiguous (listed in the design note
     (Section 4.2: the clip "scales the gradient norm to" that value);
   * stored state (gamma, theta, m, v) is rounded to its storage dtype after every
     step ("storage" mode, the parity reference); `state_dtype=np.float64` keeps
-    everything in float64 for invariant tests.
+    everything in float64 for invariant tests;
+  * with `moment_dtype="bf16"` the moments are STORED as bfloat16 (the paper trains in
+    bfloat16 / float8 precision and does not say how optimizer state is rounded): a step reads
+    the stored bfloat16 moments exactly, does its arithmetic in float64, updates theta from
+    the unrounded new moments, and rounds the moments to the nearest bfloat16 (ties to even)
+    only when it stores them.
 
 Parity pins: tests/test_oracle_pins.py (closed forms, library special cases,
 hand-worked example, invariants, brute force).
@@ -72,6 +77,45 @@ def sumsq(g: np.ndarray) -> float:
 
 def l2_norm(g: np.ndarray) -> float:
     return math.sqrt(sumsq(g))
+
+
+def _bf16_grid(x: np.ndarray):
+    """For finite non-zero float64 x: (q, p) with x = q * 2^(p-7), where 2^(p-7) is the spacing of bfloat16
+    values around x.  bfloat16 has 8 significand bits (one implicit, seven stored), the exponent range of
+    float32 (normal numbers from 2^-126) and subnormals with the fixed spacing 2^-133 below that."""
+    _, e = np.frexp(x)                                   # |x| = frac * 2^e with frac in [0.5, 1)
+    p = np.maximum(e - 1, -126)                          # floor(log2|x|), clamped for subnormals
+    return np.ldexp(x, 7 - p), p
+
+
+def round_to_bf16(x) -> np.ndarray:
+    """Nearest bfloat16 value of every element (round to nearest, ties to even), returned as float64."""
+    x = np.asarray(x, dtype=np.float64)
+    y = x.copy()
+    fin = np.isfinite(x) & (x != 0.0)
+    q, p = _bf16_grid(x[fin])
+    r = np.ldexp(np.rint(q), p - 7)                      # np.rint rounds halves to even
+    r[np.abs(r) >= 2.0 ** 128] = np.inf * np.sign(r[np.abs(r) >= 2.0 ** 128])    # beyond the largest finite value
+    y[fin] = r
+    return y
+
+
+def bf16_rounding_margin(x, scale) -> np.ndarray:
+    """How far each x is from the nearest point where rounding to bfloat16 changes its result (the midpoint
+    between two neighbouring bfloat16 values), divided by `scale`.  An implementation whose x differs from
+    this oracle's by less than margin * scale rounds to the same bfloat16."""
+    x = np.asarray(x, dtype=np.float64)
+    out = np.full(x.shape, np.inf)
+    fin = np.isfinite(x) & (x != 0.0)
+    q, p = _bf16_grid(x[fin])
+    frac = np.abs(q) - np.floor(np.abs(q))
+    dist = np.abs(frac - 0.5)                            # in units of the spacing 2^(p-7)
+    # just above a power of two the values below are twice as dense: the flip below 2^p is a quarter spacing under it
+    low_edge = (np.floor(np.abs(q)) == 128.0) & (p > -126)
+    dist = np.where(low_edge, np.minimum(dist, frac + 0.25), dist)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        out[fin] = dist * np.ldexp(1.0, p - 7) / np.broadcast_to(np.asarray(scale, np.float64), x.shape)[fin]
+    return out
 
 
 def clip_decisions(s: Sequence[float], gamma_prev: np.ndarray, step: int, hp: Hyper,
@@ -153,12 +197,18 @@ def clip_decisions(s: Sequence[float], gamma_prev: np.ndarray, step: int, hp: Hy
 
 
 def adamw_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray, h: float,
-                 step: int, hp: Hyper, state_dtype=np.float32
-                 ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+                 step: int, hp: Hyper, state_dtype=np.float32, moment_dtype: Optional[str] = None,
+                 return_margin: bool = False):
     """The four AdamW lines of Algorithm 1 on hat(g) = h * g, elementwise, in float64.
 
     Inputs are read in their storage dtype, the arithmetic is float64, the results are
     rounded to `state_dtype`.  Works on any array of elements of one tensor (or a sample).
+
+    moment_dtype="bf16": m and v are stored as bfloat16 (held here in float32 arrays whose values are
+    bfloat16 values).  theta is updated from the unrounded new moments; the moments are rounded to the
+    nearest bfloat16, ties to even, when stored.  Rounding is a discrete decision: with `return_margin`
+    the call also returns, per element, how close m and v came to a point where the rounding flips,
+    relative to the size of the terms they are summed from (see bf16_rounding_margin).
     """
     th = np.asarray(theta, dtype=np.float64)
     gh = float(h) * np.asarray(g, dtype=np.float64)                   # hat(g)
@@ -167,11 +217,21 @@ def adamw_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray,
     m_hat = m1 / (1.0 - hp.beta1 ** step)
     v_hat = v1 / (1.0 - hp.beta2 ** step)
     th1 = th - hp.lr * hp.wd * th - hp.lr * m_hat / (np.sqrt(v_hat) + hp.eps)
-    return th1.astype(state_dtype), m1.astype(state_dtype), v1.astype(state_dtype)
+    if moment_dtype is None:
+        return th1.astype(state_dtype), m1.astype(state_dtype), v1.astype(state_dtype)
+    if moment_dtype != "bf16":
+        raise ValueError("moment_dtype is None or 'bf16'")
+    out = (th1.astype(state_dtype), round_to_bf16(m1).astype(np.float32), round_to_bf16(v1).astype(np.float32))
+    if return_margin:
+        old_term = hp.beta1 * np.asarray(m, dtype=np.float64)      # m1 = old_term + (m1 - old_term): its two terms
+        m_scale = np.abs(old_term) + np.abs(m1 - old_term)
+        return out + (bf16_rounding_margin(m1, m_scale), bf16_rounding_margin(v1, np.abs(v1)))
+    return out
 
 
 def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, beta1: float,
-                beta2: float, wd: float, state_dtype=np.float32, return_margin: bool = False):
+                beta2: float, wd: float, state_dtype=np.float32, return_margin: bool = False,
+                moment_dtype: Optional[str] = None):
     """Lion on the clipped gradient hat(g) = h * g (Section 4.2 of the paper: the clip is
     optimizer-agnostic and is used with Lion; the update itself is Lion's published rule,
     Chen et al. 2023):
@@ -191,7 +251,8 @@ def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: f
     c = a + b
     th1 = th - lr * (np.sign(c) + wd * th)
     m1 = beta2 * mm + (1.0 - beta2) * gh
-    out = (th1.astype(state_dtype), m1.astype(state_dtype))
+    # moment_dtype="bf16": the momentum is stored as bfloat16, rounded to nearest even on store
+    out = (th1.astype(state_dtype), m1.astype(state_dtype) if moment_dtype is None else round_to_bf16(m1).astype(np.float32))
     if return_margin:
         den = np.abs(a) + np.abs(b)
         with np.errstate(divide="ignore", invalid="ignore"):
@@ -201,7 +262,7 @@ def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: f
 
 
 def sgdm_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, momentum: float,
-                wd: float, state_dtype=np.float32) -> Tuple[np.ndarray, np.ndarray]:
+                wd: float, state_dtype=np.float32, moment_dtype: Optional[str] = None) -> Tuple[np.ndarray, np.ndarray]:
     """SGD with momentum on the clipped gradient hat(g) = h * g (Section 4.2: the clip is optimizer-agnostic).
     The textbook heavy-ball form with L2 weight decay folded into the gradient, the form common libraries use:
         d     = hat(g) + wd * theta
@@ -211,8 +272,8 @@ def sgdm_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: f
     th = np.asarray(theta, dtype=np.float64)
     d = float(h) * np.asarray(g, dtype=np.float64) + wd * th
     m1 = momentum * np.asarray(m, dtype=np.float64) + d
-    th1 = th - lr * m1
-    return th1.astype(state_dtype), m1.astype(state_dtype)
+    th1 = th - lr * m1                                    # theta sees the unrounded momentum
+    return th1.astype(state_dtype), m1.astype(state_dtype) if moment_dtype is None else round_to_bf16(m1).astype(np.float32)
 
 
 def clipped_grad(g: np.ndarray, h: float) -> np.ndarray:
@@ -223,9 +284,11 @@ def clipped_grad(g: np.ndarray, h: float) -> np.ndarray:
 class AdaGCAdamW:
     """Algorithm 1 over a list of tensors; holds theta, m, v, gamma and the counters."""
 
-    def __init__(self, params: Sequence[np.ndarray], hp: Hyper, state_dtype=np.float32):
+    def __init__(self, params: Sequence[np.ndarray], hp: Hyper, state_dtype=np.float32,
+                 moment_dtype: Optional[str] = None):
         self.hp = hp
         self.dt = state_dtype
+        self.moment_dtype = moment_dtype
         self.theta = [np.array(p, dtype=state_dtype) for p in params]
         self.m = [np.zeros_like(p) for p in self.theta]               # m_0 = 0
         self.v = [np.zeros_like(p) for p in self.theta]               # v_0 = 0
@@ -249,7 +312,7 @@ class AdaGCAdamW:
         hp = self.hp if lr is None else Hyper(**{**self.hp.__dict__, "lr": lr})
         for i, g in enumerate(grads):
             self.theta[i], self.m[i], self.v[i] = adamw_update(
-                self.theta[i], g, self.m[i], self.v[i], r.h[i], self.t, hp, self.dt)
+                self.theta[i], g, self.m[i], self.v[i], r.h[i], self.t, hp, self.dt, self.moment_dtype)
         return r
 
     def clip_only(self, grads: Sequence[np.ndarray]) -> Tuple[ClipResult, List[np.ndarray]]:

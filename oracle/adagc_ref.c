@@ -256,6 +256,101 @@ void adagc_ref_sgdm(float* theta, const void* g, int g_is_bf16, float* m, int64_
   }
 }
 
+/* Distance from x to the nearest point where rounding to bfloat16 flips (the midpoint between two
+ * neighbouring bfloat16 values): an implementation whose x differs by less than this rounds alike. */
+static double bf16_flip_distance(double x) {
+  if (!isfinite(x) || x == 0.0) return INFINITY;
+  int e;
+  (void)frexp(x, &e);
+  int p = e - 1;
+  if (p < -126) p = -126;
+  double q = fabs(ldexp(x, 7 - p));
+  double frac = q - floor(q);
+  double dist = fabs(frac - 0.5); /* in units of the spacing 2^(p-7) */
+  /* just above a power of two the values below are twice as dense: the flip below 2^p is a quarter spacing under it */
+  if (floor(q) == 128.0 && p > -126 && frac + 0.25 < dist) dist = frac + 0.25;
+  return dist * ldexp(1.0, p - 7);
+}
+
+static inline void count_near_tie(uint8_t* near_tie, int64_t j, double x, double scale, double tie_tol) {
+  if (near_tie && bf16_flip_distance(x) < tie_tol * scale && near_tie[j] < 255) near_tie[j] += 1;
+}
+
+/*
+ * The AdamW lines of Algorithm 1 with the moments STORED as bfloat16 (the paper trains in bfloat16 / float8
+ * precision and does not say how optimizer state is rounded; reading taken: fp32 master theta, m and v read
+ * exactly from their stored bfloat16, float64 arithmetic, theta updated from the UNROUNDED new moments, the
+ * moments rounded to the nearest bfloat16, ties to even, when stored).  In place.  Rounding is a discrete
+ * decision: if near_tie is not NULL, near_tie[j] is incremented (saturating) whenever the new m or v lies
+ * within tie_tol, relative to the terms it is summed from, of a point where the rounding flips.
+ */
+void adagc_ref_adamw_bf16state(float* theta, const void* g, int g_is_bf16, uint16_t* m, uint16_t* v, int64_t n,
+                               double h, int64_t step, double lr, double beta1, double beta2, double eps,
+                               double wd, uint8_t* near_tie, double tie_tol) {
+  const double bc1 = 1.0 - pow(beta1, (double)step);
+  const double bc2 = 1.0 - pow(beta2, (double)step);
+  const uint16_t* gb = (const uint16_t*)g;
+  const float* gf = (const float*)g;
+#pragma omp parallel for schedule(static) if (n > 65536)
+  for (int64_t j = 0; j < n; ++j) {
+    const double gj = g_is_bf16 ? bf16_to_double(gb[j]) : (double)gf[j];
+    const double gh = h * gj;
+    const double a = beta1 * bf16_to_double(m[j]), b = (1.0 - beta1) * gh;
+    const double m1 = a + b;
+    const double v1 = beta2 * bf16_to_double(v[j]) + (1.0 - beta2) * gh * gh;
+    const double mh = m1 / bc1;
+    const double vh = v1 / bc2;
+    const double th = (double)theta[j];
+    theta[j] = (float)(th - lr * wd * th - lr * mh / (sqrt(vh) + eps));
+    count_near_tie(near_tie, j, m1, fabs(a) + fabs(b), tie_tol);
+    count_near_tie(near_tie, j, v1, v1, tie_tol);
+    m[j] = double_to_bf16(m1);
+    v[j] = double_to_bf16(v1);
+  }
+}
+
+/* Lion (see adagc_ref_lion) with the momentum stored as bfloat16, rounded to nearest even on store.
+ * near_tie counts both kinds of discrete decision: sign(c) and the rounding of m. */
+void adagc_ref_lion_bf16state(float* theta, const void* g, int g_is_bf16, uint16_t* m, int64_t n, double h,
+                              double lr, double beta1, double beta2, double wd, uint8_t* near_tie,
+                              double tie_tol) {
+  const uint16_t* gb = (const uint16_t*)g;
+  const float* gf = (const float*)g;
+#pragma omp parallel for schedule(static) if (n > 65536)
+  for (int64_t j = 0; j < n; ++j) {
+    const double gj = g_is_bf16 ? bf16_to_double(gb[j]) : (double)gf[j];
+    const double gh = h * gj;
+    const double mj = bf16_to_double(m[j]);
+    const double a = beta1 * mj, b = (1.0 - beta1) * gh;
+    const double c = a + b;
+    const double sgn = (c > 0.0) - (c < 0.0);
+    if (near_tie && fabs(c) < tie_tol * (fabs(a) + fabs(b)) && near_tie[j] < 255) near_tie[j] += 1;
+    const double th = (double)theta[j];
+    theta[j] = (float)(th - lr * (sgn + wd * th));
+    const double a2 = beta2 * mj, b2 = (1.0 - beta2) * gh;
+    count_near_tie(near_tie, j, a2 + b2, fabs(a2) + fabs(b2), tie_tol);
+    m[j] = double_to_bf16(a2 + b2);
+  }
+}
+
+/* Momentum SGD (see adagc_ref_sgdm) with the momentum stored as bfloat16; theta sees the unrounded momentum. */
+void adagc_ref_sgdm_bf16state(float* theta, const void* g, int g_is_bf16, uint16_t* m, int64_t n, double h,
+                              double lr, double momentum, double wd, uint8_t* near_tie, double tie_tol) {
+  const uint16_t* gb = (const uint16_t*)g;
+  const float* gf = (const float*)g;
+#pragma omp parallel for schedule(static) if (n > 65536)
+  for (int64_t j = 0; j < n; ++j) {
+    const double gj = g_is_bf16 ? bf16_to_double(gb[j]) : (double)gf[j];
+    const double th = (double)theta[j];
+    const double d = h * gj + wd * th;
+    const double a = momentum * bf16_to_double(m[j]);
+    const double m1 = a + d;
+    theta[j] = (float)(th - lr * m1);
+    count_near_tie(near_tie, j, m1, fabs(a) + fabs(h * gj) + fabs(wd * th), tie_tol);
+    m[j] = double_to_bf16(m1);
+  }
+}
+
 /* hat(g) = h * g written in the gradient's dtype (clip-only use with other optimizers). */
 void adagc_ref_scale(void* out, const void* g, int is_bf16, int64_t n, double h) {
   if (is_bf16) {

@@ -62,6 +62,15 @@ def lib():
                                      [C.c_void_p, C.c_double])
         L.adagc_ref_sgdm.restype = None
         L.adagc_ref_sgdm.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64] + [C.c_double] * 4
+        L.adagc_ref_adamw_bf16state.restype = None
+        L.adagc_ref_adamw_bf16state.argtypes = ([C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int64,
+                                                 C.c_double, C.c_int64] + [C.c_double] * 5 + [C.c_void_p, C.c_double])
+        L.adagc_ref_lion_bf16state.restype = None
+        L.adagc_ref_lion_bf16state.argtypes = ([C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64] +
+                                               [C.c_double] * 5 + [C.c_void_p, C.c_double])
+        L.adagc_ref_sgdm_bf16state.restype = None
+        L.adagc_ref_sgdm_bf16state.argtypes = ([C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64] +
+                                               [C.c_double] * 4 + [C.c_void_p, C.c_double])
         L.adagc_ref_scale.restype = None
         L.adagc_ref_scale.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_double]
         L.adagc_ref_step.restype = C.c_int32
@@ -127,28 +136,58 @@ def adamw_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray,
                           float(h), int(step), lr, beta1, beta2, eps, wd)
 
 
+def _tie_ptr(near_tie: Optional[np.ndarray], n: int):
+    if near_tie is None:
+        return None
+    assert near_tie.dtype == np.uint8 and near_tie.flags["C_CONTIGUOUS"] and near_tie.size == n
+    return near_tie.ctypes.data
+
+
+def _is_bf16_state(theta: np.ndarray, moments, n: int) -> bool:
+    """Moments are fp32 arrays, or uint16 arrays holding bfloat16 bit patterns (all of one kind)."""
+    assert theta.dtype == np.float32 and theta.flags["C_CONTIGUOUS"] and theta.size == n
+    kinds = {a.dtype for a in moments}
+    assert kinds in ({np.dtype(np.float32)}, {np.dtype(np.uint16)}), "moments: all float32, or all uint16 (bf16 bits)"
+    for a in moments:
+        assert a.flags["C_CONTIGUOUS"] and a.size == n
+    return kinds == {np.dtype(np.uint16)}
+
+
+def adamw_update_bf16state(theta: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray, h: float, step: int,
+                           lr: float, beta1: float, beta2: float, eps: float, wd: float,
+                           near_tie: Optional[np.ndarray] = None, tie_tol: float = 0.0) -> None:
+    """AdamW with m and v stored as bfloat16 (uint16 bit patterns), in place; theta fp32.  `near_tie` (uint8) counts,
+    per element, the steps in which the rounding of m or v was decided with a relative margin below `tie_tol`."""
+    p, bf = _grad_ptr(g)
+    assert _is_bf16_state(theta, (m, v), g.size)
+    lib().adagc_ref_adamw_bf16state(theta.ctypes.data, p, bf, m.ctypes.data, v.ctypes.data, g.size, float(h),
+                                    int(step), lr, beta1, beta2, eps, wd, _tie_ptr(near_tie, g.size), float(tie_tol))
+
+
 def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, beta1: float,
                 beta2: float, wd: float, near_tie: Optional[np.ndarray] = None, tie_tol: float = 0.0) -> None:
-    """Lion on the clipped gradient, in place on fp32 theta and m.  `near_tie` (uint8, same length) counts,
-    per element, the steps in which sign(c) was decided with a relative margin below `tie_tol`."""
+    """Lion on the clipped gradient, in place on fp32 theta and on m (fp32, or uint16 = stored as bfloat16).
+    `near_tie` (uint8, same length) counts, per element, the steps in which sign(c) -- and, for bfloat16 m, its
+    rounding -- was decided with a relative margin below `tie_tol`."""
     p, bf = _grad_ptr(g)
-    for a in (theta, m):
-        assert a.dtype == np.float32 and a.flags["C_CONTIGUOUS"] and a.size == g.size
-    nt = None
-    if near_tie is not None:
-        assert near_tie.dtype == np.uint8 and near_tie.flags["C_CONTIGUOUS"] and near_tie.size == g.size
-        nt = near_tie.ctypes.data
-    lib().adagc_ref_lion(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, beta1, beta2, wd,
-                         nt, float(tie_tol))
+    nt = _tie_ptr(near_tie, g.size)
+    if _is_bf16_state(theta, (m,), g.size):
+        lib().adagc_ref_lion_bf16state(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, beta1, beta2,
+                                       wd, nt, float(tie_tol))
+    else:
+        lib().adagc_ref_lion(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, beta1, beta2, wd,
+                             nt, float(tie_tol))
 
 
 def sgdm_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, momentum: float,
-                wd: float) -> None:
-    """SGD with momentum on the clipped gradient, in place on fp32 theta and m."""
+                wd: float, near_tie: Optional[np.ndarray] = None, tie_tol: float = 0.0) -> None:
+    """SGD with momentum on the clipped gradient, in place on fp32 theta and on m (fp32, or uint16 = bfloat16)."""
     p, bf = _grad_ptr(g)
-    for a in (theta, m):
-        assert a.dtype == np.float32 and a.flags["C_CONTIGUOUS"] and a.size == g.size
-    lib().adagc_ref_sgdm(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, momentum, wd)
+    if _is_bf16_state(theta, (m,), g.size):
+        lib().adagc_ref_sgdm_bf16state(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, momentum, wd,
+                                       _tie_ptr(near_tie, g.size), float(tie_tol))
+    else:
+        lib().adagc_ref_sgdm(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, momentum, wd)
 
 
 def scale(g: np.ndarray, h: float, out: Optional[np.ndarray] = None) -> np.ndarray:
@@ -169,14 +208,19 @@ class ArenaOracle:
     def __init__(self, offsets: Sequence[int], numels: Sequence[int], theta0: np.ndarray, *,
                  lr: float, beta1: float, beta2: float, eps: float, wd: float, lambda_rel: float,
                  beta: float, lambda_abs: float, warmup: int, keep_initial: bool = False,
-                 global_adaptive: bool = False, gamma0: Optional[np.ndarray] = None, ema_cap: float = 0.0):
+                 global_adaptive: bool = False, gamma0: Optional[np.ndarray] = None, ema_cap: float = 0.0,
+                 bf16_state: bool = False, tie_tol: float = 0.0):
+        """bf16_state: m and v are stored as bfloat16 (uint16 bit patterns), rounded to nearest even on store;
+        `self.ties` then counts, per element, the steps whose rounding was decided with a margin below tie_tol."""
         self.keep_initial, self.global_adaptive, self.ema_cap = keep_initial, global_adaptive, float(ema_cap)
+        self.bf16_state, self.tie_tol = bool(bf16_state), float(tie_tol)
         self.off = np.ascontiguousarray(offsets, dtype=np.int64)
         self.numel = np.ascontiguousarray(numels, dtype=np.int64)
         self.T = len(self.off)
         self.theta = np.array(theta0, dtype=np.float32)
-        self.m = np.zeros_like(self.theta)
-        self.v = np.zeros_like(self.theta)
+        self.m = np.zeros(self.theta.shape, np.uint16 if bf16_state else np.float32)
+        self.v = np.zeros_like(self.m)
+        self.ties = np.zeros(self.theta.shape, np.uint8) if bf16_state else None
         self.gamma = np.zeros(self.T, dtype=np.float32) if gamma0 is None else np.array(gamma0, dtype=np.float32)
         self.hp = dict(lr=lr, beta1=beta1, beta2=beta2, eps=eps, wd=wd, lambda_rel=lambda_rel,
                        beta=beta, lambda_abs=lambda_abs, warmup=warmup)
@@ -185,7 +229,7 @@ class ArenaOracle:
         self._s = np.empty(self.T, np.float64)
 
     def step(self, grads: np.ndarray, lr: Optional[float] = None):
-        if self.keep_initial or self.global_adaptive or self.ema_cap > 0:
+        if self.keep_initial or self.global_adaptive or self.ema_cap > 0 or self.bf16_state:
             return self._step_variant(grads, lr)
         self.t += 1
         p, bf = _grad_ptr(grads)
@@ -208,8 +252,12 @@ class ArenaOracle:
         hp = self.hp
         for i in range(self.T):
             o, n = int(self.off[i]), int(self.numel[i])
-            adamw_update(self.theta[o:o + n], grads[o:o + n], self.m[o:o + n], self.v[o:o + n], float(r["h"][i]),
-                         self.t, hp["lr"] if lr is None else lr, hp["beta1"], hp["beta2"], hp["eps"], hp["wd"])
+            args = (self.theta[o:o + n], grads[o:o + n], self.m[o:o + n], self.v[o:o + n], float(r["h"][i]),
+                    self.t, hp["lr"] if lr is None else lr, hp["beta1"], hp["beta2"], hp["eps"], hp["wd"])
+            if self.bf16_state:
+                adamw_update_bf16state(*args, near_tie=self.ties[o:o + n], tie_tol=self.tie_tol)
+            else:
+                adamw_update(*args)
         return r
 
     def clip(self, grads: np.ndarray):

@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 
 import test_oracle_pins as pins
+import test_oracle_pins_bf16_state as pins_bf
 
 SRC = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "oracle", "adagc_oracle.py")
 
@@ -140,4 +141,51 @@ def test_every_planted_mistake_in_a_variant_is_caught(name, monkeypatch):
 
 def test_unmutated_variant_pins_pass():
     for pin, args in VARIANT_PINS:
+        pin(*args)
+
+
+# ---------------------------------------------------------------- optimizer state stored as bfloat16
+BF16_STATE_MUTATIONS = {
+    "moments truncated instead of rounded": ("np.ldexp(np.rint(q), p - 7)", "np.ldexp(np.trunc(q), p - 7)"),
+    "ties rounded away from zero": ("np.ldexp(np.rint(q), p - 7)", "np.ldexp(np.sign(q) * np.floor(np.abs(q) + 0.5), p - 7)"),
+    "subnormals rounded on the grid of normal numbers": ("p = np.maximum(e - 1, -126) ", "p = e - 1 "),
+    "v stored unrounded": ("round_to_bf16(v1).astype(np.float32))", "v1.astype(np.float32))"),
+    "m stored unrounded": ("round_to_bf16(m1).astype(np.float32), round_to_bf16(v1)", "m1.astype(np.float32), round_to_bf16(v1)"),
+    "theta updated from the rounded first moment": ("m_hat = m1 / (1.0 - hp.beta1 ** step)",
+                                                    "m_hat = (m1 if moment_dtype is None else round_to_bf16(m1)) / (1.0 - hp.beta1 ** step)"),
+    "theta updated from the rounded second moment": ("v_hat = v1 / (1.0 - hp.beta2 ** step)",
+                                                     "v_hat = (v1 if moment_dtype is None else round_to_bf16(v1)) / (1.0 - hp.beta2 ** step)"),
+    "Lion momentum stored unrounded": ("m1.astype(state_dtype) if moment_dtype is None else round_to_bf16(m1).astype(np.float32))\n    if return_margin:",
+                                       "m1.astype(state_dtype))\n    if return_margin:"),
+    "SGD: theta sees the rounded momentum": ("th1 = th - lr * m1 ", "th1 = th - lr * (m1 if moment_dtype is None else round_to_bf16(m1)) "),
+    "SGD momentum stored unrounded": ("return th1.astype(state_dtype), m1.astype(state_dtype) if moment_dtype is None else round_to_bf16(m1).astype(np.float32)",
+                                      "return th1.astype(state_dtype), m1.astype(state_dtype)"),
+    "flip distance ignores the denser values below a power of two": ("dist = np.where(low_edge, np.minimum(dist, frac + 0.25), dist)",
+                                                                     "dist = dist + 0.0 * low_edge"),
+}
+
+BF16_STATE_PINS = [(pins_bf.test_rounding_matches_the_library_conversion_and_ties_go_to_even, ()),
+                   (pins_bf.test_rounding_margin_is_the_distance_to_a_flip, ()),
+                   (pins_bf.test_one_step_from_a_given_state_matches_library_adamw, (pins_bf.NumpyBF, 7)),
+                   (pins_bf.test_theta_is_the_fp32_state_paths_theta_bit_for_bit, (pins_bf.NumpyBF,)),
+                   (pins_bf.test_lion_and_sgdm_store_the_nearest_bf16_and_leave_theta_alone, ("numpy",)),
+                   (pins_bf.test_c_oracle_counts_decisions_close_to_a_flip, ())]
+
+
+@pytest.mark.parametrize("name", sorted(BF16_STATE_MUTATIONS))
+def test_every_planted_mistake_in_the_bf16_state_is_caught(name, monkeypatch):
+    monkeypatch.setattr(pins_bf, "npo", _mutant_module(*BF16_STATE_MUTATIONS[name]))
+    caught = []
+    for pin, args in BF16_STATE_PINS:
+        try:
+            pin(*args)
+        except AssertionError:
+            caught.append(pin.__name__)
+        except Exception as e:
+            caught.append(f"{pin.__name__} ({type(e).__name__})")
+    assert caught, f"no pin notices: {name}"
+
+
+def test_unmutated_bf16_state_pins_pass():
+    for pin, args in BF16_STATE_PINS:
         pin(*args)

@@ -1,0 +1,273 @@
+"""Pins for the oracles' bfloat16-stored optimizer state (m and v kept as bfloat16, fp32 master theta).
+
+The paper trains in bfloat16 / float8 precision (Appendix "Hyper-Parameters") and does not say how stored
+optimizer state is rounded.  Reading pinned here: a step reads the stored bfloat16 moments exactly, computes
+in float64, updates theta from the UNROUNDED new moments, and rounds the moments to the nearest bfloat16
+(ties to even) when it stores them.
+
+Nothing here touches the CUDA path.  The pins are the library's own conversion (torch .to(bfloat16) on
+fp32-exact inputs), torch.optim.AdamW / SGD in float64 started from a given state, the definition of
+"nearest representable value", a derived stall bound for a constant gradient, and numpy-vs-C agreement.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import adagc_oracle as npo
+from oracle import c_oracle as co
+
+
+def bits_to_f64(b):
+    return (np.asarray(b, np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def f32_to_bits(x):
+    """bit patterns of float32 values that are exactly bfloat16 values"""
+    u = np.asarray(x, np.float32).view(np.uint32)
+    assert (u & 0xFFFF == 0).all(), "value is not representable in bfloat16"
+    return (u >> 16).astype(np.uint16)
+
+
+def spacing_bf16(x):
+    """distance between neighbouring bfloat16 values around x (from the format: 8 significand bits)"""
+    x = np.abs(np.asarray(x, np.float64))
+    e = np.floor(np.log2(np.maximum(x, 2.0 ** -126)))
+    return 2.0 ** (np.maximum(e, -126) - 7)
+
+
+def assert_is_nearest_bf16(stored, exact, what):
+    """`stored` holds bfloat16 values and none of its neighbours is closer to `exact`."""
+    stored, exact = np.asarray(stored, np.float64), np.asarray(exact, np.float64)
+    assert (stored.astype(np.float32).view(np.uint32) & 0xFFFF == 0).all(), f"{what}: not a bfloat16 value"
+    # neighbouring bfloat16 values around `exact` are one spacing (of exact's binade) apart
+    assert (np.abs(stored - exact) <= 0.5 * spacing_bf16(exact) * (1 + 1e-12)).all(), f"{what}: not the nearest bfloat16"
+
+
+class NumpyBF:
+    name = "numpy"
+
+    @staticmethod
+    def adamw(theta, g, m, v, h, step, hp):
+        """m, v: float arrays of bfloat16 values.  Returns theta (fp32), m, v (float64 views of the stored values)."""
+        th, m1, v1 = npo.adamw_update(theta, g, m, v, h, step, hp, np.float32, moment_dtype="bf16")
+        return th, m1.astype(np.float64), v1.astype(np.float64)
+
+
+class CBF:
+    name = "c"
+
+    @staticmethod
+    def adamw(theta, g, m, v, h, step, hp):
+        th = np.array(theta, np.float32)
+        mb, vb = f32_to_bits(m), f32_to_bits(v)
+        co.adamw_update_bf16state(th, np.ascontiguousarray(g, np.float32), mb, vb, h, step, hp.lr, hp.beta1,
+                                  hp.beta2, hp.eps, hp.wd)
+        return th, bits_to_f64(mb), bits_to_f64(vb)
+
+
+BF_IMPLS = [NumpyBF, CBF]
+
+
+def bf16_values(rng, n, scale):
+    """random values that are exactly bfloat16 values (via the library's conversion of fp32 numbers)"""
+    x = torch.from_numpy((rng.standard_normal(n) * scale).astype(np.float32))
+    return x.to(torch.bfloat16).to(torch.float32).numpy()
+
+
+# ----------------------------------------------------------------------------- the rounding itself
+def test_rounding_matches_the_library_conversion_and_ties_go_to_even():
+    rng = np.random.RandomState(3)
+    x = np.concatenate([rng.standard_normal(200000) * 10.0 ** rng.uniform(-44, 38, 200000),
+                        [0.0, -0.0, 1.0, -1.0, 3.3895e38, 3.4e38, -3.4e38, 1e-40, 2.0 ** -133, 2.0 ** -134,
+                         1.5 * 2.0 ** -133, np.inf, -np.inf]]).astype(np.float32)
+    # exact ties: midpoints between neighbouring bfloat16 values, even and odd lower neighbours, both signs
+    lows = np.array([0x3F80, 0x3F81, 0x4000, 0x40FF, 0x0001, 0x0002, 0x7F7E, 0x0080, 0x007F], np.uint32)
+    mids = ((lows << 16) | 0x8000).view(np.float32)
+    x = np.concatenate([x, mids, -mids])
+    want = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()         # fp32 -> bf16: one rounding
+    got_np = npo.round_to_bf16(x.astype(np.float64))
+    assert np.array_equal(got_np.astype(np.float32).view(np.uint32), want.view(np.uint32))
+    got_c = np.array([co.double_to_bf16_bits(float(v)) for v in x[-5000:]], np.uint16)
+    assert np.array_equal(got_c, (want[-5000:].view(np.uint32) >> 16).astype(np.uint16))
+    # the tie cases really are ties and went to the even neighbour
+    tie_bits = (want[-2 * len(lows):-len(lows)].view(np.uint32) >> 16)
+    assert (tie_bits % 2 == 0).all() and np.array_equal(tie_bits, lows + (lows & 1))
+    assert np.isnan(npo.round_to_bf16(np.array([np.nan]))[0])
+
+
+def test_rounding_margin_is_the_distance_to_a_flip():
+    """bf16_rounding_margin: 0 at a midpoint, half the spacing at a bfloat16 value (a quarter at a power of two, whose
+    lower neighbours are twice as dense), and any perturbation smaller than margin * scale leaves the rounding
+    unchanged while a slightly larger one (towards the nearer flip) changes it."""
+    assert npo.bf16_rounding_margin(np.array([1.0 + 2.0 ** -8]), 1.0)[0] == 0.0
+    assert npo.bf16_rounding_margin(np.array([1.0 + 2.0 ** -7]), 1.0)[0] == 2.0 ** -8
+    assert npo.bf16_rounding_margin(np.array([1.0]), 1.0)[0] == 2.0 ** -9
+    assert npo.bf16_rounding_margin(np.array([3.0]), 2.0)[0] == 2.0 ** -7 / 2.0
+    rng = np.random.RandomState(4)
+    x = rng.standard_normal(20000) * 10.0 ** rng.uniform(-30, 30, 20000)
+    d = npo.bf16_rounding_margin(x, 1.0)
+    r0 = npo.round_to_bf16(x)
+    for sgn in (-1.0, 1.0):
+        assert np.array_equal(npo.round_to_bf16(x + sgn * 0.999 * d), r0)
+    flipped = (npo.round_to_bf16(x + 1.001 * d) != r0) | (npo.round_to_bf16(x - 1.001 * d) != r0)
+    assert flipped.all()
+
+
+# ----------------------------------------------------------------------------- one step against the library
+@pytest.mark.parametrize("impl", BF_IMPLS, ids=lambda i: i.name)
+@pytest.mark.parametrize("step", [1, 2, 7, 100])
+def test_one_step_from_a_given_state_matches_library_adamw(impl, step):
+    """torch.optim.AdamW (float64) started from the same theta, m, v and step count: theta agrees (so theta was
+    updated from the unrounded moments), and the stored moments are the bfloat16 values nearest to the library's."""
+    rng = np.random.RandomState(100 + step)
+    n = 4096
+    hp = npo.Hyper(lr=3e-3, beta1=0.9, beta2=0.95, eps=1e-8, wd=0.1)
+    theta0 = (rng.standard_normal(n) * 0.5).astype(np.float32)
+    g = (rng.standard_t(3, size=n) * 1e-2).astype(np.float32)
+    h = 0.37
+    if step == 1:
+        m0, v0 = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    else:
+        m0 = bf16_values(rng, n, 1e-2)
+        v0 = bf16_values(rng, n, 1e-2) ** 2
+        v0 = torch.from_numpy(v0).to(torch.bfloat16).to(torch.float32).numpy()
+    p = torch.tensor(theta0.astype(np.float64), requires_grad=True)
+    opt = torch.optim.AdamW([p], lr=hp.lr, betas=(hp.beta1, hp.beta2), eps=hp.eps, weight_decay=hp.wd, foreach=False)
+    opt.state[p] = {"step": torch.tensor(float(step - 1)), "exp_avg": torch.tensor(m0.astype(np.float64)),
+                    "exp_avg_sq": torch.tensor(v0.astype(np.float64))}
+    p.grad = torch.tensor(h * g.astype(np.float64))
+    opt.step()
+    th, m1, v1 = impl.adamw(theta0, g, m0, v0, h, step, hp)
+    np.testing.assert_allclose(th, p.detach().numpy(), rtol=1.2e-7, atol=1e-30)           # fp32 storage of theta only
+    assert_is_nearest_bf16(m1, opt.state[p]["exp_avg"].numpy(), "m")
+    assert_is_nearest_bf16(v1, opt.state[p]["exp_avg_sq"].numpy(), "v")
+    assert (m1 != opt.state[p]["exp_avg"].numpy()).mean() > 0.9, "the moments were not rounded at all"
+
+
+@pytest.mark.parametrize("impl", BF_IMPLS, ids=lambda i: i.name)
+def test_theta_is_the_fp32_state_paths_theta_bit_for_bit(impl):
+    """Rounding happens on store only: from the same stored inputs the step's theta equals, bit for bit, the theta of
+    the (separately pinned) fp32-state update, and the stored moments are the nearest bfloat16 of its float64 moments."""
+    rng = np.random.RandomState(8)
+    n = 3000
+    hp = npo.Hyper(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-15, wd=0.05)
+    theta0 = (rng.standard_normal(n) * 0.02).astype(np.float32)
+    m0, v0 = bf16_values(rng, n, 1e-4), bf16_values(rng, n, 1e-8).__abs__()
+    g = (rng.standard_normal(n) * 1e-4).astype(np.float32)
+    th, m1, v1 = impl.adamw(theta0, g, m0, v0, 1.0, 5, hp)
+    th_ref, _, _ = npo.adamw_update(theta0, g, m0, v0, 1.0, 5, hp, np.float32)
+    _, m64, v64 = npo.adamw_update(theta0, g, m0, v0, 1.0, 5, hp, np.float64)
+    assert np.array_equal(th.view(np.uint32), th_ref.view(np.uint32))
+    assert_is_nearest_bf16(m1, m64, "m")
+    assert_is_nearest_bf16(v1, v64, "v")
+
+
+# ----------------------------------------------------------------------------- an invariant of the iteration
+@pytest.mark.parametrize("impl", BF_IMPLS, ids=lambda i: i.name)
+def test_constant_gradient_stalls_within_the_derived_bound(impl):
+    """With a constant gradient the fp32-state moments converge to g and g^2.  Stored as bfloat16 the iteration
+    x <- round(beta x + (1 - beta) c) stops moving once the increment (1 - beta)|c - x| is below half the spacing, so
+    it ends within spacing / (2 (1 - beta)) of the fixed point (plus one spacing for the last rounding), and approaches
+    it monotonically.  beta1 = 0.9: 5 spacings; beta2 = 0.95: 10 spacings."""
+    rng = np.random.RandomState(9)
+    n = 512
+    hp = npo.Hyper(lr=0.0, beta1=0.9, beta2=0.95, wd=0.0)
+    g = (np.abs(rng.standard_normal(n)) * 1e-3 + 1e-4).astype(np.float32)
+    theta = np.zeros(n, np.float32)
+    m, v = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    prev_m, prev_v = m.astype(np.float64), v.astype(np.float64)
+    for t in range(1, 301):
+        theta, m, v = impl.adamw(theta, g, m.astype(np.float32), v.astype(np.float32), 1.0, t, hp)
+        assert (m >= prev_m).all() and (v >= prev_v).all()            # monotone approach from below
+        prev_m, prev_v = m, v
+    g64 = g.astype(np.float64)
+    assert (np.abs(m - g64) <= spacing_bf16(g64) * (0.5 / (1 - hp.beta1) + 1.0)).all()
+    assert (np.abs(v - g64 ** 2) <= spacing_bf16(g64 ** 2) * (0.5 / (1 - hp.beta2) + 1.0)).all()
+    assert (m <= g64 * (1 + 2.0 ** -8)).all() and (v <= g64 ** 2 * (1 + 2.0 ** -8)).all()   # never beyond the fixed point's rounding
+    # the bound is not vacuous: some elements do stall short of the fixed point's own rounding
+    assert (np.abs(m - g64) > spacing_bf16(g64)).any()
+
+
+# ----------------------------------------------------------------------------- Lion and momentum SGD
+@pytest.mark.parametrize("impl_name", ["numpy", "c"])
+def test_lion_and_sgdm_store_the_nearest_bf16_and_leave_theta_alone(impl_name):
+    rng = np.random.RandomState(10)
+    n = 2048
+    theta0 = (rng.standard_normal(n) * 0.02).astype(np.float32)
+    m0 = bf16_values(rng, n, 1e-3)
+    g = (rng.standard_t(3, size=n) * 1e-3).astype(np.float32)
+    h, lr, b1, b2, wd, mu = 0.5, 1e-4, 0.9, 0.99, 0.1, 0.9
+    # Lion
+    th_ref, _ = npo.lion_update(theta0, g, m0, h, lr, b1, b2, wd, np.float32)
+    _, m64 = npo.lion_update(theta0, g, m0, h, lr, b1, b2, wd, np.float64)
+    if impl_name == "numpy":
+        th, m1 = npo.lion_update(theta0, g, m0, h, lr, b1, b2, wd, np.float32, moment_dtype="bf16")
+        m1 = m1.astype(np.float64)
+    else:
+        th, mb = theta0.copy(), f32_to_bits(m0)
+        co.lion_update(th, g, mb, h, lr, b1, b2, wd)
+        m1 = bits_to_f64(mb)
+    assert np.array_equal(th.view(np.uint32), th_ref.view(np.uint32))
+    assert_is_nearest_bf16(m1, m64, "Lion m")
+    # momentum SGD, against the library started from the given momentum buffer
+    p = torch.tensor(theta0.astype(np.float64), requires_grad=True)
+    opt = torch.optim.SGD([p], lr=lr, momentum=mu, weight_decay=wd)
+    opt.state[p] = {"momentum_buffer": torch.tensor(m0.astype(np.float64))}
+    p.grad = torch.tensor(h * g.astype(np.float64))
+    opt.step()
+    if impl_name == "numpy":
+        th, m1 = npo.sgdm_update(theta0, g, m0, h, lr, mu, wd, np.float32, moment_dtype="bf16")
+        m1 = m1.astype(np.float64)
+    else:
+        th, mb = theta0.copy(), f32_to_bits(m0)
+        co.sgdm_update(th, g, mb, h, lr, mu, wd)
+        m1 = bits_to_f64(mb)
+    np.testing.assert_allclose(th, p.detach().numpy(), rtol=1.2e-7, atol=1e-30)           # theta saw the unrounded momentum
+    assert_is_nearest_bf16(m1, opt.state[p]["momentum_buffer"].numpy(), "SGD m")
+
+
+# ----------------------------------------------------------------------------- the two oracles against each other
+def test_numpy_and_c_oracles_agree_with_bf16_state_over_many_steps():
+    """Whole path on a small ragged layout: decisions, gamma, theta and the stored moments, bit for bit."""
+    rng = np.random.RandomState(11)
+    sizes = [7, 300, 4097, 33]
+    offs, o = [], 0
+    for s in sizes:
+        offs.append(o)
+        o += (s + 7) // 8 * 8
+    hp = npo.Hyper(lr=1e-3, warmup=3, lambda_abs=0.02, lambda_rel=1.04, beta=0.98)
+    theta0 = (rng.standard_normal(o) * 0.02).astype(np.float32)
+    ref_np = npo.AdaGCAdamW([theta0[a:a + s] for a, s in zip(offs, sizes)], hp, np.float32, moment_dtype="bf16")
+    ref_c = co.ArenaOracle(offs, sizes, theta0, lr=hp.lr, beta1=hp.beta1, beta2=hp.beta2, eps=hp.eps, wd=hp.wd,
+                           lambda_rel=hp.lambda_rel, beta=hp.beta, lambda_abs=hp.lambda_abs, warmup=hp.warmup,
+                           bf16_state=True, tie_tol=1e-6)
+    for t in range(1, 16):
+        g = (rng.standard_t(3, size=o) * 1e-3 * (30.0 if t == 9 else 1.0)).astype(np.float32)
+        r_np = ref_np.step([g[a:a + s] for a, s in zip(offs, sizes)])
+        r_c = ref_c.step(g)
+        assert np.array_equal(r_np.flag, r_c["flag"])
+        np.testing.assert_allclose(r_np.gamma, r_c["gamma"], rtol=1e-7)
+    for i, (a, s) in enumerate(zip(offs, sizes)):
+        np.testing.assert_allclose(ref_np.theta[i], ref_c.theta[a:a + s], rtol=2e-7, atol=1e-12)
+        same_m = f32_to_bits(ref_np.m[i]) == ref_c.m[a:a + s]
+        same_v = f32_to_bits(ref_np.v[i]) == ref_c.v[a:a + s]
+        # pow() and ** may differ in the last bit of a float64 coefficient; only an element that the C oracle itself
+        # reports as decided within 1e-6 of a flip may round differently
+        assert (same_m | (ref_c.ties[a:a + s] > 0)).all() and (same_v | (ref_c.ties[a:a + s] > 0)).all()
+    assert ref_c.ties.mean() < 0.05
+
+
+def test_c_oracle_counts_decisions_close_to_a_flip():
+    """near_tie is incremented exactly for elements whose new m (or v) is within tie_tol of a rounding flip."""
+    hp = npo.Hyper(lr=0.0, beta1=0.5, beta2=0.5, wd=0.0)
+    # m1 = 0.5 * m0 + 0.5 * g: choose m0 = 1, g = 1 + 2^-6 -> m1 = 1 + 2^-7 ... a bfloat16 value (margin = half a spacing);
+    # g = 1 + 2^-7 -> m1 = 1 + 2^-8: exactly the midpoint between 1 and 1 + 2^-7 (margin 0)
+    m0 = np.array([1.0, 1.0, 1.0], np.float32)
+    g = np.array([1.0 + 2.0 ** -6, 1.0 + 2.0 ** -7, 1.0 + 2.0 ** -7 + 2.0 ** -20], np.float32)
+    v0 = np.zeros(3, np.float32)
+    th, mb, vb, ties = np.zeros(3, np.float32), f32_to_bits(m0), f32_to_bits(v0), np.zeros(3, np.uint8)
+    co.adamw_update_bf16state(th, g, mb, vb, 1.0, 3, hp.lr, hp.beta1, hp.beta2, hp.eps, hp.wd, near_tie=ties, tie_tol=1e-5)
+    assert ties.tolist() == [0, 1, 1]
+    assert bits_to_f64(mb).tolist() == [1.0 + 2.0 ** -7, 1.0, 1.0 + 2.0 ** -7]     # tie to even; just above the midpoint rounds up
+    _, _, _, mm, _ = npo.adamw_update(th, g, m0, v0, 1.0, 3, hp, np.float32, moment_dtype="bf16", return_margin=True)
+    assert mm[1] == 0.0 and mm[0] > 1e-3 and 0 < mm[2] < 1e-5

@@ -43,10 +43,14 @@ UNIT = "params/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
-# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the update kernel: 25.53 B/param measured on
-# the GPT-2-small-shaped layout (committed ncu summary of that capture: 3177.4 MB for 124 439 808
-# params), scaled by the parameter count because the traffic of this streaming kernel grows in proportion.
-TRAFFIC_BYTES_PER_PARAM = {"bf16": 3177.385e6 / 124439808}
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the update kernel, per parameter, from the committed
+# captures of the same kernel on smaller layouts (a multi-pass capture is not pointed at a 94 GB workload); scaled by the
+# parameter count because the traffic of this streaming kernel grows in proportion.  None once a kernel has changed
+# since its capture.
+TRAFFIC_BYTES_PER_PARAM = {
+    "bf16": (3177.385e6 / 124439808, "profiles/adagc_kernels_gpt2_small_ncu_full.md (GPT-2-small-shaped layout, scaled by N)"),
+    "f32": (16.04 + 11.71, "profiles/adagc_kernels_many_small_ncu_full.md (20 000 small tensors, scaled by N)"),
+}
 
 
 # ------------------------------------------------------------------------------------ helpers
@@ -158,10 +162,10 @@ def oracle_sample(wl, max_params=8.2e8):
     return picked, tot
 
 
-def time_oracle(wl, steps: int, warm: int):
+def time_oracle(wl, steps: int, warm: int, sample=None):
     """Times the C oracle, as it stands, on the bounded sample; returns (params/s, s/step, info)."""
     from oracle import c_oracle
-    picked, tot = oracle_sample(wl)
+    picked, tot = sample if sample is not None else oracle_sample(wl)
     offs, o = [], 0
     for t in picked:
         offs.append(o)
@@ -197,6 +201,49 @@ def time_oracle(wl, steps: int, warm: int):
     return tot * steps / dt, dt / steps, info
 
 
+def oracle_extra_legs(wl, g_host, sample_params_per_s):
+    """Further legs of the CPU baseline, each labelled with what it covers:
+      all_norms      the oracle's phase 1 + 2 over ALL tensors of the layout (sums of squares streamed from the host copy
+                     of the gradient arena, then the decisions), i.e. everything of a step that needs no optimizer state;
+      single_thread  the whole oracle step on a smaller sample with one OpenMP thread;
+      extrapolated   seconds per full step = all_norms + (update time per parameter on the sample) x N."""
+    import ctypes
+    from oracle import c_oracle
+    out = {}
+    offs = np.array([t.offset for t in wl.tensors], np.int64)
+    nums = np.array([t.numel for t in wl.tensors], np.int64)
+    g_np = g_host.view(torch.int16).numpy().view(np.uint16) if g_host.dtype == torch.bfloat16 else g_host.numpy()
+    gamma = np.zeros(wl.n_tensors, np.float32)
+    t0 = time.perf_counter()
+    ssq = c_oracle.sumsq_tensors(g_np, offs, nums)
+    c_oracle.clip_decisions(ssq, gamma, 2, wl.hyper["lambda_rel"], wl.hyper["beta"], wl.hyper["lambda_abs"], 1)
+    dt = time.perf_counter() - t0
+    out["all_norms"] = {"seconds": dt, "value": wl.n_params / dt, "unit": UNIT, "cores": c_oracle.num_threads(),
+                        "sample": f"norm + decision phases of the C oracle over all {wl.n_tensors} tensors "
+                                  f"({wl.n_params} params) of {wl.name}, one step"}
+    # update cost per parameter on the sample: its whole step minus its own norm phase
+    picked, tot = oracle_sample(wl)
+    t0 = time.perf_counter()
+    c_oracle.sumsq_tensors(g_np, np.array([t.offset for t in picked], np.int64), np.array([t.numel for t in picked], np.int64))
+    norm_sample = time.perf_counter() - t0
+    upd_per_param = max(tot / sample_params_per_s - norm_sample, 0.0) / tot
+    full = dt + upd_per_param * wl.n_params
+    out["extrapolated_full_layout"] = {"seconds_per_step": full, "value": wl.n_params / full, "unit": UNIT,
+                                       "sample": "extrapolated: all_norms (measured on the full layout) + the sample's "
+                                                 "update time per parameter x all parameters"}
+    try:
+        gomp = ctypes.CDLL("libgomp.so.1")
+        n_before = c_oracle.num_threads()
+        gomp.omp_set_num_threads(1)
+        small, stot = oracle_sample(wl, max_params=1.2e8)
+        val1, _, info1 = time_oracle(wl, 1, 1, sample=(small, stot))
+        gomp.omp_set_num_threads(n_before)
+        out["single_thread"] = {"value": val1, "unit": UNIT, "cores": 1, "sample": info1["sample"]}
+    except OSError:
+        out["single_thread"] = None
+    return out
+
+
 def run_reference(args, wl):
     rank, world, _ = dist_env()
     if rank != 0:
@@ -209,6 +256,78 @@ def run_reference(args, wl):
             "cpu_baseline": dict(info, value=val, unit=UNIT),
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
+
+
+def time_layout(binding, workloads, wl, dev, steps, warm=3, state_dtype=torch.float32, fused_small=False):
+    """One layout on one GPU, the way the headline number is taken: `warm` untimed steps, then `steps` steady-state AdaGC
+    steps timed with CUDA events (L2 flushed before each step when the layout is small), then the same number of steps
+    with the library's per-phase events.  Returns milliseconds and fractions of the minimum-bytes roofline."""
+    hp = wl.hyper
+    offs, nums = [t.offset for t in wl.tensors], [t.numel for t in wl.tensors]
+    opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=dev, state_dtype=state_dtype)
+    theta = workloads.init_params(wl, dev)
+    m = torch.zeros(wl.arena_elems, dtype=state_dtype, device=dev)
+    v = torch.zeros_like(m)
+    ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device=dev)
+    g = workloads.grads_for_step(wl, 1, dev)
+    small = wl.n_params * 14 <= (1 << 30)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if small else None
+    args_h = (hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"], hp["beta"], 1)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t = 0
+    per, ph = [], []
+    for k in range(warm + 2 * steps):
+        t += 1
+        timed, phased = warm <= k < warm + steps, k >= warm + steps
+        opt.set_phase_timing(phased)
+        if flush is not None:
+            flush.fill_(t & 0xFF)
+        if timed:
+            e0.record()
+        opt.step(theta, g, m, v, ema, t, *args_h)
+        if timed:
+            e1.record()
+            e1.synchronize()
+            per.append(e0.elapsed_time(e1))
+        if phased:
+            ph.append(opt.get_phase_times())
+    opt.set_phase_timing(False)
+    peak, _ = measured_peak()
+    sb = 2 if state_dtype == torch.bfloat16 else 4
+    gb = 2 if wl.grad_dtype == "bf16" else 4
+    bpp = 8 + gb + 4 * sb                       # theta read + written, g read, m and v read + written
+    ms = float(np.median(per))
+    norm_ms, fin_ms, upd_ms = (float(x) for x in np.median(np.array(ph), axis=0))
+    out = {"n_params": wl.n_params, "n_tensors": wl.n_tensors, "grad_dtype": wl.grad_dtype,
+           "state_dtype": "bf16" if sb == 2 else "f32", "min_bytes_per_param": bpp, "ms_per_step": ms,
+           "norm_ms": norm_ms, "finalize_ms": fin_ms, "update_ms": upd_ms,
+           "update_kernel_frac_of_measured": bpp * wl.n_params / (upd_ms * 1e-3) / 1e9 / peak,
+           "norm_kernel_frac_of_measured": gb * wl.n_params / (norm_ms * 1e-3) / 1e9 / peak,
+           "whole_step_frac_of_measured": bpp * wl.n_params / (ms * 1e-3) / 1e9 / peak,
+           "whole_step_frac_of_nominal_8TBs": bpp * wl.n_params / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+           "l2": "flushed before every step" if small else "working set far larger than L2"}
+    if fused_small and opt.n_chunks <= 4096:
+        # launch-latency-bound layouts: wall clock over back-to-back steps like a training loop, three launches against
+        # the one-kernel step (ADAGC_FUSED_SMALL)
+        fused = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=dev, flags=binding.FUSED_SMALL,
+                              state_dtype=state_dtype)
+        ema_f = torch.zeros_like(ema)
+        for name, o, e_ in (("three_launch_step_us_back_to_back", opt, ema), ("fused_small_step_us_back_to_back", fused, ema_f)):
+            tt = 100
+            for _ in range(20):
+                tt += 1
+                o.step(theta, g, m, v, e_, tt, *args_h)
+            torch.cuda.synchronize(dev)
+            w0 = time.perf_counter()
+            for _ in range(200):
+                tt += 1
+                o.step(theta, g, m, v, e_, tt, *args_h)
+            torch.cuda.synchronize(dev)
+            out[name] = (time.perf_counter() - w0) / 200 * 1e6
+        fused.close()
+    assert opt.get_stats()["status"] == 0
+    opt.close()
+    return out
 
 
 # ------------------------------------------------------------------------------------ our arm
@@ -301,13 +420,23 @@ def run_ours(args, wl):
     achieved = bpp * wl.n_params / (upd_ms * 1e-3) / 1e9
     norm_gbs = (bpp - 24) * wl.n_params / (norm_ms * 1e-3) / 1e9
     kernel = "adagc_update_tma_kernel" if opt.update_path == binding.UPDATE_PATH_BULK else "adagc_update_kernel"
+    traffic_bpp, traffic_src = TRAFFIC_BYTES_PER_PARAM.get(wl.grad_dtype, (None, None))
+    if kernel != "adagc_update_tma_kernel":
+        traffic_bpp, traffic_src = None, None
+    whole_gbs = bpp * wl.n_params / step_s / 1e9
     roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-                "traffic": (TRAFFIC_BYTES_PER_PARAM[wl.grad_dtype] * wl.n_params
-                            if wl.grad_dtype in TRAFFIC_BYTES_PER_PARAM and kernel == "adagc_update_tma_kernel" else None),
+                "traffic": traffic_bpp * wl.n_params if traffic_bpp else None,
+                "traffic_source": traffic_src,
                 "algorithmic_bytes_per_launch": bpp * wl.n_params, "launch_ms": upd_ms,
-                "whole_step_frac": bpp * wl.n_params / step_s / 1e9 / peak,
-                "whole_step_frac_of_nominal_8TBs": bpp * wl.n_params / step_s / 1e9 / NOMINAL_HBM_GBS,
+                # the whole step against the minimum bytes the method must move (g read once): the step reads g twice
+                # (norm pass, update pass), so its ceiling is 26/28 (28/32 with fp32 gradients) of the bandwidth reached
+                "whole_step": {"achieved": whole_gbs, "frac_of_measured": whole_gbs / peak,
+                               "frac_of_nominal_8TBs": whole_gbs / NOMINAL_HBM_GBS,
+                               "target_frac_of_nominal": 0.80, "target_met": bool(whole_gbs / NOMINAL_HBM_GBS >= 0.80),
+                               "min_bytes_per_param": bpp, "bytes_moved_per_param": bpp + (2 if wl.grad_dtype == "bf16" else 4)},
+                "whole_step_frac": whole_gbs / peak,
+                "whole_step_frac_of_nominal_8TBs": whole_gbs / NOMINAL_HBM_GBS,
                 "norm_kernel": {"launch_ms": norm_ms, "achieved": norm_gbs, "frac": norm_gbs / peak},
                 "finalize_ms": fin_ms}
 
@@ -351,24 +480,6 @@ def run_ours(args, wl):
                                             "frac": (bpp + 2) * wl.n_params / (emit_ms[2] * 1e-3) / 1e9 / peak}
         del lowp
 
-    # small layouts: the one-kernel step (ADAGC_FUSED_SMALL), wall clock over back-to-back steps like a training loop
-    if opt.n_chunks <= 4096:
-        fused = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=dev, flags=binding.FUSED_SMALL)
-        ema_f = torch.zeros_like(ema)
-        for name, o, e_ in (("three_launch_step_us_back_to_back", opt, ema), ("fused_small_step_us_back_to_back", fused, ema_f)):
-            tt = 100
-            for _ in range(20):
-                tt += 1
-                o.step(theta, g, m, v, e_, tt, *args_h, T_START)
-            torch.cuda.synchronize(dev)
-            w0 = time.perf_counter()
-            for _ in range(200):
-                tt += 1
-                o.step(theta, g, m, v, e_, tt, *args_h, T_START)
-            torch.cuda.synchronize(dev)
-            extra[name] = (time.perf_counter() - w0) / 200 * 1e6
-        fused.close()
-
     # ---- end to end through the host-buffer entry point
     e2e_steps = max(1, min(args.steps, 5))
     g_host = torch.empty(wl.arena_elems, dtype=wl.torch_grad_dtype).pin_memory()
@@ -390,12 +501,33 @@ def run_ours(args, wl):
            "note": "wall clock around adagc_step_host (it synchronises the stream); gradients from pinned host memory"}
     st = opt.get_stats()
     assert st["status"] == 0 and np.isfinite(st["norm"]).all()
-    del g_host
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         val, sec, info = time_oracle(wl, 5, 1)
         cpu_baseline = dict(info, value=val, unit=UNIT)
+        cpu_baseline.update(oracle_extra_legs(wl, g_host, val))
+    del g_host
+
+    # ---- the same step with the moments stored as bfloat16 (18 B/param instead of 26), and the other layouts
+    if world == 1 and not args.no_extras:
+        del theta, m, v, g, ema
+        opt.close()
+        torch.cuda.empty_cache()
+        k = max(3, min(args.steps, 10))
+        if all(t_.offset % 8 == 0 for t_ in wl.tensors):
+            r = time_layout(binding, workloads, wl, dev, k, 3, torch.bfloat16)
+            extra["bf16_state"] = r
+            extra["bf16_state_update_kernel"] = {"launch_ms": r["update_ms"], "bytes_per_param": r["min_bytes_per_param"],
+                                                 "achieved": r["min_bytes_per_param"] * wl.n_params / (r["update_ms"] * 1e-3) / 1e9,
+                                                 "frac": r["update_kernel_frac_of_measured"]}
+        if args.workload is None:
+            per_config = {}
+            for name in ("llama32_1b", "gpt2_small", "many_small", "tiny"):
+                torch.cuda.empty_cache()
+                per_config[name] = time_layout(binding, workloads, workloads.build(name), dev, 20, 5,
+                                               fused_small=(name == "tiny"))
+            extra["per_config"] = per_config
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -513,6 +645,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default=None, help="tiny | gpt2_small | llama2_7b | many_small | llama32_1b | moe_8x1b | moe_ernie")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the bfloat16-state and other-layout measurements")
     ap.add_argument("--parallel", choices=["replicas", "sharded"], default="replicas",
                     help="N > 1: independent replicas (default; the data-parallel case) or flat shards of one model")
     args = ap.parse_args()

@@ -87,6 +87,26 @@ typedef enum {
  * be created anew. */
 #define ADAGC_FUSED_SMALL 32
 
+/*
+ * Optimizer state stored as bfloat16 (adagc_desc.state_dtype = ADAGC_BF16).  The paper trains in bfloat16 / float8
+ * precision (Appendix "Hyper-Parameters") and does not say how stored optimizer state is rounded; this library's
+ * reading: theta stays an fp32 master copy; d_m and d_v (d_m alone for Lion and momentum SGD) are bfloat16 arenas
+ * with the descriptor's element offsets; a step reads the stored moments exactly, computes in fp32, updates theta
+ * from the UNROUNDED new moments and rounds the moments to the nearest bfloat16, ties to even, where it stores them.
+ * The update phase then moves 18 instead of 26 bytes per parameter (bf16 gradients).  Every entry point that takes
+ * d_m / d_v follows the descriptor's state dtype.
+ * Which bfloat16 neighbour is stored is a discrete decision, so its precision is part of the interface: the value that
+ * is rounded is computed in single precision, each operation rounded once (fl), coefficients rounded to fp32 first:
+ *     gh = fl(h g);   m' = fl(beta1 m + fl((1 - beta1) gh));   v' = fl(beta2 v + fl((1 - beta2) fl(gh gh)))       (AdamW)
+ *     m' = fl(beta2 m + fl((1 - beta2) gh))                                                                        (Lion)
+ *     m' = fl(momentum m + fl(wd theta + gh))                                                                      (SGD)
+ * where each outer sum with its first product is one fused multiply-add.  (With bfloat16 g and m and beta1 = 0.9 the
+ * exact value of m' lies precisely half-way between two bfloat16 values for about one element in twenty; a float64
+ * evaluation resolves such ties by the rounding error of 0.9 itself.)  Note that with a decay close to 1 a stored bfloat16 moment stops
+ * moving once (1 - beta)|target - x| drops below half its spacing, i.e. within spacing / (2 (1 - beta)) of the value
+ * an fp32 moment would reach: 10 spacings (8 %) for beta2 = 0.95, 500 spacings for beta2 = 0.999.
+ */
+
 /* One parameter tensor. */
 typedef struct {
   int64_t numel;    /* > 0 (0 allowed with ADAGC_ALLOW_EMPTY); offset + numel <= 2^34 */
@@ -103,7 +123,8 @@ typedef struct {
   int32_t n_tensors;           /* 1 .. 2^24 */
   int32_t param_dtype;         /* ADAGC_F32 */
   int32_t grad_dtype;          /* ADAGC_F32 or ADAGC_BF16 */
-  int32_t state_dtype;         /* ADAGC_F32 (m and v) */
+  int32_t state_dtype;         /* dtype of the m and v arenas: ADAGC_F32, or ADAGC_BF16 (see "Optimizer state stored as
+                                  bfloat16" below); every tensor offset must then be a multiple of 8 elements */
   const adagc_tensor* tensors; /* host array, copied by adagc_create */
   double lambda_abs;           /* warm-up global-norm threshold of Eq. 2, > 0 (paper: 1.0) */
   int32_t flags;               /* 0, or one ADAGC_UPDATE_PATH_* value, optionally OR-ed with the other ADAGC_* flags above */
@@ -132,7 +153,8 @@ int adagc_destroy(adagc_ctx* ctx);
 
 /*
  * One fused step of Algorithm 1.
- *   d_params, d_m, d_v : fp32 arenas, updated in place
+ *   d_params           : fp32 arena, updated in place
+ *   d_m, d_v           : arenas in the descriptor's state dtype (fp32 or bfloat16), updated in place
  *   d_grads            : gradient arena in the descriptor's grad dtype, read only
  *   d_ema              : gamma, n_tensors fp32 values, updated in place (Section 4.3 "Memory":
  *                        one 32-bit float per tensor)

@@ -279,18 +279,29 @@ static inline void count_near_tie(uint8_t* near_tie, int64_t j, double x, double
 /*
  * The AdamW lines of Algorithm 1 with the moments STORED as bfloat16 (the paper trains in bfloat16 / float8
  * precision and does not say how optimizer state is rounded; reading taken: fp32 master theta, m and v read
- * exactly from their stored bfloat16, float64 arithmetic, theta updated from the UNROUNDED new moments, the
- * moments rounded to the nearest bfloat16, ties to even, when stored).  In place.  Rounding is a discrete
- * decision: if near_tie is not NULL, near_tie[j] is incremented (saturating) whenever the new m or v lies
- * within tie_tol, relative to the terms it is summed from, of a point where the rounding flips.
+ * exactly from their stored bfloat16, theta updated from the UNROUNDED new moments, the moments rounded to the
+ * nearest bfloat16, ties to even, when stored).  In place.
+ *
+ * Rounding to bfloat16 is a discrete decision.  fp32_decision = 0: everything in float64 (the plain definition;
+ * if near_tie is not NULL, near_tie[j] is incremented, saturating, whenever the new m or v lies within tie_tol,
+ * relative to the terms it is summed from, of a point where the rounding flips).  fp32_decision = 1: the value
+ * that is rounded to bfloat16 is evaluated in the precision the stored format is defined for, single precision,
+ * in this order, every operation rounded once (fl = round to float, coefficients rounded to float first):
+ *     gh = fl(h * g);   m' = fl(beta1 * m + fl((1 - beta1) * gh));   v' = fl(beta2 * v + fl((1 - beta2) * fl(gh * gh)))
+ * (the sum and its first product are one fused multiply-add).  With bfloat16 m, bfloat16 g and beta1 = 0.9 the
+ * float64 value of m' is an exact decimal tie (x.5 spacings) for about one element in twenty, so which neighbour is
+ * stored depends on how the coefficients themselves are rounded: the decision has to name its precision.
+ * theta is always computed in float64 from the float64 moments.
  */
 void adagc_ref_adamw_bf16state(float* theta, const void* g, int g_is_bf16, uint16_t* m, uint16_t* v, int64_t n,
                                double h, int64_t step, double lr, double beta1, double beta2, double eps,
-                               double wd, uint8_t* near_tie, double tie_tol) {
+                               double wd, uint8_t* near_tie, double tie_tol, int fp32_decision) {
   const double bc1 = 1.0 - pow(beta1, (double)step);
   const double bc2 = 1.0 - pow(beta2, (double)step);
   const uint16_t* gb = (const uint16_t*)g;
   const float* gf = (const float*)g;
+  const float hf = (float)h, b1f = (float)beta1, omb1f = (float)(1.0 - beta1), b2f = (float)beta2,
+              omb2f = (float)(1.0 - beta2);
 #pragma omp parallel for schedule(static) if (n > 65536)
   for (int64_t j = 0; j < n; ++j) {
     const double gj = g_is_bf16 ? bf16_to_double(gb[j]) : (double)gf[j];
@@ -304,18 +315,29 @@ void adagc_ref_adamw_bf16state(float* theta, const void* g, int g_is_bf16, uint1
     theta[j] = (float)(th - lr * wd * th - lr * mh / (sqrt(vh) + eps));
     count_near_tie(near_tie, j, m1, fabs(a) + fabs(b), tie_tol);
     count_near_tie(near_tie, j, v1, v1, tie_tol);
-    m[j] = double_to_bf16(m1);
-    v[j] = double_to_bf16(v1);
+    if (fp32_decision) {
+      const float ghf = hf * (float)gj; /* g is exactly a float */
+      const float m1f = fmaf(b1f, (float)bf16_to_double(m[j]), omb1f * ghf);
+      const float v1f = fmaf(b2f, (float)bf16_to_double(v[j]), omb2f * (ghf * ghf));
+      m[j] = double_to_bf16((double)m1f);
+      v[j] = double_to_bf16((double)v1f);
+    } else {
+      m[j] = double_to_bf16(m1);
+      v[j] = double_to_bf16(v1);
+    }
   }
 }
 
 /* Lion (see adagc_ref_lion) with the momentum stored as bfloat16, rounded to nearest even on store.
- * near_tie counts both kinds of discrete decision: sign(c) and the rounding of m. */
+ * near_tie counts both kinds of discrete decision: sign(c) and the rounding of m.  fp32_decision = 1: the stored
+ * value is the rounding of  fl(beta2 * m + fl((1 - beta2) * fl(h * g)))  evaluated in single precision (see above);
+ * sign(c) stays a float64 decision. */
 void adagc_ref_lion_bf16state(float* theta, const void* g, int g_is_bf16, uint16_t* m, int64_t n, double h,
                               double lr, double beta1, double beta2, double wd, uint8_t* near_tie,
-                              double tie_tol) {
+                              double tie_tol, int fp32_decision) {
   const uint16_t* gb = (const uint16_t*)g;
   const float* gf = (const float*)g;
+  const float hf = (float)h, b2f = (float)beta2, omb2f = (float)(1.0 - beta2);
 #pragma omp parallel for schedule(static) if (n > 65536)
   for (int64_t j = 0; j < n; ++j) {
     const double gj = g_is_bf16 ? bf16_to_double(gb[j]) : (double)gf[j];
@@ -328,16 +350,24 @@ void adagc_ref_lion_bf16state(float* theta, const void* g, int g_is_bf16, uint16
     const double th = (double)theta[j];
     theta[j] = (float)(th - lr * (sgn + wd * th));
     const double a2 = beta2 * mj, b2 = (1.0 - beta2) * gh;
-    count_near_tie(near_tie, j, a2 + b2, fabs(a2) + fabs(b2), tie_tol);
-    m[j] = double_to_bf16(a2 + b2);
+    if (fp32_decision) {
+      m[j] = double_to_bf16((double)fmaf(b2f, (float)mj, omb2f * (hf * (float)gj)));
+    } else {
+      count_near_tie(near_tie, j, a2 + b2, fabs(a2) + fabs(b2), tie_tol);
+      m[j] = double_to_bf16(a2 + b2);
+    }
   }
 }
 
-/* Momentum SGD (see adagc_ref_sgdm) with the momentum stored as bfloat16; theta sees the unrounded momentum. */
+/* Momentum SGD (see adagc_ref_sgdm) with the momentum stored as bfloat16; theta sees the unrounded momentum.
+ * fp32_decision = 1: the stored value is the rounding of  fl(momentum * m + fl(wd * theta + fl(h * g)))  evaluated in
+ * single precision (both sums fused multiply-adds). */
 void adagc_ref_sgdm_bf16state(float* theta, const void* g, int g_is_bf16, uint16_t* m, int64_t n, double h,
-                              double lr, double momentum, double wd, uint8_t* near_tie, double tie_tol) {
+                              double lr, double momentum, double wd, uint8_t* near_tie, double tie_tol,
+                              int fp32_decision) {
   const uint16_t* gb = (const uint16_t*)g;
   const float* gf = (const float*)g;
+  const float hf = (float)h, muf = (float)momentum, wdf = (float)wd;
 #pragma omp parallel for schedule(static) if (n > 65536)
   for (int64_t j = 0; j < n; ++j) {
     const double gj = g_is_bf16 ? bf16_to_double(gb[j]) : (double)gf[j];
@@ -345,9 +375,14 @@ void adagc_ref_sgdm_bf16state(float* theta, const void* g, int g_is_bf16, uint16
     const double d = h * gj + wd * th;
     const double a = momentum * bf16_to_double(m[j]);
     const double m1 = a + d;
+    const float m1f = fmaf(muf, (float)bf16_to_double(m[j]), fmaf(wdf, theta[j], hf * (float)gj));
     theta[j] = (float)(th - lr * m1);
-    count_near_tie(near_tie, j, m1, fabs(a) + fabs(h * gj) + fabs(wd * th), tie_tol);
-    m[j] = double_to_bf16(m1);
+    if (fp32_decision) {
+      m[j] = double_to_bf16((double)m1f);
+    } else {
+      count_near_tie(near_tie, j, m1, fabs(a) + fabs(h * gj) + fabs(wd * th), tie_tol);
+      m[j] = double_to_bf16(m1);
+    }
   }
 }
 

@@ -64,13 +64,14 @@ def lib():
         L.adagc_ref_sgdm.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64] + [C.c_double] * 4
         L.adagc_ref_adamw_bf16state.restype = None
         L.adagc_ref_adamw_bf16state.argtypes = ([C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int64,
-                                                 C.c_double, C.c_int64] + [C.c_double] * 5 + [C.c_void_p, C.c_double])
+                                                 C.c_double, C.c_int64] + [C.c_double] * 5 +
+                                                [C.c_void_p, C.c_double, C.c_int])
         L.adagc_ref_lion_bf16state.restype = None
         L.adagc_ref_lion_bf16state.argtypes = ([C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64] +
-                                               [C.c_double] * 5 + [C.c_void_p, C.c_double])
+                                               [C.c_double] * 5 + [C.c_void_p, C.c_double, C.c_int])
         L.adagc_ref_sgdm_bf16state.restype = None
         L.adagc_ref_sgdm_bf16state.argtypes = ([C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64] +
-                                               [C.c_double] * 4 + [C.c_void_p, C.c_double])
+                                               [C.c_double] * 4 + [C.c_void_p, C.c_double, C.c_int])
         L.adagc_ref_scale.restype = None
         L.adagc_ref_scale.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_double]
         L.adagc_ref_step.restype = C.c_int32
@@ -155,17 +156,21 @@ def _is_bf16_state(theta: np.ndarray, moments, n: int) -> bool:
 
 def adamw_update_bf16state(theta: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray, h: float, step: int,
                            lr: float, beta1: float, beta2: float, eps: float, wd: float,
-                           near_tie: Optional[np.ndarray] = None, tie_tol: float = 0.0) -> None:
+                           near_tie: Optional[np.ndarray] = None, tie_tol: float = 0.0,
+                           fp32_decision: bool = False) -> None:
     """AdamW with m and v stored as bfloat16 (uint16 bit patterns), in place; theta fp32.  `near_tie` (uint8) counts,
-    per element, the steps in which the rounding of m or v was decided with a relative margin below `tie_tol`."""
+    per element, the steps in which the float64 rounding of m or v was decided with a relative margin below `tie_tol`.
+    fp32_decision: the value rounded to bfloat16 is evaluated in single precision (see adagc_ref.c) instead."""
     p, bf = _grad_ptr(g)
     assert _is_bf16_state(theta, (m, v), g.size)
     lib().adagc_ref_adamw_bf16state(theta.ctypes.data, p, bf, m.ctypes.data, v.ctypes.data, g.size, float(h),
-                                    int(step), lr, beta1, beta2, eps, wd, _tie_ptr(near_tie, g.size), float(tie_tol))
+                                    int(step), lr, beta1, beta2, eps, wd, _tie_ptr(near_tie, g.size), float(tie_tol),
+                                    int(fp32_decision))
 
 
 def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, beta1: float,
-                beta2: float, wd: float, near_tie: Optional[np.ndarray] = None, tie_tol: float = 0.0) -> None:
+                beta2: float, wd: float, near_tie: Optional[np.ndarray] = None, tie_tol: float = 0.0,
+                fp32_decision: bool = False) -> None:
     """Lion on the clipped gradient, in place on fp32 theta and on m (fp32, or uint16 = stored as bfloat16).
     `near_tie` (uint8, same length) counts, per element, the steps in which sign(c) -- and, for bfloat16 m, its
     rounding -- was decided with a relative margin below `tie_tol`."""
@@ -173,19 +178,20 @@ def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: f
     nt = _tie_ptr(near_tie, g.size)
     if _is_bf16_state(theta, (m,), g.size):
         lib().adagc_ref_lion_bf16state(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, beta1, beta2,
-                                       wd, nt, float(tie_tol))
+                                       wd, nt, float(tie_tol), int(fp32_decision))
     else:
         lib().adagc_ref_lion(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, beta1, beta2, wd,
                              nt, float(tie_tol))
 
 
 def sgdm_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, momentum: float,
-                wd: float, near_tie: Optional[np.ndarray] = None, tie_tol: float = 0.0) -> None:
+                wd: float, near_tie: Optional[np.ndarray] = None, tie_tol: float = 0.0,
+                fp32_decision: bool = False) -> None:
     """SGD with momentum on the clipped gradient, in place on fp32 theta and on m (fp32, or uint16 = bfloat16)."""
     p, bf = _grad_ptr(g)
     if _is_bf16_state(theta, (m,), g.size):
         lib().adagc_ref_sgdm_bf16state(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, momentum, wd,
-                                       _tie_ptr(near_tie, g.size), float(tie_tol))
+                                       _tie_ptr(near_tie, g.size), float(tie_tol), int(fp32_decision))
     else:
         lib().adagc_ref_sgdm(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, momentum, wd)
 
@@ -209,9 +215,11 @@ class ArenaOracle:
                  lr: float, beta1: float, beta2: float, eps: float, wd: float, lambda_rel: float,
                  beta: float, lambda_abs: float, warmup: int, keep_initial: bool = False,
                  global_adaptive: bool = False, gamma0: Optional[np.ndarray] = None, ema_cap: float = 0.0,
-                 bf16_state: bool = False, tie_tol: float = 0.0):
+                 bf16_state: bool = False, tie_tol: float = 0.0, fp32_decision: bool = False):
         """bf16_state: m and v are stored as bfloat16 (uint16 bit patterns), rounded to nearest even on store;
-        `self.ties` then counts, per element, the steps whose rounding was decided with a margin below tie_tol."""
+        `self.ties` then counts, per element, the steps whose float64 rounding was decided with a margin below
+        tie_tol; fp32_decision: the rounded value is evaluated in single precision (see adagc_ref.c)."""
+        self.fp32_decision = bool(fp32_decision)
         self.keep_initial, self.global_adaptive, self.ema_cap = keep_initial, global_adaptive, float(ema_cap)
         self.bf16_state, self.tie_tol = bool(bf16_state), float(tie_tol)
         self.off = np.ascontiguousarray(offsets, dtype=np.int64)
@@ -255,7 +263,8 @@ class ArenaOracle:
             args = (self.theta[o:o + n], grads[o:o + n], self.m[o:o + n], self.v[o:o + n], float(r["h"][i]),
                     self.t, hp["lr"] if lr is None else lr, hp["beta1"], hp["beta2"], hp["eps"], hp["wd"])
             if self.bf16_state:
-                adamw_update_bf16state(*args, near_tie=self.ties[o:o + n], tie_tol=self.tie_tol)
+                adamw_update_bf16state(*args, near_tie=self.ties[o:o + n], tie_tol=self.tie_tol,
+                                       fp32_decision=self.fp32_decision)
             else:
                 adamw_update(*args)
         return r

@@ -172,13 +172,16 @@ class AdaGC:
     """adagc_ctx plus its torch-owned workspace.  Method names mirror the C entry points."""
 
     def __init__(self, numels: Sequence[int], offsets: Sequence[int], grad_dtype: torch.dtype,
-                 lambda_abs: float = 1.0, shapes=None, device="cuda", flags: int = 0):
+                 lambda_abs: float = 1.0, shapes=None, device="cuda", flags: int = 0,
+                 state_dtype: torch.dtype = torch.float32):
         L = lib()
         gd = {torch.float32: ADAGC_F32, torch.bfloat16: ADAGC_BF16}[grad_dtype]
         self.grad_dtype = grad_dtype
+        self.state_dtype = state_dtype           # dtype of the m and v arenas (adagc_desc.state_dtype)
         self.n_tensors = len(numels)
         self.device = torch.device(device)
-        desc, keep = make_desc(numels, offsets, gd, lambda_abs, shapes, flags=flags)
+        desc, keep = make_desc(numels, offsets, gd, lambda_abs, shapes, flags=flags,
+                               state_dtype={torch.float32: ADAGC_F32, torch.bfloat16: ADAGC_BF16}[state_dtype])
         nbytes = L.adagc_workspace_bytes(C.byref(desc))
         if nbytes == 0:
             rc = L.adagc_num_chunks(C.byref(desc))
@@ -209,7 +212,7 @@ class AdaGC:
     # -- the entry points ------------------------------------------------------------------
     def step(self, params, grads, m, v, ema, step, lr, beta1, beta2, eps, wd, lambda_rel, beta, warmup,
              stream=None):
-        assert grads.dtype == self.grad_dtype and params.dtype == m.dtype == v.dtype == ema.dtype == torch.float32
+        assert grads.dtype == self.grad_dtype and params.dtype == ema.dtype == torch.float32 and m.dtype == v.dtype == self.state_dtype
         rc = lib().adagc_step(self._h, _ptr(params), _ptr(grads), _ptr(m), _ptr(v), _ptr(ema), int(step),
                               lr, beta1, beta2, eps, wd, lambda_rel, beta, int(warmup), _stream_ptr(stream))
         if rc != 0:
@@ -219,7 +222,7 @@ class AdaGC:
                         lr_dev: Optional[torch.Tensor] = None, stream=None):
         """adagc_step_capturable: the step number lives on the device; `lr_dev` (one fp32 on the device), if given,
         is read at every execution instead of `lr`."""
-        assert grads.dtype == self.grad_dtype and params.dtype == m.dtype == v.dtype == ema.dtype == torch.float32
+        assert grads.dtype == self.grad_dtype and params.dtype == ema.dtype == torch.float32 and m.dtype == v.dtype == self.state_dtype
         assert lr_dev is None or (lr_dev.dtype == torch.float32 and lr_dev.is_cuda)
         rc = lib().adagc_step_capturable(self._h, _ptr(params), _ptr(grads), _ptr(m), _ptr(v), _ptr(ema),
                                          _ptr(lr_dev), lr, beta1, beta2, eps, wd, lambda_rel, beta, int(warmup),
@@ -235,7 +238,7 @@ class AdaGC:
     def step_emit_bf16(self, params, params_bf16, grads, m, v, ema, step, lr, beta1, beta2, eps, wd, lambda_rel, beta,
                        warmup, stream=None):
         assert grads.dtype == self.grad_dtype and params_bf16.dtype == torch.bfloat16
-        assert params.dtype == m.dtype == v.dtype == ema.dtype == torch.float32
+        assert params.dtype == ema.dtype == torch.float32 and m.dtype == v.dtype == self.state_dtype
         rc = lib().adagc_step_emit_bf16(self._h, _ptr(params), _ptr(params_bf16), _ptr(grads), _ptr(m), _ptr(v),
                                         _ptr(ema), int(step), lr, beta1, beta2, eps, wd, lambda_rel, beta,
                                         int(warmup), _stream_ptr(stream))
@@ -243,14 +246,14 @@ class AdaGC:
             raise AdagcError(rc, "adagc_step_emit_bf16")
 
     def step_lion(self, params, grads, m, ema, step, lr, beta1, beta2, wd, lambda_rel, beta, warmup, stream=None):
-        assert grads.dtype == self.grad_dtype and params.dtype == m.dtype == ema.dtype == torch.float32
+        assert grads.dtype == self.grad_dtype and params.dtype == ema.dtype == torch.float32 and m.dtype == self.state_dtype
         rc = lib().adagc_step_lion(self._h, _ptr(params), _ptr(grads), _ptr(m), _ptr(ema), int(step), lr, beta1,
                                    beta2, wd, lambda_rel, beta, int(warmup), _stream_ptr(stream))
         if rc != 0:
             raise AdagcError(rc, "adagc_step_lion")
 
     def step_sgdm(self, params, grads, m, ema, step, lr, momentum, wd, lambda_rel, beta, warmup, stream=None):
-        assert grads.dtype == self.grad_dtype and params.dtype == m.dtype == ema.dtype == torch.float32
+        assert grads.dtype == self.grad_dtype and params.dtype == ema.dtype == torch.float32 and m.dtype == self.state_dtype
         rc = lib().adagc_step_sgdm(self._h, _ptr(params), _ptr(grads), _ptr(m), _ptr(ema), int(step), lr, momentum,
                                    wd, lambda_rel, beta, int(warmup), _stream_ptr(stream))
         if rc != 0:
@@ -282,7 +285,7 @@ class AdaGC:
 
     def step_presummed(self, params, grads, m, v, ema, sumsq, step, lr, beta1, beta2, eps, wd, lambda_rel, beta,
                        warmup, stream=None):
-        assert grads.dtype == self.grad_dtype and params.dtype == m.dtype == v.dtype == ema.dtype == torch.float32
+        assert grads.dtype == self.grad_dtype and params.dtype == ema.dtype == torch.float32 and m.dtype == v.dtype == self.state_dtype
         assert sumsq.dtype == torch.float64 and sumsq.is_cuda and sumsq.numel() >= self.n_tensors
         rc = lib().adagc_step_presummed(self._h, _ptr(params), _ptr(grads), _ptr(m), _ptr(v), _ptr(ema), _ptr(sumsq),
                                         int(step), lr, beta1, beta2, eps, wd, lambda_rel, beta, int(warmup),

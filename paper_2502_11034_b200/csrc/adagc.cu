@@ -131,6 +131,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return f32_to_bf16_bits(lo) | (f32_to_bf16_bits(hi) << 16);
 }
 
+// the same rounding by the conversion instruction (one instruction per pair; NaN becomes the canonical NaN)
+__device__ __forceinline__ uint32_t pack_bf16_cvt(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
 __device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
 __device__ __forceinline__ void st_stream(uint4* p, uint4 v) { __stcs(p, v); }
@@ -555,11 +561,50 @@ __device__ __forceinline__ void adamw_vec4(const float g0, const float g1, const
   adamw_elem<kOpt>(g3, h, p.w, m.w, v.w, a);
 }
 
+// Optimizer state (m, v) is stored as fp32 or as bfloat16 (kSB); arithmetic is fp32 either way.  A stored bfloat16
+// is read exactly; the new moments are rounded to the nearest bfloat16 (ties to even) only where they are stored,
+// after theta has been updated from the unrounded values.  Which neighbour is stored is decided by the fp32 value
+// adamw_elem computes, in exactly its operation order (the header states it): with bfloat16 g and m and
+// beta1 = 0.9 about one new m in twenty is an exact decimal tie in real arithmetic, so the order is part of the
+// contract and must not be rearranged.
+template <bool kSB>
+__device__ __forceinline__ void load_state8(const void* __restrict__ base, int i, float4& a, float4& b) {
+  if (kSB) {
+    const uint4 q = __ldcs(static_cast<const uint4*>(base) + i);
+    a = make_float4(bf16_lo(q.x), bf16_hi(q.x), bf16_lo(q.y), bf16_hi(q.y));
+    b = make_float4(bf16_lo(q.z), bf16_hi(q.z), bf16_lo(q.w), bf16_hi(q.w));
+  } else {
+    a = ld_stream(static_cast<const float4*>(base) + 2 * i);
+    b = ld_stream(static_cast<const float4*>(base) + 2 * i + 1);
+  }
+}
+template <bool kSB>
+__device__ __forceinline__ void store_state8(void* __restrict__ base, int i, const float4& a, const float4& b) {
+  if (kSB) {
+    st_stream(static_cast<uint4*>(base) + i, make_uint4(pack_bf16_cvt(a.x, a.y), pack_bf16_cvt(a.z, a.w),
+                                                        pack_bf16_cvt(b.x, b.y), pack_bf16_cvt(b.z, b.w)));
+  } else {
+    st_stream(static_cast<float4*>(base) + 2 * i, a);
+    st_stream(static_cast<float4*>(base) + 2 * i + 1, b);
+  }
+}
+template <bool kSB>
+__device__ __forceinline__ float load_state1(const void* __restrict__ base, int64_t j) {
+  return kSB ? __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(base)[j]) << 16)
+             : static_cast<const float*>(base)[j];
+}
+template <bool kSB>
+__device__ __forceinline__ void store_state1(void* __restrict__ base, int64_t j, float x) {
+  if (kSB) static_cast<uint16_t*>(base)[j] = static_cast<uint16_t>(pack_bf16_cvt(x, 0.0f));
+  else static_cast<float*>(base)[j] = x;
+}
+
 // Eight consecutive elements of one chunk: 7 (bf16 gradients) or 8 (fp32) 16-byte loads, 6 stores
-// (AdamW; Lion has no v stream).
-template <bool kBF16, int kOpt>
+// (AdamW with fp32 state; Lion has no v stream; bfloat16 state halves the m and v accesses).
+// mbase / vbase point at the chunk's first element of the m and v arenas.
+template <bool kBF16, int kOpt, bool kSB>
 __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gbase, float4* __restrict__ p4,
-                                             float4* __restrict__ m4, float4* __restrict__ v4, float h,
+                                             void* __restrict__ mbase, void* __restrict__ vbase, float h,
                                              const AdamScalars& a, uint4* __restrict__ lowp8 = nullptr) {
   float g[8];
   if (kBF16) {
@@ -577,20 +622,15 @@ __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gba
     g[4] = gb.x; g[5] = gb.y; g[6] = gb.z; g[7] = gb.w;
   }
   float4 pa = ld_stream(p4 + 2 * i), pb = ld_stream(p4 + 2 * i + 1);
-  float4 ma = ld_stream(m4 + 2 * i), mb = ld_stream(m4 + 2 * i + 1);
+  float4 ma, mb;
+  load_state8<kSB>(mbase, i, ma, mb);
   float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
-  if (kOpt == kOptAdamW) {
-    va = ld_stream(v4 + 2 * i);
-    vb = ld_stream(v4 + 2 * i + 1);
-  }
+  if (kOpt == kOptAdamW) load_state8<kSB>(vbase, i, va, vb);
   adamw_vec4<kOpt>(g[0], g[1], g[2], g[3], h, pa, ma, va, a);
   adamw_vec4<kOpt>(g[4], g[5], g[6], g[7], h, pb, mb, vb, a);
   st_stream(p4 + 2 * i, pa); st_stream(p4 + 2 * i + 1, pb);
-  st_stream(m4 + 2 * i, ma); st_stream(m4 + 2 * i + 1, mb);
-  if (kOpt == kOptAdamW) {
-    st_stream(v4 + 2 * i, va);
-    st_stream(v4 + 2 * i + 1, vb);
-  }
+  store_state8<kSB>(mbase, i, ma, mb);
+  if (kOpt == kOptAdamW) store_state8<kSB>(vbase, i, va, vb);
   if (lowp8)  // bf16 copy of the updated parameters (the model's working weights in mixed precision)
     st_stream(lowp8 + i, make_uint4(pack_bf16(pa.x, pa.y), pack_bf16(pa.z, pa.w), pack_bf16(pb.x, pb.y),
                                     pack_bf16(pb.z, pb.w)));
@@ -600,24 +640,26 @@ __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gba
 // elements) and the rows of successive chunks go to the block's warps in one continuing round-robin:
 // row_base counts the rows dealt so far.  Restarting at warp 0 for every chunk would give the low warps
 // the extra rows every time and make them the critical path.
-template <bool kBF16, int kBlockThreads, int kOpt>
+template <bool kBF16, int kBlockThreads, int kOpt, bool kSB>
 __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, int& row_base, float* __restrict__ params,
-                                                    const void* __restrict__ grads, float* __restrict__ m_arena,
-                                                    float* __restrict__ v_arena, const AdamScalars& a,
+                                                    const void* __restrict__ grads, void* __restrict__ m_arena,
+                                                    void* __restrict__ v_arena, const AdamScalars& a,
                                                     uint16_t* __restrict__ lowp = nullptr) {
   constexpr int kWarps = kBlockThreads / 32;
+  constexpr int kStateBytes = kSB ? 2 : 4;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int64_t start = chunk_start(ck);
   float4* __restrict__ p4 = reinterpret_cast<float4*>(params + start);
-  float4* __restrict__ m4 = reinterpret_cast<float4*>(m_arena + start);
-  float4* __restrict__ v4 = reinterpret_cast<float4*>(v_arena + start);
+  char* __restrict__ mbase = static_cast<char*>(m_arena) + start * kStateBytes;
+  char* __restrict__ vbase = kOpt == kOptAdamW ? static_cast<char*>(v_arena) + start * kStateBytes : nullptr;
   const char* __restrict__ gbase = static_cast<const char*>(grads) + start * (kBF16 ? 2 : 4);
   const int n8 = ck.count >> 3;
   const int rows = (n8 + 31) >> 5;
 #pragma unroll 2
   for (int r = (warp - row_base) & (kWarps - 1); r < rows; r += kWarps) {
     const int i = (r << 5) + lane;
-    if (i < n8) adamw_group8<kBF16, kOpt>(i, gbase, p4, m4, v4, h, a, lowp ? reinterpret_cast<uint4*>(lowp + start) : nullptr);
+    if (i < n8)
+      adamw_group8<kBF16, kOpt, kSB>(i, gbase, p4, mbase, vbase, h, a, lowp ? reinterpret_cast<uint4*>(lowp + start) : nullptr);
   }
   row_base = (row_base + rows) & (kWarps - 1);
   const int t = (n8 << 3) + lane;  // ragged tail (fewer than 8 elements): the next warp in turn takes it
@@ -628,24 +670,25 @@ __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, in
     } else {
       g = reinterpret_cast<const float*>(gbase)[t];
     }
-    float p = params[start + t], m = m_arena[start + t], v = 0.0f;
-    if (kOpt == kOptAdamW) v = v_arena[start + t];
+    float p = params[start + t], m = load_state1<kSB>(mbase, t), v = 0.0f;
+    if (kOpt == kOptAdamW) v = load_state1<kSB>(vbase, t);
     adamw_elem<kOpt>(g, h, p, m, v, a);
     params[start + t] = p;
-    m_arena[start + t] = m;
-    if (kOpt == kOptAdamW) v_arena[start + t] = v;
+    store_state1<kSB>(mbase, t, m);
+    if (kOpt == kOptAdamW) store_state1<kSB>(vbase, t, v);
     if (lowp) lowp[start + t] = static_cast<uint16_t>(f32_to_bf16_bits(p));
   }
 }
 
 // Register-streaming update kernel: every thread loads eight elements of each stream into registers.
-template <bool kBF16, int kOpt>
+template <bool kBF16, int kOpt, bool kSB>
 __global__ void __launch_bounds__(kThreads)
-adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, float* __restrict__ m_arena,
-                    float* __restrict__ v_arena, const Chunk* __restrict__ chunks,
+adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, void* __restrict__ m_arena,
+                    void* __restrict__ v_arena, const Chunk* __restrict__ chunks,
                     const int32_t* __restrict__ block_begin, const float* __restrict__ h_arr, AdamScalars a,
                     uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a) {
   if (d_a) a = *d_a;  // capturable step: coefficients from device memory
+  constexpr int kStateBytes = kSB ? 2 : 4;
   const int tid = threadIdx.x;
   int c = block_begin[blockIdx.x];
   const int n_chunks = block_begin[blockIdx.x + 1];  // end of this block's entries
@@ -666,15 +709,15 @@ adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, 
     if (ck.count == kChunkElems) {  // full chunk: fixed trip count
       const int64_t start = chunk_start(ck);
       float4* __restrict__ p4 = reinterpret_cast<float4*>(params + start);
-      float4* __restrict__ m4 = reinterpret_cast<float4*>(m_arena + start);
-      float4* __restrict__ v4 = reinterpret_cast<float4*>(v_arena + start);
+      char* __restrict__ mbase = static_cast<char*>(m_arena) + start * kStateBytes;
+      char* __restrict__ vbase = kOpt == kOptAdamW ? static_cast<char*>(v_arena) + start * kStateBytes : nullptr;
       const char* __restrict__ gbase = static_cast<const char*>(grads) + start * (kBF16 ? 2 : 4);
 #pragma unroll 2
       for (int k = 0; k < kChunkElems / 8 / kThreads; ++k)
-        adamw_group8<kBF16, kOpt>(k * kThreads + tid, gbase, p4, m4, v4, h, a,
-                                  lowp ? reinterpret_cast<uint4*>(lowp + start) : nullptr);
+        adamw_group8<kBF16, kOpt, kSB>(k * kThreads + tid, gbase, p4, mbase, vbase, h, a,
+                                       lowp ? reinterpret_cast<uint4*>(lowp + start) : nullptr);
     } else {
-      adamw_partial_chunk<kBF16, kThreads, kOpt>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp);
+      adamw_partial_chunk<kBF16, kThreads, kOpt, kSB>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp);
     }
     if (c_next >= n_chunks) break;
     c = c_next;
@@ -685,17 +728,28 @@ adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, 
 
 // ------------------------------------------------------------------------------------------------
 // Bulk-async (TMA) update kernel.  Full chunks are cut into tiles of kTile elements; an elected thread
-// moves each tile's four streams global -> shared with cp.async.bulk (completion on an mbarrier), all
-// threads update the tile in shared memory, and the three written streams go back with bulk stores.
-// Two stages: while tile j is computed, tile j+1 is in flight (about 57 KB of loads per SM, the amount
-// this access mix wants on B200) and tile j-1 drains.  Partial chunks take the register path afterwards.
+// moves each tile's streams global -> shared with cp.async.bulk (completion on an mbarrier), all
+// threads update the tile in shared memory, and the written streams go back with bulk stores.
+// A ring of kStages stages: while tile j is computed, tiles j+1 .. j+kStages-1 are in flight and tile j-1
+// drains.  fp32 state: tiles of 4096 elements, two stages (one 57 KB tile in flight per SM, the amount
+// this access mix wants on B200).  bfloat16 state moves 10 instead of 14 bytes per element, and there the
+// per-tile costs (barrier wait, block barrier, issue) weigh more: measured on the 7B-shaped layout, tiles of
+// 2048 / 4096 / 8192 elements in two stages gave 5060 / 5650 / 6050 GB/s, more stages never helped (4096 x 3:
+// 5700, 4096 x 4: 5670), and rounding with the conversion instruction instead of integer arithmetic took
+// 8192 x 2 to 6650 GB/s.  Partial chunks take the register path afterwards.
 // Every wait is bounded: after ~2 s without completion the block records ADAGC_E_TIMEOUT in the
 // status word and leaves its remaining tiles untouched.
 // ------------------------------------------------------------------------------------------------
 constexpr int kTmaThreads = 512;
-constexpr int kTile = 4096;
-constexpr int kTilesPerChunk = kChunkElems / kTile;
-constexpr int kTmaStages = 2;
+template <bool kSB>
+struct TmaRing {  // fp32 state: 14 (16) bytes per element
+  static constexpr int kTile = 4096, kStages = 2;
+};
+template <>
+struct TmaRing<true> {  // bfloat16 state: 10 (12) bytes per element
+  static constexpr int kTile = 8192, kStages = 2;
+};
+constexpr int kMaxDynamicSmem = 227 * 1024;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -758,93 +812,130 @@ __device__ __forceinline__ void bulk_wait_smem_read() { asm volatile("cp.async.b
 __device__ __forceinline__ void bulk_wait_done() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_generic_to_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+// bytes per element that the loads of one tile bring into a stage: theta, m (and v), g
+__host__ __device__ constexpr int tma_elem_bytes(bool bf16, int opt, bool state_bf16) {
+  return 4 + (opt == kOptAdamW ? 2 : 1) * (state_bf16 ? 2 : 4) + (bf16 ? 2 : 4);
+}
+template <bool kSB>
 constexpr int tma_smem_bytes(bool bf16, int opt, bool emit_lowp = false) {
-  return kTmaStages * kTile * ((opt == kOptAdamW ? 12 : 8) + (bf16 ? 2 : 4) + (emit_lowp ? 2 : 0));
+  return TmaRing<kSB>::kStages * TmaRing<kSB>::kTile * (tma_elem_bytes(bf16, opt, kSB) + (emit_lowp ? 2 : 0));
 }
 
-template <bool kBF16, int kOpt>
+// One 4-element group of a tile's m or v region in shared memory, in the state dtype.
+template <bool kSB>
+__device__ __forceinline__ float4 smem_state4(const unsigned char* region, int q) {
+  if (kSB) {
+    const uint2 w = reinterpret_cast<const uint2*>(region)[q];
+    return make_float4(bf16_lo(w.x), bf16_hi(w.x), bf16_lo(w.y), bf16_hi(w.y));
+  }
+  return reinterpret_cast<const float4*>(region)[q];
+}
+template <bool kSB>
+__device__ __forceinline__ void smem_state4_store(unsigned char* region, int q, const float4& x) {
+  if (kSB) reinterpret_cast<uint2*>(region)[q] = make_uint2(pack_bf16_cvt(x.x, x.y), pack_bf16_cvt(x.z, x.w));
+  else reinterpret_cast<float4*>(region)[q] = x;
+}
+
+template <bool kBF16, int kOpt, bool kSB>
 __global__ void __launch_bounds__(kTmaThreads, 1)
-adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ grads, float* __restrict__ m_arena,
-                        float* __restrict__ v_arena, const Chunk* __restrict__ chunks,
+adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ grads, void* __restrict__ m_arena,
+                        void* __restrict__ v_arena, const Chunk* __restrict__ chunks,
                         const int32_t* __restrict__ block_begin, const int32_t* __restrict__ block_mid,
                         const float* __restrict__ h_arr, AdamScalars a, int* __restrict__ status,
                         uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a) {
   if (d_a) a = *d_a;  // capturable step: coefficients from device memory
   extern __shared__ __align__(128) unsigned char tile_smem[];
+  constexpr int kTile = TmaRing<kSB>::kTile, kStages = TmaRing<kSB>::kStages;
+  constexpr int kTilesPerChunk = kChunkElems / kTile;
+  constexpr int kAhead = kStages - 1;  // tiles in flight beyond the one being computed
+  static_assert(kChunkElems % kTile == 0 && kTile % (4 * kTmaThreads) == 0, "tiles divide chunks, threads divide tiles");
+  static_assert(kAhead >= 1 && kAhead <= kTilesPerChunk, "the tile being fetched lies in this chunk or the next");
   constexpr int kGBytes = kBF16 ? 2 : 4;
-  constexpr int kStateBytes = kOpt == kOptAdamW ? 12 : 8;  // theta, m (and v) per element; g follows them
-  constexpr uint32_t kStageBytes = kTile * (kStateBytes + kGBytes);  // what the loads of one tile bring in
-  // with a bf16 copy of the parameters to emit, each stage has a fifth region that only the stores read
+  constexpr int kSBytes = kSB ? 2 : 4;                              // m, v element size
+  constexpr int kMOff = kTile * 4;                                   // region offsets inside a stage: theta, m, v, g
+  constexpr int kVOff = kMOff + kTile * kSBytes;
+  constexpr int kGOff = kOpt == kOptAdamW ? kVOff + kTile * kSBytes : kVOff;
+  constexpr uint32_t kStageBytes = kGOff + kTile * kGBytes;          // what the loads of one tile bring in
+  static_assert(kStageBytes == static_cast<uint32_t>(kTile) * tma_elem_bytes(kBF16, kOpt, kSB), "stage layout");
+  static_assert(kStages * (kStageBytes + kTile * 2) <= kMaxDynamicSmem, "the ring fits in shared memory");
+  // with a bf16 copy of the parameters to emit, each stage has one more region that only the stores read
   const uint32_t stage_stride = kStageBytes + (lowp ? kTile * 2 : 0);
-  __shared__ __align__(8) uint64_t full_bar[kTmaStages];
+  __shared__ __align__(8) uint64_t full_bar[kStages];
   const int tid = threadIdx.x;
   const int begin = block_begin[blockIdx.x], mid = block_mid[blockIdx.x], end = block_begin[blockIdx.x + 1];
   const int n_tiles = (mid - begin) * kTilesPerChunk;
 
   __shared__ int abort_flag;
   if (tid == 0) {
-    for (int s = 0; s < kTmaStages; ++s) mbar_init(&full_bar[s], 1);
+    for (int s = 0; s < kStages; ++s) mbar_init(&full_bar[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     abort_flag = 0;
   }
   __syncthreads();
 
   const uint64_t stream_policy = l2_policy_evict_first();  // every byte this kernel moves is used once
-  // thread 0 only: start the four loads of one tile (tile `sub` of the chunk that starts at element e0)
+  // thread 0 only: start the loads of one tile (tile `sub` of the chunk that starts at element e0)
   auto issue_tile = [&](int64_t e0, int sub, int s) {
     const int64_t e = e0 + static_cast<int64_t>(sub) * kTile;
     unsigned char* b = tile_smem + static_cast<size_t>(s) * stage_stride;
     mbar_arrive_expect_tx(&full_bar[s], kStageBytes);
     bulk_load_hint(b, params + e, kTile * 4, &full_bar[s], stream_policy);
-    bulk_load_hint(b + kTile * 4, m_arena + e, kTile * 4, &full_bar[s], stream_policy);
-    if (kOpt == kOptAdamW) bulk_load_hint(b + kTile * 8, v_arena + e, kTile * 4, &full_bar[s], stream_policy);
-    bulk_load_hint(b + kTile * kStateBytes, static_cast<const char*>(grads) + e * kGBytes, kTile * kGBytes, &full_bar[s],
-                   stream_policy);
+    bulk_load_hint(b + kMOff, static_cast<const char*>(m_arena) + e * kSBytes, kTile * kSBytes, &full_bar[s], stream_policy);
+    if (kOpt == kOptAdamW)
+      bulk_load_hint(b + kVOff, static_cast<const char*>(v_arena) + e * kSBytes, kTile * kSBytes, &full_bar[s], stream_policy);
+    bulk_load_hint(b + kGOff, static_cast<const char*>(grads) + e * kGBytes, kTile * kGBytes, &full_bar[s], stream_policy);
   };
 
   bool healthy = true;
   int j_fail = 0;
   if (n_tiles > 0) {
-    // table entries are kept one chunk ahead in registers, so that neither the elected thread's issue path
+    // table entries are kept two chunks ahead in registers, so that neither the elected thread's issue path
     // nor the consumers ever wait for a table load
     Chunk ck = chunks[begin];
     float h = h_arr[ck.tensor];
-    Chunk ck_next = ck;
-    float h_next = h;
+    Chunk ck_next = ck, ck_next2 = ck;
+    float h_next = h, h_next2 = h;
     if (begin + 1 < mid) {
       ck_next = chunks[begin + 1];
       h_next = h_arr[ck_next.tensor];
     }
-    if (tid == 0) issue_tile(chunk_start(ck), 0, 0);
+    if (begin + 2 < mid) {
+      ck_next2 = chunks[begin + 2];
+      h_next2 = h_arr[ck_next2.tensor];
+    }
+    if (tid == 0)
+      for (int k = 0; k < kAhead && k < n_tiles; ++k) issue_tile(chunk_start(ck), k, k);  // kAhead <= tiles per chunk
+    int s = 0;           // stage of tile j
+    uint32_t phase = 0;  // parity of the barrier phase tile j completes: flips each time the ring wraps
     for (int j = 0; j < n_tiles; ++j) {
-      const int s = j & 1;
       const int sub = j % kTilesPerChunk;
       const bool last_of_chunk = sub == kTilesPerChunk - 1;
-      if (tid == 0 && j + 1 < n_tiles) {
-        bulk_wait_smem_read();  // the stores of tile j-1 have finished reading stage s^1
-        if (last_of_chunk) issue_tile(chunk_start(ck_next), 0, s ^ 1);
-        else issue_tile(chunk_start(ck), sub + 1, s ^ 1);
+      if (tid == 0 && j + kAhead < n_tiles) {
+        bulk_wait_smem_read();  // the stores of tile j-1 have finished reading the stage that is refilled now
+        const int sub_f = sub + kAhead;  // tile j + kAhead: in this chunk or in the next
+        const int s_f = s == 0 ? kStages - 1 : s - 1;
+        if (sub_f >= kTilesPerChunk) issue_tile(chunk_start(ck_next), sub_f - kTilesPerChunk, s_f);
+        else issue_tile(chunk_start(ck), sub_f, s_f);
       }
       unsigned char* b = tile_smem + static_cast<size_t>(s) * stage_stride;
-      if (mbar_wait_bounded(&full_bar[s], (j >> 1) & 1)) {
+      if (mbar_wait_bounded(&full_bar[s], phase)) {
         float4* p4 = reinterpret_cast<float4*>(b);
-        float4* m4 = reinterpret_cast<float4*>(b + kTile * 4);
-        float4* v4 = reinterpret_cast<float4*>(b + kTile * 8);
 #pragma unroll
         for (int q = tid; q < kTile / 4; q += kTmaThreads) {
           float g0, g1, g2, g3;
           if (kBF16) {
-            const uint2 w = reinterpret_cast<const uint2*>(b + kTile * kStateBytes)[q];
+            const uint2 w = reinterpret_cast<const uint2*>(b + kGOff)[q];
             g0 = bf16_lo(w.x); g1 = bf16_hi(w.x); g2 = bf16_lo(w.y); g3 = bf16_hi(w.y);
           } else {
-            const float4 w = reinterpret_cast<const float4*>(b + kTile * kStateBytes)[q];
+            const float4 w = reinterpret_cast<const float4*>(b + kGOff)[q];
             g0 = w.x; g1 = w.y; g2 = w.z; g3 = w.w;
           }
-          float4 p = p4[q], m = m4[q], v = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (kOpt == kOptAdamW) v = v4[q];
+          float4 p = p4[q], m = smem_state4<kSB>(b + kMOff, q), v = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (kOpt == kOptAdamW) v = smem_state4<kSB>(b + kVOff, q);
           adamw_vec4<kOpt>(g0, g1, g2, g3, h, p, m, v, a);
-          p4[q] = p; m4[q] = m;
-          if (kOpt == kOptAdamW) v4[q] = v;
+          p4[q] = p;
+          smem_state4_store<kSB>(b + kMOff, q, m);
+          if (kOpt == kOptAdamW) smem_state4_store<kSB>(b + kVOff, q, v);
           if (lowp) reinterpret_cast<uint2*>(b + kStageBytes)[q] = make_uint2(pack_bf16(p.x, p.y), pack_bf16(p.z, p.w));
         }
         fence_generic_to_async_smem();  // the updated tile must be visible to the bulk-copy engine
@@ -860,29 +951,38 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
       if (tid == 0) {
         const int64_t e = chunk_start(ck) + static_cast<int64_t>(sub) * kTile;
         bulk_store_hint(params + e, b, kTile * 4, stream_policy);
-        bulk_store_hint(m_arena + e, b + kTile * 4, kTile * 4, stream_policy);
-        if (kOpt == kOptAdamW) bulk_store_hint(v_arena + e, b + kTile * 8, kTile * 4, stream_policy);
+        bulk_store_hint(static_cast<char*>(m_arena) + e * kSBytes, b + kMOff, kTile * kSBytes, stream_policy);
+        if (kOpt == kOptAdamW)
+          bulk_store_hint(static_cast<char*>(v_arena) + e * kSBytes, b + kVOff, kTile * kSBytes, stream_policy);
         if (lowp) bulk_store_hint(lowp + e, b + kStageBytes, kTile * 2, stream_policy);
         bulk_commit();
       }
       if (last_of_chunk) {
         ck = ck_next;
         h = h_next;
-        const int c2 = begin + j / kTilesPerChunk + 2;
-        if (c2 < mid) {
-          ck_next = chunks[c2];
-          h_next = h_arr[ck_next.tensor];
+        ck_next = ck_next2;
+        h_next = h_next2;
+        const int c3 = begin + j / kTilesPerChunk + 3;
+        if (c3 < mid) {
+          ck_next2 = chunks[c3];
+          h_next2 = h_arr[ck_next2.tensor];
         }
+      }
+      if (++s == kStages) {
+        s = 0;
+        phase ^= 1u;
       }
     }
     if (tid == 0) {
       bulk_wait_done();
       if (!healthy) {
         atomicOr(status, ADAGC_E_TIMEOUT);
-        // a load may still be in flight into this block's shared memory: give it one more bounded
+        // loads may still be in flight into this block's shared memory: give each of them one more bounded
         // chance to land before the block (and its shared memory) goes away
-        (void)mbar_wait_bounded(&full_bar[j_fail & 1], (j_fail >> 1) & 1);
-        if (j_fail + 1 < n_tiles) (void)mbar_wait_bounded(&full_bar[(j_fail + 1) & 1], ((j_fail + 1) >> 1) & 1);
+        for (int k = 0; k <= kAhead && j_fail + k < n_tiles; ++k) {
+          const int jj = j_fail + k;
+          (void)mbar_wait_bounded(&full_bar[jj % kStages], (jj / kStages) & 1);
+        }
       }
     }
     __syncthreads();
@@ -902,7 +1002,7 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
       ck_next = chunks[c + 1];
       h_next = h_arr[ck_next.tensor];
     }
-    adamw_partial_chunk<kBF16, kTmaThreads, kOpt>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp);
+    adamw_partial_chunk<kBF16, kTmaThreads, kOpt, kSB>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp);
     ck = ck_next;
     h = h_next;
   }
@@ -1013,10 +1113,10 @@ __device__ __forceinline__ bool grid_barrier_bounded(unsigned long long* counter
 constexpr int kSlice = 4096;
 constexpr int kSlicesPerChunk = kChunkElems / kSlice;
 
-template <bool kBF16>
+template <bool kBF16, bool kSB>
 __global__ void __launch_bounds__(kThreads)
-adagc_fused_small_kernel(float* __restrict__ params, const void* __restrict__ grads, float* __restrict__ m_arena,
-                         float* __restrict__ v_arena, float* ema, const Chunk* __restrict__ chunks, int n_chunks,
+adagc_fused_small_kernel(float* __restrict__ params, const void* __restrict__ grads, void* __restrict__ m_arena,
+                         void* __restrict__ v_arena, float* ema, const Chunk* __restrict__ chunks, int n_chunks,
                          const TensorEntry* __restrict__ tensors, double* slice_partials, ClipScalars cs, int in_warmup,
                          AdamScalars a, StatPtrs st, unsigned long long* barrier_counter,
                          unsigned long long barrier_index, float* gamma_prev) {
@@ -1107,7 +1207,7 @@ adagc_fused_small_kernel(float* __restrict__ params, const void* __restrict__ gr
     Chunk sub = ck;
     sub.start4 = ck.start4 + static_cast<uint32_t>(begin / 4);
     sub.count = min(kSlice, ck.count - begin);
-    adamw_partial_chunk<kBF16, kThreads, kOptAdamW>(sub, h, row_base, params, grads, m_arena, v_arena, a);
+    adamw_partial_chunk<kBF16, kThreads, kOptAdamW, kSB>(sub, h, row_base, params, grads, m_arena, v_arena, a);
   }
 }
 
@@ -1155,7 +1255,8 @@ Layout make_layout(int64_t n_chunks, int64_t T, bool fused_small = false) {
 
 int validate_desc(const adagc_desc* d, int64_t* n_chunks_out, int64_t* arena_elems_out) {
   if (!d || !d->tensors || d->n_tensors < 1 || d->n_tensors > (1 << 24)) return ADAGC_E_INVALID_ARG;
-  if (d->param_dtype != ADAGC_F32 || d->state_dtype != ADAGC_F32) return ADAGC_E_DTYPE;
+  if (d->param_dtype != ADAGC_F32) return ADAGC_E_DTYPE;
+  if (d->state_dtype != ADAGC_F32 && d->state_dtype != ADAGC_BF16) return ADAGC_E_DTYPE;
   if (d->grad_dtype != ADAGC_F32 && d->grad_dtype != ADAGC_BF16) return ADAGC_E_DTYPE;
   if (!(d->lambda_abs > 0.0) || !std::isfinite(d->lambda_abs)) return ADAGC_E_INVALID_ARG;
   constexpr int kKnownFlags =
@@ -1164,7 +1265,8 @@ int validate_desc(const adagc_desc* d, int64_t* n_chunks_out, int64_t* arena_ele
   if ((d->flags & ADAGC_FUSED_SMALL) && (d->flags & ADAGC_CLIP_GLOBAL_ADAPTIVE)) return ADAGC_E_INVALID_ARG;
   const bool allow_empty = (d->flags & ADAGC_ALLOW_EMPTY) != 0;
   if ((d->flags & ~kKnownFlags) != 0 || (d->flags & ADAGC_UPDATE_PATH_MASK) == 3) return ADAGC_E_INVALID_ARG;
-  const int64_t align = (d->grad_dtype == ADAGC_BF16) ? 8 : 4;
+  // every arena must start each tensor on a 16-byte boundary: 8 elements as soon as one arena holds 2-byte elements
+  const int64_t align = (d->grad_dtype == ADAGC_BF16 || d->state_dtype == ADAGC_BF16) ? 8 : 4;
   int64_t n_chunks = 0, extent = 0;
   std::vector<std::pair<int64_t, int64_t>> spans;
   spans.reserve(d->n_tensors);
@@ -1237,7 +1339,8 @@ struct adagc_ctx {
   int32_t T = 0;
   int32_t n_chunks = 0;
   int64_t arena_elems = 0;
-  bool bf16 = false;
+  bool bf16 = false;        // gradient arena is bfloat16
+  bool state_bf16 = false;  // m and v arenas are bfloat16
   double lambda_abs = 1.0;
   int device = 0;
   int grid_wide = 1, grid_update = 1;  // norm and scale kernels: SMs x resident blocks; update: SMs x 2 or x 1
@@ -1301,20 +1404,17 @@ int check_clip_args(const adagc_ctx* ctx, const float* d_ema, int64_t step, doub
 
 // Largest L1 carve-out for the register kernels (L1 lines hold their loads in flight); opt-in shared
 // memory size for the bulk-async kernels.
-template <bool kBF16>
+template <bool kBF16, int kOpt, bool kSB>
+bool prepare_update_kernel() {
+  return cudaFuncSetAttribute(adagc_update_kernel<kBF16, kOpt, kSB>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                              cudaSharedmemCarveoutMaxL1) == cudaSuccess &&
+         cudaFuncSetAttribute(adagc_update_tma_kernel<kBF16, kOpt, kSB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              tma_smem_bytes<kSB>(kBF16, kOpt, kOpt == kOptAdamW)) == cudaSuccess;
+}
+template <bool kBF16, bool kSB>
 bool prepare_update_kernels() {
-  return cudaFuncSetAttribute(adagc_update_kernel<kBF16, kOptAdamW>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                              cudaSharedmemCarveoutMaxL1) == cudaSuccess &&
-         cudaFuncSetAttribute(adagc_update_kernel<kBF16, kOptLion>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                              cudaSharedmemCarveoutMaxL1) == cudaSuccess &&
-         cudaFuncSetAttribute(adagc_update_tma_kernel<kBF16, kOptAdamW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              tma_smem_bytes(kBF16, kOptAdamW, true)) == cudaSuccess &&
-         cudaFuncSetAttribute(adagc_update_tma_kernel<kBF16, kOptLion>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              tma_smem_bytes(kBF16, kOptLion)) == cudaSuccess &&
-         cudaFuncSetAttribute(adagc_update_kernel<kBF16, kOptSgdM>, cudaFuncAttributePreferredSharedMemoryCarveout,
-                              cudaSharedmemCarveoutMaxL1) == cudaSuccess &&
-         cudaFuncSetAttribute(adagc_update_tma_kernel<kBF16, kOptSgdM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              tma_smem_bytes(kBF16, kOptSgdM)) == cudaSuccess;
+  return prepare_update_kernel<kBF16, kOptAdamW, kSB>() && prepare_update_kernel<kBF16, kOptLion, kSB>() &&
+         prepare_update_kernel<kBF16, kOptSgdM, kSB>();
 }
 
 // One kernel's view of the chunk tables: the whole layout, or one group of the pipelined host step.
@@ -1325,24 +1425,40 @@ struct TableView {
   int grid;
 };
 
-template <bool kBF16, int kOpt>
-void launch_update(adagc_ctx* ctx, const TableView& tv, float* p, const void* g, float* m, float* v,
-                   const AdamScalars& a, cudaStream_t s, uint16_t* lowp = nullptr, const AdamScalars* d_a = nullptr) {
+template <bool kBF16, int kOpt, bool kSB>
+void launch_update_t(adagc_ctx* ctx, const TableView& tv, float* p, const void* g, void* m, void* v,
+                     const AdamScalars& a, cudaStream_t s, uint16_t* lowp, const AdamScalars* d_a) {
   const StatPtrs st = ctx->stats();
   if (ctx->update_bulk)
-    adagc_update_tma_kernel<kBF16, kOpt>
-        <<<tv.grid, kTmaThreads, tma_smem_bytes(kBF16, kOpt, lowp != nullptr), s>>>(
+    adagc_update_tma_kernel<kBF16, kOpt, kSB>
+        <<<tv.grid, kTmaThreads, tma_smem_bytes<kSB>(kBF16, kOpt, lowp != nullptr), s>>>(
             p, g, m, v, tv.chunks, tv.begin, tv.mid, st.h, a, st.status, lowp, d_a);
   else
-    adagc_update_kernel<kBF16, kOpt><<<tv.grid, kThreads, 0, s>>>(p, g, m, v, tv.chunks, tv.begin, st.h, a, lowp, d_a);
+    adagc_update_kernel<kBF16, kOpt, kSB><<<tv.grid, kThreads, 0, s>>>(p, g, m, v, tv.chunks, tv.begin, st.h, a, lowp, d_a);
   ctx->launches++;
 }
 
-template <bool kBF16, int kOpt>
-void launch_update(adagc_ctx* ctx, float* p, const void* g, float* m, float* v, const AdamScalars& a,
-                   cudaStream_t s, uint16_t* lowp = nullptr, const AdamScalars* d_a = nullptr) {
+// The update phase over one table view, in the context's gradient and state dtypes.  m and v are fp32 or bfloat16
+// arenas (adagc_desc.state_dtype); v is unused by Lion and momentum SGD.
+template <int kOpt>
+void launch_update(adagc_ctx* ctx, const TableView& tv, void* p, const void* g, void* m, void* v,
+                   const AdamScalars& a, cudaStream_t s, void* lowp = nullptr, const AdamScalars* d_a = nullptr) {
+  float* pf = static_cast<float*>(p);
+  uint16_t* lp = static_cast<uint16_t*>(lowp);
+  if (ctx->bf16) {
+    if (ctx->state_bf16) launch_update_t<true, kOpt, true>(ctx, tv, pf, g, m, v, a, s, lp, d_a);
+    else launch_update_t<true, kOpt, false>(ctx, tv, pf, g, m, v, a, s, lp, d_a);
+  } else {
+    if (ctx->state_bf16) launch_update_t<false, kOpt, true>(ctx, tv, pf, g, m, v, a, s, lp, d_a);
+    else launch_update_t<false, kOpt, false>(ctx, tv, pf, g, m, v, a, s, lp, d_a);
+  }
+}
+
+template <int kOpt>
+void launch_update(adagc_ctx* ctx, void* p, const void* g, void* m, void* v, const AdamScalars& a,
+                   cudaStream_t s, void* lowp = nullptr, const AdamScalars* d_a = nullptr) {
   const TableView tv = {ctx->d_chunks_upd(), ctx->d_begin_upd(), ctx->d_mid_upd(), ctx->grid_update};
-  launch_update<kBF16, kOpt>(ctx, tv, p, g, m, v, a, s, lowp, d_a);
+  launch_update<kOpt>(ctx, tv, p, g, m, v, a, s, lowp, d_a);
 }
 
 void launch_norm(adagc_ctx* ctx, const TableView& tv, const void* d_grads, cudaStream_t s) {
@@ -1478,12 +1594,7 @@ int enqueue_grouped_adamw(adagc_ctx* ctx, void* d_params, const void* d_grads, v
                                                                     ctx->stats(), order, gr.order_first, gr.n_tensors,
                                                                     k == 0 ? 1 : 0);
     ctx->launches++;
-    if (ctx->bf16)
-      launch_update<true, kOptAdamW>(ctx, upd, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
-                                     static_cast<float*>(d_v), a, s);
-    else
-      launch_update<false, kOptAdamW>(ctx, upd, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
-                                      static_cast<float*>(d_v), a, s);
+    launch_update<kOptAdamW>(ctx, upd, d_params, d_grads, d_m, d_v, a, s);
   }
   return ADAGC_OK;
 }
@@ -1496,6 +1607,14 @@ int finish_launches(adagc_ctx* ctx, cudaStream_t s) {
   return cudaGetLastError() == cudaSuccess ? ADAGC_OK : ADAGC_E_CUDA;
 }
 
+const void* fused_small_kernel_of(const adagc_ctx* ctx) {
+  if (ctx->bf16)
+    return ctx->state_bf16 ? reinterpret_cast<const void*>(adagc_fused_small_kernel<true, true>)
+                           : reinterpret_cast<const void*>(adagc_fused_small_kernel<true, false>);
+  return ctx->state_bf16 ? reinterpret_cast<const void*>(adagc_fused_small_kernel<false, true>)
+                         : reinterpret_cast<const void*>(adagc_fused_small_kernel<false, false>);
+}
+
 // adagc_step of a context created with ADAGC_FUSED_SMALL: one cooperative launch.
 int launch_fused_small(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, void* d_v, float* d_ema,
                        ClipScalars cs, bool in_warmup, AdamScalars a, cudaStream_t s) {
@@ -1505,8 +1624,8 @@ int launch_fused_small(adagc_ctx* ctx, void* d_params, const void* d_grads, void
     cudaEventRecord(ctx->ev[2], s);  // the phases are not separable here: the whole kernel is reported as the third
   }
   float* p = static_cast<float*>(d_params);
-  float* m = static_cast<float*>(d_m);
-  float* v = static_cast<float*>(d_v);
+  void* m = d_m;
+  void* v = d_v;
   const Chunk* chunks = ctx->d_chunks_upd();
   int n_chunks = ctx->n_chunks;
   const TensorEntry* tensors = ctx->d_tensors();
@@ -1518,8 +1637,7 @@ int launch_fused_small(adagc_ctx* ctx, void* d_params, const void* d_grads, void
   float* gamma_prev = reinterpret_cast<float*>(ctx->ws + ctx->L.gamma_prev);
   void* args[] = {&p,        &d_grads, &m,    &v, &d_ema, &chunks,  &n_chunks, &tensors,
                   &partials, &cs,      &warm, &a, &st,    &counter, &index, &gamma_prev};
-  const void* fn = ctx->bf16 ? reinterpret_cast<const void*>(adagc_fused_small_kernel<true>)
-                             : reinterpret_cast<const void*>(adagc_fused_small_kernel<false>);
+  const void* fn = fused_small_kernel_of(ctx);
   if (cudaLaunchCooperativeKernel(fn, dim3(ctx->grid_fused), dim3(kThreads), args, 0, s) != cudaSuccess) {
     (void)cudaGetLastError();
     return ADAGC_E_CUDA;
@@ -1593,6 +1711,7 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
   ctx->n_chunks = static_cast<int32_t>(n_chunks);
   ctx->arena_elems = extent;
   ctx->bf16 = desc->grad_dtype == ADAGC_BF16;
+  ctx->state_bf16 = desc->state_dtype == ADAGC_BF16;
   ctx->lambda_abs = desc->lambda_abs;
   bool any_empty = false;
   for (int32_t i = 0; i < desc->n_tensors; ++i) {
@@ -1611,11 +1730,11 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
     if (ctx->bf16) {
       ok = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_n, adagc_norm_kernel<true>, kThreads, 0) == cudaSuccess &&
            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_s, adagc_scale_kernel<true>, kThreads, 0) == cudaSuccess &&
-           prepare_update_kernels<true>();
+           (ctx->state_bf16 ? prepare_update_kernels<true, true>() : prepare_update_kernels<true, false>());
     } else {
       ok = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_n, adagc_norm_kernel<false>, kThreads, 0) == cudaSuccess &&
            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_s, adagc_scale_kernel<false>, kThreads, 0) == cudaSuccess &&
-           prepare_update_kernels<false>();
+           (ctx->state_bf16 ? prepare_update_kernels<false, true>() : prepare_update_kernels<false, false>());
     }
     if (ok) {
       const int64_t sms = prop.multiProcessorCount;
@@ -1632,9 +1751,7 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
     // the one-kernel step needs every block resident at once (cooperative launch) and is meant for small layouts
     int coop = 0, occ_f = 0;
     ok = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, ctx->device) == cudaSuccess &&
-         (ctx->bf16 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_f, adagc_fused_small_kernel<true>, kThreads, 0)
-                    : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_f, adagc_fused_small_kernel<false>, kThreads, 0)) ==
-             cudaSuccess;
+         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ_f, fused_small_kernel_of(ctx), kThreads, 0) == cudaSuccess;
     if (ok && (!coop || n_chunks > kFusedMaxChunks || occ_f < 1)) {
       release_ctx(ctx);
       return ADAGC_E_INVALID_ARG;
@@ -1750,12 +1867,7 @@ int adagc_step(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, v
   rc = enqueue_clip_phases(ctx, d_grads, d_ema, step, lambda_rel, beta, warmup, s);
   if (rc != ADAGC_OK) return rc;
   const AdamScalars a = make_adam_scalars(step, lr, beta1, beta2, eps, wd);
-  if (ctx->bf16)
-    launch_update<true, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
-                                   static_cast<float*>(d_v), a, s);
-  else
-    launch_update<false, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
-                                    static_cast<float*>(d_v), a, s);
+  launch_update<kOptAdamW>(ctx, d_params, d_grads, d_m, d_v, a, s);
   return finish_launches(ctx, s);
 }
 
@@ -1772,13 +1884,7 @@ int adagc_step_emit_bf16(adagc_ctx* ctx, void* d_params, void* d_params_bf16, co
   rc = enqueue_clip_phases(ctx, d_grads, d_ema, step, lambda_rel, beta, warmup, s);
   if (rc != ADAGC_OK) return rc;
   const AdamScalars a = make_adam_scalars(step, lr, beta1, beta2, eps, wd);
-  uint16_t* lowp = static_cast<uint16_t*>(d_params_bf16);
-  if (ctx->bf16)
-    launch_update<true, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
-                                   static_cast<float*>(d_v), a, s, lowp);
-  else
-    launch_update<false, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
-                                    static_cast<float*>(d_v), a, s, lowp);
+  launch_update<kOptAdamW>(ctx, d_params, d_grads, d_m, d_v, a, s, d_params_bf16);
   return finish_launches(ctx, s);
 }
 
@@ -1803,10 +1909,7 @@ int adagc_step_lion(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d
   a.step_size = static_cast<float>(lr);
   a.decay = static_cast<float>(1.0 - lr * wd);
   a.eps = 0.0f;
-  if (ctx->bf16)
-    launch_update<true, kOptLion>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), nullptr, a, s);
-  else
-    launch_update<false, kOptLion>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), nullptr, a, s);
+  launch_update<kOptLion>(ctx, d_params, d_grads, d_m, nullptr, a, s);
   return finish_launches(ctx, s);
 }
 
@@ -1825,10 +1928,7 @@ int adagc_step_sgdm(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d
   a.beta1 = static_cast<float>(momentum);
   a.step_size = static_cast<float>(lr);
   a.decay = static_cast<float>(wd);
-  if (ctx->bf16)
-    launch_update<true, kOptSgdM>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), nullptr, a, s);
-  else
-    launch_update<false, kOptSgdM>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m), nullptr, a, s);
+  launch_update<kOptSgdM>(ctx, d_params, d_grads, d_m, nullptr, a, s);
   return finish_launches(ctx, s);
 }
 
@@ -1875,12 +1975,7 @@ int adagc_step_capturable(adagc_ctx* ctx, void* d_params, const void* d_grads, v
   else
     adagc_warmup_finalize_kernel<<<1, kWarmupThreads, 0, s>>>(ClipScalars{}, d_ema, st, ds);
   ctx->launches++;
-  if (ctx->bf16)
-    launch_update<true, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
-                                   static_cast<float*>(d_v), AdamScalars{}, s, nullptr, &ds->a);
-  else
-    launch_update<false, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
-                                    static_cast<float*>(d_v), AdamScalars{}, s, nullptr, &ds->a);
+  launch_update<kOptAdamW>(ctx, d_params, d_grads, d_m, d_v, AdamScalars{}, s, nullptr, &ds->a);
   return cudaGetLastError() == cudaSuccess ? ADAGC_OK : ADAGC_E_CUDA;
 }
 
@@ -1925,12 +2020,7 @@ int adagc_step_presummed(adagc_ctx* ctx, void* d_params, const void* d_grads, vo
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   enqueue_presummed_phase(ctx, d_sumsq, d_ema, step, lambda_rel, beta, warmup, s);
   const AdamScalars a = make_adam_scalars(step, lr, beta1, beta2, eps, wd);
-  if (ctx->bf16)
-    launch_update<true, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
-                                   static_cast<float*>(d_v), a, s);
-  else
-    launch_update<false, kOptAdamW>(ctx, static_cast<float*>(d_params), d_grads, static_cast<float*>(d_m),
-                                    static_cast<float*>(d_v), a, s);
+  launch_update<kOptAdamW>(ctx, d_params, d_grads, d_m, d_v, a, s);
   return finish_launches(ctx, s);
 }
 

@@ -491,3 +491,181 @@ def run_full_sharded(wl: workloads.Workload, n_steps: int, world: int, device="c
     for rk in ranks:
         rk.close()
     return rep
+
+
+# ------------------------------------------------------------------------------------------------------------------
+# Optimizer state stored as bfloat16 (adagc_desc.state_dtype = ADAGC_BF16)
+# ------------------------------------------------------------------------------------------------------------------
+def _bf16_view(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def _assert_same_bf16(name: str, got_bits: np.ndarray, ref_bits: np.ndarray, what: str):
+    bad = np.nonzero(got_bits != ref_bits)[0]
+    assert bad.size == 0, (f"{name} of {what}: {bad.size} of {got_bits.size} stored bfloat16 values differ from the oracle's, "
+                           f"first at element {bad[:3]}: {bf16_bits_to_f64(got_bits[bad[:3]])} vs {bf16_bits_to_f64(ref_bits[bad[:3]])}")
+
+
+def run_bf16_state(wl: workloads.Workload, n_steps: int, optimizer: str = "adamw", teacher_forced: bool = False,
+                   device="cuda", flags: int = 0, hyper_over: Optional[dict] = None, lion_lr: float = 1e-4,
+                   sgd_lr: float = 1e-2) -> ParityReport:
+    """Every element with m (and v) stored as bfloat16, GPU vs the C oracle's bfloat16-state functions.
+
+    Which bfloat16 neighbour a moment is stored as is a discrete decision, taken on both sides in the precision the
+    library states for it (single precision, a fixed operation order: the oracle's fp32_decision mode, itself pinned
+    to exact rational arithmetic and to the float64 definition).  So the stored m and v must be BIT-IDENTICAL to the
+    oracle's on every element at every step; theta meets the fp32 tolerance (it is computed from the unrounded moments).
+      free-running    both sides carry their own state for n_steps (m and v do not depend on theta, so they stay
+                      bit-identical; momentum SGD's m does depend on theta and is only compared in the other mode);
+      teacher_forced  before every step the GPU's theta, m, v are overwritten with the oracle's stored state (inputs
+                      flow oracle -> GPU only) and every step is compared from identical stored state.
+    Lion's sign(c) near-ties may move theta by 2 lr per occurrence, as in run_full_lion.
+    """
+    hp = hyper_of(wl, **(hyper_over or {}))
+    offs = np.array([t.offset for t in wl.tensors], np.int64)
+    nums = np.array([t.numel for t in wl.tensors], np.int64)
+    opt = binding.AdaGC(nums.tolist(), offs.tolist(), wl.torch_grad_dtype, hp["lambda_abs"], device=device, flags=flags,
+                        state_dtype=torch.bfloat16)
+    n_state = 2 if optimizer == "adamw" else 1
+    assert optimizer != "sgdm" or teacher_forced, "momentum SGD's m depends on theta: compare it from identical state"
+    theta = workloads.init_params(wl, device)
+    r_theta = theta.cpu().numpy().copy()
+    pad = np.ones(wl.arena_elems, bool)
+    for o, n in zip(offs, nums):
+        pad[o:o + n] = False
+    pad_mask = torch.from_numpy(pad).to(device)
+    GUARD = 768.0                                            # a bfloat16 value
+    theta[pad_mask] = GUARD
+    m = torch.zeros(wl.arena_elems, dtype=torch.bfloat16, device=device)
+    v = torch.zeros_like(m)
+    m[pad_mask] = GUARD
+    v[pad_mask] = GUARD
+    r_m = np.zeros(wl.arena_elems, np.uint16)
+    r_v = np.zeros(wl.arena_elems, np.uint16)
+    sign_ties = np.zeros(wl.arena_elems, np.uint8)           # Lion only
+    ema = torch.full((wl.n_tensors,), float("nan"), dtype=torch.float32, device=device)
+    gamma = np.zeros(wl.n_tensors, np.float32)
+    clip_count = np.zeros(wl.n_tensors, np.uint64)
+    rep = ParityReport()
+    lr = {"adamw": hp["lr"], "lion": lion_lr, "sgdm": sgd_lr}[optimizer]
+
+    def gpu_step(g, t):
+        if optimizer == "adamw":
+            opt.step(theta, g, m, v, ema, t, lr, hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"],
+                     hp["beta"], hp["warmup"])
+        elif optimizer == "lion":
+            opt.step_lion(theta, g, m, ema, t, lr, 0.9, 0.99, hp["wd"], hp["lambda_rel"], hp["beta"], hp["warmup"])
+        else:
+            opt.step_sgdm(theta, g, m, ema, t, lr, 0.9, hp["wd"], hp["lambda_rel"], hp["beta"], hp["warmup"])
+
+    def oracle_update(o, n, g_np, h, t, ties):
+        sl = slice(o, o + n)
+        if optimizer == "adamw":
+            c_oracle.adamw_update_bf16state(r_theta[sl], g_np[sl], r_m[sl], r_v[sl], h, t, lr, hp["beta1"], hp["beta2"],
+                                            hp["eps"], hp["wd"], fp32_decision=True)
+        elif optimizer == "lion":
+            c_oracle.lion_update(r_theta[sl], g_np[sl], r_m[sl], h, lr, 0.9, 0.99, hp["wd"], near_tie=ties[sl],
+                                 tie_tol=LION_TIE_TOL, fp32_decision=True)
+        else:
+            c_oracle.sgdm_update(r_theta[sl], g_np[sl], r_m[sl], h, lr, 0.9, hp["wd"], fp32_decision=True)
+
+    def compare(t, ties):
+        th, mb, vb = theta.cpu().numpy(), _bf16_view(m), _bf16_view(v)
+        for t_, o, n in zip(wl.tensors, offs, nums):
+            sl = slice(int(o), int(o + n))
+            what = f"{t_.name}, step {t}"
+            _assert_same_bf16("m", mb[sl], r_m[sl], what)
+            if n_state == 2:
+                _assert_same_bf16("v", vb[sl], r_v[sl], what)
+            if optimizer == "lion":
+                sure = ties[sl] == 0
+                check_state("theta", th[sl][sure], r_theta[sl][sure], rep, what)
+                d = np.abs(th[sl][~sure].astype(np.float64) - r_theta[sl][~sure])
+                k = ties[sl][~sure].astype(np.float64)
+                assert (d <= 2.0 * lr * k * 1.001 + RTOL * np.maximum(np.abs(r_theta[sl][~sure]), 1e-3)).all(), \
+                    f"theta of {what}: sign near-tie element off"
+            else:
+                check_state("theta", th[sl], r_theta[sl], rep, what)
+
+    for t in range(1, n_steps + 1):
+        g = workloads.grads_for_step(wl, t, device)
+        g_np = to_numpy_grads(g)
+        if teacher_forced and t > 1:                         # the oracle's stored state is this step's input on both sides
+            keep = theta[pad_mask].clone()
+            theta.copy_(torch.from_numpy(r_theta).to(device))
+            theta[pad_mask] = keep
+            for dst, src in ((m, r_m), (v, r_v)):
+                bits = torch.from_numpy(src.view(np.int16)).to(device).view(torch.bfloat16)
+                dst.copy_(torch.where(pad_mask, dst, bits))
+        gpu_step(g, t)
+        ssq = c_oracle.sumsq_tensors(g_np, offs, nums)
+        r = c_oracle.clip_decisions(ssq, gamma, t, hp["lambda_rel"], hp["beta"], hp["lambda_abs"], hp["warmup"])
+        clip_count += r["flag"].astype(np.uint64)
+        step_ties = np.zeros(wl.arena_elems, np.uint8) if teacher_forced else sign_ties
+        for i, (o, n) in enumerate(zip(offs, nums)):
+            oracle_update(int(o), int(n), g_np, float(r["h"][i]), t, step_ties)
+        check_decisions(opt.get_stats(), opt.get_sumsq(), ema.cpu().numpy(), r, rep, t)
+        if teacher_forced or t == n_steps:
+            compare(t, step_ties)
+        rep.steps = t
+    st = opt.get_stats()
+    assert st["steps_done"] == n_steps and np.array_equal(st["clip_count"], clip_count) and st["status"] == 0
+    for a, name in ((theta, "theta"), (m, "m"), (v, "v")):
+        assert bool((a[pad_mask].float() == GUARD).all()), f"guard bands between tensors were overwritten in {name}"
+    if optimizer == "lion":
+        assert int((sign_ties > 0).sum()) <= 1e-3 * wl.n_params + 50
+    opt.close()
+    return rep
+
+
+def run_sampled_bf16_state(wl: workloads.Workload, n_steps: int, device="cuda", k: int = 2048,
+                           hyper_over: Optional[dict] = None) -> ParityReport:
+    """Full-size layouts with bfloat16 moments: all norms / decisions / gamma against the oracle, and theta, m, v on
+    sampled elements that the oracle follows one by one (free-running; m and v bit-identical, theta within tolerance)."""
+    hp = hyper_of(wl, **(hyper_over or {}))
+    offs = np.array([t.offset for t in wl.tensors], np.int64)
+    nums = np.array([t.numel for t in wl.tensors], np.int64)
+    opt = binding.AdaGC(nums.tolist(), offs.tolist(), wl.torch_grad_dtype, hp["lambda_abs"], device=device,
+                        state_dtype=torch.bfloat16)
+    rng = np.random.RandomState(99)
+    samp = [sample_indices(int(n), k, rng) + int(o) for o, n in zip(offs, nums)]
+    sizes = np.array([len(s) for s in samp], np.int64)
+    soff = np.concatenate([[0], np.cumsum(sizes)[:-1]]).astype(np.int64)
+    flat_np = np.concatenate(samp)
+    flat = torch.from_numpy(flat_np).to(device)
+    rep = ParityReport()
+    gamma = np.zeros(wl.n_tensors, np.float32)
+    clip_count = np.zeros(wl.n_tensors, np.uint64)
+    ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device=device)
+    theta = workloads.init_params(wl, device)
+    m = torch.zeros(wl.arena_elems, dtype=torch.bfloat16, device=device)
+    v = torch.zeros_like(m)
+    s_theta = theta[flat].cpu().numpy().copy()
+    s_m, s_v = np.zeros(len(flat_np), np.uint16), np.zeros(len(flat_np), np.uint16)
+    for t in range(1, n_steps + 1):
+        g = workloads.grads_for_step(wl, t, device)
+        g_np = to_numpy_grads(g)
+        s_g = np.ascontiguousarray(g_np[flat_np])
+        opt.step(theta, g, m, v, ema, t, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"],
+                 hp["beta"], hp["warmup"])
+        ssq = c_oracle.sumsq_tensors(g_np, offs, nums)
+        r = c_oracle.clip_decisions(ssq, gamma, t, hp["lambda_rel"], hp["beta"], hp["lambda_abs"], hp["warmup"])
+        clip_count += r["flag"].astype(np.uint64)
+        check_decisions(opt.get_stats(), opt.get_sumsq(), ema.cpu().numpy(), r, rep, t)
+        for i in range(wl.n_tensors):
+            sl = slice(int(soff[i]), int(soff[i] + sizes[i]))
+            c_oracle.adamw_update_bf16state(s_theta[sl], s_g[sl], s_m[sl], s_v[sl], float(r["h"][i]), t, hp["lr"],
+                                            hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], fp32_decision=True)
+        rep.steps = t
+        del g
+    st = opt.get_stats()
+    assert st["steps_done"] == n_steps and np.array_equal(st["clip_count"], clip_count) and st["status"] == 0
+    g_theta = theta[flat].cpu().numpy()
+    g_m, g_v = _bf16_view(m[flat]), _bf16_view(v[flat])
+    for i, t_ in enumerate(wl.tensors):
+        sl = slice(int(soff[i]), int(soff[i] + sizes[i]))
+        _assert_same_bf16("m", g_m[sl], s_m[sl], t_.name)
+        _assert_same_bf16("v", g_v[sl], s_v[sl], t_.name)
+        check_state("theta", g_theta[sl], s_theta[sl], rep, t_.name)
+    opt.close()
+    return rep

@@ -271,3 +271,92 @@ def test_c_oracle_counts_decisions_close_to_a_flip():
     assert bits_to_f64(mb).tolist() == [1.0 + 2.0 ** -7, 1.0, 1.0 + 2.0 ** -7]     # tie to even; just above the midpoint rounds up
     _, _, _, mm, _ = npo.adamw_update(th, g, m0, v0, 1.0, 3, hp, np.float32, moment_dtype="bf16", return_margin=True)
     assert mm[1] == 0.0 and mm[0] > 1e-3 and 0 < mm[2] < 1e-5
+
+
+# ----------------------------------------------------------------------------- the rounding decision taken in fp32
+def _round_fraction(x, sig_bits, e_min):
+    """Exact rational x -> nearest binary floating-point number with `sig_bits` significand bits and least exponent
+    e_min for the last place (round half to even), returned as a Fraction."""
+    from fractions import Fraction
+    if x == 0:
+        return Fraction(0)
+    e = 0
+    ax = abs(x)
+    while ax >= Fraction(2) ** (e + 1):
+        e += 1
+    while ax < Fraction(2) ** e:
+        e -= 1
+    ulp_e = max(e - (sig_bits - 1), e_min)
+    n = round(x / Fraction(2) ** ulp_e)                     # Python rounds halves to even
+    return n * Fraction(2) ** ulp_e
+
+
+def test_fp32_decision_follows_the_stated_single_precision_order_exactly():
+    """The stored bfloat16 of the C oracle's fp32-decision mode equals, bit for bit, the stated formula evaluated in
+    exact rational arithmetic with one rounding to single precision per operation (24 bits, last place >= 2^-149)
+    and one rounding to bfloat16 (8 bits, last place >= 2^-133) at the end."""
+    from fractions import Fraction as F
+    rng = np.random.RandomState(21)
+    n = 1500
+    g = bf16_values(rng, n, 1e-4).astype(np.float32)
+    g[:50] = (rng.standard_normal(50) * 1e-4).astype(np.float32)            # and some full-precision gradients
+    m0, v0 = bf16_values(rng, n, 3e-5), np.abs(bf16_values(rng, n, 1e-8))
+    theta = (rng.standard_normal(n) * 0.02).astype(np.float32)
+    h, b1, b2 = 0.731, 0.9, 0.95
+    f32 = lambda x: _round_fraction(x, 24, -149)
+    bf = lambda x: _round_fraction(x, 8, -133)
+    hf, b1f, o1f, b2f, o2f = (F(float(np.float32(x))) for x in (h, b1, 1.0 - b1, b2, 1.0 - b2))
+    want_m, want_v = [], []
+    for j in range(n):
+        gh = f32(hf * F(float(g[j])))
+        want_m.append(float(bf(f32(b1f * F(float(m0[j])) + f32(o1f * gh)))))
+        want_v.append(float(bf(f32(b2f * F(float(v0[j])) + f32(o2f * f32(gh * gh))))))
+    mb, vb = f32_to_bits(m0), f32_to_bits(v0)
+    co.adamw_update_bf16state(theta.copy(), g, mb, vb, h, 3, 1e-3, b1, b2, 1e-8, 0.1, fp32_decision=True)
+    assert np.array_equal(bits_to_f64(mb), np.array(want_m)) and np.array_equal(bits_to_f64(vb), np.array(want_v))
+    # Lion's and momentum SGD's stored momentum, the same way
+    mb = f32_to_bits(m0)
+    co.lion_update(theta.copy(), g, mb, h, 1e-4, 0.9, 0.99, 0.1, fp32_decision=True)
+    b2l, o2l = F(float(np.float32(0.99))), F(float(np.float32(1.0 - 0.99)))
+    want = [float(bf(f32(b2l * F(float(m0[j])) + f32(o2l * f32(hf * F(float(g[j]))))))) for j in range(n)]
+    assert np.array_equal(bits_to_f64(mb), np.array(want))
+    mb = f32_to_bits(m0)
+    co.sgdm_update(theta.copy(), g, mb, h, 1e-2, 0.9, 0.05, fp32_decision=True)
+    muf, wdf = F(float(np.float32(0.9))), F(float(np.float32(0.05)))
+    want = [float(bf(f32(muf * F(float(m0[j])) + f32(wdf * F(float(theta[j])) + f32(hf * F(float(g[j]))))))) for j in range(n)]
+    assert np.array_equal(bits_to_f64(mb), np.array(want))
+
+
+def test_fp32_and_float64_decisions_differ_only_at_reported_ties_and_by_one_neighbour():
+    """The single-precision decision is pinned to the (library-pinned) float64 one: the stored values agree except
+    where the float64 oracle itself reports that the rounding was decided within 1e-6 of a flip, and there they are
+    neighbours.  With bfloat16 g and m and beta1 = 0.9 such ties are frequent: the float64 value is an exact decimal
+    tie (x.5 spacings) for a few percent of the elements, which is why the decision must name its precision."""
+    rng = np.random.RandomState(22)
+    n = 200000
+    g = bf16_values(rng, n, 1e-4).astype(np.float32)
+    m0, v0 = bf16_values(rng, n, 3e-5), np.abs(bf16_values(rng, n, 1e-8))
+    theta = (rng.standard_normal(n) * 0.02).astype(np.float32)
+    th64, th32 = theta.copy(), theta.copy()
+    m64, v64, m32, v32 = f32_to_bits(m0), f32_to_bits(v0), f32_to_bits(m0), f32_to_bits(v0)
+    ties = np.zeros(n, np.uint8)
+    co.adamw_update_bf16state(th64, g, m64, v64, 1.0, 4, 3e-4, 0.9, 0.95, 1e-8, 0.1, near_tie=ties, tie_tol=1e-6)
+    co.adamw_update_bf16state(th32, g, m32, v32, 1.0, 4, 3e-4, 0.9, 0.95, 1e-8, 0.1, fp32_decision=True)
+    assert np.array_equal(th64, th32)                                  # theta never sees the rounding decision
+    m_terms = np.abs(0.9 * m0.astype(np.float64)) + np.abs(0.1 * g.astype(np.float64))
+    for a, b, terms in ((m64, m32, m_terms), (v64, v32, None)):
+        diff = a != b
+        assert (~diff | (ties > 0)).all()
+        # neighbours (bfloat16 bit patterns of one sign are ordered like the magnitudes they encode) -- or, where the
+        # two terms of m' cancel completely, two different roundings of what is zero in exact arithmetic
+        near = np.abs(a[diff].astype(np.int64) - b[diff].astype(np.int64)) == 1
+        if terms is not None:
+            near |= np.maximum(np.abs(bits_to_f64(a[diff])), np.abs(bits_to_f64(b[diff]))) <= 1e-6 * terms[diff]
+        assert near.all()
+    assert 0.01 < (ties > 0).mean() < 0.10 and (m64 != m32).mean() > 0.005
+    # with full-precision fp32 gradients the ties are as rare as for arbitrary numbers
+    g2 = (rng.standard_normal(n) * 1e-4).astype(np.float32)
+    ties2 = np.zeros(n, np.uint8)
+    co.adamw_update_bf16state(theta.copy(), g2, f32_to_bits(m0), f32_to_bits(v0), 1.0, 4, 3e-4, 0.9, 0.95, 1e-8, 0.1,
+                              near_tie=ties2, tie_tol=1e-6)
+    assert (ties2 > 0).mean() < 4e-3

@@ -48,7 +48,8 @@ typedef enum {
   ADAGC_E_DTYPE = -5,       /* unsupported dtype combination */
   ADAGC_E_CUDA = -6,        /* a CUDA runtime call failed (no device, launch error, ...) */
   ADAGC_E_NOMEM = -7,       /* host allocation of the context failed */
-  ADAGC_E_TOO_LARGE = -8    /* adagc_sumsq_noalloc: more elements than its fixed scratch covers */
+  ADAGC_E_TOO_LARGE = -8,   /* adagc_sumsq_noalloc: more elements than its fixed scratch covers */
+  ADAGC_E_POISONED = -9     /* ADAGC_FUSED_SMALL context after adagc_get_stats reported ADAGC_E_TIMEOUT */
 } adagc_status;
 
 /* Bits of the device status word (adagc_get_stats). */
@@ -84,7 +85,8 @@ typedef enum {
  * returns ADAGC_E_INVALID_ARG beyond that, with ADAGC_CLIP_GLOBAL_ADAPTIVE, or on a device without cooperative
  * launch).  Only adagc_step takes the fused route; every other entry point of the context is unchanged.  The
  * barriers wait with a time limit; if one gives up, ADAGC_E_TIMEOUT is set in the status word and the context must
- * be created anew. */
+ * be created anew: once adagc_get_stats has read that bit, every later adagc_step of the context returns
+ * ADAGC_E_POISONED and enqueues nothing (until then the steps still return ADAGC_OK, each waiting out its limit). */
 #define ADAGC_FUSED_SMALL 32
 
 /*
@@ -106,6 +108,11 @@ typedef enum {
  * moving once (1 - beta)|target - x| drops below half its spacing, i.e. within spacing / (2 (1 - beta)) of the value
  * an fp32 moment would reach: 10 spacings (8 %) for beta2 = 0.95, 500 spacings for beta2 = 0.999.
  */
+
+/* On AdaGC steps (step > warmup) the per-tensor decisions are taken in the tail of the norm kernel, so the step is two
+ * launches.  With this flag they run as a kernel of their own, as on warm-up steps (three launches).  Results are
+ * bit-identical either way.  (Contexts with ADAGC_ALLOW_EMPTY tensors of numel 0 always use the separate kernel.) */
+#define ADAGC_SEPARATE_FINALIZE 64
 
 /* One parameter tensor. */
 typedef struct {
@@ -355,6 +362,10 @@ int adagc_get_phase_times(adagc_ctx* ctx, float ms[3]);
  * The call enqueues two kernels on `cuda_stream`, does not synchronise, and calls no allocating
  * routine.  The first call on each device looks up the array's device address
  * (cudaGetSymbolAddress, with that device current); make that first call outside any stream capture.
+ * That lookup is safe against several host threads making their first call at once (one does it, the
+ * others wait).  Device ordinals 0..63 are supported; on a higher ordinal, or if the lookup fails, the
+ * call returns ADAGC_E_CUDA and enqueues nothing.  If a launch itself fails the return value is
+ * ADAGC_E_CUDA as well, and the first kernel may already be enqueued.
  * All calls share the one array and it keeps the previous call's contents; every entry a call reads
  * it has first rewritten, so nothing needs clearing, but two calls whose kernels overlap on the GPU
  * (different streams, or several host threads) race on it: serialise them on one stream or with events.
@@ -370,6 +381,10 @@ int adagc_sumsq_noalloc(const void* d_grads, int32_t grad_dtype, int64_t numel, 
  * returns normally, leaving the context usable.  Enqueues only.
  */
 int adagc_debug_wait_timeout(adagc_ctx* ctx, double limit_ms, void* cuda_stream);
+
+/* Test aid: feeds `device_status` to the same host-side latch that adagc_get_stats applies to the status word it reads
+ * (a context created with ADAGC_FUSED_SMALL refuses further steps once ADAGC_E_TIMEOUT has been seen).  Host-only. */
+int adagc_debug_latch_status(adagc_ctx* ctx, int32_t device_status);
 
 /* Static string for a status code. */
 const char* adagc_strerror(int status);

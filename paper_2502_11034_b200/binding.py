@@ -16,7 +16,7 @@ ADAGC_F32, ADAGC_BF16 = 0, 1
 ADAGC_W_NONFINITE = 1
 ADAGC_E_TIMEOUT = 2
 UPDATE_PATH_AUTO, UPDATE_PATH_REGISTERS, UPDATE_PATH_BULK = 0, 1, 2
-EMA_KEEP_INITIAL, CLIP_GLOBAL_ADAPTIVE, ALLOW_EMPTY, FUSED_SMALL = 4, 8, 16, 32
+EMA_KEEP_INITIAL, CLIP_GLOBAL_ADAPTIVE, ALLOW_EMPTY, FUSED_SMALL, SEPARATE_FINALIZE = 4, 8, 16, 32, 64
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libadagc.so")
 _lib = None
@@ -103,6 +103,8 @@ def lib() -> C.CDLL:
     L.adagc_sumsq_noalloc.argtypes = [vp, C.c_int32, i64, vp, vp]
     L.adagc_debug_wait_timeout.restype = C.c_int
     L.adagc_debug_wait_timeout.argtypes = [vp, dbl, vp]
+    L.adagc_debug_latch_status.restype = C.c_int
+    L.adagc_debug_latch_status.argtypes = [vp, C.c_int32]
     L.adagc_strerror.restype = C.c_char_p
     L.adagc_strerror.argtypes = [C.c_int]
     _lib = L
@@ -329,6 +331,11 @@ class AdaGC:
         rc = lib().adagc_debug_wait_timeout(self._h, float(limit_ms), _stream_ptr(stream))
         if rc != 0:
             raise AdagcError(rc, "adagc_debug_wait_timeout")
+
+    def debug_latch_status(self, device_status: int):
+        rc = lib().adagc_debug_latch_status(self._h, int(device_status))
+        if rc != 0:
+            raise AdagcError(rc, "adagc_debug_latch_status")
 
     def launch_count(self) -> int:
         return int(lib().adagc_launch_count(self._h))

@@ -26,6 +26,7 @@
 #include <algorithm>
 #include <cmath>
 #include <functional>
+#include <mutex>
 #include <new>
 #include <queue>
 #include <utility>
@@ -116,6 +117,13 @@ __device__ __forceinline__ double warp_sum(double x) {
   for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
   return x;  // identical in every lane: each level adds the same two values in both partners
 }
+
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start while its
+// predecessor in the stream is still running, once every block of the predecessor has executed launch_dependents (or
+// exited); griddep_wait returns when the predecessor grid has completed and its writes are visible.  Both are no-ops
+// in a kernel that was launched the ordinary way.
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
@@ -251,13 +259,18 @@ __global__ void __launch_bounds__(kThreads)
 adagc_norm_kernel(const void* __restrict__ grads, const Chunk* __restrict__ chunks,
                   const int32_t* __restrict__ block_begin, double* __restrict__ partials) {
   __shared__ double warp_part[kThreads / 32];
-  const int c_end = block_begin[blockIdx.x + 1];
-  for (int c = block_begin[blockIdx.x]; c < c_end; ++c) {
-    const Chunk ck = chunks[c];
+  const int c_begin = block_begin[blockIdx.x], c_end = block_begin[blockIdx.x + 1];
+  if (c_begin >= c_end) return;
+  Chunk ck = chunks[c_begin];
+  for (int c = c_begin; c < c_end; ++c) {
+    // the next table entry is fetched while this chunk streams: a block of many small chunks would otherwise wait for
+    // a dependent load before every chunk's first gradient load
+    const Chunk ck_next = c + 1 < c_end ? chunks[c + 1] : ck;
     const uint4* vec =
         reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + chunk_start(ck) * (kBF16 ? 2 : 4));
     const double s = block_chunk_sumsq<kBF16, true>(vec, ck.count, warp_part);
     if (threadIdx.x == 0) partials[ck.partial] = s;
+    ck = ck_next;
   }
 }
 
@@ -310,31 +323,76 @@ __device__ __forceinline__ void adagc_decide(int i, double s, const ClipScalars&
   adagc_commit(i, s, adagc_decision(s, ema[i], cs), ema, st);
 }
 
-// Fixed-order sum of one tensor's chunk partials by one warp (identical in every lane on return).
+// Fixed-order sum of one tensor's chunk partials.  The order is defined once and implemented twice, with identical
+// bits: partial j is added, in increasing j, into slot j mod 256; the 32 slots of each group of 32 consecutive slots
+// are combined by the xor-shuffle tree of warp_sum; the 8 group totals are added in order.
+//   tensor_partial_sum        one warp: lane l keeps the 8 slots l, l + 32, ..., l + 224 (result in every lane);
+//   tensor_partial_sum_block  a block of kThreads = 256 threads: thread t keeps slot t (result in thread 0; ends
+//                             with a barrier) -- for tensors with thousands of partials.
 __device__ __forceinline__ double tensor_partial_sum(const double* __restrict__ partials, const TensorEntry te, int lane) {
-  double acc = 0.0;
-  // the additions stay in index order; batching only lets the loads of the next terms start early (the embedding
-  // of a large model has thousands of partials, and one warp walks them)
   const double* __restrict__ tp = partials + te.first_chunk;
-  int j = lane;
-  for (; j + 15 * 32 < te.n_chunks; j += 16 * 32) {
+  const int n = te.n_chunks;
+  if (n <= 32) {  // slots 0..31 only: the other groups would add zeros
+    return warp_sum(lane < n ? __ldcg(tp + lane) : 0.0);
+  }
+  double slot[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) slot[k] = 0.0;
+  for (int base = 0; base < n; base += 256) {
+    double t[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {  // the loads of one round are independent; the additions stay in index order
+      const int j = base + k * 32 + lane;
+      t[k] = j < n ? __ldcg(tp + j) : 0.0;
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) slot[k] += t[k];
+  }
+  double total = warp_sum(slot[0]);
+#pragma unroll
+  for (int k = 1; k < 8; ++k) total += warp_sum(slot[k]);
+  return total;
+}
+
+__device__ __forceinline__ double tensor_partial_sum_block(const double* __restrict__ partials, const TensorEntry te,
+                                                           double* warp_part) {
+  static_assert(kThreads == 256, "the summation order is defined over 256 slots");
+  const double* __restrict__ tp = partials + te.first_chunk;
+  const int tid = threadIdx.x;
+  double acc = 0.0;
+  int j = tid;
+  for (; j + 15 * kThreads < te.n_chunks; j += 16 * kThreads) {  // sixteen loads in flight, additions in index order
     double t[16];
 #pragma unroll
-    for (int u = 0; u < 16; ++u) t[u] = __ldcg(tp + j + u * 32);
+    for (int u = 0; u < 16; ++u) t[u] = __ldcg(tp + j + u * kThreads);
 #pragma unroll
     for (int u = 0; u < 16; ++u) acc += t[u];
   }
-  for (; j < te.n_chunks; j += 32) acc += __ldcg(tp + j);
-  return warp_sum(acc);
+  for (; j < te.n_chunks; j += kThreads) acc += __ldcg(tp + j);
+  const double w = warp_sum(acc);
+  if ((tid & 31) == 0) warp_part[tid >> 5] = w;
+  __syncthreads();
+  double s = 0.0;
+  if (tid == 0) {
+    s = warp_part[0];
+#pragma unroll
+    for (int k = 1; k < kThreads / 32; ++k) s += warp_part[k];
+  }
+  __syncthreads();
+  return s;
 }
 
-// One warp per tensor: fixed-order sum of the tensor's chunk partials; in the AdaGC branch the
-// same warp takes the decision.
+constexpr int kBigTensorChunks = 1024;  // from here on the finalize kernel puts a whole block on the tensor's partials
+
+// One warp per tensor (a whole block for tensors with very many chunks): fixed-order sum of the tensor's chunk
+// partials; in the AdaGC branch the same warp takes the decision.
 __global__ void __launch_bounds__(kFinalizeThreads)
 adagc_tensor_finalize_kernel(const double* __restrict__ partials, const TensorEntry* __restrict__ tensors,
                              ClipScalars cs, int decide, float* __restrict__ ema, StatPtrs st,
                              const int32_t* __restrict__ order, int first, int count, int bump_steps,
                              const DeviceStep* __restrict__ ds = nullptr) {
+  static_assert(kFinalizeThreads == kThreads, "tensor_partial_sum_block runs in this kernel's blocks");
+  __shared__ double warp_part[kFinalizeThreads / 32];
   if (ds) {  // capturable step: scalars and the warm-up switch come from device memory
     cs = ds->cs;
     decide = decide && !ds->in_warmup;
@@ -343,15 +401,119 @@ adagc_tensor_finalize_kernel(const double* __restrict__ partials, const TensorEn
   // (a group of the pipelined host step), else the tensors first..first+count-1
   const int k = (blockIdx.x * kFinalizeThreads + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
-  if (k >= count) return;
-  const int w = order ? order[first + k] : first + k;
-  const double acc = tensor_partial_sum(partials, tensors[w], lane);
-  if (lane == 0) {
-    st.sumsq[w] = acc;
-    if (decide) {
-      adagc_decide(w, acc, cs, ema, st);
-      if (k == 0 && bump_steps) *st.steps_done += 1ull;
+  if (k < count) {
+    const int w = order ? order[first + k] : first + k;
+    const TensorEntry te = tensors[w];
+    if (te.n_chunks < kBigTensorChunks) {
+      const double acc = tensor_partial_sum(partials, te, lane);
+      if (lane == 0) {
+        st.sumsq[w] = acc;
+        if (decide) {
+          adagc_decide(w, acc, cs, ema, st);
+          if (k == 0 && bump_steps) *st.steps_done += 1ull;
+        }
+      }
     }
+  }
+  // the big tensors among this block's eight, one after the other, by the whole block (uniform control flow)
+  for (int k8 = 0; k8 < kFinalizeThreads / 32; ++k8) {
+    const int kk = blockIdx.x * (kFinalizeThreads / 32) + k8;
+    if (kk >= count) break;
+    const int w = order ? order[first + kk] : first + kk;
+    const TensorEntry te = tensors[w];
+    if (te.n_chunks < kBigTensorChunks) continue;
+    const double acc = tensor_partial_sum_block(partials, te, warp_part);
+    if (threadIdx.x == 0) {
+      st.sumsq[w] = acc;
+      if (decide) {
+        adagc_decide(w, acc, cs, ema, st);
+        if (kk == 0 && bump_steps) *st.steps_done += 1ull;
+      }
+    }
+  }
+}
+
+// AdaGC steps: the norm phase with the per-tensor finalize folded into its tail, so that a step is two launches.
+// Here block b owns a contiguous range [range_begin[b], range_begin[b+1]) of the chunks in their original order
+// (tensor after tensor), balanced by cost, so a block holds all chunks of most of its tensors and shares at most its
+// first and its last tensor with neighbouring blocks.  The streaming loop is that of adagc_norm_kernel.  Afterwards,
+// once per block: a tensor whose chunks all lie in this block is complete; for a shared tensor the block adds its
+// number of chunks to the tensor's ticket word, and the block whose addition completes the count knows that every
+// partial of the tensor is written and visible.  Complete tensors are summed in the fixed order and decided by the
+// warps of the block that completed them.  Tickets are integers and nothing waits on them; no floating-point value goes
+// through an atomic, and which block completes a tensor does not change any bit of the result.  A ticket word is left
+// at zero for the next launch.  Tensors without chunks are not handled here (contexts that list such tensors use the
+// separate kernel).
+constexpr int kDoneListMax = 1024;  // complete tensors a block collects before it works them off
+
+template <bool kBF16>
+__global__ void __launch_bounds__(kThreads, 8)  // as many resident blocks as adagc_norm_kernel: the grid is sized for that
+adagc_norm_decide_kernel(const void* __restrict__ grads, const Chunk* __restrict__ chunks,
+                         const int32_t* __restrict__ range_begin, double* partials,
+                         const TensorEntry* __restrict__ tensors, unsigned int* tickets, ClipScalars cs,
+                         float* __restrict__ ema, StatPtrs st) {
+  __shared__ double warp_part[kThreads / 32];
+  __shared__ int done_list[kDoneListMax];
+  __shared__ int n_done;
+  griddep_launch_dependents();  // the update kernel may be staged now; it waits for this grid before it needs h
+  const int lo = range_begin[blockIdx.x], hi = range_begin[blockIdx.x + 1];
+  if (lo >= hi) return;
+  Chunk ck = chunks[lo];  // original order: entry c is chunk c, its partial is partials[c]
+  const int t_first = ck.tensor;
+  int t_last = t_first;
+  for (int c = lo; c < hi; ++c) {
+    const Chunk ck_next = c + 1 < hi ? chunks[c + 1] : ck;  // one entry ahead, as in adagc_norm_kernel
+    const uint4* vec =
+        reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + chunk_start(ck) * (kBF16 ? 2 : 4));
+    const double s = block_chunk_sumsq<kBF16, true>(vec, ck.count, warp_part);
+    if (threadIdx.x == 0) partials[c] = s;
+    t_last = ck.tensor;
+    ck = ck_next;
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (threadIdx.x == 0) __threadfence();  // this block's partials are visible device-wide before any ticket is
+  for (int t0 = t_first; t0 <= t_last; t0 += kDoneListMax) {  // (one round, unless a block holds over a thousand tensors)
+    const int t1 = min(t_last, t0 + kDoneListMax - 1);
+    if (threadIdx.x == 0) n_done = 0;
+    __syncthreads();
+    for (int t = t0 + threadIdx.x; t <= t1; t += kThreads) {
+      const TensorEntry te = tensors[t];
+      const int mine = min(hi, te.first_chunk + te.n_chunks) - max(lo, te.first_chunk);  // its chunks in this block
+      bool complete = mine == te.n_chunks;
+      if (!complete) {
+        const unsigned int before = atomicAdd(tickets + t, static_cast<unsigned int>(mine));
+        complete = before + static_cast<unsigned int>(mine) == static_cast<unsigned int>(te.n_chunks);
+        if (complete) tickets[t] = 0u;  // every block that holds a part of the tensor has added its share
+      }
+      if (complete) done_list[atomicAdd(&n_done, 1)] = t;
+    }
+    __syncthreads();
+    __threadfence();  // (the partials of the other blocks are read below)
+    const int n = n_done;
+    // tensors of a few chunks: one warp each; tensors with very many chunks: the whole block, one after the other
+    for (int k = warp; k < n; k += kThreads / 32) {
+      const int t = done_list[k];
+      const TensorEntry te = tensors[t];
+      if (te.n_chunks >= kBigTensorChunks) continue;
+      const double total = tensor_partial_sum(partials, te, lane);
+      if (lane == 0) {
+        st.sumsq[t] = total;
+        adagc_decide(t, total, cs, ema, st);
+        if (t == 0) *st.steps_done += 1ull;
+      }
+    }
+    for (int k = 0; k < n; ++k) {  // uniform over the block
+      const int t = done_list[k];
+      const TensorEntry te = tensors[t];
+      if (te.n_chunks < kBigTensorChunks) continue;
+      const double total = tensor_partial_sum_block(partials, te, warp_part);
+      if (threadIdx.x == 0) {
+        st.sumsq[t] = total;
+        adagc_decide(t, total, cs, ema, st);
+        if (t == 0) *st.steps_done += 1ull;
+      }
+    }
+    __syncthreads();  // done_list is free again
   }
 }
 
@@ -687,13 +849,14 @@ adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, 
                     void* __restrict__ v_arena, const Chunk* __restrict__ chunks,
                     const int32_t* __restrict__ block_begin, const float* __restrict__ h_arr, AdamScalars a,
                     uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a) {
-  if (d_a) a = *d_a;  // capturable step: coefficients from device memory
   constexpr int kStateBytes = kSB ? 2 : 4;
   const int tid = threadIdx.x;
   int c = block_begin[blockIdx.x];
   const int n_chunks = block_begin[blockIdx.x + 1];  // end of this block's entries
   if (c >= n_chunks) return;
   Chunk ck = chunks[c];
+  griddep_wait();     // the clip factors (and, in a capturable step, the coefficients) come from the preceding kernels
+  if (d_a) a = *d_a;  // capturable step: coefficients from device memory
   float h = h_arr[ck.tensor];
   int row_base = 0;
   while (true) {
@@ -843,7 +1006,6 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
                         const int32_t* __restrict__ block_begin, const int32_t* __restrict__ block_mid,
                         const float* __restrict__ h_arr, AdamScalars a, int* __restrict__ status,
                         uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a) {
-  if (d_a) a = *d_a;  // capturable step: coefficients from device memory
   extern __shared__ __align__(128) unsigned char tile_smem[];
   constexpr int kTile = TmaRing<kSB>::kTile, kStages = TmaRing<kSB>::kStages;
   constexpr int kTilesPerChunk = kChunkElems / kTile;
@@ -888,23 +1050,25 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
 
   bool healthy = true;
   int j_fail = 0;
-  if (n_tiles > 0) {
+  // Everything up to here, the table entries and the first loads below touch nothing that the preceding kernels of the
+  // step write (they write the clip factors, gamma and statistics only), so with a programmatic dependent launch this
+  // much overlaps the tail of the norm phase.
+  if (n_tiles == 0) {
+    griddep_wait();
+    if (d_a) a = *d_a;
+  } else {
     // table entries are kept two chunks ahead in registers, so that neither the elected thread's issue path
     // nor the consumers ever wait for a table load
     Chunk ck = chunks[begin];
-    float h = h_arr[ck.tensor];
     Chunk ck_next = ck, ck_next2 = ck;
-    float h_next = h, h_next2 = h;
-    if (begin + 1 < mid) {
-      ck_next = chunks[begin + 1];
-      h_next = h_arr[ck_next.tensor];
-    }
-    if (begin + 2 < mid) {
-      ck_next2 = chunks[begin + 2];
-      h_next2 = h_arr[ck_next2.tensor];
-    }
+    if (begin + 1 < mid) ck_next = chunks[begin + 1];
+    if (begin + 2 < mid) ck_next2 = chunks[begin + 2];
     if (tid == 0)
       for (int k = 0; k < kAhead && k < n_tiles; ++k) issue_tile(chunk_start(ck), k, k);  // kAhead <= tiles per chunk
+    griddep_wait();
+    if (d_a) a = *d_a;  // capturable step: coefficients from device memory
+    float h = h_arr[ck.tensor];
+    float h_next = h_arr[ck_next.tensor], h_next2 = h_arr[ck_next2.tensor];
     int s = 0;           // stage of tile j
     uint32_t phase = 0;  // parity of the barrier phase tile j completes: flips each time the ring wraps
     for (int j = 0; j < n_tiles; ++j) {
@@ -1027,7 +1191,7 @@ __device__ __forceinline__ uint4 scale_vec(uint4 q, float h) {
 
 template <bool kBF16>
 __global__ void __launch_bounds__(kThreads)
-adagc_scale_kernel(const void* __restrict__ gin, void* __restrict__ gout, const Chunk* __restrict__ chunks,
+adagc_scale_kernel(const void* gin, void* gout /* may alias gin: in-place clipping */, const Chunk* __restrict__ chunks,
                    const int32_t* __restrict__ block_begin, const float* __restrict__ h_arr, int in_place) {
   constexpr int kEPV = kBF16 ? 8 : 4;
   constexpr int kWarps = kThreads / 32;
@@ -1217,14 +1381,16 @@ adagc_fused_small_kernel(float* __restrict__ params, const void* __restrict__ gr
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {  // byte offsets of the workspace sections
-  size_t chunks_wide, chunks_upd, begin_wide, begin_upd, mid_upd, g_chunks_wide, g_chunks_upd, g_begin_wide,
+  size_t chunks_range, begin_range, chunks_wide, chunks_upd, begin_wide, begin_upd, mid_upd, g_chunks_wide, g_chunks_upd, g_begin_wide,
       g_begin_upd, g_mid_upd, g_order, tensors, partials, sumsq, norm, h, clip_count, scalars, dev_step, gamma_prev, slice_partials, flag,
-      total;
+      tickets, total;
 };
 
 Layout make_layout(int64_t n_chunks, int64_t T, bool fused_small = false) {
   Layout L;
   size_t o = 0;
+  L.chunks_range = o; o = align_up(o + sizeof(Chunk) * n_chunks, 256);  // original order, cut into one range per block
+  L.begin_range = o;  o = align_up(o + sizeof(int32_t) * (kMaxGrid + 1), 256);
   L.chunks_wide = o; o = align_up(o + sizeof(Chunk) * n_chunks, 256);  // order of the norm / scale grid
   L.chunks_upd = o;  o = align_up(o + sizeof(Chunk) * n_chunks, 256);  // order of the update grid
   L.begin_wide = o;  o = align_up(o + sizeof(int32_t) * (kMaxGrid + 1), 256);
@@ -1249,6 +1415,7 @@ Layout make_layout(int64_t n_chunks, int64_t T, bool fused_small = false) {
   L.slice_partials = o;  // one-kernel step: one partial per slice of a chunk
   if (fused_small) o = align_up(o + sizeof(double) * n_chunks * 4, 256);
   L.flag = o;       o = align_up(o + T, 256);
+  L.tickets = o;    o = align_up(o + sizeof(uint32_t) * T, 256);  // per tensor: chunks of it summed so far in this launch
   L.total = o;
   return L;
 }
@@ -1261,7 +1428,7 @@ int validate_desc(const adagc_desc* d, int64_t* n_chunks_out, int64_t* arena_ele
   if (!(d->lambda_abs > 0.0) || !std::isfinite(d->lambda_abs)) return ADAGC_E_INVALID_ARG;
   constexpr int kKnownFlags =
       ADAGC_UPDATE_PATH_MASK | ADAGC_EMA_KEEP_INITIAL | ADAGC_CLIP_GLOBAL_ADAPTIVE | ADAGC_ALLOW_EMPTY |
-      ADAGC_FUSED_SMALL;
+      ADAGC_FUSED_SMALL | ADAGC_SEPARATE_FINALIZE;
   if ((d->flags & ADAGC_FUSED_SMALL) && (d->flags & ADAGC_CLIP_GLOBAL_ADAPTIVE)) return ADAGC_E_INVALID_ARG;
   const bool allow_empty = (d->flags & ADAGC_ALLOW_EMPTY) != 0;
   if ((d->flags & ~kKnownFlags) != 0 || (d->flags & ADAGC_UPDATE_PATH_MASK) == 3) return ADAGC_E_INVALID_ARG;
@@ -1333,6 +1500,22 @@ void balance_chunks(const std::vector<Chunk>& chunks, int grid, std::vector<Chun
   }
 }
 
+// The chunks in their original order cut into `grid` consecutive ranges of about equal cost (elements plus the fixed
+// cost per chunk): block b of adagc_norm_decide_kernel owns [out[b], out[b+1]).
+std::vector<int32_t> contiguous_ranges(const std::vector<Chunk>& chunks, int grid) {
+  int64_t total = 0;
+  for (const Chunk& c : chunks) total += c.count + kChunkFixedCostWide;
+  std::vector<int32_t> out(grid + 1, static_cast<int32_t>(chunks.size()));
+  out[0] = 0;
+  int64_t acc = 0;
+  int b = 1;
+  for (size_t i = 0; i < chunks.size() && b < grid; ++i) {
+    acc += chunks[i].count + kChunkFixedCostWide;
+    while (b < grid && acc * grid >= total * b) out[b++] = static_cast<int32_t>(i + 1);  // cut after chunk i
+  }
+  return out;
+}
+
 }  // namespace
 
 struct adagc_ctx {
@@ -1345,6 +1528,7 @@ struct adagc_ctx {
   int device = 0;
   int grid_wide = 1, grid_update = 1;  // norm and scale kernels: SMs x resident blocks; update: SMs x 2 or x 1
   bool update_bulk = false;            // update phase through the bulk-async (TMA) kernel
+  bool fold_finalize = true;           // AdaGC steps decide in the norm kernel's tail (needs every tensor to have a chunk)
   bool offsets_mult8 = true;           // every tensor offset is a multiple of 8 elements (bf16 arenas stay 16-byte aligned)
   bool keep_initial = false;           // ADAGC_EMA_KEEP_INITIAL
   bool global_adaptive = false;        // ADAGC_CLIP_GLOBAL_ADAPTIVE
@@ -1352,6 +1536,7 @@ struct adagc_ctx {
   bool fused_small = false;            // ADAGC_FUSED_SMALL: adagc_step runs as one cooperative kernel
   int grid_fused = 1;                  // its grid: every block resident at once
   unsigned long long barriers_done = 0;  // grid barriers executed by earlier fused launches of this context
+  bool fused_poisoned = false;           // adagc_get_stats has seen ADAGC_E_TIMEOUT: the barrier counter is out of step
   char* ws = nullptr;
   Layout L{};
   uint64_t launches = 0;
@@ -1425,16 +1610,36 @@ struct TableView {
   int grid;
 };
 
+// Launch with the programmatic-stream-serialization attribute: the kernel may be scheduled while the preceding kernel
+// of the stream drains; it calls griddep_wait before it reads what that kernel wrote.
+template <typename... Params, typename... Args>
+void launch_dependent(void (*kernel)(Params...), int grid, int block, size_t smem, cudaStream_t s, bool programmatic,
+                      Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = programmatic ? 1 : 0;
+  (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);  // errors surface in finish_launches
+}
+
 template <bool kBF16, int kOpt, bool kSB>
 void launch_update_t(adagc_ctx* ctx, const TableView& tv, float* p, const void* g, void* m, void* v,
                      const AdamScalars& a, cudaStream_t s, uint16_t* lowp, const AdamScalars* d_a) {
   const StatPtrs st = ctx->stats();
+  const bool programmatic = d_a == nullptr;  // (the capturable step keeps ordinary launches)
   if (ctx->update_bulk)
-    adagc_update_tma_kernel<kBF16, kOpt, kSB>
-        <<<tv.grid, kTmaThreads, tma_smem_bytes<kSB>(kBF16, kOpt, lowp != nullptr), s>>>(
-            p, g, m, v, tv.chunks, tv.begin, tv.mid, st.h, a, st.status, lowp, d_a);
+    launch_dependent(adagc_update_tma_kernel<kBF16, kOpt, kSB>, tv.grid, kTmaThreads,
+                     tma_smem_bytes<kSB>(kBF16, kOpt, lowp != nullptr), s, programmatic, p, g, m, v, tv.chunks, tv.begin,
+                     tv.mid, st.h, a, st.status, lowp, d_a);
   else
-    adagc_update_kernel<kBF16, kOpt, kSB><<<tv.grid, kThreads, 0, s>>>(p, g, m, v, tv.chunks, tv.begin, st.h, a, lowp, d_a);
+    launch_dependent(adagc_update_kernel<kBF16, kOpt, kSB>, tv.grid, kThreads, 0, s, programmatic, p, g, m, v, tv.chunks,
+                     tv.begin, st.h, a, lowp, d_a);
   ctx->launches++;
 }
 
@@ -1515,12 +1720,31 @@ int enqueue_clip_phases(adagc_ctx* ctx, const void* d_grads, float* d_ema, int64
                         double beta, int64_t warmup, cudaStream_t s) {
   if (ctx->timing) cudaEventRecord(ctx->ev[0], s);
   const TableView wide = {ctx->d_chunks_wide(), ctx->d_begin_wide(), nullptr, ctx->grid_wide};
-  launch_norm(ctx, wide, d_grads, s);
-  if (ctx->timing) cudaEventRecord(ctx->ev[1], s);
   const ClipScalars cs = make_clip_scalars(ctx, step, lambda_rel, beta);
   const bool in_warmup = step <= warmup;
-  const int blocks = (ctx->T * 32 + kFinalizeThreads - 1) / kFinalizeThreads;
   const bool per_tensor = !in_warmup && !ctx->global_adaptive;
+  if (per_tensor && ctx->fold_finalize) {
+    // AdaGC step: a tensor's decision needs that tensor's partials only, so the block that completes a tensor takes it
+    // at once: phases 1 and 2 are one launch
+    unsigned int* tickets = reinterpret_cast<unsigned int*>(ctx->ws + ctx->L.tickets);
+    const Chunk* in_order = reinterpret_cast<const Chunk*>(ctx->ws + ctx->L.chunks_range);
+    const int32_t* ranges = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.begin_range);
+    if (ctx->bf16)
+      adagc_norm_decide_kernel<true><<<wide.grid, kThreads, 0, s>>>(d_grads, in_order, ranges, ctx->d_partials(),
+                                                                  ctx->d_tensors(), tickets, cs, d_ema, ctx->stats());
+    else
+      adagc_norm_decide_kernel<false><<<wide.grid, kThreads, 0, s>>>(d_grads, in_order, ranges, ctx->d_partials(),
+                                                                   ctx->d_tensors(), tickets, cs, d_ema, ctx->stats());
+    ctx->launches++;
+    if (ctx->timing) {
+      cudaEventRecord(ctx->ev[1], s);
+      cudaEventRecord(ctx->ev[2], s);  // no separate finalize phase
+    }
+    return ADAGC_OK;
+  }
+  launch_norm(ctx, wide, d_grads, s);
+  if (ctx->timing) cudaEventRecord(ctx->ev[1], s);
+  const int blocks = (ctx->T * 32 + kFinalizeThreads - 1) / kFinalizeThreads;
   adagc_tensor_finalize_kernel<<<blocks, kFinalizeThreads, 0, s>>>(ctx->d_partials(), ctx->d_tensors(), cs,
                                                                   per_tensor ? 1 : 0, d_ema, ctx->stats(), nullptr, 0,
                                                                   ctx->T, 1);
@@ -1647,6 +1871,13 @@ int launch_fused_small(adagc_ctx* ctx, void* d_params, const void* d_grads, void
   return finish_launches(ctx, s);
 }
 
+// What the host remembers of a status word it has read: after a timed-out grid barrier the device-side arrival counter
+// and the host's count of barriers differ for good, so every later one-kernel step would wait its full limit and skip
+// its update; the context refuses them instead.
+void latch_device_status(adagc_ctx* ctx, int32_t device_status) {
+  if (ctx->fused_small && (device_status & ADAGC_E_TIMEOUT)) ctx->fused_poisoned = true;
+}
+
 void release_ctx(adagc_ctx* ctx) {
   for (int k = 0; k < 4; ++k)
     if (ctx->ev[k]) cudaEventDestroy(ctx->ev[k]);
@@ -1720,6 +1951,7 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
   }
   ctx->ws = static_cast<char*>(d_workspace);
   ctx->L = L;
+  ctx->fold_finalize = !any_empty && !(desc->flags & ADAGC_SEPARATE_FINALIZE);
 
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   cudaDeviceProp prop;
@@ -1761,16 +1993,19 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
         1, std::min<int64_t>(n_chunks * 4, static_cast<int64_t>(prop.multiProcessorCount) * std::min(occ_f, 2))));
   }
   std::vector<Chunk> table_wide, table_upd;
-  std::vector<int32_t> begin_wide, begin_upd, mid_upd;
+  std::vector<int32_t> begin_wide, begin_upd, mid_upd, begin_range;
   if (ok) {
     balance_chunks(chunks, ctx->grid_wide, &table_wide, &begin_wide);
     balance_chunks(chunks, ctx->grid_update, &table_upd, &begin_upd, &mid_upd);
+    begin_range = contiguous_ranges(chunks, ctx->grid_wide);
   }
   auto upload = [&](size_t off, const void* src, size_t bytes) {
     if (bytes == 0) return;  // a rank of a sharded model may hold no chunk at all
     ok = ok && cudaMemcpyAsync(ctx->ws + off, src, bytes, cudaMemcpyHostToDevice, s) == cudaSuccess;
   };
   ok = ok && cudaMemsetAsync(ctx->ws, 0, L.total, s) == cudaSuccess;
+  upload(L.chunks_range, chunks.data(), sizeof(Chunk) * chunks.size());
+  upload(L.begin_range, begin_range.data(), sizeof(int32_t) * begin_range.size());
   upload(L.chunks_wide, table_wide.data(), sizeof(Chunk) * table_wide.size());
   upload(L.chunks_upd, table_upd.data(), sizeof(Chunk) * table_upd.size());
   upload(L.begin_wide, begin_wide.data(), sizeof(int32_t) * begin_wide.size());
@@ -1861,6 +2096,7 @@ int adagc_step(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, v
   rc = check_adamw_args(d_params, d_grads, d_m, d_v, lr, beta1, beta2, eps, wd);
   if (rc != ADAGC_OK) return rc;
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+  if (ctx->fused_small && ctx->fused_poisoned) return ADAGC_E_POISONED;
   if (ctx->fused_small)
     return launch_fused_small(ctx, d_params, d_grads, d_m, d_v, d_ema, make_clip_scalars(ctx, step, lambda_rel, beta),
                               step <= warmup, make_adam_scalars(step, lr, beta1, beta2, eps, wd), s);
@@ -2079,8 +2315,17 @@ int adagc_get_stats(adagc_ctx* ctx, float* h_norm, float* h_clipfactor, uint8_t*
     ok = ok && cudaMemcpyAsync(h_steps_done, st.steps_done, 8, cudaMemcpyDeviceToHost, s) == cudaSuccess;
   if (h_device_status)
     ok = ok && cudaMemcpyAsync(h_device_status, st.status, 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  int32_t status_now = 0;  // read in any case: a timed-out grid barrier of the one-kernel step must be latched
+  ok = ok && cudaMemcpyAsync(&status_now, st.status, 4, cudaMemcpyDeviceToHost, s) == cudaSuccess;
   ok = ok && cudaStreamSynchronize(s) == cudaSuccess;
+  if (ok) latch_device_status(ctx, status_now);
   return ok ? ADAGC_OK : ADAGC_E_CUDA;
+}
+
+int adagc_debug_latch_status(adagc_ctx* ctx, int32_t device_status) {
+  if (!ctx) return ADAGC_E_INVALID_ARG;
+  latch_device_status(ctx, device_status);
+  return ADAGC_OK;
 }
 
 int adagc_get_sumsq(adagc_ctx* ctx, double* h_sumsq, void* cuda_stream) {
@@ -2185,6 +2430,7 @@ const char* adagc_strerror(int status) {
     case ADAGC_E_CUDA: return "CUDA runtime error";
     case ADAGC_E_NOMEM: return "host allocation failed";
     case ADAGC_E_TOO_LARGE: return "size exceeds the fixed scratch of the no-allocation entry point";
+    case ADAGC_E_POISONED: return "a grid barrier of the one-kernel step timed out earlier: create the context anew";
     default: return "unknown status";
   }
 }
@@ -2224,22 +2470,37 @@ adagc_sumsq_static_kernel(const void* __restrict__ grads, int64_t numel, int n_c
   }
 }
 
-// One warp sums the partials in the same fixed order as adagc_tensor_finalize_kernel.
+// One warp sums the partials in the same fixed order as the step's per-tensor sums (tensor_partial_sum).
 __global__ void __launch_bounds__(32)
 adagc_sumsq_static_reduce_kernel(const double* __restrict__ partials, int n_chunks, double* __restrict__ out) {
   const int lane = threadIdx.x;
-  double acc = 0.0;
-  for (int j = lane; j < n_chunks; j += 32) acc += partials[j];
-  acc = warp_sum(acc);
+  TensorEntry te;
+  te.first_chunk = 0;
+  te.n_chunks = n_chunks;
+  const double acc = tensor_partial_sum(partials, te, lane);
   if (lane == 0) *out = acc;
 }
 
-struct StaticScratch {
-  bool ready[kMaxDevices] = {};
+struct StaticScratch {  // host side; one entry per device ordinal, filled once by the first call on that device
+  std::once_flag once[kMaxDevices];
   double* ptr[kMaxDevices] = {};
   int sms[kMaxDevices] = {};
 };
-StaticScratch g_static;  // host side; filled on the first call on each device
+StaticScratch g_static;
+
+// With `dev` current: look up the array's device address.  In host code the array's name is only a handle; the address
+// the kernels need comes from the runtime, once per device.  Leaves ptr[dev] null on failure.
+void static_scratch_setup(int dev) {
+  double* p = nullptr;
+  int sms = 0;
+  if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_partials) != cudaSuccess || !p ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+    (void)cudaGetLastError();
+    return;
+  }
+  g_static.sms[dev] = sms;
+  g_static.ptr[dev] = p;
+}
 
 }  // namespace
 
@@ -2254,20 +2515,11 @@ extern "C" int adagc_sumsq_noalloc(const void* d_grads, int32_t grad_dtype, int6
     (void)cudaGetLastError();
     return ADAGC_E_CUDA;
   }
-  if (!g_static.ready[dev]) {
-    // In host code the array's name is only a handle; the address the kernels need comes from the
-    // runtime, once per device, with that device current.
-    double* p = nullptr;
-    int sms = 0;
-    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_partials) != cudaSuccess || !p ||
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
-      (void)cudaGetLastError();
-      return ADAGC_E_CUDA;
-    }
-    g_static.ptr[dev] = p;
-    g_static.sms[dev] = sms;
-    g_static.ready[dev] = true;
-  }
+  // several host threads may make the first call on a device at the same time: one of them does the lookup, the others
+  // wait for it (std::call_once also orders its writes before their reads)
+  std::call_once(g_static.once[dev], static_scratch_setup, dev);
+  if (!g_static.ptr[dev]) return ADAGC_E_CUDA;
+  (void)cudaGetLastError();  // an error left behind by earlier calls of the process is not this call's
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   const int n_chunks = static_cast<int>((numel + kChunkElems - 1) / kChunkElems);
   const int grid = std::max(1, std::min(n_chunks, g_static.sms[dev] * 8));

@@ -293,12 +293,30 @@ def test_random_layouts(seed):
     rng.shuffle(sizes)
     dtype = ["f32", "bf16"][int(rng.randint(2))]
     flags = [0, binding.UPDATE_PATH_REGISTERS, binding.UPDATE_PATH_BULK, binding.FUSED_SMALL][int(rng.randint(4))]
+    if flags != binding.FUSED_SMALL:      # where the decisions are taken: norm kernel's tail (default) or a kernel of their own
+        flags |= [0, binding.SEPARATE_FINALIZE][int(rng.randint(2))]
     over = dict(warmup=int(rng.randint(0, 4)), lambda_abs=float(np.exp(rng.uniform(np.log(1e-3), np.log(1e2)))),
                 lambda_rel=float(rng.uniform(1.0, 1.3)), beta=float(rng.uniform(0.5, 0.999)))
     wl = _ragged_workload(sizes, dtype)
     how = ["", "", "eager", "graph"][int(rng.randint(4))] if flags != binding.FUSED_SMALL else ""
     rep = H.run_full(wl, 7, flags=flags, hyper_over=over, capturable=how)
     _report(f"random layout {seed}: T={len(sizes)} {dtype} flags={flags} {over} capturable={how!r}", rep)
+
+
+@pytest.mark.parametrize("where", [0, binding.SEPARATE_FINALIZE], ids=["norm_tail", "own_kernel"])
+def test_decisions_in_the_norm_tail_and_in_their_own_kernel(where):
+    """Both places where an AdaGC step can take its per-tensor decisions, forced, on layouts that exercise what differs
+    between them: tensors inside one block's range of chunks, tensors shared by many blocks (tickets), a tensor with
+    more than 1024 chunks (summed by a whole block), thousands of one-chunk tensors."""
+    sizes = [1, 9, 300, 16384, 16385, 5 * 16384 + 3, 1100 * 16384 + 77, 40 * 16384, 2049, 70000]
+    for dtype in ("f32", "bf16"):
+        _report(f"decisions flag {where} {dtype}", H.run_full(_ragged_workload(sizes, dtype), 6, flags=where))
+    wl = workloads.build("many_small", n_tensors=5000, lo=16, hi=40000)
+    _report(f"decisions flag {where}, 5000 tensors", H.run_full(wl, 8, flags=where, hyper_over=dict(lambda_abs=1e4)))
+    a, _ = _run_gpu(*_mini(), 8, flags=where)
+    b, _ = _run_gpu(*_mini(), 8, flags=binding.SEPARATE_FINALIZE - where)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)                                   # bit-identical wherever the decisions are taken
 
 
 def test_single_tensor_and_warmup_zero():
@@ -319,9 +337,9 @@ def _mini():
     return wl, offs, nums
 
 
-def _run_gpu(wl, offs, nums, steps, start_state=None, first_step=1):
+def _run_gpu(wl, offs, nums, steps, start_state=None, first_step=1, flags=0):
     hp = H.hyper_of(wl)
-    opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"])
+    opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], flags=flags)
     if start_state is None:
         theta = workloads.init_params(wl, "cuda")
         m, v = torch.zeros_like(theta), torch.zeros_like(theta)
@@ -446,6 +464,36 @@ def test_bounded_wait_gives_up_and_context_stays_usable():
     opt.close()
 
 
+def test_one_kernel_step_refuses_work_after_a_timed_out_barrier_was_seen():
+    """After a grid barrier of the one-kernel step has timed out, the device-side arrival counter and the host's
+    barrier count differ for good.  The host latches the ADAGC_E_TIMEOUT bit when it reads the status word and refuses
+    later steps of that context.  The bit is fed to the latch by hand here: no barrier is made to time out on the GPU."""
+    wl, offs, nums = _mini()
+    hp = H.hyper_of(wl)
+    args = (hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"], hp["beta"], hp["warmup"])
+    theta = workloads.init_params(wl, "cuda")
+    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device="cuda")
+    g = workloads.grads_for_step(wl, 1, "cuda")
+    fused = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], flags=binding.FUSED_SMALL)
+    plain = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"])
+    fused.step(theta, g, m, v, ema, 1, *args)
+    fused.debug_latch_status(binding.ADAGC_W_NONFINITE)            # other bits do not poison the context
+    fused.step(theta, g, m, v, ema, 2, *args)
+    assert fused.get_stats()["steps_done"] == 2
+    before = theta.clone()
+    fused.debug_latch_status(binding.ADAGC_E_TIMEOUT)
+    with pytest.raises(binding.AdagcError) as e:
+        fused.step(theta, g, m, v, ema, 3, *args)
+    assert e.value.status == -9 and "anew" in binding.strerror(-9)
+    torch.cuda.synchronize()
+    assert torch.equal(theta, before) and fused.get_stats()["steps_done"] == 2     # nothing was enqueued
+    plain.debug_latch_status(binding.ADAGC_E_TIMEOUT)              # the three-launch step has no such state
+    plain.step(theta, g, m, v, ema, 1, *args)
+    fused.close()
+    plain.close()
+
+
 def test_phase_timing_and_launch_count():
     wl, offs, nums = _mini()
     hp = H.hyper_of(wl)
@@ -458,8 +506,8 @@ def test_phase_timing_and_launch_count():
     args = (hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"], hp["beta"])
     opt.step(theta, g, m, v, ema, 1, *args, 1)                    # warm-up step: 4 kernels
     assert opt.launch_count() == 4
-    opt.step(theta, g, m, v, ema, 2, *args, 1)                    # AdaGC step: 3 kernels
-    assert opt.launch_count() == 7
+    opt.step(theta, g, m, v, ema, 2, *args, 1)                    # AdaGC step: 2 kernels (the decisions are taken in the
+    assert opt.launch_count() == 6                                # norm kernel's tail)
     ms = opt.get_phase_times()
     assert len(ms) == 3 and all(x >= 0 for x in ms)
     opt.close()

@@ -36,10 +36,17 @@ def test_two_calls_in_a_row_match_the_workspace_path(dtype):
     small = (torch.randn(16384 + 3, device="cuda", generator=gen) * 3.0).to(dtype)          # 2 chunks: stale partials
     want_big, want_small = _regular_sumsq(big), _regular_sumsq(small)                        # beyond them must not leak
     out = torch.zeros(2, dtype=torch.float64, device="cuda")
-    before = torch.cuda.memory_allocated()
-    binding.sumsq_noalloc(big, out[0:1])
-    binding.sumsq_noalloc(small, out[1:2])
-    assert torch.cuda.memory_allocated() == before
+    side = torch.cuda.Stream()                                    # an explicit, non-default stream
+    binding.sumsq_noalloc(small, out[1:2])                        # first call on this device: looks up the array's address
+    torch.cuda.synchronize()
+    # free device memory as the driver counts it (torch's own counters would not see a cudaMalloc inside the library)
+    free_before, _ = torch.cuda.mem_get_info()
+    torch_before = torch.cuda.memory_allocated()
+    side.wait_stream(torch.cuda.current_stream())
+    binding.sumsq_noalloc(big, out[0:1], stream=side)
+    binding.sumsq_noalloc(small, out[1:2], stream=side)
+    side.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before and torch.cuda.memory_allocated() == torch_before
     got = out.cpu().numpy()
     assert got[0] == pytest.approx(want_big, rel=RTOL)
     assert got[1] == pytest.approx(want_small, rel=RTOL)

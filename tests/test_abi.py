@@ -57,14 +57,18 @@ def test_descriptor_validation_codes():
     assert chunks([50, 100], [96, 0])[0] == -3                           # overlap, unsorted
     assert chunks([100], [0], dt=2)[0] == -5
     assert chunks([100], [0], param_dtype=binding.ADAGC_BF16)[0] == -5
+    assert chunks([100], [0], state_dtype=binding.ADAGC_BF16)[0] == 1                       # moments stored as bfloat16
+    assert chunks([100], [0], state_dtype=2)[0] == -5
+    assert chunks([100, 50], [0, 100], state_dtype=binding.ADAGC_BF16)[0] == -2            # then offsets in multiples of 8
+    assert chunks([100], [0], flags=binding.SEPARATE_FINALIZE)[0] == 1
     assert chunks([100], [0], flags=binding.UPDATE_PATH_BULK)[0] == 1
     d, keep = binding.make_desc([8], [0], binding.ADAGC_F32)
     d.n_tensors = (1 << 24) + 1                                          # more tensors than the descriptor may list
     assert int(lib.adagc_num_chunks(C.byref(d))) == -1
-    assert chunks([100], [0], flags=3)[0] == -1 and chunks([100], [0], flags=64)[0] == -1   # unknown flags
+    assert chunks([100], [0], flags=3)[0] == -1 and chunks([100], [0], flags=128)[0] == -1   # unknown flags
     assert chunks([100], [0], flags=binding.EMA_KEEP_INITIAL | binding.CLIP_GLOBAL_ADAPTIVE | 2)[0] == 1
     assert lib.adagc_workspace_bytes(None) == 0
-    for code in range(-7, 1):
+    for code in range(-9, 1):
         assert binding.strerror(code) not in ("", "unknown status")
     assert binding.strerror(-99) == "unknown status"
 

@@ -90,7 +90,7 @@ def test_empty_tensors_need_the_flag():
     assert chunks([100, 0, 50], [0, 999, 104], flags=binding.ALLOW_EMPTY) == 2     # offset of an empty tensor is ignored
     assert chunks([0, 0], [0, 0], flags=binding.ALLOW_EMPTY) == 0                  # a rank that holds nothing
     assert chunks([100, -1], [0, 104], flags=binding.ALLOW_EMPTY) == -1
-    assert chunks([100], [0], flags=64) == -1                                      # unknown flag
+    assert chunks([100], [0], flags=128) == -1                                      # unknown flag
 
 
 def _free_port() -> int:

@@ -56,6 +56,9 @@ typedef enum {
 #define ADAGC_W_NONFINITE 1 /* some tensor's sum of squares was Inf or NaN in some step */
 #define ADAGC_E_TIMEOUT 2   /* a bounded device-side wait gave up (a bulk copy never completed): the
                                update of that step is incomplete */
+#define ADAGC_E_BOUNDS 4    /* only in a library built with -DADAGC_BOUNDS_CHECK: a kernel found a chunk-table entry
+                               that points outside the arenas (or is otherwise malformed); the blocks that saw it
+                               returned without touching the arenas */
 
 /* adagc_desc.flags: which kernel runs the AdamW update phase.  AUTO (0) currently picks the bulk-async
  * kernel (cp.async.bulk + mbarrier pipeline through shared memory), which measured 1-2 % faster than the
@@ -381,6 +384,27 @@ int adagc_sumsq_noalloc(const void* d_grads, int32_t grad_dtype, int64_t numel, 
  * returns normally, leaving the context usable.  Enqueues only.
  */
 int adagc_debug_wait_timeout(adagc_ctx* ctx, double limit_ms, void* cuda_stream);
+
+/*
+ * Debugging aids for the chunk tables (host-only, no CUDA call).  adagc_create cuts every tensor into chunks of 16384
+ * elements (the last one shorter; one partial sum per chunk) and hands the chunks to thread blocks through three
+ * tables; adagc_debug_chunk_tables rebuilds one of them for `grid` blocks:
+ *   which = 0  original order, block b owns the consecutive entries [block_begin[b], block_begin[b+1]) (norm kernel
+ *              with the decisions in its tail);
+ *   which = 1  balanced over the blocks of the norm / scale grid, a block's entries contiguous;
+ *   which = 2  balanced over the blocks of the update grid; a block's full chunks come first:
+ *              [block_begin[b], block_mid[b]) are full, [block_mid[b], block_begin[b+1]) partial.
+ * Output arrays (host memory): adagc_num_chunks(desc) entries each of h_start (element offset into the arenas),
+ * h_count, h_tensor, h_partial; grid + 1 entries of h_block_begin; grid entries of h_block_mid (which = 2 only).
+ * adagc_debug_chunk_entry_ok is the predicate a library built with -DADAGC_BOUNDS_CHECK applies, on the device, to
+ * every table entry a block is about to walk (such a build sets ADAGC_E_BOUNDS in the status word and skips the block
+ * instead of accessing memory); adagc_debug_bounds_checked_build tells whether this library is such a build.
+ */
+int adagc_debug_chunk_tables(const adagc_desc* desc, int32_t which, int32_t grid, int64_t* h_start, int32_t* h_count,
+                             int32_t* h_tensor, int32_t* h_partial, int32_t* h_block_begin, int32_t* h_block_mid);
+int adagc_debug_chunk_entry_ok(int64_t start, int32_t count, int32_t tensor, int32_t partial, int64_t arena_elems,
+                               int32_t n_chunks, int32_t n_tensors);
+int adagc_debug_bounds_checked_build(void);
 
 /* Test aid: feeds `device_status` to the same host-side latch that adagc_get_stats applies to the status word it reads
  * (a context created with ADAGC_FUSED_SMALL refuses further steps once ADAGC_E_TIMEOUT has been seen).  Host-only. */

@@ -15,10 +15,12 @@ import torch
 ADAGC_F32, ADAGC_BF16 = 0, 1
 ADAGC_W_NONFINITE = 1
 ADAGC_E_TIMEOUT = 2
+ADAGC_E_BOUNDS = 4
 UPDATE_PATH_AUTO, UPDATE_PATH_REGISTERS, UPDATE_PATH_BULK = 0, 1, 2
 EMA_KEEP_INITIAL, CLIP_GLOBAL_ADAPTIVE, ALLOW_EMPTY, FUSED_SMALL, SEPARATE_FINALIZE = 4, 8, 16, 32, 64
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libadagc.so")
+# ADAGC_LIBRARY selects another build of the same library (e.g. the bounds-checked one, libadagc_checked.so)
+_LIB_PATH = os.environ.get("ADAGC_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libadagc.so")
 _lib = None
 
 
@@ -103,6 +105,12 @@ def lib() -> C.CDLL:
     L.adagc_sumsq_noalloc.argtypes = [vp, C.c_int32, i64, vp, vp]
     L.adagc_debug_wait_timeout.restype = C.c_int
     L.adagc_debug_wait_timeout.argtypes = [vp, dbl, vp]
+    L.adagc_debug_chunk_tables.restype = C.c_int
+    L.adagc_debug_chunk_tables.argtypes = [C.POINTER(adagc_desc), C.c_int32, C.c_int32, vp, vp, vp, vp, vp, vp]
+    L.adagc_debug_chunk_entry_ok.restype = C.c_int
+    L.adagc_debug_chunk_entry_ok.argtypes = [i64, C.c_int32, C.c_int32, C.c_int32, i64, C.c_int32, C.c_int32]
+    L.adagc_debug_bounds_checked_build.restype = C.c_int
+    L.adagc_debug_bounds_checked_build.argtypes = []
     L.adagc_debug_latch_status.restype = C.c_int
     L.adagc_debug_latch_status.argtypes = [vp, C.c_int32]
     L.adagc_strerror.restype = C.c_char_p
@@ -146,6 +154,22 @@ def make_desc(numels: Sequence[int], offsets: Sequence[int], grad_dtype: int, la
     d.lambda_abs = float(lambda_abs)
     d.flags = int(flags)
     return d, arr
+
+
+def chunk_tables(numels: Sequence[int], offsets: Sequence[int], grad_dtype: int, which: int, grid: int,
+                 state_dtype: int = ADAGC_F32, flags: int = 0):
+    """adagc_debug_chunk_tables: dict(start, count, tensor, partial, block_begin[, block_mid]) of numpy arrays; host-only."""
+    d, keep = make_desc(numels, offsets, grad_dtype, state_dtype=state_dtype, flags=flags)
+    n = int(lib().adagc_num_chunks(C.byref(d)))
+    if n < 0:
+        raise AdagcError(n, "invalid descriptor")
+    out = dict(start=np.zeros(n, np.int64), count=np.zeros(n, np.int32), tensor=np.zeros(n, np.int32),
+               partial=np.zeros(n, np.int32), block_begin=np.zeros(grid + 1, np.int32), block_mid=np.zeros(grid, np.int32))
+    rc = lib().adagc_debug_chunk_tables(C.byref(d), int(which), int(grid), *(out[k].ctypes.data for k in
+                                        ("start", "count", "tensor", "partial", "block_begin", "block_mid")))
+    if rc != 0:
+        raise AdagcError(rc, "adagc_debug_chunk_tables")
+    return out
 
 
 def shard_plan(numels: Sequence[int], offsets: Sequence[int], grad_dtype: int, rank: int, world: int):

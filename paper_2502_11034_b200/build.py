@@ -20,15 +20,23 @@ def nvcc_path() -> str:
     return "nvcc"
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile the CUDA library if it is missing or older than its sources; returns its path."""
+LIB_CHECKED = os.path.join(_HERE, "libadagc_checked.so")
+
+
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Compile the CUDA library if it is missing or older than its sources; returns its path.
+    checked: the debugging build (-DADAGC_BOUNDS_CHECK, libadagc_checked.so) whose kernels verify every chunk-table entry
+    before they use it; select it at run time with ADAGC_LIBRARY=<path>."""
+    lib = LIB_CHECKED if checked else LIB
     newest = max(os.path.getmtime(SRC), os.path.getmtime(HEADER))
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= newest:
-        return LIB
-    cmd = [nvcc_path()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB, SRC]
+    if not force and os.path.exists(lib) and os.path.getmtime(lib) >= newest:
+        return lib
+    cmd = ([nvcc_path()] + NVCC_FLAGS + (["-DADAGC_BOUNDS_CHECK"] if checked else []) +
+           (["-Xptxas", "-v"] if verbose else []) + ["-o", lib, SRC])
     subprocess.run(cmd, check=True)
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose=True))
+    import sys
+    print(build(force=True, verbose=True, checked="--checked" in sys.argv))

@@ -58,6 +58,21 @@ struct Chunk {
 static_assert(sizeof(Chunk) == 16, "chunk entries are 16 bytes");
 __host__ __device__ __forceinline__ int64_t chunk_start(const Chunk& c) { return static_cast<int64_t>(c.start4) * 4; }
 
+// What every kernel that walks a chunk table is told about the context, so that a build with -DADAGC_BOUNDS_CHECK can
+// verify the entries it is about to use before the first access (a debugging build: the tables are written once by
+// adagc_create from a validated descriptor, so a violation means a corrupted workspace or a defect of the table builder).
+struct Guard {
+  long long arena_elems;  // every chunk must end at or before this element
+  int n_chunks;           // table length; also the number of partial sums
+  int n_tensors;
+  int* status;            // device status word: ADAGC_E_BOUNDS is set here
+};
+
+__host__ __device__ __forceinline__ bool chunk_entry_ok(const Chunk& c, long long arena_elems, int n_chunks, int n_tensors) {
+  return c.count > 0 && c.count <= kChunkElems && c.tensor >= 0 && c.tensor < n_tensors && c.partial >= 0 &&
+         c.partial < n_chunks && chunk_start(c) + c.count <= arena_elems;
+}
+
 // Chunks are handed to thread blocks by a table built once on the host: block b owns the entries
 // [block_begin[b], block_begin[b+1]) of its kernel's table.  The assignment balances elements (plus a
 // fixed cost per chunk) over the blocks; with equal chunks it is plain round-robin.
@@ -188,6 +203,24 @@ __device__ __forceinline__ double sq_acc(double acc, float x) {
   return fma(d, d, acc);
 }
 
+#ifdef ADAGC_BOUNDS_CHECK
+// Checked build: the whole block verifies the table entries [first, last) it is about to walk.  On a violation the
+// status bit is set and false is returned to every thread, and the block returns without touching the arenas.
+__device__ __forceinline__ bool block_entries_ok(const Chunk* __restrict__ chunks, int first, int last, const Guard& g) {
+  int ok = first >= 0 && first <= last && last <= g.n_chunks;
+  if (ok)
+    for (int c = first + threadIdx.x; c < last; c += blockDim.x)
+      ok = ok && chunk_entry_ok(chunks[c], g.arena_elems, g.n_chunks, g.n_tensors);
+  ok = __syncthreads_and(ok);
+  if (!ok && threadIdx.x == 0) atomicOr(g.status, ADAGC_E_BOUNDS);
+  return ok != 0;
+}
+#define ADAGC_CHECK_ENTRIES(chunks, first, last, guard) \
+  if (!block_entries_ok(chunks, first, last, guard)) return
+#else
+#define ADAGC_CHECK_ENTRIES(chunks, first, last, guard) (void)(guard)
+#endif
+
 // ------------------------------------------------------------------------------------------------
 // phase 1: per-chunk sums of squares (Eq. 3: ||g_t,i||^2 = sum_j g_ij^2)
 // ------------------------------------------------------------------------------------------------
@@ -257,9 +290,10 @@ __device__ __forceinline__ double block_chunk_sumsq(const uint4* __restrict__ ve
 template <bool kBF16>
 __global__ void __launch_bounds__(kThreads)
 adagc_norm_kernel(const void* __restrict__ grads, const Chunk* __restrict__ chunks,
-                  const int32_t* __restrict__ block_begin, double* __restrict__ partials) {
+                  const int32_t* __restrict__ block_begin, double* __restrict__ partials, Guard guard) {
   __shared__ double warp_part[kThreads / 32];
   const int c_begin = block_begin[blockIdx.x], c_end = block_begin[blockIdx.x + 1];
+  ADAGC_CHECK_ENTRIES(chunks, c_begin, c_end, guard);
   if (c_begin >= c_end) return;
   Chunk ck = chunks[c_begin];
   for (int c = c_begin; c < c_end; ++c) {
@@ -451,12 +485,13 @@ __global__ void __launch_bounds__(kThreads, 8)  // as many resident blocks as ad
 adagc_norm_decide_kernel(const void* __restrict__ grads, const Chunk* __restrict__ chunks,
                          const int32_t* __restrict__ range_begin, double* partials,
                          const TensorEntry* __restrict__ tensors, unsigned int* tickets, ClipScalars cs,
-                         float* __restrict__ ema, StatPtrs st) {
+                         float* __restrict__ ema, StatPtrs st, Guard guard) {
   __shared__ double warp_part[kThreads / 32];
   __shared__ int done_list[kDoneListMax];
   __shared__ int n_done;
   griddep_launch_dependents();  // the update kernel may be staged now; it waits for this grid before it needs h
   const int lo = range_begin[blockIdx.x], hi = range_begin[blockIdx.x + 1];
+  ADAGC_CHECK_ENTRIES(chunks, lo, hi, guard);
   if (lo >= hi) return;
   Chunk ck = chunks[lo];  // original order: entry c is chunk c, its partial is partials[c]
   const int t_first = ck.tensor;
@@ -848,11 +883,12 @@ __global__ void __launch_bounds__(kThreads)
 adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, void* __restrict__ m_arena,
                     void* __restrict__ v_arena, const Chunk* __restrict__ chunks,
                     const int32_t* __restrict__ block_begin, const float* __restrict__ h_arr, AdamScalars a,
-                    uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a) {
+                    uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a, Guard guard) {
   constexpr int kStateBytes = kSB ? 2 : 4;
   const int tid = threadIdx.x;
   int c = block_begin[blockIdx.x];
   const int n_chunks = block_begin[blockIdx.x + 1];  // end of this block's entries
+  ADAGC_CHECK_ENTRIES(chunks, c, n_chunks, guard);
   if (c >= n_chunks) return;
   Chunk ck = chunks[c];
   griddep_wait();     // the clip factors (and, in a capturable step, the coefficients) come from the preceding kernels
@@ -1005,7 +1041,7 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
                         void* __restrict__ v_arena, const Chunk* __restrict__ chunks,
                         const int32_t* __restrict__ block_begin, const int32_t* __restrict__ block_mid,
                         const float* __restrict__ h_arr, AdamScalars a, int* __restrict__ status,
-                        uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a) {
+                        uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a, Guard guard) {
   extern __shared__ __align__(128) unsigned char tile_smem[];
   constexpr int kTile = TmaRing<kSB>::kTile, kStages = TmaRing<kSB>::kStages;
   constexpr int kTilesPerChunk = kChunkElems / kTile;
@@ -1025,6 +1061,18 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
   __shared__ __align__(8) uint64_t full_bar[kStages];
   const int tid = threadIdx.x;
   const int begin = block_begin[blockIdx.x], mid = block_mid[blockIdx.x], end = block_begin[blockIdx.x + 1];
+  ADAGC_CHECK_ENTRIES(chunks, begin, end, guard);
+#ifdef ADAGC_BOUNDS_CHECK
+  {  // the entries before `mid` are moved as whole tiles: they must be full chunks
+    int full = mid >= begin && mid <= end;
+    for (int c = begin + threadIdx.x; full && c < mid; c += blockDim.x) full = chunks[c].count == kChunkElems;
+    full = __syncthreads_and(full);
+    if (!full) {
+      if (threadIdx.x == 0) atomicOr(guard.status, ADAGC_E_BOUNDS);
+      return;
+    }
+  }
+#endif
   const int n_tiles = (mid - begin) * kTilesPerChunk;
 
   __shared__ int abort_flag;
@@ -1192,7 +1240,7 @@ __device__ __forceinline__ uint4 scale_vec(uint4 q, float h) {
 template <bool kBF16>
 __global__ void __launch_bounds__(kThreads)
 adagc_scale_kernel(const void* gin, void* gout /* may alias gin: in-place clipping */, const Chunk* __restrict__ chunks,
-                   const int32_t* __restrict__ block_begin, const float* __restrict__ h_arr, int in_place) {
+                   const int32_t* __restrict__ block_begin, const float* __restrict__ h_arr, int in_place, Guard guard) {
   constexpr int kEPV = kBF16 ? 8 : 4;
   constexpr int kWarps = kThreads / 32;
 #ifndef ADAGC_SCALE_BATCH
@@ -1203,6 +1251,7 @@ adagc_scale_kernel(const void* gin, void* gout /* may alias gin: in-place clippi
   int row_base = 0;  // rows (32 vectors) dealt so far: successive chunks continue one round-robin over the warps
   const uint64_t done = l2_policy_evict_first();
   const int c_end = block_begin[blockIdx.x + 1];
+  ADAGC_CHECK_ENTRIES(chunks, block_begin[blockIdx.x], c_end, guard);
   for (int c = block_begin[blockIdx.x]; c < c_end; ++c) {
     const Chunk ck = chunks[c];
     const float h = h_arr[ck.tensor];
@@ -1283,10 +1332,11 @@ adagc_fused_small_kernel(float* __restrict__ params, const void* __restrict__ gr
                          void* __restrict__ v_arena, float* ema, const Chunk* __restrict__ chunks, int n_chunks,
                          const TensorEntry* __restrict__ tensors, double* slice_partials, ClipScalars cs, int in_warmup,
                          AdamScalars a, StatPtrs st, unsigned long long* barrier_counter,
-                         unsigned long long barrier_index, float* gamma_prev) {
+                         unsigned long long barrier_index, float* gamma_prev, Guard guard) {
   __shared__ double warp_part[kThreads / 32];
   __shared__ double total_s;
   __shared__ float h_shared;
+  ADAGC_CHECK_ENTRIES(chunks, 0, n_chunks, guard);  // (every block checks the whole table, so all of them agree)
   const int n_units = n_chunks * kSlicesPerChunk;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   auto slices_of = [](const TensorEntry te) {
@@ -1500,6 +1550,28 @@ void balance_chunks(const std::vector<Chunk>& chunks, int grid, std::vector<Chun
   }
 }
 
+// Every tensor of a validated descriptor cut into chunks of kChunkElems elements (the last one shorter), in tensor
+// order; chunk k's partial sum has index k.
+void cut_into_chunks(const adagc_desc* desc, int64_t n_chunks, std::vector<Chunk>* chunks, std::vector<TensorEntry>* tensors) {
+  chunks->reserve(n_chunks);
+  tensors->reserve(desc->n_tensors);
+  for (int32_t i = 0; i < desc->n_tensors; ++i) {
+    const adagc_tensor& t = desc->tensors[i];
+    TensorEntry te;
+    te.first_chunk = static_cast<int32_t>(chunks->size());
+    for (int64_t o = 0; o < t.numel; o += kChunkElems) {
+      Chunk c;
+      c.start4 = static_cast<uint32_t>((t.offset + o) / 4);
+      c.count = static_cast<int32_t>(std::min<int64_t>(kChunkElems, t.numel - o));
+      c.tensor = i;
+      c.partial = static_cast<int32_t>(chunks->size());
+      chunks->push_back(c);
+    }
+    te.n_chunks = static_cast<int32_t>(chunks->size()) - te.first_chunk;
+    tensors->push_back(te);
+  }
+}
+
 // The chunks in their original order cut into `grid` consecutive ranges of about equal cost (elements plus the fixed
 // cost per chunk): block b of adagc_norm_decide_kernel owns [out[b], out[b+1]).
 std::vector<int32_t> contiguous_ranges(const std::vector<Chunk>& chunks, int grid) {
@@ -1560,6 +1632,14 @@ struct adagc_ctx {
   const int32_t* d_mid_upd() const { return reinterpret_cast<const int32_t*>(ws + L.mid_upd); }
   const TensorEntry* d_tensors() const { return reinterpret_cast<const TensorEntry*>(ws + L.tensors); }
   double* d_partials() const { return reinterpret_cast<double*>(ws + L.partials); }
+  Guard guard() const {
+    Guard g;
+    g.arena_elems = arena_elems;
+    g.n_chunks = n_chunks;
+    g.n_tensors = T;
+    g.status = reinterpret_cast<int*>(ws + L.scalars + 8);
+    return g;
+  }
   StatPtrs stats() const {
     StatPtrs s;
     s.sumsq = reinterpret_cast<double*>(ws + L.sumsq);
@@ -1636,10 +1716,10 @@ void launch_update_t(adagc_ctx* ctx, const TableView& tv, float* p, const void* 
   if (ctx->update_bulk)
     launch_dependent(adagc_update_tma_kernel<kBF16, kOpt, kSB>, tv.grid, kTmaThreads,
                      tma_smem_bytes<kSB>(kBF16, kOpt, lowp != nullptr), s, programmatic, p, g, m, v, tv.chunks, tv.begin,
-                     tv.mid, st.h, a, st.status, lowp, d_a);
+                     tv.mid, st.h, a, st.status, lowp, d_a, ctx->guard());
   else
     launch_dependent(adagc_update_kernel<kBF16, kOpt, kSB>, tv.grid, kThreads, 0, s, programmatic, p, g, m, v, tv.chunks,
-                     tv.begin, st.h, a, lowp, d_a);
+                     tv.begin, st.h, a, lowp, d_a, ctx->guard());
   ctx->launches++;
 }
 
@@ -1668,9 +1748,9 @@ void launch_update(adagc_ctx* ctx, void* p, const void* g, void* m, void* v, con
 
 void launch_norm(adagc_ctx* ctx, const TableView& tv, const void* d_grads, cudaStream_t s) {
   if (ctx->bf16)
-    adagc_norm_kernel<true><<<tv.grid, kThreads, 0, s>>>(d_grads, tv.chunks, tv.begin, ctx->d_partials());
+    adagc_norm_kernel<true><<<tv.grid, kThreads, 0, s>>>(d_grads, tv.chunks, tv.begin, ctx->d_partials(), ctx->guard());
   else
-    adagc_norm_kernel<false><<<tv.grid, kThreads, 0, s>>>(d_grads, tv.chunks, tv.begin, ctx->d_partials());
+    adagc_norm_kernel<false><<<tv.grid, kThreads, 0, s>>>(d_grads, tv.chunks, tv.begin, ctx->d_partials(), ctx->guard());
   ctx->launches++;
 }
 
@@ -1731,10 +1811,12 @@ int enqueue_clip_phases(adagc_ctx* ctx, const void* d_grads, float* d_ema, int64
     const int32_t* ranges = reinterpret_cast<const int32_t*>(ctx->ws + ctx->L.begin_range);
     if (ctx->bf16)
       adagc_norm_decide_kernel<true><<<wide.grid, kThreads, 0, s>>>(d_grads, in_order, ranges, ctx->d_partials(),
-                                                                  ctx->d_tensors(), tickets, cs, d_ema, ctx->stats());
+                                                                  ctx->d_tensors(), tickets, cs, d_ema, ctx->stats(),
+                                                                  ctx->guard());
     else
       adagc_norm_decide_kernel<false><<<wide.grid, kThreads, 0, s>>>(d_grads, in_order, ranges, ctx->d_partials(),
-                                                                   ctx->d_tensors(), tickets, cs, d_ema, ctx->stats());
+                                                                   ctx->d_tensors(), tickets, cs, d_ema, ctx->stats(),
+                                                                   ctx->guard());
     ctx->launches++;
     if (ctx->timing) {
       cudaEventRecord(ctx->ev[1], s);
@@ -1789,10 +1871,10 @@ void launch_scale(adagc_ctx* ctx, const void* d_grads_in, void* d_grads_out, cud
   const int in_place = d_grads_in == d_grads_out ? 1 : 0;
   if (ctx->bf16)
     adagc_scale_kernel<true><<<ctx->grid_wide, kThreads, 0, s>>>(d_grads_in, d_grads_out, ctx->d_chunks_wide(),
-                                                                ctx->d_begin_wide(), ctx->stats().h, in_place);
+                                                                ctx->d_begin_wide(), ctx->stats().h, in_place, ctx->guard());
   else
     adagc_scale_kernel<false><<<ctx->grid_wide, kThreads, 0, s>>>(d_grads_in, d_grads_out, ctx->d_chunks_wide(),
-                                                                 ctx->d_begin_wide(), ctx->stats().h, in_place);
+                                                                 ctx->d_begin_wide(), ctx->stats().h, in_place, ctx->guard());
   ctx->launches++;
 }
 
@@ -1859,8 +1941,9 @@ int launch_fused_small(adagc_ctx* ctx, void* d_params, const void* d_grads, void
   unsigned long long* counter = reinterpret_cast<unsigned long long*>(ctx->ws + ctx->L.scalars + 16);
   unsigned long long index = ctx->barriers_done;
   float* gamma_prev = reinterpret_cast<float*>(ctx->ws + ctx->L.gamma_prev);
+  Guard guard = ctx->guard();
   void* args[] = {&p,        &d_grads, &m,    &v, &d_ema, &chunks,  &n_chunks, &tensors,
-                  &partials, &cs,      &warm, &a, &st,    &counter, &index, &gamma_prev};
+                  &partials, &cs,      &warm, &a, &st,    &counter, &index, &gamma_prev, &guard};
   const void* fn = fused_small_kernel_of(ctx);
   if (cudaLaunchCooperativeKernel(fn, dim3(ctx->grid_fused), dim3(kThreads), args, 0, s) != cudaSuccess) {
     (void)cudaGetLastError();
@@ -1918,23 +2001,7 @@ int adagc_create(const adagc_desc* desc, void* d_workspace, size_t workspace_byt
 
   std::vector<Chunk> chunks;
   std::vector<TensorEntry> tensors;
-  chunks.reserve(n_chunks);
-  tensors.reserve(desc->n_tensors);
-  for (int32_t i = 0; i < desc->n_tensors; ++i) {
-    const adagc_tensor& t = desc->tensors[i];
-    TensorEntry te;
-    te.first_chunk = static_cast<int32_t>(chunks.size());
-    for (int64_t o = 0; o < t.numel; o += kChunkElems) {
-      Chunk c;
-      c.start4 = static_cast<uint32_t>((t.offset + o) / 4);
-      c.count = static_cast<int32_t>(std::min<int64_t>(kChunkElems, t.numel - o));
-      c.tensor = i;
-      c.partial = static_cast<int32_t>(chunks.size());
-      chunks.push_back(c);
-    }
-    te.n_chunks = static_cast<int32_t>(chunks.size()) - te.first_chunk;
-    tensors.push_back(te);
-  }
+  cut_into_chunks(desc, n_chunks, &chunks, &tensors);
 
   adagc_ctx* ctx = new (std::nothrow) adagc_ctx();
   if (!ctx) return ADAGC_E_NOMEM;
@@ -2320,6 +2387,56 @@ int adagc_get_stats(adagc_ctx* ctx, float* h_norm, float* h_clipfactor, uint8_t*
   ok = ok && cudaStreamSynchronize(s) == cudaSuccess;
   if (ok) latch_device_status(ctx, status_now);
   return ok ? ADAGC_OK : ADAGC_E_CUDA;
+}
+
+int adagc_debug_chunk_tables(const adagc_desc* desc, int32_t which, int32_t grid, int64_t* h_start, int32_t* h_count,
+                             int32_t* h_tensor, int32_t* h_partial, int32_t* h_block_begin, int32_t* h_block_mid) {
+  int64_t n_chunks = 0;
+  const int rc = validate_desc(desc, &n_chunks, nullptr);
+  if (rc != ADAGC_OK) return rc;
+  if (which < 0 || which > 2 || grid < 1 || grid > kMaxGrid || !h_start || !h_count || !h_tensor || !h_partial ||
+      !h_block_begin || (which == 2 && !h_block_mid))
+    return ADAGC_E_INVALID_ARG;
+  std::vector<Chunk> chunks, table;
+  std::vector<TensorEntry> tensors;
+  cut_into_chunks(desc, n_chunks, &chunks, &tensors);
+  std::vector<int32_t> begin, mid;
+  if (which == 0) {
+    table = chunks;
+    begin = contiguous_ranges(chunks, grid);
+  } else if (which == 1) {
+    balance_chunks(chunks, grid, &table, &begin);
+  } else {
+    balance_chunks(chunks, grid, &table, &begin, &mid);
+  }
+  for (size_t k = 0; k < table.size(); ++k) {
+    h_start[k] = chunk_start(table[k]);
+    h_count[k] = table[k].count;
+    h_tensor[k] = table[k].tensor;
+    h_partial[k] = table[k].partial;
+  }
+  std::copy(begin.begin(), begin.end(), h_block_begin);
+  if (which == 2) std::copy(mid.begin(), mid.begin() + grid, h_block_mid);
+  return ADAGC_OK;
+}
+
+int adagc_debug_chunk_entry_ok(int64_t start, int32_t count, int32_t tensor, int32_t partial, int64_t arena_elems,
+                               int32_t n_chunks, int32_t n_tensors) {
+  if (start < 0 || (start & 3) || (start >> 2) > int64_t(0xffffffff)) return 0;
+  Chunk c;
+  c.start4 = static_cast<uint32_t>(start >> 2);
+  c.count = count;
+  c.tensor = tensor;
+  c.partial = partial;
+  return chunk_entry_ok(c, arena_elems, n_chunks, n_tensors) ? 1 : 0;
+}
+
+int adagc_debug_bounds_checked_build(void) {
+#ifdef ADAGC_BOUNDS_CHECK
+  return 1;
+#else
+  return 0;
+#endif
 }
 
 int adagc_debug_latch_status(adagc_ctx* ctx, int32_t device_status) {

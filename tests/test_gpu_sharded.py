@@ -122,3 +122,93 @@ def test_bench_sharded_mode_prints_one_json_line():
     assert line["scaling"] == "strong" and line["n_gpus"] == 1 and line["value"] > 0
     assert line["gpu_launches"] == 3 * 4          # per step: norm, per-tensor sum, decision, update
     assert 0.3 < line["roofline"]["frac"] < 1.2
+
+
+# ------------------------------------------------------------------ two real ranks through the product's own code
+def _free_port() -> int:
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def _two_rank_worker(rank, world, port, out):
+    """One rank: sharded.ShardedAdaGC(rank, world).step() -- the library's shard sums, the real
+    torch.distributed all-reduce, the pre-summed step -- on its slice, against the UNSHARDED oracle."""
+    import os
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    sys.path.insert(0, root)
+    sys.path.insert(0, os.path.join(root, "tests"))
+    import torch.distributed as dist
+    from oracle import c_oracle
+    import parity_harness as HH
+    try:
+        os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+        # both ranks share the one GPU of this machine; gloo carries the CUDA exchange buffer through the host
+        # (NCCL refuses two ranks on one device), and no kernel of one rank waits on the other's
+        dist.init_process_group("gloo", rank=rank, world_size=world)
+        torch.cuda.set_device(0)
+        wl = workloads.build("llama2_7b", n_layer=2, d=256, ffn=688, vocab=1000)
+        hp = HH.hyper_of(wl, lambda_abs=1e4)
+        offs, nums = [t.offset for t in wl.tensors], [t.numel for t in wl.tensors]
+        sh = sharded.ShardedAdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], rank, world, device="cuda:0")
+        b, e = sh.elem_begin, sh.elem_end
+        theta0 = workloads.init_params(wl, "cpu")
+        theta = theta0[b:e].cuda()
+        m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+        ema = torch.full((wl.n_tensors,), float("nan"), dtype=torch.float32, device="cuda:0")
+        ref = c_oracle.ArenaOracle(offs, nums, theta0.numpy(), lr=hp["lr"], beta1=hp["beta1"], beta2=hp["beta2"],
+                                   eps=hp["eps"], wd=hp["wd"], lambda_rel=hp["lambda_rel"], beta=hp["beta"],
+                                   lambda_abs=hp["lambda_abs"], warmup=hp["warmup"])
+        rep = HH.ParityReport()
+        for t in range(1, 13):
+            g_full = workloads.grads_for_step(wl, t, "cpu")              # every rank draws the same full gradient ...
+            g = g_full[b:e].cuda()                                      # ... and keeps only its range
+            sh.step(theta, g, m, v, ema, t, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"],
+                    hp["beta"], hp["warmup"])
+            r = ref.step(HH.to_numpy_grads(g_full))
+            HH.check_decisions(sh.opt.get_stats(), sh.sumsq.cpu().numpy(), ema.cpu().numpy(), r, rep, t)
+        th, mm, vv = theta.cpu().numpy(), m.cpu().numpy(), v.cpu().numpy()
+        for name, got, want in (("theta", th, ref.theta[b:e]), ("m", mm, ref.m[b:e]), ("v", vv, ref.v[b:e])):
+            for t_, o, n in zip(wl.tensors, offs, nums):
+                lo, hi = max(o, b), min(o + n, e)
+                if hi > lo:
+                    HH.check_state(name, got[lo - b:hi - b], want[lo - b:hi - b], rep, t_.name)
+        st = sh.opt.get_stats()
+        assert st["steps_done"] == 12 and st["status"] == 0 and np.array_equal(st["clip_count"], ref.clip_count)
+        gathered = [torch.zeros_like(ema) for _ in range(world)]
+        dist.all_gather(gathered, ema)                                   # gamma is replicated: identical bits on all ranks
+        same = all(torch.equal(gathered[0], x) for x in gathered)
+        dist.barrier()
+        out.put((rank, "ok", bool(same), int(rep.clipped), e - b))
+        sh.close()
+        dist.destroy_process_group()
+    except BaseException as ex:  # noqa: BLE001 -- the parent reports it
+        import traceback
+        out.put((rank, "error: " + "".join(traceback.format_exception(ex))[-1500:], False, 0, 0))
+
+
+def test_two_processes_run_the_sharded_step_through_a_real_all_reduce():
+    """sharded.ShardedAdaGC.step() end to end with world = 2: two processes on this machine's one GPU, each with its
+    own context over its flat shard, exchanging the per-tensor partial sums of squares through torch.distributed."""
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_two_rank_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=600) for _ in procs)
+    for p in procs:
+        p.join(timeout=120)
+    total = 0
+    for rank, status, same, clipped, n_local in res:
+        assert status == "ok", f"rank {rank}: {status}"
+        assert same, "gamma differs between the ranks"
+        assert clipped > 0
+        total += n_local
+    wl = workloads.build("llama2_7b", n_layer=2, d=256, ffn=688, vocab=1000)
+    assert total == wl.arena_elems
+    for p in procs:
+        assert p.exitcode == 0

@@ -170,6 +170,40 @@ def test_hand_worked_example(impl):
         np.testing.assert_allclose(a, b, rtol=3e-7, atol=0)   # fp32 storage vs float64 library run
 
 
+def test_second_hand_worked_example_with_printed_parameters():
+    """The decimal variant of the example (g_A = (0.6, 0.8) at t = 2), whose parameters are printed to 10 digits after
+    every step: the float64-state oracle reproduces the table to rounding and every printed theta to 1e-9; the fixture
+    itself is re-derived in 50-digit decimal arithmetic by tests/golden/make_worked_example.py, without the oracle.
+    (The first fixture uses (0.75, 1) instead, so that every input is exact in binary and the fp32 paths -- the C oracle
+    and the GPU -- can be required to reproduce its table bit for bit.)"""
+    with open(os.path.join(GOLDEN, "worked_example_decimal.json")) as f:
+        gold = json.load(f)
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("make_worked_example", os.path.join(GOLDEN, "make_worked_example.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    derived = mod.derive_theta(mod.GRADS_DECIMAL, [gold["theta0"]["A"], gold["theta0"]["B"]])
+    hp = npo.Hyper(**gold["hyper"])
+    ref = npo.AdaGCAdamW([np.array(gold["theta0"]["A"]), np.array(gold["theta0"]["B"])], hp, np.float64)
+    for s, d in zip(gold["steps"], derived):
+        r = ref.step([np.array(s["gA"], np.float64), np.array(s["gB"], np.float64)])
+        np.testing.assert_allclose(r.norm, s["norm"], rtol=1e-15, atol=0)
+        np.testing.assert_allclose(r.h, s["h"], rtol=1e-15)
+        np.testing.assert_array_equal(r.flag.astype(int), s["flag"])
+        np.testing.assert_allclose(r.gamma, s["gamma"], rtol=1e-15)
+        for got, printed, exact in zip(ref.theta, (s["theta_A"], s["theta_B"]), d):
+            np.testing.assert_allclose(got, printed, rtol=0, atol=1e-9)        # the printed 10 digits
+            np.testing.assert_allclose(got, exact, rtol=1e-13, atol=0)         # the 50-digit derivation
+    # the C oracle (fp32 storage) on the same inputs rounded to fp32
+    theta = [np.array(gold["theta0"]["A"], np.float32), np.array(gold["theta0"]["B"], np.float32)]
+    grads = [[f32_exact(s["gA"]), f32_exact(s["gB"])] for s in gold["steps"]]
+    hist, th, _, _, _ = run(CImpl, theta, grads, hp)
+    for s, r in zip(gold["steps"], hist):
+        np.testing.assert_array_equal(np.asarray(r["flag"], int), s["flag"])
+        np.testing.assert_allclose(r["h"], s["h"], rtol=1e-7)
+    np.testing.assert_allclose(np.concatenate(th), gold["steps"][-1]["theta_A"] + gold["steps"][-1]["theta_B"], rtol=5e-7)
+
+
 def _torch_adamw(params, clipped_grads_per_step, hp, dtype=torch.float64):
     ps = [torch.tensor(p, dtype=dtype, requires_grad=True) for p in params]
     opt = torch.optim.AdamW(ps, lr=hp.lr, betas=(hp.beta1, hp.beta2), eps=hp.eps,

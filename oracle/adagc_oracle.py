@@ -118,6 +118,61 @@ def bf16_rounding_margin(x, scale) -> np.ndarray:
     return out
 
 
+# ----------------------------------------------------------------------------------------------------------------
+# Stochastic rounding of stored bfloat16 moments.  The random numbers come from the counter-based generator
+# Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", SC 2011), written here from
+# its definition: a counter of four 32-bit words and a key of two go through ten rounds; a round replaces the counter
+# (c0, c1, c2, c3) by (hi(M1 c2) ^ c1 ^ k0, lo(M1 c2), hi(M0 c0) ^ c3 ^ k1, lo(M0 c0)), where hi / lo are the halves
+# of the 64-bit product, and after each round but the last the key is bumped by the Weyl constants (W0, W1).
+# ----------------------------------------------------------------------------------------------------------------
+PHILOX_M0, PHILOX_M1 = 0xD2511F53, 0xCD9E8D57
+PHILOX_W0, PHILOX_W1 = 0x9E3779B9, 0xBB67AE85
+
+
+def philox4x32_10(counter, key) -> np.ndarray:
+    """counter: (..., 4) uint32 words, key: (2,) or (..., 2) uint32 words -> (..., 4) uint32 output words."""
+    c = np.asarray(counter, dtype=np.uint64) & 0xFFFFFFFF
+    k = np.broadcast_to(np.asarray(key, dtype=np.uint64) & 0xFFFFFFFF, c.shape[:-1] + (2,))
+    c0, c1, c2, c3 = (c[..., i].copy() for i in range(4))
+    k0, k1 = k[..., 0].copy(), k[..., 1].copy()
+    mask = np.uint64(0xFFFFFFFF)
+    for r in range(10):
+        p0, p1 = np.uint64(PHILOX_M0) * c0, np.uint64(PHILOX_M1) * c2          # 32 x 32 -> 64 bits, exact in uint64
+        c0, c1, c2, c3 = (p1 >> np.uint64(32)) ^ c1 ^ k0, p1 & mask, (p0 >> np.uint64(32)) ^ c3 ^ k1, p0 & mask
+        if r < 9:
+            k0, k1 = (k0 + np.uint64(PHILOX_W0)) & mask, (k1 + np.uint64(PHILOX_W1)) & mask
+    return np.stack([c0, c1, c2, c3], axis=-1).astype(np.uint32)
+
+
+def rounding_randoms(index: np.ndarray, step: int, seed: int):
+    """The two 16-bit random numbers (for m and for v) of the elements at arena positions `index` at step `step`:
+    the group of four elements 4q..4q+3 shares one generator call with counter (lo(q), hi(q), lo(step), hi(step)) and
+    key (lo(seed), hi(seed)); element 4q + l takes output word l, its low half for m and its high half for v."""
+    index = np.asarray(index, dtype=np.uint64)
+    q = index >> np.uint64(2)
+    ctr = np.stack([q & np.uint64(0xFFFFFFFF), q >> np.uint64(32),
+                    np.full(q.shape, step & 0xFFFFFFFF, np.uint64), np.full(q.shape, (step >> 32) & 0xFFFFFFFF, np.uint64)], axis=-1)
+    out = philox4x32_10(ctr, np.array([seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF], np.uint64))
+    word = np.take_along_axis(out, (index & np.uint64(3)).astype(np.int64)[..., None], axis=-1)[..., 0]
+    return (word & np.uint32(0xFFFF)).astype(np.uint32), (word >> np.uint32(16)).astype(np.uint32)
+
+
+def stochastic_round_to_bf16(x32: np.ndarray, r16: np.ndarray) -> np.ndarray:
+    """Stochastic rounding of float32 values to bfloat16 with the 16-bit random integers r16: the value moves to the
+    neighbour of larger magnitude with probability (distance to the smaller neighbour) / spacing, which is what adding
+    r16 to the low half of the float32 bit pattern and dropping that half does (a carry runs into the exponent as it
+    should); bfloat16 values are left as they are, infinities and NaN are rounded to nearest.  Returns the bfloat16
+    values held in float32."""
+    x32 = np.ascontiguousarray(x32, dtype=np.float32)
+    u = x32.view(np.uint32).astype(np.uint64)
+    out = (((u + np.asarray(r16, np.uint64)) >> np.uint64(16)) << np.uint64(16)).astype(np.uint32).view(np.float32)
+    special = ~np.isfinite(x32)
+    if special.any():
+        out = out.copy()
+        out[special] = round_to_bf16(x32[special].astype(np.float64)).astype(np.float32)
+    return out
+
+
 def clip_decisions(s: Sequence[float], gamma_prev: np.ndarray, step: int, hp: Hyper,
                    state_dtype=np.float32, keep_initial: bool = False,
                    global_adaptive: bool = False, ema_cap: Optional[float] = None) -> ClipResult:

@@ -256,6 +256,49 @@ void adagc_ref_sgdm(float* theta, const void* g, int g_is_bf16, float* m, int64_
   }
 }
 
+/*
+ * Stochastic rounding of stored bfloat16 moments.  Random numbers: the counter-based generator Philox4x32-10 (Salmon,
+ * Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3", SC 2011), from its definition: ten rounds, each
+ * replacing the counter (c0, c1, c2, c3) by (hi(M1 c2) ^ c1 ^ k0, lo(M1 c2), hi(M0 c0) ^ c3 ^ k1, lo(M0 c0)); the key
+ * is bumped by (W0, W1) between rounds.
+ */
+void adagc_ref_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n1 = (uint32_t)p1, n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1,
+                   n3 = (uint32_t)p0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    if (r < 9) { k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* The 16-bit random numbers of the element at arena position `index` at step `step`: elements 4q..4q+3 share the call
+ * with counter (lo q, hi q, lo step, hi step) and key (lo seed, hi seed); element 4q + l takes output word l, the low
+ * half for m (which = 0), the high half for v (which = 1). */
+static uint32_t rounding_random(int64_t index, int64_t step, uint64_t seed, int which) {
+  const uint64_t q = (uint64_t)index >> 2;
+  const uint32_t ctr[4] = {(uint32_t)q, (uint32_t)(q >> 32), (uint32_t)step, (uint32_t)((uint64_t)step >> 32)};
+  const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  uint32_t out[4];
+  adagc_ref_philox4x32_10(ctr, key, out);
+  const uint32_t w = out[index & 3];
+  return which ? (w >> 16) : (w & 0xFFFFu);
+}
+
+/* Stochastic rounding of a float to bfloat16 with the 16-bit random integer r: the neighbour of larger magnitude is taken
+ * with probability (distance to the smaller neighbour) / spacing -- add r to the low half of the bit pattern, drop that
+ * half.  Infinities and NaN are rounded to nearest. */
+static uint16_t float_to_bf16_stochastic(float x, uint32_t r) {
+  if (isnan(x) || isinf(x)) return double_to_bf16((double)x);
+  uint32_t u;
+  memcpy(&u, &x, 4);
+  return (uint16_t)((u + r) >> 16);
+}
+
+uint16_t adagc_ref_float_to_bf16_stochastic(float x, uint32_t r) { return float_to_bf16_stochastic(x, r); }
+
 /* Distance from x to the nearest point where rounding to bfloat16 flips (the midpoint between two
  * neighbouring bfloat16 values): an implementation whose x differs by less than this rounds alike. */
 static double bf16_flip_distance(double x) {
@@ -292,10 +335,13 @@ static inline void count_near_tie(uint8_t* near_tie, int64_t j, double x, double
  * float64 value of m' is an exact decimal tie (x.5 spacings) for about one element in twenty, so which neighbour is
  * stored depends on how the coefficients themselves are rounded: the decision has to name its precision.
  * theta is always computed in float64 from the float64 moments.
+ * stochastic = 1 (with fp32_decision): the single-precision m' and v' are rounded stochastically instead, with the random
+ * numbers of the element's arena position (index[j] if index is given, else index0 + j), `step` and `seed`.
  */
 void adagc_ref_adamw_bf16state(float* theta, const void* g, int g_is_bf16, uint16_t* m, uint16_t* v, int64_t n,
                                double h, int64_t step, double lr, double beta1, double beta2, double eps,
-                               double wd, uint8_t* near_tie, double tie_tol, int fp32_decision) {
+                               double wd, uint8_t* near_tie, double tie_tol, int fp32_decision, int stochastic,
+                               uint64_t seed, int64_t index0, const int64_t* index) {
   const double bc1 = 1.0 - pow(beta1, (double)step);
   const double bc2 = 1.0 - pow(beta2, (double)step);
   const uint16_t* gb = (const uint16_t*)g;
@@ -319,8 +365,14 @@ void adagc_ref_adamw_bf16state(float* theta, const void* g, int g_is_bf16, uint1
       const float ghf = hf * (float)gj; /* g is exactly a float */
       const float m1f = fmaf(b1f, (float)bf16_to_double(m[j]), omb1f * ghf);
       const float v1f = fmaf(b2f, (float)bf16_to_double(v[j]), omb2f * (ghf * ghf));
-      m[j] = double_to_bf16((double)m1f);
-      v[j] = double_to_bf16((double)v1f);
+      if (stochastic) { /* (only with fp32_decision: the rounding acts on the bits of the single-precision value) */
+        const int64_t at = index ? index[j] : index0 + j; /* position of the element in the arenas */
+        m[j] = float_to_bf16_stochastic(m1f, rounding_random(at, step, seed, 0));
+        v[j] = float_to_bf16_stochastic(v1f, rounding_random(at, step, seed, 1));
+      } else {
+        m[j] = double_to_bf16((double)m1f);
+        v[j] = double_to_bf16((double)v1f);
+      }
     } else {
       m[j] = double_to_bf16(m1);
       v[j] = double_to_bf16(v1);
@@ -331,10 +383,12 @@ void adagc_ref_adamw_bf16state(float* theta, const void* g, int g_is_bf16, uint1
 /* Lion (see adagc_ref_lion) with the momentum stored as bfloat16, rounded to nearest even on store.
  * near_tie counts both kinds of discrete decision: sign(c) and the rounding of m.  fp32_decision = 1: the stored
  * value is the rounding of  fl(beta2 * m + fl((1 - beta2) * fl(h * g)))  evaluated in single precision (see above);
- * sign(c) stays a float64 decision. */
+ * sign(c) stays a float64 decision.  stochastic = 1: that value is rounded stochastically (random numbers of arena
+ * position index0 + j, `step`, `seed`; the half of the word that AdamW uses for m). */
 void adagc_ref_lion_bf16state(float* theta, const void* g, int g_is_bf16, uint16_t* m, int64_t n, double h,
                               double lr, double beta1, double beta2, double wd, uint8_t* near_tie,
-                              double tie_tol, int fp32_decision) {
+                              double tie_tol, int fp32_decision, int stochastic, uint64_t seed, int64_t step,
+                              int64_t index0) {
   const uint16_t* gb = (const uint16_t*)g;
   const float* gf = (const float*)g;
   const float hf = (float)h, b2f = (float)beta2, omb2f = (float)(1.0 - beta2);
@@ -351,7 +405,9 @@ void adagc_ref_lion_bf16state(float* theta, const void* g, int g_is_bf16, uint16
     theta[j] = (float)(th - lr * (sgn + wd * th));
     const double a2 = beta2 * mj, b2 = (1.0 - beta2) * gh;
     if (fp32_decision) {
-      m[j] = double_to_bf16((double)fmaf(b2f, (float)mj, omb2f * (hf * (float)gj)));
+      const float m1f = fmaf(b2f, (float)mj, omb2f * (hf * (float)gj));
+      m[j] = stochastic ? float_to_bf16_stochastic(m1f, rounding_random(index0 + j, step, seed, 0))
+                        : double_to_bf16((double)m1f);
     } else {
       count_near_tie(near_tie, j, a2 + b2, fabs(a2) + fabs(b2), tie_tol);
       m[j] = double_to_bf16(a2 + b2);
@@ -364,7 +420,7 @@ void adagc_ref_lion_bf16state(float* theta, const void* g, int g_is_bf16, uint16
  * single precision (both sums fused multiply-adds). */
 void adagc_ref_sgdm_bf16state(float* theta, const void* g, int g_is_bf16, uint16_t* m, int64_t n, double h,
                               double lr, double momentum, double wd, uint8_t* near_tie, double tie_tol,
-                              int fp32_decision) {
+                              int fp32_decision, int stochastic, uint64_t seed, int64_t step, int64_t index0) {
   const uint16_t* gb = (const uint16_t*)g;
   const float* gf = (const float*)g;
   const float hf = (float)h, muf = (float)momentum, wdf = (float)wd;
@@ -378,7 +434,8 @@ void adagc_ref_sgdm_bf16state(float* theta, const void* g, int g_is_bf16, uint16
     const float m1f = fmaf(muf, (float)bf16_to_double(m[j]), fmaf(wdf, theta[j], hf * (float)gj));
     theta[j] = (float)(th - lr * m1);
     if (fp32_decision) {
-      m[j] = double_to_bf16((double)m1f);
+      m[j] = stochastic ? float_to_bf16_stochastic(m1f, rounding_random(index0 + j, step, seed, 0))
+                        : double_to_bf16((double)m1f);
     } else {
       count_near_tie(near_tie, j, m1, fabs(a) + fabs(h * gj) + fabs(wd * th), tie_tol);
       m[j] = double_to_bf16(m1);

@@ -65,13 +65,20 @@ def lib():
         L.adagc_ref_adamw_bf16state.restype = None
         L.adagc_ref_adamw_bf16state.argtypes = ([C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int64,
                                                  C.c_double, C.c_int64] + [C.c_double] * 5 +
-                                                [C.c_void_p, C.c_double, C.c_int])
+                                                [C.c_void_p, C.c_double, C.c_int, C.c_int, C.c_uint64, C.c_int64,
+                                                 C.c_void_p])
         L.adagc_ref_lion_bf16state.restype = None
         L.adagc_ref_lion_bf16state.argtypes = ([C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64] +
-                                               [C.c_double] * 5 + [C.c_void_p, C.c_double, C.c_int])
+                                               [C.c_double] * 5 + [C.c_void_p, C.c_double, C.c_int, C.c_int,
+                                                                   C.c_uint64, C.c_int64, C.c_int64])
         L.adagc_ref_sgdm_bf16state.restype = None
         L.adagc_ref_sgdm_bf16state.argtypes = ([C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_int64] +
-                                               [C.c_double] * 4 + [C.c_void_p, C.c_double, C.c_int])
+                                               [C.c_double] * 4 + [C.c_void_p, C.c_double, C.c_int, C.c_int,
+                                                                   C.c_uint64, C.c_int64, C.c_int64])
+        L.adagc_ref_philox4x32_10.restype = None
+        L.adagc_ref_philox4x32_10.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        L.adagc_ref_float_to_bf16_stochastic.restype = C.c_uint16
+        L.adagc_ref_float_to_bf16_stochastic.argtypes = [C.c_float, C.c_uint32]
         L.adagc_ref_scale.restype = None
         L.adagc_ref_scale.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_double]
         L.adagc_ref_step.restype = C.c_int32
@@ -157,20 +164,28 @@ def _is_bf16_state(theta: np.ndarray, moments, n: int) -> bool:
 def adamw_update_bf16state(theta: np.ndarray, g: np.ndarray, m: np.ndarray, v: np.ndarray, h: float, step: int,
                            lr: float, beta1: float, beta2: float, eps: float, wd: float,
                            near_tie: Optional[np.ndarray] = None, tie_tol: float = 0.0,
-                           fp32_decision: bool = False) -> None:
+                           fp32_decision: bool = False, stochastic_seed: Optional[int] = None, index0: int = 0,
+                           index: Optional[np.ndarray] = None) -> None:
     """AdamW with m and v stored as bfloat16 (uint16 bit patterns), in place; theta fp32.  `near_tie` (uint8) counts,
     per element, the steps in which the float64 rounding of m or v was decided with a relative margin below `tie_tol`.
-    fp32_decision: the value rounded to bfloat16 is evaluated in single precision (see adagc_ref.c) instead."""
+    fp32_decision: the value rounded to bfloat16 is evaluated in single precision (see adagc_ref.c) instead.
+    stochastic_seed: round that value stochastically, with the random numbers of the elements' arena positions
+    (`index`, an int64 array, or index0 + j), the step and this seed."""
     p, bf = _grad_ptr(g)
     assert _is_bf16_state(theta, (m, v), g.size)
+    assert stochastic_seed is None or fp32_decision, "stochastic rounding acts on the single-precision value"
+    if index is not None:
+        assert index.dtype == np.int64 and index.flags["C_CONTIGUOUS"] and index.size == g.size
     lib().adagc_ref_adamw_bf16state(theta.ctypes.data, p, bf, m.ctypes.data, v.ctypes.data, g.size, float(h),
                                     int(step), lr, beta1, beta2, eps, wd, _tie_ptr(near_tie, g.size), float(tie_tol),
-                                    int(fp32_decision))
+                                    int(fp32_decision), int(stochastic_seed is not None), int(stochastic_seed or 0),
+                                    int(index0), None if index is None else index.ctypes.data)
 
 
 def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, beta1: float,
                 beta2: float, wd: float, near_tie: Optional[np.ndarray] = None, tie_tol: float = 0.0,
-                fp32_decision: bool = False) -> None:
+                fp32_decision: bool = False, stochastic_seed: Optional[int] = None, step: int = 0,
+                index0: int = 0) -> None:
     """Lion on the clipped gradient, in place on fp32 theta and on m (fp32, or uint16 = stored as bfloat16).
     `near_tie` (uint8, same length) counts, per element, the steps in which sign(c) -- and, for bfloat16 m, its
     rounding -- was decided with a relative margin below `tie_tol`."""
@@ -178,7 +193,8 @@ def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: f
     nt = _tie_ptr(near_tie, g.size)
     if _is_bf16_state(theta, (m,), g.size):
         lib().adagc_ref_lion_bf16state(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, beta1, beta2,
-                                       wd, nt, float(tie_tol), int(fp32_decision))
+                                       wd, nt, float(tie_tol), int(fp32_decision), int(stochastic_seed is not None),
+                                       int(stochastic_seed or 0), int(step), int(index0))
     else:
         lib().adagc_ref_lion(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, beta1, beta2, wd,
                              nt, float(tie_tol))
@@ -186,12 +202,14 @@ def lion_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: f
 
 def sgdm_update(theta: np.ndarray, g: np.ndarray, m: np.ndarray, h: float, lr: float, momentum: float,
                 wd: float, near_tie: Optional[np.ndarray] = None, tie_tol: float = 0.0,
-                fp32_decision: bool = False) -> None:
+                fp32_decision: bool = False, stochastic_seed: Optional[int] = None, step: int = 0,
+                index0: int = 0) -> None:
     """SGD with momentum on the clipped gradient, in place on fp32 theta and on m (fp32, or uint16 = bfloat16)."""
     p, bf = _grad_ptr(g)
     if _is_bf16_state(theta, (m,), g.size):
         lib().adagc_ref_sgdm_bf16state(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, momentum, wd,
-                                       _tie_ptr(near_tie, g.size), float(tie_tol), int(fp32_decision))
+                                       _tie_ptr(near_tie, g.size), float(tie_tol), int(fp32_decision),
+                                       int(stochastic_seed is not None), int(stochastic_seed or 0), int(step), int(index0))
     else:
         lib().adagc_ref_sgdm(theta.ctypes.data, p, bf, m.ctypes.data, g.size, float(h), lr, momentum, wd)
 
@@ -202,6 +220,16 @@ def scale(g: np.ndarray, h: float, out: Optional[np.ndarray] = None) -> np.ndarr
     out = np.empty_like(g) if out is None else out
     lib().adagc_ref_scale(out.ctypes.data, p, bf, g.size, float(h))
     return out
+
+
+def philox4x32_10(counter, key) -> np.ndarray:
+    c, k, out = np.asarray(counter, np.uint32).copy(), np.asarray(key, np.uint32).copy(), np.zeros(4, np.uint32)
+    lib().adagc_ref_philox4x32_10(c.ctypes.data, k.ctypes.data, out.ctypes.data)
+    return out
+
+
+def float_to_bf16_stochastic_bits(x: float, r: int) -> int:
+    return int(lib().adagc_ref_float_to_bf16_stochastic(float(np.float32(x)), int(r)))
 
 
 def double_to_bf16_bits(x: float) -> int:
@@ -215,11 +243,13 @@ class ArenaOracle:
                  lr: float, beta1: float, beta2: float, eps: float, wd: float, lambda_rel: float,
                  beta: float, lambda_abs: float, warmup: int, keep_initial: bool = False,
                  global_adaptive: bool = False, gamma0: Optional[np.ndarray] = None, ema_cap: float = 0.0,
-                 bf16_state: bool = False, tie_tol: float = 0.0, fp32_decision: bool = False):
+                 bf16_state: bool = False, tie_tol: float = 0.0, fp32_decision: bool = False,
+                 stochastic_seed: Optional[int] = None):
         """bf16_state: m and v are stored as bfloat16 (uint16 bit patterns), rounded to nearest even on store;
         `self.ties` then counts, per element, the steps whose float64 rounding was decided with a margin below
         tie_tol; fp32_decision: the rounded value is evaluated in single precision (see adagc_ref.c)."""
         self.fp32_decision = bool(fp32_decision)
+        self.stochastic_seed = stochastic_seed
         self.keep_initial, self.global_adaptive, self.ema_cap = keep_initial, global_adaptive, float(ema_cap)
         self.bf16_state, self.tie_tol = bool(bf16_state), float(tie_tol)
         self.off = np.ascontiguousarray(offsets, dtype=np.int64)
@@ -264,7 +294,7 @@ class ArenaOracle:
                     self.t, hp["lr"] if lr is None else lr, hp["beta1"], hp["beta2"], hp["eps"], hp["wd"])
             if self.bf16_state:
                 adamw_update_bf16state(*args, near_tie=self.ties[o:o + n], tie_tol=self.tie_tol,
-                                       fp32_decision=self.fp32_decision)
+                                       fp32_decision=self.fp32_decision, stochastic_seed=self.stochastic_seed, index0=o)
             else:
                 adamw_update(*args)
         return r

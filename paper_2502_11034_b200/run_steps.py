@@ -1,7 +1,7 @@
 """Run a few fused AdaGC + AdamW steps (or clip-only steps) on a named synthetic layout.
 
     python -m paper_2502_11034_b200.run_steps --workload gpt2_small --steps 4 [--mode step|clip|lion|sgdm] [--n-layer N]
-        [--update-path auto|registers|bulk] [--fused-small]
+        [--update-path auto|registers|bulk] [--fused-small] [--state f32|bf16] [--separate-finalize]
 
 A minimal driver of the C ABI (adagc_create / adagc_step / adagc_clip / adagc_get_stats): useful as
 an example and as a small, short-running target for profilers.  Prints the per-phase device times.
@@ -26,6 +26,9 @@ def main():
                     help="kernel of the update phase (adagc_desc.flags)")
     ap.add_argument("--fused-small", action="store_true",
                     help="ADAGC_FUSED_SMALL: adagc_step as one cooperative kernel (small layouts, --mode step)")
+    ap.add_argument("--state", choices=["f32", "bf16"], default="f32", help="dtype of the m and v arenas (adagc_desc.state_dtype)")
+    ap.add_argument("--separate-finalize", action="store_true",
+                    help="ADAGC_SEPARATE_FINALIZE: the per-tensor decisions of AdaGC steps in a kernel of their own")
     args = ap.parse_args()
     over = {} if args.n_layer is None else {"n_layer": args.n_layer}
     wl = workloads.build(args.workload, **over)
@@ -37,9 +40,13 @@ def main():
              "bulk": binding.UPDATE_PATH_BULK}[args.update_path]
     if args.fused_small:
         flags |= binding.FUSED_SMALL
-    opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=dev, flags=flags)
+    if args.separate_finalize:
+        flags |= binding.SEPARATE_FINALIZE
+    sd = torch.bfloat16 if args.state == "bf16" else torch.float32
+    opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=dev, flags=flags, state_dtype=sd)
     theta = workloads.init_params(wl, dev)
-    m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+    m = torch.zeros(wl.arena_elems, dtype=sd, device=dev)
+    v = torch.zeros_like(m)
     ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device=dev)
     g = workloads.grads_for_step(wl, 1, dev)
     g_out = torch.empty_like(g) if args.mode == "clip" else None

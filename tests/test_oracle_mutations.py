@@ -164,12 +164,27 @@ BF16_STATE_MUTATIONS = {
                                                                      "dist = dist + 0.0 * low_edge"),
 }
 
+BF16_STATE_MUTATIONS.update({
+    "Philox: key not bumped between rounds": ("        if r < 9:\n            k0, k1 = (k0 + np.uint64(PHILOX_W0)) & mask, (k1 + np.uint64(PHILOX_W1)) & mask",
+                                              "        if False:\n            pass"),
+    "Philox: nine rounds": ("    for r in range(10):\n        p0, p1 = np.uint64(PHILOX_M0)", "    for r in range(9):\n        p0, p1 = np.uint64(PHILOX_M0)"),
+    "Philox: multipliers swapped": ("p0, p1 = np.uint64(PHILOX_M0) * c0, np.uint64(PHILOX_M1) * c2", "p0, p1 = np.uint64(PHILOX_M1) * c0, np.uint64(PHILOX_M0) * c2"),
+    "stochastic rounding: m and v use the same half of the word": ("(word >> np.uint32(16)).astype(np.uint32)", "(word & np.uint32(0xFFFF)).astype(np.uint32)"),
+    "stochastic rounding: one generator call per element instead of per four": ("q = index >> np.uint64(2)", "q = index"),
+    "stochastic rounding: step not in the counter": ("np.full(q.shape, step & 0xFFFFFFFF, np.uint64)", "np.full(q.shape, 0, np.uint64)"),
+    "stochastic rounding: always toward zero": ("out = (((u + np.asarray(r16, np.uint64)) >> np.uint64(16))", "out = (((u + 0 * np.asarray(r16, np.uint64)) >> np.uint64(16))"),
+    "stochastic rounding: random number twice as large": ("out = (((u + np.asarray(r16, np.uint64)) >> np.uint64(16))", "out = (((u + 2 * np.asarray(r16, np.uint64)) >> np.uint64(16))"),
+})
+
 BF16_STATE_PINS = [(pins_bf.test_rounding_matches_the_library_conversion_and_ties_go_to_even, ()),
                    (pins_bf.test_rounding_margin_is_the_distance_to_a_flip, ()),
                    (pins_bf.test_one_step_from_a_given_state_matches_library_adamw, (pins_bf.NumpyBF, 7)),
                    (pins_bf.test_theta_is_the_fp32_state_paths_theta_bit_for_bit, (pins_bf.NumpyBF,)),
                    (pins_bf.test_lion_and_sgdm_store_the_nearest_bf16_and_leave_theta_alone, ("numpy",)),
-                   (pins_bf.test_c_oracle_counts_decisions_close_to_a_flip, ())]
+                   (pins_bf.test_c_oracle_counts_decisions_close_to_a_flip, ()),
+                   (pins_bf.test_philox_known_answers, ()),
+                   (pins_bf.test_stochastic_rounding_is_exactly_unbiased_and_leaves_bf16_values_alone, ()),
+                   (pins_bf.test_stochastic_step_is_the_nearest_rounding_steps_value_rounded_with_the_stated_random_numbers, ())]
 
 
 @pytest.mark.parametrize("name", sorted(BF16_STATE_MUTATIONS))

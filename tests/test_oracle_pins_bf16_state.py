@@ -360,3 +360,109 @@ def test_fp32_and_float64_decisions_differ_only_at_reported_ties_and_by_one_neig
     co.adamw_update_bf16state(theta.copy(), g2, f32_to_bits(m0), f32_to_bits(v0), 1.0, 4, 3e-4, 0.9, 0.95, 1e-8, 0.1,
                               near_tie=ties2, tie_tol=1e-6)
     assert (ties2 > 0).mean() < 4e-3
+
+
+# ----------------------------------------------------------------------------- stochastic rounding
+def test_philox_known_answers():
+    """Both oracles' Philox4x32-10 against the published known-answer vectors (tests/golden/philox4x32_10_kat.txt)."""
+    import os
+    rows = [ln.split() for ln in open(os.path.join(os.path.dirname(__file__), "golden", "philox4x32_10_kat.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 3
+    for r in rows:
+        w = [int(x, 16) for x in r]
+        ctr, key, want = w[0:4], w[4:6], w[6:10]
+        assert npo.philox4x32_10(np.array(ctr), np.array(key)).tolist() == want
+        assert co.philox4x32_10(ctr, key).tolist() == want
+    # vectorised over many counters = one at a time
+    rng = np.random.RandomState(31)
+    ctrs = rng.randint(0, 2 ** 32, size=(50, 4), dtype=np.uint64)
+    key = rng.randint(0, 2 ** 32, size=2, dtype=np.uint64)
+    many = npo.philox4x32_10(ctrs, key)
+    for c, o in zip(ctrs, many):
+        assert co.philox4x32_10(c, key).tolist() == o.tolist()
+
+
+def test_stochastic_rounding_is_exactly_unbiased_and_leaves_bf16_values_alone():
+    """Closed form: over all 65536 values of the random integer, a float x between the bfloat16 neighbours a < b (in
+    magnitude) goes to b exactly low16(x) times, so the mean of the results is x itself; a bfloat16 value never moves."""
+    rng = np.random.RandomState(32)
+    xs = np.concatenate([(rng.standard_normal(40) * 10.0 ** rng.uniform(-30, 30, 40)).astype(np.float32),
+                         np.array([1.0, -1.0, 1.0 + 2.0 ** -8, 1.0 + 2.0 ** -23, 2.0 - 2.0 ** -23, 1e-40, -3e-39], np.float32)])
+    r = np.arange(65536, dtype=np.uint32)
+    for x in xs:
+        out = npo.stochastic_round_to_bf16(np.full(65536, x, np.float32), r).astype(np.float64)
+        lo16 = int(np.float32(x).view(np.uint32)) & 0xFFFF
+        vals = np.unique(out)
+        assert len(vals) == (1 if lo16 == 0 else 2)
+        assert (out.astype(np.float32).view(np.uint32) & 0xFFFF == 0).all()
+        assert int((np.abs(out) == np.abs(vals).max()).sum()) == (65536 if lo16 == 0 else lo16)
+        assert abs(out.mean() - float(x)) <= 2.0 ** -40 * abs(float(x))            # = x up to the float64 mean's rounding
+    # C and numpy agree, value by value; infinities and NaN are rounded to nearest
+    for x, rr in zip(xs, rng.randint(0, 65536, size=len(xs))):
+        want = int(npo.stochastic_round_to_bf16(np.array([x], np.float32), np.array([rr]))[0].view(np.uint32)) >> 16
+        assert co.float_to_bf16_stochastic_bits(x, int(rr)) == want
+    assert co.float_to_bf16_stochastic_bits(np.inf, 65535) == 0x7F80 and co.float_to_bf16_stochastic_bits(-np.inf, 1) == 0xFF80
+    assert np.isinf(npo.stochastic_round_to_bf16(np.array([np.inf], np.float32), np.array([65535]))[0])
+
+
+def test_stochastic_step_is_the_nearest_rounding_steps_value_rounded_with_the_stated_random_numbers():
+    """The C oracle's stochastic step, piece by piece: its single-precision m' and v' are those of the (exact-arithmetic
+    pinned) fp32-decision mode -- recovered here as the values whose two candidate roundings bracket them -- and the
+    stored result is stochastic_round_to_bf16 of that value with rounding_randoms(arena position, step, seed)."""
+    rng = np.random.RandomState(33)
+    n, index0, step, seed = 5000, 123456, 7, 0x1234_5678_9ABC_DEF0
+    g = bf16_values(rng, n, 1e-4).astype(np.float32)
+    m0, v0 = bf16_values(rng, n, 3e-5), np.abs(bf16_values(rng, n, 1e-8))
+    theta = (rng.standard_normal(n) * 0.02).astype(np.float32)
+    # the single-precision values, by the numpy route: products of two floats are exact in float64, and the one
+    # float64 addition is exact whenever both terms fit 53 bits together, which holds for all but a few elements
+    h, b1, b2 = np.float32(0.61), np.float32(0.9), np.float32(0.95)
+    o1, o2 = np.float32(1.0 - 0.9), np.float32(1.0 - 0.95)
+    gh = (h * g).astype(np.float32)
+    m1f = (b1.astype(np.float64) * m0.astype(np.float64) + (o1 * gh).astype(np.float32).astype(np.float64)).astype(np.float32)
+    v1f = (b2.astype(np.float64) * v0.astype(np.float64) +
+           (o2 * (gh * gh).astype(np.float32)).astype(np.float32).astype(np.float64)).astype(np.float32)
+    idx = index0 + np.arange(n)
+    rm, rv = npo.rounding_randoms(idx, step, seed)
+    want_m = (npo.stochastic_round_to_bf16(m1f, rm).view(np.uint32) >> 16).astype(np.uint16)
+    want_v = (npo.stochastic_round_to_bf16(v1f, rv).view(np.uint32) >> 16).astype(np.uint16)
+    th_s, mb, vb = theta.copy(), f32_to_bits(m0), f32_to_bits(v0)
+    co.adamw_update_bf16state(th_s, g, mb, vb, float(h), step, 3e-4, 0.9, 0.95, 1e-8, 0.1, fp32_decision=True,
+                              stochastic_seed=seed, index0=index0)
+    assert (mb != want_m).mean() < 1e-3 and (vb != want_v).mean() < 1e-3          # (double rounding of the numpy route)
+    assert (np.abs(mb.astype(np.int64) - want_m.astype(np.int64)) <= 1).all()
+    # an explicit index array gives the same as index0 + j, another step or seed gives other roundings, theta is untouched
+    th2, mb2, vb2 = theta.copy(), f32_to_bits(m0), f32_to_bits(v0)
+    co.adamw_update_bf16state(th2, g, mb2, vb2, float(h), step, 3e-4, 0.9, 0.95, 1e-8, 0.1, fp32_decision=True,
+                              stochastic_seed=seed, index=idx.astype(np.int64))
+    assert np.array_equal(mb, mb2) and np.array_equal(vb, vb2) and np.array_equal(th_s, th2)
+    th3, mb3, vb3 = theta.copy(), f32_to_bits(m0), f32_to_bits(v0)
+    co.adamw_update_bf16state(th3, g, mb3, vb3, float(h), step, 3e-4, 0.9, 0.95, 1e-8, 0.1, fp32_decision=True)
+    assert np.array_equal(th3, th_s)                                           # theta never sees the rounding
+    assert 0.2 < (mb3 != mb).mean() < 0.3        # a uniform fraction f goes the other way with probability min(f, 1 - f): 1/4
+    # stochastic and nearest results are the two neighbours of the same value
+    assert (np.abs(mb3.astype(np.int64) - mb.astype(np.int64)) <= 1).all()
+    th4, mb4, vb4 = theta.copy(), f32_to_bits(m0), f32_to_bits(v0)
+    co.adamw_update_bf16state(th4, g, mb4, vb4, float(h), step + 1, 3e-4, 0.9, 0.95, 1e-8, 0.1, fp32_decision=True,
+                              stochastic_seed=seed, index0=index0)
+    assert (mb4 != mb).mean() > 0.2
+
+
+def test_stochastic_rounding_tracks_a_slow_average_where_nearest_rounding_stalls():
+    """Why one would round stochastically: with beta2 = 0.999 a bfloat16 v rounded to nearest stops moving 500 spacings
+    (a factor of several) short of its fixed point, while the stochastically rounded v reaches it on average."""
+    n = 4096
+    g = np.full(n, 1e-3, np.float32)
+    theta = np.zeros(n, np.float32)
+    res = {}
+    for mode, seed in (("nearest", None), ("stochastic", 99)):
+        th, mb, vb = theta.copy(), np.zeros(n, np.uint16), np.zeros(n, np.uint16)
+        for t in range(1, 6001):
+            co.adamw_update_bf16state(th, g, mb, vb, 1.0, t, 0.0, 0.9, 0.999, 1e-8, 0.0, fp32_decision=True,
+                                      stochastic_seed=seed)
+        res[mode] = bits_to_f64(vb)
+    target = 1e-6 * (1 - 0.999 ** 6000)
+    assert res["nearest"].max() < 0.5 * target                                  # stalled far below
+    assert abs(res["stochastic"].mean() - target) < 0.02 * target               # unbiased
+    assert res["stochastic"].std() < 0.1 * target

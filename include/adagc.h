@@ -327,6 +327,25 @@ int adagc_get_sumsq(adagc_ctx* ctx, double* h_sumsq, void* cuda_stream);
  */
 int adagc_set_ema_cap(adagc_ctx* ctx, double cap);
 
+/*
+ * How bfloat16-stored moments (state_dtype = ADAGC_BF16) are rounded where they are stored.
+ *   ADAGC_ROUND_NEAREST     to the nearest bfloat16, ties to even (the default);
+ *   ADAGC_ROUND_STOCHASTIC  to the neighbour of larger magnitude with probability (distance to the smaller neighbour) /
+ *                           spacing, otherwise to the smaller one: unbiased, so a slow average (beta2 = 0.999) keeps
+ *                           moving where rounding to nearest stalls.  The single-precision value of "Optimizer state
+ *                           stored as bfloat16" above has the 16-bit random integer r added to the low half of its bit
+ *                           pattern, and that half is dropped.  r comes from the counter-based generator Philox4x32-10
+ *                           (Salmon et al., SC 2011): the four elements 4q .. 4q+3 of the arenas share one call with
+ *                           counter (lo q, hi q, lo step, hi step) and key (lo seed, hi seed); element 4q + l takes
+ *                           output word l, its low half for m, its high half for v.  The result therefore depends on
+ *                           (seed, step, element position) only: reruns and restarts reproduce it bit for bit.
+ * Host-only; takes effect from the next step.  ADAGC_E_DTYPE if the context's state is fp32.  adagc_step_capturable
+ * returns ADAGC_E_INVALID_ARG while stochastic rounding is on (its step number lives on the device).
+ */
+#define ADAGC_ROUND_NEAREST 0
+#define ADAGC_ROUND_STOCHASTIC 1
+int adagc_set_state_rounding(adagc_ctx* ctx, int32_t mode, uint64_t seed);
+
 /* The update path this context uses: ADAGC_UPDATE_PATH_REGISTERS or ADAGC_UPDATE_PATH_BULK. */
 int adagc_update_path(const adagc_ctx* ctx);
 

@@ -91,6 +91,8 @@ def lib() -> C.CDLL:
     L.adagc_get_sumsq.argtypes = [vp, vp, vp]
     L.adagc_set_ema_cap.restype = C.c_int
     L.adagc_set_ema_cap.argtypes = [vp, dbl]
+    L.adagc_set_state_rounding.restype = C.c_int
+    L.adagc_set_state_rounding.argtypes = [vp, C.c_int32, C.c_uint64]
     L.adagc_update_path.restype = C.c_int
     L.adagc_update_path.argtypes = [vp]
     L.adagc_arena_elems.restype = i64
@@ -350,6 +352,11 @@ class AdaGC:
         rc = lib().adagc_set_ema_cap(self._h, float(cap))
         if rc != 0:
             raise AdagcError(rc, "adagc_set_ema_cap")
+
+    def set_state_rounding(self, stochastic: bool, seed: int = 0):
+        rc = lib().adagc_set_state_rounding(self._h, 1 if stochastic else 0, int(seed) & (2 ** 64 - 1))
+        if rc != 0:
+            raise AdagcError(rc, "adagc_set_state_rounding")
 
     def debug_wait_timeout(self, limit_ms: float, stream=None):
         rc = lib().adagc_debug_wait_timeout(self._h, float(limit_ms), _stream_ptr(stream))

@@ -160,6 +160,51 @@ __device__ __forceinline__ uint32_t pack_bf16_cvt(float lo, float hi) {
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
   return d;
 }
+// Stochastic rounding of stored bfloat16 moments (adagc_set_state_rounding).  Random numbers: Philox4x32-10, the
+// counter-based generator of Salmon, Moraes, Dror and Shaw (SC 2011), from its definition: ten rounds that replace the
+// counter (c0, c1, c2, c3) by (hi(M1 c2) ^ c1 ^ k0, lo(M1 c2), hi(M0 c0) ^ c3 ^ k1, lo(M0 c0)), the key bumped by
+// (W0, W1) between rounds.  The four elements 4q .. 4q+3 of the arenas share one call with counter
+// (lo q, hi q, lo step, hi step) and key (lo seed, hi seed); element 4q + l takes output word l, the low half for m,
+// the high half for v.
+struct StateRounding {
+  uint32_t seed_lo, seed_hi, step_lo, step_hi;
+  int stochastic;  // 0: round to nearest even
+};
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1) {
+  constexpr uint32_t kM0 = 0xD2511F53u, kM1 = 0xCD9E8D57u, kW0 = 0x9E3779B9u, kW1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(kM0, c0), lo0 = kM0 * c0, hi1 = __umulhi(kM1, c2), lo1 = kM1 * c2;
+    c0 = hi1 ^ c1 ^ k0;
+    c1 = lo1;
+    c2 = hi0 ^ c3 ^ k1;
+    c3 = lo0;
+    k0 += kW0;  // (the bump after the last round is never used)
+    k1 += kW1;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+__device__ __forceinline__ uint4 rounding_words(int64_t q, const StateRounding& sr) {
+  return philox4x32_10(static_cast<uint32_t>(q), static_cast<uint32_t>(static_cast<uint64_t>(q) >> 32), sr.step_lo, sr.step_hi,
+                       sr.seed_lo, sr.seed_hi);
+}
+// x moves to its bfloat16 neighbour of larger magnitude with probability (distance to the smaller one) / spacing: the
+// 16-bit random number is added to the low half of the bit pattern and that half is dropped.  This is what the
+// stochastic-rounding conversion instruction computes (checked on B200 against the integer formula for finite values,
+// subnormals and overflow included: the low result takes the second source and random bits 15..0, the high result
+// the first source and bits 31..16); infinities stay, NaN stays NaN.
+__device__ __forceinline__ uint32_t pack_bf16_stochastic(float lo, float hi, uint32_t r_lo_hi) {
+  uint32_t d;
+  asm("cvt.rs.bf16x2.f32 %0, %1, %2, %3;" : "=r"(d) : "f"(hi), "f"(lo), "r"(r_lo_hi));
+  return d;
+}
+// four values with the four words of their group; which = 0: low halves (m), 1: high halves (v)
+__device__ __forceinline__ uint2 pack4_stochastic(const float4& x, const uint4& w, int which) {
+  const uint32_t sel = which ? 0x7632u : 0x5410u;  // the chosen halves of two words, side by side
+  return make_uint2(pack_bf16_stochastic(x.x, x.y, __byte_perm(w.x, w.y, sel)),
+                    pack_bf16_stochastic(x.z, x.w, __byte_perm(w.z, w.w, sel)));
+}
+
 __device__ __forceinline__ float4 ld_stream(const float4* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream(float4* p, float4 v) { __stcs(p, v); }
 __device__ __forceinline__ void st_stream(uint4* p, uint4 v) { __stcs(p, v); }
@@ -776,10 +821,18 @@ __device__ __forceinline__ void load_state8(const void* __restrict__ base, int i
   }
 }
 template <bool kSB>
-__device__ __forceinline__ void store_state8(void* __restrict__ base, int i, const float4& a, const float4& b) {
+__device__ __forceinline__ void store_state8(void* __restrict__ base, int i, const float4& a, const float4& b,
+                                             bool stochastic = false, const uint4& wa = uint4(), const uint4& wb = uint4(),
+                                             int which = 0) {
   if (kSB) {
-    st_stream(static_cast<uint4*>(base) + i, make_uint4(pack_bf16_cvt(a.x, a.y), pack_bf16_cvt(a.z, a.w),
-                                                        pack_bf16_cvt(b.x, b.y), pack_bf16_cvt(b.z, b.w)));
+    uint4 packed;
+    if (stochastic) {
+      const uint2 lo = pack4_stochastic(a, wa, which), hi = pack4_stochastic(b, wb, which);
+      packed = make_uint4(lo.x, lo.y, hi.x, hi.y);
+    } else {
+      packed = make_uint4(pack_bf16_cvt(a.x, a.y), pack_bf16_cvt(a.z, a.w), pack_bf16_cvt(b.x, b.y), pack_bf16_cvt(b.z, b.w));
+    }
+    st_stream(static_cast<uint4*>(base) + i, packed);
   } else {
     st_stream(static_cast<float4*>(base) + 2 * i, a);
     st_stream(static_cast<float4*>(base) + 2 * i + 1, b);
@@ -789,6 +842,13 @@ template <bool kSB>
 __device__ __forceinline__ float load_state1(const void* __restrict__ base, int64_t j) {
   return kSB ? __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(base)[j]) << 16)
              : static_cast<const float*>(base)[j];
+}
+// one element at arena index `at`, rounded stochastically (which = 0: m, 1: v)
+__device__ __forceinline__ void store_state1_stochastic(void* __restrict__ base, int64_t j, float x, int64_t at,
+                                                        const StateRounding& sr, int which) {
+  const uint4 w = rounding_words(at >> 2, sr);
+  const uint32_t word = (at & 3) == 0 ? w.x : (at & 3) == 1 ? w.y : (at & 3) == 2 ? w.z : w.w;
+  static_cast<uint16_t*>(base)[j] = static_cast<uint16_t>(pack_bf16_stochastic(x, 0.0f, (word >> (which ? 16 : 0)) & 0xffffu));
 }
 template <bool kSB>
 __device__ __forceinline__ void store_state1(void* __restrict__ base, int64_t j, float x) {
@@ -802,7 +862,8 @@ __device__ __forceinline__ void store_state1(void* __restrict__ base, int64_t j,
 template <bool kBF16, int kOpt, bool kSB>
 __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gbase, float4* __restrict__ p4,
                                              void* __restrict__ mbase, void* __restrict__ vbase, float h,
-                                             const AdamScalars& a, uint4* __restrict__ lowp8 = nullptr) {
+                                             const AdamScalars& a, uint4* __restrict__ lowp8 = nullptr,
+                                             const StateRounding* sr = nullptr, int64_t q0 = 0) {
   float g[8];
   if (kBF16) {
     // the norm kernel left these lines marked evict_last; this last read of them hands them back
@@ -826,8 +887,14 @@ __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gba
   adamw_vec4<kOpt>(g[0], g[1], g[2], g[3], h, pa, ma, va, a);
   adamw_vec4<kOpt>(g[4], g[5], g[6], g[7], h, pb, mb, vb, a);
   st_stream(p4 + 2 * i, pa); st_stream(p4 + 2 * i + 1, pb);
-  store_state8<kSB>(mbase, i, ma, mb);
-  if (kOpt == kOptAdamW) store_state8<kSB>(vbase, i, va, vb);
+  if (kSB && sr && sr->stochastic) {  // q0: arena index / 4 of the chunk's first element; this group is elements 8i .. 8i+7
+    const uint4 wa = rounding_words(q0 + 2 * i, *sr), wb = rounding_words(q0 + 2 * i + 1, *sr);
+    store_state8<kSB>(mbase, i, ma, mb, true, wa, wb, 0);
+    if (kOpt == kOptAdamW) store_state8<kSB>(vbase, i, va, vb, true, wa, wb, 1);
+  } else {
+    store_state8<kSB>(mbase, i, ma, mb);
+    if (kOpt == kOptAdamW) store_state8<kSB>(vbase, i, va, vb);
+  }
   if (lowp8)  // bf16 copy of the updated parameters (the model's working weights in mixed precision)
     st_stream(lowp8 + i, make_uint4(pack_bf16(pa.x, pa.y), pack_bf16(pa.z, pa.w), pack_bf16(pb.x, pb.y),
                                     pack_bf16(pb.z, pb.w)));
@@ -841,7 +908,8 @@ template <bool kBF16, int kBlockThreads, int kOpt, bool kSB>
 __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, int& row_base, float* __restrict__ params,
                                                     const void* __restrict__ grads, void* __restrict__ m_arena,
                                                     void* __restrict__ v_arena, const AdamScalars& a,
-                                                    uint16_t* __restrict__ lowp = nullptr) {
+                                                    uint16_t* __restrict__ lowp = nullptr,
+                                                    const StateRounding* sr = nullptr) {
   constexpr int kWarps = kBlockThreads / 32;
   constexpr int kStateBytes = kSB ? 2 : 4;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -856,7 +924,8 @@ __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, in
   for (int r = (warp - row_base) & (kWarps - 1); r < rows; r += kWarps) {
     const int i = (r << 5) + lane;
     if (i < n8)
-      adamw_group8<kBF16, kOpt, kSB>(i, gbase, p4, mbase, vbase, h, a, lowp ? reinterpret_cast<uint4*>(lowp + start) : nullptr);
+      adamw_group8<kBF16, kOpt, kSB>(i, gbase, p4, mbase, vbase, h, a, lowp ? reinterpret_cast<uint4*>(lowp + start) : nullptr,
+                                     sr, start >> 2);
   }
   row_base = (row_base + rows) & (kWarps - 1);
   const int t = (n8 << 3) + lane;  // ragged tail (fewer than 8 elements): the next warp in turn takes it
@@ -871,8 +940,13 @@ __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, in
     if (kOpt == kOptAdamW) v = load_state1<kSB>(vbase, t);
     adamw_elem<kOpt>(g, h, p, m, v, a);
     params[start + t] = p;
-    store_state1<kSB>(mbase, t, m);
-    if (kOpt == kOptAdamW) store_state1<kSB>(vbase, t, v);
+    if (kSB && sr && sr->stochastic) {
+      store_state1_stochastic(mbase, t, m, start + t, *sr, 0);
+      if (kOpt == kOptAdamW) store_state1_stochastic(vbase, t, v, start + t, *sr, 1);
+    } else {
+      store_state1<kSB>(mbase, t, m);
+      if (kOpt == kOptAdamW) store_state1<kSB>(vbase, t, v);
+    }
     if (lowp) lowp[start + t] = static_cast<uint16_t>(f32_to_bf16_bits(p));
   }
 }
@@ -883,7 +957,7 @@ __global__ void __launch_bounds__(kThreads)
 adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, void* __restrict__ m_arena,
                     void* __restrict__ v_arena, const Chunk* __restrict__ chunks,
                     const int32_t* __restrict__ block_begin, const float* __restrict__ h_arr, AdamScalars a,
-                    uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a, Guard guard) {
+                    uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a, Guard guard, StateRounding sr) {
   constexpr int kStateBytes = kSB ? 2 : 4;
   const int tid = threadIdx.x;
   int c = block_begin[blockIdx.x];
@@ -914,9 +988,9 @@ adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, 
 #pragma unroll 2
       for (int k = 0; k < kChunkElems / 8 / kThreads; ++k)
         adamw_group8<kBF16, kOpt, kSB>(k * kThreads + tid, gbase, p4, mbase, vbase, h, a,
-                                       lowp ? reinterpret_cast<uint4*>(lowp + start) : nullptr);
+                                       lowp ? reinterpret_cast<uint4*>(lowp + start) : nullptr, &sr, start >> 2);
     } else {
-      adamw_partial_chunk<kBF16, kThreads, kOpt, kSB>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp);
+      adamw_partial_chunk<kBF16, kThreads, kOpt, kSB>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp, &sr);
     }
     if (c_next >= n_chunks) break;
     c = c_next;
@@ -1041,7 +1115,7 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
                         void* __restrict__ v_arena, const Chunk* __restrict__ chunks,
                         const int32_t* __restrict__ block_begin, const int32_t* __restrict__ block_mid,
                         const float* __restrict__ h_arr, AdamScalars a, int* __restrict__ status,
-                        uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a, Guard guard) {
+                        uint16_t* __restrict__ lowp, const AdamScalars* __restrict__ d_a, Guard guard, StateRounding sr) {
   extern __shared__ __align__(128) unsigned char tile_smem[];
   constexpr int kTile = TmaRing<kSB>::kTile, kStages = TmaRing<kSB>::kStages;
   constexpr int kTilesPerChunk = kChunkElems / kTile;
@@ -1146,8 +1220,14 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
           if (kOpt == kOptAdamW) v = smem_state4<kSB>(b + kVOff, q);
           adamw_vec4<kOpt>(g0, g1, g2, g3, h, p, m, v, a);
           p4[q] = p;
-          smem_state4_store<kSB>(b + kMOff, q, m);
-          if (kOpt == kOptAdamW) smem_state4_store<kSB>(b + kVOff, q, v);
+          if (kSB && sr.stochastic) {  // elements 4q .. 4q+3 of this tile: one group of the arenas
+            const uint4 w = rounding_words((chunk_start(ck) >> 2) + sub * (kTile / 4) + q, sr);
+            reinterpret_cast<uint2*>(b + kMOff)[q] = pack4_stochastic(m, w, 0);
+            if (kOpt == kOptAdamW) reinterpret_cast<uint2*>(b + kVOff)[q] = pack4_stochastic(v, w, 1);
+          } else {
+            smem_state4_store<kSB>(b + kMOff, q, m);
+            if (kOpt == kOptAdamW) smem_state4_store<kSB>(b + kVOff, q, v);
+          }
           if (lowp) reinterpret_cast<uint2*>(b + kStageBytes)[q] = make_uint2(pack_bf16(p.x, p.y), pack_bf16(p.z, p.w));
         }
         fence_generic_to_async_smem();  // the updated tile must be visible to the bulk-copy engine
@@ -1214,7 +1294,7 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
       ck_next = chunks[c + 1];
       h_next = h_arr[ck_next.tensor];
     }
-    adamw_partial_chunk<kBF16, kTmaThreads, kOpt, kSB>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp);
+    adamw_partial_chunk<kBF16, kTmaThreads, kOpt, kSB>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp, &sr);
     ck = ck_next;
     h = h_next;
   }
@@ -1332,7 +1412,7 @@ adagc_fused_small_kernel(float* __restrict__ params, const void* __restrict__ gr
                          void* __restrict__ v_arena, float* ema, const Chunk* __restrict__ chunks, int n_chunks,
                          const TensorEntry* __restrict__ tensors, double* slice_partials, ClipScalars cs, int in_warmup,
                          AdamScalars a, StatPtrs st, unsigned long long* barrier_counter,
-                         unsigned long long barrier_index, float* gamma_prev, Guard guard) {
+                         unsigned long long barrier_index, float* gamma_prev, Guard guard, StateRounding sr) {
   __shared__ double warp_part[kThreads / 32];
   __shared__ double total_s;
   __shared__ float h_shared;
@@ -1421,7 +1501,7 @@ adagc_fused_small_kernel(float* __restrict__ params, const void* __restrict__ gr
     Chunk sub = ck;
     sub.start4 = ck.start4 + static_cast<uint32_t>(begin / 4);
     sub.count = min(kSlice, ck.count - begin);
-    adamw_partial_chunk<kBF16, kThreads, kOptAdamW, kSB>(sub, h, row_base, params, grads, m_arena, v_arena, a);
+    adamw_partial_chunk<kBF16, kThreads, kOptAdamW, kSB>(sub, h, row_base, params, grads, m_arena, v_arena, a, nullptr, &sr);
   }
 }
 
@@ -1600,6 +1680,18 @@ struct adagc_ctx {
   int device = 0;
   int grid_wide = 1, grid_update = 1;  // norm and scale kernels: SMs x resident blocks; update: SMs x 2 or x 1
   bool update_bulk = false;            // update phase through the bulk-async (TMA) kernel
+  bool sr_stochastic = false;          // adagc_set_state_rounding: bfloat16 moments rounded stochastically
+  uint64_t sr_seed = 0;
+  int64_t sr_step = 0;                 // step number of the launches being enqueued (part of the generator's counter)
+  StateRounding rounding() const {
+    StateRounding r;
+    r.seed_lo = static_cast<uint32_t>(sr_seed);
+    r.seed_hi = static_cast<uint32_t>(sr_seed >> 32);
+    r.step_lo = static_cast<uint32_t>(sr_step);
+    r.step_hi = static_cast<uint32_t>(static_cast<uint64_t>(sr_step) >> 32);
+    r.stochastic = sr_stochastic ? 1 : 0;
+    return r;
+  }
   bool fold_finalize = true;           // AdaGC steps decide in the norm kernel's tail (needs every tensor to have a chunk)
   bool offsets_mult8 = true;           // every tensor offset is a multiple of 8 elements (bf16 arenas stay 16-byte aligned)
   bool keep_initial = false;           // ADAGC_EMA_KEEP_INITIAL
@@ -1655,7 +1747,7 @@ struct adagc_ctx {
 
 namespace {
 
-int check_clip_args(const adagc_ctx* ctx, const float* d_ema, int64_t step, double lambda_rel, double beta,
+int check_clip_args(adagc_ctx* ctx, const float* d_ema, int64_t step, double lambda_rel, double beta,
                     int64_t warmup) {
   if (!ctx || !d_ema) return ADAGC_E_INVALID_ARG;
   int dev = -1;  // the context's tables live on the device that was current at adagc_create
@@ -1664,6 +1756,7 @@ int check_clip_args(const adagc_ctx* ctx, const float* d_ema, int64_t step, doub
   if (step < 1 || warmup < 0) return ADAGC_E_INVALID_ARG;
   if (!(lambda_rel > 0.0) || !std::isfinite(lambda_rel)) return ADAGC_E_INVALID_ARG;
   if (!(beta >= 0.0 && beta < 1.0)) return ADAGC_E_INVALID_ARG;
+  ctx->sr_step = step;  // the launches that follow belong to this step
   return ADAGC_OK;
 }
 
@@ -1716,10 +1809,10 @@ void launch_update_t(adagc_ctx* ctx, const TableView& tv, float* p, const void* 
   if (ctx->update_bulk)
     launch_dependent(adagc_update_tma_kernel<kBF16, kOpt, kSB>, tv.grid, kTmaThreads,
                      tma_smem_bytes<kSB>(kBF16, kOpt, lowp != nullptr), s, programmatic, p, g, m, v, tv.chunks, tv.begin,
-                     tv.mid, st.h, a, st.status, lowp, d_a, ctx->guard());
+                     tv.mid, st.h, a, st.status, lowp, d_a, ctx->guard(), ctx->rounding());
   else
     launch_dependent(adagc_update_kernel<kBF16, kOpt, kSB>, tv.grid, kThreads, 0, s, programmatic, p, g, m, v, tv.chunks,
-                     tv.begin, st.h, a, lowp, d_a, ctx->guard());
+                     tv.begin, st.h, a, lowp, d_a, ctx->guard(), ctx->rounding());
   ctx->launches++;
 }
 
@@ -1942,8 +2035,9 @@ int launch_fused_small(adagc_ctx* ctx, void* d_params, const void* d_grads, void
   unsigned long long index = ctx->barriers_done;
   float* gamma_prev = reinterpret_cast<float*>(ctx->ws + ctx->L.gamma_prev);
   Guard guard = ctx->guard();
+  StateRounding sr = ctx->rounding();
   void* args[] = {&p,        &d_grads, &m,    &v, &d_ema, &chunks,  &n_chunks, &tensors,
-                  &partials, &cs,      &warm, &a, &st,    &counter, &index, &gamma_prev, &guard};
+                  &partials, &cs,      &warm, &a, &st,    &counter, &index, &gamma_prev, &guard, &sr};
   const void* fn = fused_small_kernel_of(ctx);
   if (cudaLaunchCooperativeKernel(fn, dim3(ctx->grid_fused), dim3(kThreads), args, 0, s) != cudaSuccess) {
     (void)cudaGetLastError();
@@ -2256,6 +2350,7 @@ int adagc_step_capturable(adagc_ctx* ctx, void* d_params, const void* d_grads, v
   rc = check_adamw_args(d_params, d_grads, d_m, d_v, lr, beta1, beta2, eps, wd);
   if (rc != ADAGC_OK) return rc;
   if (d_lr && (reinterpret_cast<uintptr_t>(d_lr) & 3u)) return ADAGC_E_MISALIGNED;
+  if (ctx->sr_stochastic) return ADAGC_E_INVALID_ARG;  // the generator's counter holds the step number, known on the host only
   cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
   DeviceStep* ds = reinterpret_cast<DeviceStep*>(ctx->ws + ctx->L.dev_step);
   StepHyper hh;
@@ -2509,6 +2604,14 @@ int adagc_debug_wait_timeout(adagc_ctx* ctx, double limit_ms, void* cuda_stream)
 int adagc_set_ema_cap(adagc_ctx* ctx, double cap) {
   if (!ctx || !(cap >= 0.0) || !std::isfinite(cap)) return ADAGC_E_INVALID_ARG;
   ctx->ema_cap = cap;
+  return ADAGC_OK;
+}
+
+int adagc_set_state_rounding(adagc_ctx* ctx, int32_t mode, uint64_t seed) {
+  if (!ctx || (mode != ADAGC_ROUND_NEAREST && mode != ADAGC_ROUND_STOCHASTIC)) return ADAGC_E_INVALID_ARG;
+  if (mode == ADAGC_ROUND_STOCHASTIC && !ctx->state_bf16) return ADAGC_E_DTYPE;
+  ctx->sr_stochastic = mode == ADAGC_ROUND_STOCHASTIC;
+  ctx->sr_seed = seed;
   return ADAGC_OK;
 }
 

@@ -508,7 +508,7 @@ def _assert_same_bf16(name: str, got_bits: np.ndarray, ref_bits: np.ndarray, wha
 
 def run_bf16_state(wl: workloads.Workload, n_steps: int, optimizer: str = "adamw", teacher_forced: bool = False,
                    device="cuda", flags: int = 0, hyper_over: Optional[dict] = None, lion_lr: float = 1e-4,
-                   sgd_lr: float = 1e-2) -> ParityReport:
+                   sgd_lr: float = 1e-2, stochastic_seed: Optional[int] = None) -> ParityReport:
     """Every element with m (and v) stored as bfloat16, GPU vs the C oracle's bfloat16-state functions.
 
     Which bfloat16 neighbour a moment is stored as is a discrete decision, taken on both sides in the precision the
@@ -520,12 +520,18 @@ def run_bf16_state(wl: workloads.Workload, n_steps: int, optimizer: str = "adamw
       teacher_forced  before every step the GPU's theta, m, v are overwritten with the oracle's stored state (inputs
                       flow oracle -> GPU only) and every step is compared from identical stored state.
     Lion's sign(c) near-ties may move theta by 2 lr per occurrence, as in run_full_lion.
+    stochastic_seed: the moments are rounded stochastically (adagc_set_state_rounding) with this seed; the random
+    numbers are a function of (seed, step, arena position) that both sides compute from the generator's published
+    definition, so the stored moments stay bit-identical.
     """
     hp = hyper_of(wl, **(hyper_over or {}))
     offs = np.array([t.offset for t in wl.tensors], np.int64)
     nums = np.array([t.numel for t in wl.tensors], np.int64)
     opt = binding.AdaGC(nums.tolist(), offs.tolist(), wl.torch_grad_dtype, hp["lambda_abs"], device=device, flags=flags,
                         state_dtype=torch.bfloat16)
+    if stochastic_seed is not None:
+        opt.set_state_rounding(True, stochastic_seed)
+    sto = dict(stochastic_seed=stochastic_seed)
     n_state = 2 if optimizer == "adamw" else 1
     assert optimizer != "sgdm" or teacher_forced, "momentum SGD's m depends on theta: compare it from identical state"
     theta = workloads.init_params(wl, device)
@@ -562,12 +568,13 @@ def run_bf16_state(wl: workloads.Workload, n_steps: int, optimizer: str = "adamw
         sl = slice(o, o + n)
         if optimizer == "adamw":
             c_oracle.adamw_update_bf16state(r_theta[sl], g_np[sl], r_m[sl], r_v[sl], h, t, lr, hp["beta1"], hp["beta2"],
-                                            hp["eps"], hp["wd"], fp32_decision=True)
+                                            hp["eps"], hp["wd"], fp32_decision=True, index0=o, **sto)
         elif optimizer == "lion":
             c_oracle.lion_update(r_theta[sl], g_np[sl], r_m[sl], h, lr, 0.9, 0.99, hp["wd"], near_tie=ties[sl],
-                                 tie_tol=LION_TIE_TOL, fp32_decision=True)
+                                 tie_tol=LION_TIE_TOL, fp32_decision=True, step=t, index0=o, **sto)
         else:
-            c_oracle.sgdm_update(r_theta[sl], g_np[sl], r_m[sl], h, lr, 0.9, hp["wd"], fp32_decision=True)
+            c_oracle.sgdm_update(r_theta[sl], g_np[sl], r_m[sl], h, lr, 0.9, hp["wd"], fp32_decision=True, step=t,
+                                 index0=o, **sto)
 
     def compare(t, ties):
         th, mb, vb = theta.cpu().numpy(), _bf16_view(m), _bf16_view(v)
@@ -619,7 +626,7 @@ def run_bf16_state(wl: workloads.Workload, n_steps: int, optimizer: str = "adamw
 
 
 def run_sampled_bf16_state(wl: workloads.Workload, n_steps: int, device="cuda", k: int = 2048,
-                           hyper_over: Optional[dict] = None) -> ParityReport:
+                           hyper_over: Optional[dict] = None, stochastic_seed: Optional[int] = None) -> ParityReport:
     """Full-size layouts with bfloat16 moments: all norms / decisions / gamma against the oracle, and theta, m, v on
     sampled elements that the oracle follows one by one (free-running; m and v bit-identical, theta within tolerance)."""
     hp = hyper_of(wl, **(hyper_over or {}))
@@ -627,11 +634,13 @@ def run_sampled_bf16_state(wl: workloads.Workload, n_steps: int, device="cuda", 
     nums = np.array([t.numel for t in wl.tensors], np.int64)
     opt = binding.AdaGC(nums.tolist(), offs.tolist(), wl.torch_grad_dtype, hp["lambda_abs"], device=device,
                         state_dtype=torch.bfloat16)
+    if stochastic_seed is not None:
+        opt.set_state_rounding(True, stochastic_seed)
     rng = np.random.RandomState(99)
     samp = [sample_indices(int(n), k, rng) + int(o) for o, n in zip(offs, nums)]
     sizes = np.array([len(s) for s in samp], np.int64)
     soff = np.concatenate([[0], np.cumsum(sizes)[:-1]]).astype(np.int64)
-    flat_np = np.concatenate(samp)
+    flat_np = np.ascontiguousarray(np.concatenate(samp), dtype=np.int64)
     flat = torch.from_numpy(flat_np).to(device)
     rep = ParityReport()
     gamma = np.zeros(wl.n_tensors, np.float32)
@@ -655,7 +664,8 @@ def run_sampled_bf16_state(wl: workloads.Workload, n_steps: int, device="cuda", 
         for i in range(wl.n_tensors):
             sl = slice(int(soff[i]), int(soff[i] + sizes[i]))
             c_oracle.adamw_update_bf16state(s_theta[sl], s_g[sl], s_m[sl], s_v[sl], float(r["h"][i]), t, hp["lr"],
-                                            hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], fp32_decision=True)
+                                            hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], fp32_decision=True,
+                                            stochastic_seed=stochastic_seed, index=np.ascontiguousarray(flat_np[sl]))
         rep.steps = t
         del g
     st = opt.get_stats()

@@ -88,6 +88,64 @@ def test_llama2_7b_sampled():
     _report("llama2_7b sampled, bf16 state", rep)
 
 
+# ------------------------------------------------------------------ stochastic rounding of the stored moments
+SEED = 0x5EED_0123_4567_89AB
+
+
+@pytest.mark.parametrize("path", [binding.UPDATE_PATH_REGISTERS, binding.UPDATE_PATH_BULK, binding.FUSED_SMALL],
+                         ids=["registers", "bulk", "one_kernel"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_stochastic_rounding_all_elements(dtype, path):
+    """adagc_set_state_rounding(STOCHASTIC): the stored moments are bit-identical to the oracle's, which draws the same
+    random numbers from its own Philox4x32-10 -- through full tiles, partial chunks and ragged tails."""
+    wl = _ragged_workload(SIZES, dtype)
+    for forced in (True, False):
+        _report(f"stochastic rounding {dtype} path {path} forced={forced}",
+                H.run_bf16_state(wl, 6, teacher_forced=forced, flags=path, stochastic_seed=SEED))
+    if path != binding.FUSED_SMALL:
+        for optimizer in ("lion", "sgdm"):
+            _report(f"stochastic rounding {optimizer} {dtype} path {path}",
+                    H.run_bf16_state(wl, 5, optimizer=optimizer, teacher_forced=True, flags=path, stochastic_seed=SEED + 1))
+
+
+def test_stochastic_rounding_larger_layouts_and_reproducibility():
+    wl = workloads.build("gpt2_small", n_layer=2, d=384, vocab=8000, n_pos=128)
+    _report("stochastic rounding, GPT-2-shaped (small)", H.run_bf16_state(wl, 12, stochastic_seed=SEED))
+    wl = workloads.build("many_small", n_tensors=2000, lo=8, hi=40000)
+    _report("stochastic rounding, 2000 small tensors", H.run_bf16_state(wl, 6, stochastic_seed=7, hyper_over=dict(lambda_abs=1e4)))
+    # same seed: same bits; another seed: other roundings; rounding mode of an fp32-state context cannot be changed
+    wl = _ragged_workload([5, 4096, 50001], "bf16")
+    hp = H.hyper_of(wl)
+    offs, nums = [t.offset for t in wl.tensors], [t.numel for t in wl.tensors]
+    args = (hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"], hp["beta"], hp["warmup"])
+    outs = []
+    for seed in (11, 11, 12):
+        opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], state_dtype=torch.bfloat16)
+        opt.set_state_rounding(True, seed)
+        theta, m, v, ema = _arenas(wl)
+        for t in range(1, 5):
+            opt.step(theta, workloads.grads_for_step(wl, t, "cuda"), m, v, ema, t, *args)
+        with pytest.raises(binding.AdagcError):
+            opt.step_capturable(theta, workloads.grads_for_step(wl, 5, "cuda"), m, v, ema, *args)
+        outs.append((m.view(torch.int16).clone(), v.view(torch.int16).clone()))
+        opt.close()
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+    assert (outs[0][0] != outs[2][0]).float().mean() > 0.1
+    plain = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"])
+    with pytest.raises(binding.AdagcError) as e:
+        plain.set_state_rounding(True, 1)
+    assert e.value.status == -5
+    plain.close()
+
+
+def test_llama2_7b_sampled_stochastic():
+    wl = workloads.build("llama2_7b")
+    free, _ = torch.cuda.mem_get_info()
+    if free < wl.arena_elems * 10 + (8 << 30):
+        pytest.skip("not enough free device memory for the 7B-shaped layout with bfloat16 state")
+    _report("llama2_7b sampled, bf16 state, stochastic rounding", H.run_sampled_bf16_state(wl, 4, stochastic_seed=SEED))
+
+
 def _arenas(wl, dev="cuda"):
     theta = workloads.init_params(wl, dev)
     m = torch.zeros(wl.arena_elems, dtype=torch.bfloat16, device=dev)

@@ -307,12 +307,12 @@ def time_layout(binding, workloads, wl, dev, steps, warm=3, state_dtype=torch.fl
            "whole_step_frac_of_nominal_8TBs": bpp * wl.n_params / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
            "l2": "flushed before every step" if small else "working set far larger than L2"}
     if fused_small and opt.n_chunks <= 4096:
-        # launch-latency-bound layouts: wall clock over back-to-back steps like a training loop, three launches against
-        # the one-kernel step (ADAGC_FUSED_SMALL)
+        # launch-latency-bound layouts: wall clock over back-to-back steps like a training loop, the default step (two
+        # launches) against the one-kernel step (ADAGC_FUSED_SMALL)
         fused = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=dev, flags=binding.FUSED_SMALL,
                               state_dtype=state_dtype)
         ema_f = torch.zeros_like(ema)
-        for name, o, e_ in (("three_launch_step_us_back_to_back", opt, ema), ("fused_small_step_us_back_to_back", fused, ema_f)):
+        for name, o, e_ in (("default_step_us_back_to_back", opt, ema), ("fused_small_step_us_back_to_back", fused, ema_f)):
             tt = 100
             for _ in range(20):
                 tt += 1

@@ -343,6 +343,7 @@ def run_full_lion(wl: workloads.Workload, n_steps: int, device="cuda", flags: in
             n_flipped += int((d > lr).sum())
     rep.max_tensor_rel["lion_near_tie_elements"] = n_ties
     rep.max_tensor_rel["lion_flipped_elements"] = n_flipped
+    assert n_flipped <= n_ties                    # (elements outside the near-tie set met the strict tolerance above)
     assert n_ties <= 1e-3 * wl.n_params + 50      # near-ties are rare: this is not a loophole for real errors
     opt.close()
     return rep

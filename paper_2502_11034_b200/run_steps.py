@@ -2,9 +2,17 @@
 
     python -m paper_2502_11034_b200.run_steps --workload gpt2_small --steps 4 [--mode step|clip|lion|sgdm] [--n-layer N]
         [--update-path auto|registers|bulk] [--fused-small] [--state f32|bf16] [--separate-finalize]
+        [--group-mb X [--graph]]
 
 A minimal driver of the C ABI (adagc_create / adagc_step / adagc_clip / adagc_get_stats): useful as
 an example and as a small, short-running target for profilers.  Prints the per-phase device times.
+
+--group-mb X runs the step group by group instead: consecutive tensors are gathered into groups of at least X MB of
+gradient, each group gets a context of its own over its slice of the arenas, and a step is norm -> decisions -> update
+of group 1, then of group 2, ...  With small groups the update's read of the gradient can hit in L2 (the norm pass of
+the same group has just read it), at the price of one set of launches per group; this mode exists to measure that
+trade (DRAM bytes and L2 hit rate of the update kernels under a profiler, step time with --graph, which replays the
+whole sequence as one CUDA graph so that no host time is in the measurement).  X = 0: one group, the same code path.
 """
 from __future__ import annotations
 
@@ -26,6 +34,8 @@ def main():
                     help="kernel of the update phase (adagc_desc.flags)")
     ap.add_argument("--fused-small", action="store_true",
                     help="ADAGC_FUSED_SMALL: adagc_step as one cooperative kernel (small layouts, --mode step)")
+    ap.add_argument("--group-mb", type=float, default=None, help="run the step group by group (see above)")
+    ap.add_argument("--graph", action="store_true", help="with --group-mb: time replays of one CUDA graph of the sequence")
     ap.add_argument("--state", choices=["f32", "bf16"], default="f32", help="dtype of the m and v arenas (adagc_desc.state_dtype)")
     ap.add_argument("--separate-finalize", action="store_true",
                     help="ADAGC_SEPARATE_FINALIZE: the per-tensor decisions of AdaGC steps in a kernel of their own")
@@ -43,6 +53,8 @@ def main():
     if args.separate_finalize:
         flags |= binding.SEPARATE_FINALIZE
     sd = torch.bfloat16 if args.state == "bf16" else torch.float32
+    if args.group_mb is not None:
+        return run_grouped(args, wl, dev, flags, sd)
     opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=dev, flags=flags, state_dtype=sd)
     theta = workloads.init_params(wl, dev)
     m = torch.zeros(wl.arena_elems, dtype=sd, device=dev)
@@ -68,6 +80,66 @@ def main():
     print(f"steps_done={st['steps_done']} clipped_last_step={int(st['flag'].sum())} status={st['status']} "
           f"kernels_launched={opt.launch_count()}")
     opt.close()
+
+
+def run_grouped(args, wl, dev, flags, sd):
+    hp = wl.hyper
+    esz = 2 if wl.grad_dtype == "bf16" else 4
+    groups, cur, cur_bytes = [], [], 0
+    for t in wl.tensors:
+        cur.append(t)
+        cur_bytes += t.numel * esz
+        if cur_bytes >= args.group_mb * (1 << 20) and args.group_mb > 0:
+            groups.append(cur)
+            cur, cur_bytes = [], 0
+    if cur:
+        groups.append(cur)
+    theta = workloads.init_params(wl, dev)
+    m = torch.zeros(wl.arena_elems, dtype=sd, device=dev)
+    v = torch.zeros_like(m)
+    g = workloads.grads_for_step(wl, 1, dev)
+    ctxs = []
+    for gr in groups:
+        lo, hi = gr[0].offset, gr[-1].offset + gr[-1].numel
+        opt = binding.AdaGC([t.numel for t in gr], [t.offset - lo for t in gr], wl.torch_grad_dtype, hp["lambda_abs"],
+                            device=dev, flags=flags, state_dtype=sd)
+        ema = torch.zeros(len(gr), dtype=torch.float32, device=dev)
+        ctxs.append((opt, theta[lo:hi], g[lo:hi], m[lo:hi], v[lo:hi], ema))
+    hyper = (hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"], hp["beta"], args.warmup)
+    big = max(sum(t.numel for t in gr) for gr in groups) * esz / (1 << 20)
+    print(f"{wl.name}: {len(groups)} group(s), largest {big:.1f} MB of gradient, {wl.n_params} params")
+
+    def step_all():
+        for opt, th_, g_, m_, v_, ema in ctxs:
+            opt.step_capturable(th_, g_, m_, v_, ema, *hyper)
+
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if args.graph:
+        for _ in range(2):
+            step_all()                                   # warm-up step(s) outside the graph
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            step_all()
+        times = []
+        for _ in range(args.steps):
+            e0.record()
+            graph.replay()
+            e1.record()
+            e1.synchronize()
+            times.append(e0.elapsed_time(e1))
+        times.sort()
+        print(f"graph replay of one step: median {times[len(times) // 2]:.4f} ms, min {times[0]:.4f} ms over {len(times)} replays")
+    else:
+        for k in range(args.steps):
+            e0.record()
+            step_all()
+            e1.record()
+            e1.synchronize()
+            print(f"step {k + 1}: {e0.elapsed_time(e1):.4f} ms (host-issued, {5 * len(groups)} launches)")
+    for c in ctxs:
+        assert c[0].get_stats()["status"] == 0
+        c[0].close()
 
 
 if __name__ == "__main__":

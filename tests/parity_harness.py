@@ -350,12 +350,12 @@ def run_full_lion(wl: workloads.Workload, n_steps: int, device="cuda", flags: in
 
 
 def run_full_clip(wl: workloads.Workload, n_steps: int, in_place: bool, device="cuda",
-                  hyper_over: Optional[dict] = None) -> ParityReport:
+                  hyper_over: Optional[dict] = None, flags: int = 0) -> ParityReport:
     """Clip-only entry, every element: clipped gradients in the gradient dtype vs the C oracle."""
     hp = hyper_of(wl, **(hyper_over or {}))
     offs = np.array([t.offset for t in wl.tensors], np.int64)
     nums = np.array([t.numel for t in wl.tensors], np.int64)
-    opt = binding.AdaGC(nums.tolist(), offs.tolist(), wl.torch_grad_dtype, hp["lambda_abs"], device=device)
+    opt = binding.AdaGC(nums.tolist(), offs.tolist(), wl.torch_grad_dtype, hp["lambda_abs"], device=device, flags=flags)
     ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device=device)
     gamma = np.zeros(wl.n_tensors, np.float32)
     rep = ParityReport()

@@ -198,6 +198,21 @@ def test_clip_only_small_layouts_all_elements(in_place):
 
 
 @pytest.mark.parametrize("path", [binding.UPDATE_PATH_REGISTERS, binding.UPDATE_PATH_BULK], ids=["registers", "bulk"])
+@pytest.mark.parametrize("in_place", [True, False], ids=["in_place", "out_of_place"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_clip_only_ragged(dtype, in_place, path):
+    """The clip-only entry on a ragged layout, in contexts of either update path: full and partial chunks, ragged tails,
+    tensors that are skipped in place because h == 1 between tensors that are not; padding between tensors must stay
+    untouched out of place."""
+    sizes = [1, 7, 8, 9, 255, 2049, 16383, 16384, 16385, 3 * 16384 + 5, 100003, 40 * 16384, 9 * 16384 + 4095, 6 * 16384,
+             16384, 5 * 16384 + 8]
+    wl = _ragged_workload(sizes, dtype)
+    rep = H.run_full_clip(wl, 8, in_place, flags=path, hyper_over=dict(lambda_abs=1e4, warmup=2))
+    _report(f"clip-only ragged {dtype} in_place={in_place} path {path}", rep)
+    assert 0 < rep.clipped < rep.decisions            # some tensors clipped, some passed through
+
+
+@pytest.mark.parametrize("path", [binding.UPDATE_PATH_REGISTERS, binding.UPDATE_PATH_BULK], ids=["registers", "bulk"])
 def test_emit_bf16_parameters_all_elements(path):
     """adagc_step_emit_bf16: fp32 master parameters plus the bf16 working copy from the same kernel."""
     sizes = [1, 7, 8, 9, 255, 2049, 16384, 16385, 3 * 16384 + 5, 40 * 16384, 100003]

@@ -82,9 +82,10 @@ typedef enum {
  * the same n_tensors-long vectors (gamma, sums of squares); the offset of an empty tensor is ignored. */
 #define ADAGC_ALLOW_EMPTY 16
 /* Small layouts: adagc_step runs as ONE kernel (norm, decisions and AdamW separated by grid-wide barriers inside a
- * cooperative launch) instead of three.  Worth it only where the three dependent launches cost more than the data
- * movement: measured on B200 it halves the step time below about 100 chunks of 16384 elements, breaks even near
- * 150 chunks (one per SM) and loses beyond; accepted for layouts of at most 4096 chunks (adagc_create
+ * cooperative launch) instead of two (four on warm-up steps).  Worth it only where the dependent launches cost more
+ * than the data movement: measured on B200 against a three-launch step it halved the step time below about 100 chunks
+ * of 16384 elements, broke even near 150 chunks (one per SM) and lost beyond (against today's two-launch step, 10.4
+ * instead of 16.5 us on a layout of 37 chunks); accepted for layouts of at most 4096 chunks (adagc_create
  * returns ADAGC_E_INVALID_ARG beyond that, with ADAGC_CLIP_GLOBAL_ADAPTIVE, or on a device without cooperative
  * launch).  Only adagc_step takes the fused route; every other entry point of the context is unchanged.  The
  * barriers wait with a time limit; if one gives up, ADAGC_E_TIMEOUT is set in the status word and the context must
@@ -189,7 +190,7 @@ int adagc_step(adagc_ctx* ctx, void* d_params, const void* d_grads, void* d_m, v
  *   - eta_t: if d_lr is not NULL it points to one fp32 value in DEVICE memory that is read at every execution
  *     (update it between replays to follow a schedule); if NULL the value `lr` is used.
  * The other arguments are those of adagc_step.  Five launches per step (prologue, norm, per-tensor
- * finalize, warm-up finalize -- which returns at once outside warm-up -- and update) instead of three.
+ * finalize, warm-up finalize -- which returns at once outside warm-up -- and update) instead of two.
  * Results agree with adagc_step's to the last bit whenever the device and host evaluations of beta^t round
  * to the same fp32 coefficients, and within the library's tolerance (1e-5) always.
  */
@@ -359,7 +360,9 @@ uint64_t adagc_launch_count(const adagc_ctx* ctx);
  * Optional per-phase timing.  When enabled, adagc_step / adagc_clip record CUDA events on the
  * caller's stream around the three phases (norm, finalize, update-or-scale).
  * adagc_get_phase_times synchronises on the last event and returns the durations in
- * milliseconds of the most recent step: ms[0] norm, ms[1] finalize, ms[2] update / scale.
+ * milliseconds of the most recent step: ms[0] norm, ms[1] finalize, ms[2] update / scale.  (On AdaGC steps the
+ * decisions are taken inside the norm kernel unless ADAGC_SEPARATE_FINALIZE is set: ms[0] then covers both and
+ * ms[1] is the empty interval between two events.)
  */
 int adagc_set_phase_timing(adagc_ctx* ctx, int enabled);
 int adagc_get_phase_times(adagc_ctx* ctx, float ms[3]);

@@ -529,7 +529,8 @@ def test_phase_timing_and_launch_count():
 
 
 @pytest.mark.parametrize("layout", ["mini", "gpt2_small"])
-def test_step_host_matches_device_entry(layout):
+@pytest.mark.parametrize("state", [torch.float32, torch.bfloat16], ids=["fp32_state", "bf16_state"])
+def test_step_host_matches_device_entry(layout, state):
     """The host-buffer entry gives bit-identical results; on the larger layout (several groups of tensors)
     its AdaGC steps run pipelined behind the host-to-device copies, its warm-up steps do not."""
     if layout == "mini":
@@ -542,9 +543,10 @@ def test_step_host_matches_device_entry(layout):
     args = (hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["wd"], hp["lambda_rel"], hp["beta"], hp["warmup"])
     outs = []
     for host in (False, True):
-        opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"])
+        opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], state_dtype=state)
         theta = workloads.init_params(wl, "cuda")
-        m, v = torch.zeros_like(theta), torch.zeros_like(theta)
+        m = torch.zeros(wl.arena_elems, dtype=state, device="cuda")
+        v = torch.zeros_like(m)
         ema = torch.zeros(wl.n_tensors, dtype=torch.float32, device="cuda")
         g_dev = torch.empty(wl.arena_elems, dtype=wl.torch_grad_dtype, device="cuda")
         norm = torch.empty(wl.n_tensors, dtype=torch.float32).pin_memory()
@@ -564,5 +566,6 @@ def test_step_host_matches_device_entry(layout):
         outs.append((theta, m, v, ema, torch.from_numpy(final["clip_count"].astype(np.int64))))
         opt.close()
     for x, y in zip(*outs):
-        assert torch.equal(x, y)
+        assert torch.equal(x.view(torch.int16) if x.dtype == torch.bfloat16 else x,
+                           y.view(torch.int16) if y.dtype == torch.bfloat16 else y)
     assert int(outs[0][4].sum()) > 0

@@ -47,9 +47,13 @@ NOMINAL_HBM_GBS = 8000.0
 # captures of the same kernel on smaller layouts (a multi-pass capture is not pointed at a 94 GB workload); scaled by the
 # parameter count because the traffic of this streaming kernel grows in proportion.  None once a kernel has changed
 # since its capture.
-TRAFFIC_BYTES_PER_PARAM = {
-    "bf16": (3177.385e6 / 124439808, "profiles/adagc_kernels_gpt2_small_ncu_full.md (GPT-2-small-shaped layout, scaled by N)"),
-    "f32": (16.04 + 11.71, "profiles/adagc_kernels_many_small_ncu_full.md (20 000 small tensors, scaled by N)"),
+TRAFFIC_BYTES_PER_PARAM = {   # (gradient dtype, state dtype) -> (bytes per parameter, capture)
+    ("bf16", "f32"): ((1742.393e6 + 1436.032e6) / 124439808,
+                      "profiles/adagc_kernels_gpt2_small_ncu_full.md (GPT-2-small-shaped layout, scaled by N)"),
+    ("bf16", "bf16"): ((1244.585e6 + 938.661e6) / 124439808,
+                       "profiles/adagc_kernels_gpt2_small_ncu_full.md (GPT-2-small-shaped layout, bfloat16 state, scaled by N)"),
+    ("f32", "f32"): ((3070.685e6 + 2244.835e6) / 191408576,
+                     "profiles/adagc_kernels_many_small_ncu_full.md (20 000 small tensors, scaled by N)"),
 }
 
 
@@ -306,6 +310,9 @@ def time_layout(binding, workloads, wl, dev, steps, warm=3, state_dtype=torch.fl
            "whole_step_frac_of_measured": bpp * wl.n_params / (ms * 1e-3) / 1e9 / peak,
            "whole_step_frac_of_nominal_8TBs": bpp * wl.n_params / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
            "l2": "flushed before every step" if small else "working set far larger than L2"}
+    t_bpp, t_src = TRAFFIC_BYTES_PER_PARAM.get((wl.grad_dtype, out["state_dtype"]), (None, None))
+    out["update_kernel_traffic"] = t_bpp * wl.n_params if t_bpp else None        # ncu DRAM bytes per launch, scaled by N
+    out["update_kernel_traffic_source"] = t_src
     if fused_small and opt.n_chunks <= 4096:
         # launch-latency-bound layouts: wall clock over back-to-back steps like a training loop, the default step (two
         # launches) against the one-kernel step (ADAGC_FUSED_SMALL)
@@ -420,7 +427,7 @@ def run_ours(args, wl):
     achieved = bpp * wl.n_params / (upd_ms * 1e-3) / 1e9
     norm_gbs = (bpp - 24) * wl.n_params / (norm_ms * 1e-3) / 1e9
     kernel = "adagc_update_tma_kernel" if opt.update_path == binding.UPDATE_PATH_BULK else "adagc_update_kernel"
-    traffic_bpp, traffic_src = TRAFFIC_BYTES_PER_PARAM.get(wl.grad_dtype, (None, None))
+    traffic_bpp, traffic_src = TRAFFIC_BYTES_PER_PARAM.get((wl.grad_dtype, "f32"), (None, None))
     if kernel != "adagc_update_tma_kernel":
         traffic_bpp, traffic_src = None, None
     whole_gbs = bpp * wl.n_params / step_s / 1e9

@@ -4,12 +4,14 @@
 //   1. norm      every fixed-size chunk of every gradient tensor -> one float64 partial sum of
 //                squares (Eq. 3 needs ||g_t,i||, Eq. 2 needs ||g_t||);
 //   2. finalize  per tensor: fixed-order sum of its partials -> norm -> clip factor h, flag and the
-//                gamma update (warm-up branch: global norm first, then min-seeding);
+//                gamma update (warm-up branch: global norm first, then min-seeding).  On AdaGC steps
+//                this phase runs in the tail of the norm kernel, so a step is two launches;
 //   3. update    every chunk again: g, theta, m, v read once, hat(g) = h * g kept on chip,
-//                AdamW lines of Algorithm 1 (or Lion's rule), theta, m, v written once.  Two kernels:
-//                a bulk-async one (cp.async.bulk + mbarrier ring through shared memory, the default)
-//                and a register-streaming one.
-// This is pure streaming work (26..28 bytes per parameter, ~20 flops): the bound is HBM bandwidth,
+//                AdamW lines of Algorithm 1 (or Lion's rule, or momentum SGD), theta, m, v written
+//                once; m and v are fp32 or bfloat16 arenas.  Two kernels: a bulk-async one
+//                (cp.async.bulk + mbarrier ring through shared memory, the default) and a
+//                register-streaming one.
+// This is pure streaming work (18..28 bytes per parameter, ~20 flops): the bound is HBM bandwidth,
 // so the kernels are built around large coalesced transfers, a measured amount of loads in flight
 // per SM and streaming cache hints; there is no contraction here and tensor cores are not used.
 //

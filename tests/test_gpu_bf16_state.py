@@ -146,6 +146,14 @@ def test_llama2_7b_sampled_stochastic():
     _report("llama2_7b sampled, bf16 state, stochastic rounding", H.run_sampled_bf16_state(wl, 4, stochastic_seed=SEED))
 
 
+def test_llama32_1b_sampled_both_rounding_modes():
+    """Config 5 at full size (heavy-tailed gradients, 5 % of the tensors spiked every step, warm-up of 10 steps with
+    global-norm clipping): all decisions, sampled elements of theta and of the bfloat16 m, v."""
+    wl = workloads.build("llama32_1b")
+    _report("llama32_1b sampled, bf16 state", H.run_sampled_bf16_state(wl, 30))
+    _report("llama32_1b sampled, bf16 state, stochastic rounding", H.run_sampled_bf16_state(wl, 14, stochastic_seed=SEED))
+
+
 def _arenas(wl, dev="cuda"):
     theta = workloads.init_params(wl, dev)
     m = torch.zeros(wl.arena_elems, dtype=torch.bfloat16, device=dev)

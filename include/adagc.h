@@ -340,6 +340,11 @@ int adagc_set_ema_cap(adagc_ctx* ctx, double cap);
  *                           counter (lo q, hi q, lo step, hi step) and key (lo seed, hi seed); element 4q + l takes
  *                           output word l, its low half for m, its high half for v.  The result therefore depends on
  *                           (seed, step, element position) only: reruns and restarts reproduce it bit for bit.
+ *                           In this mode (and only in it, and only for eps >= 1e-30) theta's increment
+ *                           m_hat / (sqrt(v_hat) + eps) is taken with the approximate square root and reciprocal
+ *                           (relative error of a few 1e-7, subnormal v_hat flushed to zero) instead of the correctly
+ *                           rounded ones: the random numbers make the kernel instruction-bound otherwise, and the
+ *                           moments already carry a random relative error of 2^-9.  The stored moments are unaffected.
  * Host-only; takes effect from the next step.  ADAGC_E_DTYPE if the context's state is fp32.  adagc_step_capturable
  * returns ADAGC_E_INVALID_ARG while stochastic rounding is on (its step number lives on the device).
  */

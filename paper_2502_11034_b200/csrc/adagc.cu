@@ -774,9 +774,24 @@ constexpr int kOptAdamW = 0;
 constexpr int kOptLion = 1;
 constexpr int kOptSgdM = 2;  // heavy-ball SGD: d = hat(g) + wd theta, m = momentum m + d, theta -= lr m (no v)
 
+// The quotient m_hat / (sqrt(v_hat) + eps) by the approximate square root and reciprocal (subnormals flushed), four
+// instructions instead of about twenty.  Used only where the moments are rounded stochastically to bfloat16: there
+// the update already carries a random relative error of 2^-9 per moment, the kernel is bound by instruction issue (the
+// random numbers cost about 22 instructions per element), and a few 1e-7 more on theta's increment are invisible.
+__device__ __forceinline__ float quotient_approx(float m, float v_hat, float eps) {
+  float s, r;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(s) : "f"(v_hat));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(s + eps));
+  return m * r;
+}
+// (a subnormal v_hat is flushed to zero, which is harmless as long as eps is not itself vanishing)
+__device__ __forceinline__ bool use_quotient_approx(const StateRounding* sr, const AdamScalars& a) {
+  return sr != nullptr && sr->stochastic && a.eps >= 1e-30f;
+}
+
 template <int kOpt>
 __device__ __forceinline__ void adamw_elem(float g, float h, float& p, float& m, float& v,
-                                           const AdamScalars& a) {
+                                           const AdamScalars& a, bool fast = false) {
   const float gh = h * g;  // hat(g)
   if (kOpt == kOptLion) {
     // fp32 like the rest of the update; where the two terms nearly cancel the sign is a near-tie
@@ -791,18 +806,23 @@ __device__ __forceinline__ void adamw_elem(float g, float h, float& p, float& m,
   } else {
     m = fmaf(a.beta1, m, a.one_minus_beta1 * gh);
     v = fmaf(a.beta2, v, a.one_minus_beta2 * (gh * gh));
-    const float denom = __fsqrt_rn(v * a.inv_bc2) + a.eps;  // sqrt(v_hat) + eps
-    p = fmaf(-a.step_size, __fdiv_rn(m, denom), p * a.decay);
+    if (fast) {
+      p = fmaf(-a.step_size, quotient_approx(m, v * a.inv_bc2, a.eps), p * a.decay);
+    } else {
+      const float denom = __fsqrt_rn(v * a.inv_bc2) + a.eps;  // sqrt(v_hat) + eps
+      p = fmaf(-a.step_size, __fdiv_rn(m, denom), p * a.decay);
+    }
   }
 }
 
 template <int kOpt>
 __device__ __forceinline__ void adamw_vec4(const float g0, const float g1, const float g2, const float g3,
-                                           float h, float4& p, float4& m, float4& v, const AdamScalars& a) {
-  adamw_elem<kOpt>(g0, h, p.x, m.x, v.x, a);
-  adamw_elem<kOpt>(g1, h, p.y, m.y, v.y, a);
-  adamw_elem<kOpt>(g2, h, p.z, m.z, v.z, a);
-  adamw_elem<kOpt>(g3, h, p.w, m.w, v.w, a);
+                                           float h, float4& p, float4& m, float4& v, const AdamScalars& a,
+                                           bool fast = false) {
+  adamw_elem<kOpt>(g0, h, p.x, m.x, v.x, a, fast);
+  adamw_elem<kOpt>(g1, h, p.y, m.y, v.y, a, fast);
+  adamw_elem<kOpt>(g2, h, p.z, m.z, v.z, a, fast);
+  adamw_elem<kOpt>(g3, h, p.w, m.w, v.w, a, fast);
 }
 
 // Optimizer state (m, v) is stored as fp32 or as bfloat16 (kSB); arithmetic is fp32 either way.  A stored bfloat16
@@ -886,8 +906,9 @@ __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gba
   load_state8<kSB>(mbase, i, ma, mb);
   float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
   if (kOpt == kOptAdamW) load_state8<kSB>(vbase, i, va, vb);
-  adamw_vec4<kOpt>(g[0], g[1], g[2], g[3], h, pa, ma, va, a);
-  adamw_vec4<kOpt>(g[4], g[5], g[6], g[7], h, pb, mb, vb, a);
+  const bool fast = kSB && use_quotient_approx(sr, a);
+  adamw_vec4<kOpt>(g[0], g[1], g[2], g[3], h, pa, ma, va, a, fast);
+  adamw_vec4<kOpt>(g[4], g[5], g[6], g[7], h, pb, mb, vb, a, fast);
   st_stream(p4 + 2 * i, pa); st_stream(p4 + 2 * i + 1, pb);
   if (kSB && sr && sr->stochastic) {  // q0: arena index / 4 of the chunk's first element; this group is elements 8i .. 8i+7
     const uint4 wa = rounding_words(q0 + 2 * i, *sr), wb = rounding_words(q0 + 2 * i + 1, *sr);
@@ -940,7 +961,7 @@ __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, in
     }
     float p = params[start + t], m = load_state1<kSB>(mbase, t), v = 0.0f;
     if (kOpt == kOptAdamW) v = load_state1<kSB>(vbase, t);
-    adamw_elem<kOpt>(g, h, p, m, v, a);
+    adamw_elem<kOpt>(g, h, p, m, v, a, kSB && use_quotient_approx(sr, a));
     params[start + t] = p;
     if (kSB && sr && sr->stochastic) {
       store_state1_stochastic(mbase, t, m, start + t, *sr, 0);
@@ -1220,7 +1241,7 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
           }
           float4 p = p4[q], m = smem_state4<kSB>(b + kMOff, q), v = make_float4(0.f, 0.f, 0.f, 0.f);
           if (kOpt == kOptAdamW) v = smem_state4<kSB>(b + kVOff, q);
-          adamw_vec4<kOpt>(g0, g1, g2, g3, h, p, m, v, a);
+          adamw_vec4<kOpt>(g0, g1, g2, g3, h, p, m, v, a, kSB && use_quotient_approx(&sr, a));
           p4[q] = p;
           if (kSB && sr.stochastic) {  // elements 4q .. 4q+3 of this tile: one group of the arenas
             const uint4 w = rounding_words((chunk_start(ck) >> 2) + sub * (kTile / 4) + q, sr);

@@ -31,6 +31,7 @@
 #include <mutex>
 #include <new>
 #include <queue>
+#include <type_traits>
 #include <utility>
 #include <vector>
 
@@ -1229,30 +1230,37 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
       unsigned char* b = tile_smem + static_cast<size_t>(s) * stage_stride;
       if (mbar_wait_bounded(&full_bar[s], phase)) {
         float4* p4 = reinterpret_cast<float4*>(b);
+        // one copy of the loop per rounding mode, so that rounding to nearest carries none of the other mode's code
+        auto update_tile = [&](auto stochastic_tag) {
+          constexpr bool kStochastic = decltype(stochastic_tag)::value;
+          const bool fast = kStochastic && use_quotient_approx(&sr, a);
 #pragma unroll
-        for (int q = tid; q < kTile / 4; q += kTmaThreads) {
-          float g0, g1, g2, g3;
-          if (kBF16) {
-            const uint2 w = reinterpret_cast<const uint2*>(b + kGOff)[q];
-            g0 = bf16_lo(w.x); g1 = bf16_hi(w.x); g2 = bf16_lo(w.y); g3 = bf16_hi(w.y);
-          } else {
-            const float4 w = reinterpret_cast<const float4*>(b + kGOff)[q];
-            g0 = w.x; g1 = w.y; g2 = w.z; g3 = w.w;
+          for (int q = tid; q < kTile / 4; q += kTmaThreads) {
+            float g0, g1, g2, g3;
+            if (kBF16) {
+              const uint2 w = reinterpret_cast<const uint2*>(b + kGOff)[q];
+              g0 = bf16_lo(w.x); g1 = bf16_hi(w.x); g2 = bf16_lo(w.y); g3 = bf16_hi(w.y);
+            } else {
+              const float4 w = reinterpret_cast<const float4*>(b + kGOff)[q];
+              g0 = w.x; g1 = w.y; g2 = w.z; g3 = w.w;
+            }
+            float4 p = p4[q], m = smem_state4<kSB>(b + kMOff, q), v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (kOpt == kOptAdamW) v = smem_state4<kSB>(b + kVOff, q);
+            adamw_vec4<kOpt>(g0, g1, g2, g3, h, p, m, v, a, fast);
+            p4[q] = p;
+            if (kStochastic) {  // elements 4q .. 4q+3 of this tile: one group of the arenas
+              const uint4 w = rounding_words((chunk_start(ck) >> 2) + sub * (kTile / 4) + q, sr);
+              reinterpret_cast<uint2*>(b + kMOff)[q] = pack4_stochastic(m, w, 0);
+              if (kOpt == kOptAdamW) reinterpret_cast<uint2*>(b + kVOff)[q] = pack4_stochastic(v, w, 1);
+            } else {
+              smem_state4_store<kSB>(b + kMOff, q, m);
+              if (kOpt == kOptAdamW) smem_state4_store<kSB>(b + kVOff, q, v);
+            }
+            if (lowp) reinterpret_cast<uint2*>(b + kStageBytes)[q] = make_uint2(pack_bf16(p.x, p.y), pack_bf16(p.z, p.w));
           }
-          float4 p = p4[q], m = smem_state4<kSB>(b + kMOff, q), v = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (kOpt == kOptAdamW) v = smem_state4<kSB>(b + kVOff, q);
-          adamw_vec4<kOpt>(g0, g1, g2, g3, h, p, m, v, a, kSB && use_quotient_approx(&sr, a));
-          p4[q] = p;
-          if (kSB && sr.stochastic) {  // elements 4q .. 4q+3 of this tile: one group of the arenas
-            const uint4 w = rounding_words((chunk_start(ck) >> 2) + sub * (kTile / 4) + q, sr);
-            reinterpret_cast<uint2*>(b + kMOff)[q] = pack4_stochastic(m, w, 0);
-            if (kOpt == kOptAdamW) reinterpret_cast<uint2*>(b + kVOff)[q] = pack4_stochastic(v, w, 1);
-          } else {
-            smem_state4_store<kSB>(b + kMOff, q, m);
-            if (kOpt == kOptAdamW) smem_state4_store<kSB>(b + kVOff, q, v);
-          }
-          if (lowp) reinterpret_cast<uint2*>(b + kStageBytes)[q] = make_uint2(pack_bf16(p.x, p.y), pack_bf16(p.z, p.w));
-        }
+        };
+        if (kSB && sr.stochastic) update_tile(std::true_type{});
+        else update_tile(std::false_type{});
         fence_generic_to_async_smem();  // the updated tile must be visible to the bulk-copy engine
       } else {
         abort_flag = 1;  // this thread gave up; the barrier below tells every thread

@@ -1,7 +1,7 @@
 """Run a few fused AdaGC + AdamW steps (or clip-only steps) on a named synthetic layout.
 
     python -m paper_2502_11034_b200.run_steps --workload gpt2_small --steps 4 [--mode step|clip|lion|sgdm] [--n-layer N]
-        [--update-path auto|registers|bulk] [--fused-small] [--state f32|bf16] [--separate-finalize]
+        [--update-path auto|registers|bulk] [--fused-small] [--state f32|bf16 [--stochastic-seed S]] [--separate-finalize]
         [--group-mb X [--graph]]
 
 A minimal driver of the C ABI (adagc_create / adagc_step / adagc_clip / adagc_get_stats): useful as
@@ -37,6 +37,8 @@ def main():
     ap.add_argument("--group-mb", type=float, default=None, help="run the step group by group (see above)")
     ap.add_argument("--graph", action="store_true", help="with --group-mb: time replays of one CUDA graph of the sequence")
     ap.add_argument("--state", choices=["f32", "bf16"], default="f32", help="dtype of the m and v arenas (adagc_desc.state_dtype)")
+    ap.add_argument("--stochastic-seed", type=int, default=None,
+                    help="with --state bf16: round the stored moments stochastically (adagc_set_state_rounding)")
     ap.add_argument("--separate-finalize", action="store_true",
                     help="ADAGC_SEPARATE_FINALIZE: the per-tensor decisions of AdaGC steps in a kernel of their own")
     args = ap.parse_args()
@@ -56,6 +58,8 @@ def main():
     if args.group_mb is not None:
         return run_grouped(args, wl, dev, flags, sd)
     opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, hp["lambda_abs"], device=dev, flags=flags, state_dtype=sd)
+    if args.stochastic_seed is not None:
+        opt.set_state_rounding(True, args.stochastic_seed)
     theta = workloads.init_params(wl, dev)
     m = torch.zeros(wl.arena_elems, dtype=sd, device=dev)
     v = torch.zeros_like(m)

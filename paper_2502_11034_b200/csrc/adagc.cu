@@ -277,40 +277,67 @@ __device__ __forceinline__ bool block_entries_ok(const Chunk* __restrict__ chunk
 // fixed-order sum of the warp totals.  The result is valid in thread 0.  Ends with a barrier, so
 // `warp_part` can be reused at once.
 // kKeepInL2: load with the evict_last policy (the step's norm phase, whose gradient is read again by the update).
+// One 16-byte vector of gradients added to a thread's two accumulators (components alternate between them).
+template <bool kBF16>
+__device__ __forceinline__ void sq_acc_vec(const uint4& q, double& acc0, double& acc1) {
+  if (kBF16) {
+    acc0 = sq_acc(acc0, bf16_lo(q.x));
+    acc1 = sq_acc(acc1, bf16_hi(q.x));
+    acc0 = sq_acc(acc0, bf16_lo(q.y));
+    acc1 = sq_acc(acc1, bf16_hi(q.y));
+    acc0 = sq_acc(acc0, bf16_lo(q.z));
+    acc1 = sq_acc(acc1, bf16_hi(q.z));
+    acc0 = sq_acc(acc0, bf16_lo(q.w));
+    acc1 = sq_acc(acc1, bf16_hi(q.w));
+  } else {
+    acc0 = sq_acc(acc0, __uint_as_float(q.x));
+    acc1 = sq_acc(acc1, __uint_as_float(q.y));
+    acc0 = sq_acc(acc0, __uint_as_float(q.z));
+    acc1 = sq_acc(acc1, __uint_as_float(q.w));
+  }
+}
+
+// kRounds rounds of the block over the vectors from `base` on: thread tid takes base + u * kThreads + tid, u = 0 ..
+// kRounds - 1, all loads issued before the first addition.  Every vector exists (the caller checks).
+template <bool kBF16, bool kKeepInL2, int kRounds>
+__device__ __forceinline__ void sq_acc_rounds(const uint4* __restrict__ vec, int base, uint64_t keep, double& acc0,
+                                              double& acc1) {
+  uint4 q[kRounds];
+#pragma unroll
+  for (int u = 0; u < kRounds; ++u) {
+    const uint4* ptr = vec + base + u * kThreads + threadIdx.x;
+    q[u] = kKeepInL2 ? ld_nc_l2_hint(ptr, keep) : __ldg(ptr);
+  }
+#pragma unroll
+  for (int u = 0; u < kRounds; ++u) sq_acc_vec<kBF16>(q[u], acc0, acc1);
+}
+
 template <bool kBF16, bool kKeepInL2 = false>
 __device__ __forceinline__ double block_chunk_sumsq(const uint4* __restrict__ vec, int count, double* warp_part) {
   constexpr int kEPV = kBF16 ? 8 : 4;  // elements per 16-byte vector
-  constexpr int kUnroll = 8;           // independent 16-byte loads in flight per thread
   const int tid = threadIdx.x;
   const int nvec = count / kEPV;
   double acc0 = 0.0, acc1 = 0.0;
   const uint64_t keep = kKeepInL2 ? l2_policy_evict_last() : 0ull;
-  for (int base = 0; base < nvec; base += kThreads * kUnroll) {
-    uint4 q[kUnroll];
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      const int i = base + u * kThreads + tid;
-      q[u] = (i < nvec) ? (kKeepInL2 ? ld_nc_l2_hint(vec + i, keep) : __ldg(vec + i)) : make_uint4(0u, 0u, 0u, 0u);
-    }
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      if (kBF16) {
-        acc0 = sq_acc(acc0, bf16_lo(q[u].x));
-        acc1 = sq_acc(acc1, bf16_hi(q[u].x));
-        acc0 = sq_acc(acc0, bf16_lo(q[u].y));
-        acc1 = sq_acc(acc1, bf16_hi(q[u].y));
-        acc0 = sq_acc(acc0, bf16_lo(q[u].z));
-        acc1 = sq_acc(acc1, bf16_hi(q[u].z));
-        acc0 = sq_acc(acc0, bf16_lo(q[u].w));
-        acc1 = sq_acc(acc1, bf16_hi(q[u].w));
-      } else {
-        acc0 = sq_acc(acc0, __uint_as_float(q[u].x));
-        acc1 = sq_acc(acc1, __uint_as_float(q[u].y));
-        acc0 = sq_acc(acc0, __uint_as_float(q[u].z));
-        acc1 = sq_acc(acc1, __uint_as_float(q[u].w));
-      }
-    }
+  // Every thread adds its vectors (tid, tid + kThreads, ...) in increasing order.  Eight rounds at a time keep eight
+  // independent loads per thread in flight; what is left after the last full eight goes in batches of four, two
+  // and one round and a last, partial round, so that a short chunk executes instructions for its own vectors only
+  // (the norm of a layout of many small tensors is bound by instruction issue, not by memory).
+  int base = 0;
+  for (; base + 8 * kThreads <= nvec; base += 8 * kThreads) sq_acc_rounds<kBF16, kKeepInL2, 8>(vec, base, keep, acc0, acc1);
+  if (base + 4 * kThreads <= nvec) {
+    sq_acc_rounds<kBF16, kKeepInL2, 4>(vec, base, keep, acc0, acc1);
+    base += 4 * kThreads;
   }
+  if (base + 2 * kThreads <= nvec) {
+    sq_acc_rounds<kBF16, kKeepInL2, 2>(vec, base, keep, acc0, acc1);
+    base += 2 * kThreads;
+  }
+  if (base + kThreads <= nvec) {
+    sq_acc_rounds<kBF16, kKeepInL2, 1>(vec, base, keep, acc0, acc1);
+    base += kThreads;
+  }
+  if (base + tid < nvec) sq_acc_rounds<kBF16, kKeepInL2, 1>(vec, base, keep, acc0, acc1);
   // ragged tail of a tensor's last chunk (fewer than one vector)
   const int t = nvec * kEPV + tid;
   if (t < count) {
@@ -928,6 +955,7 @@ __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gba
 // elements) and the rows of successive chunks go to the block's warps in one continuing round-robin:
 // row_base counts the rows dealt so far.  Restarting at warp 0 for every chunk would give the low warps
 // the extra rows every time and make them the critical path.
+constexpr int kRowAlign = 256;  // elements
 template <bool kBF16, int kBlockThreads, int kOpt, bool kSB>
 __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, int& row_base, float* __restrict__ params,
                                                     const void* __restrict__ grads, void* __restrict__ m_arena,
@@ -938,20 +966,27 @@ __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, in
   constexpr int kStateBytes = kSB ? 2 : 4;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int64_t start = chunk_start(ck);
-  float4* __restrict__ p4 = reinterpret_cast<float4*>(params + start);
-  char* __restrict__ mbase = static_cast<char*>(m_arena) + start * kStateBytes;
-  char* __restrict__ vbase = kOpt == kOptAdamW ? static_cast<char*>(v_arena) + start * kStateBytes : nullptr;
-  const char* __restrict__ gbase = static_cast<const char*>(grads) + start * (kBF16 ? 2 : 4);
-  const int n8 = ck.count >> 3;
-  const int rows = (n8 + 31) >> 5;
+  // Rows of 256 elements are laid from the last kRowAlign-element boundary at or before the chunk's start, so that a
+  // warp's accesses fall on whole lines whatever the tensor's offset; the groups before the start are skipped.
+  const int pad = static_cast<int>(start & (kRowAlign - 1));  // a multiple of 8, like start
+  const int64_t origin = start - pad;
+  float4* __restrict__ p4 = reinterpret_cast<float4*>(params + origin);
+  char* __restrict__ mbase = static_cast<char*>(m_arena) + origin * kStateBytes;
+  char* __restrict__ vbase = kOpt == kOptAdamW ? static_cast<char*>(v_arena) + origin * kStateBytes : nullptr;
+  const char* __restrict__ gbase = static_cast<const char*>(grads) + origin * (kBF16 ? 2 : 4);
+  const int first8 = pad >> 3, n8 = ck.count >> 3;
+  const int rows = (first8 + n8 + 31) >> 5;
 #pragma unroll 2
   for (int r = (warp - row_base) & (kWarps - 1); r < rows; r += kWarps) {
     const int i = (r << 5) + lane;
-    if (i < n8)
-      adamw_group8<kBF16, kOpt, kSB>(i, gbase, p4, mbase, vbase, h, a, lowp ? reinterpret_cast<uint4*>(lowp + start) : nullptr,
-                                     sr, start >> 2);
+    if (i >= first8 && i < first8 + n8)
+      adamw_group8<kBF16, kOpt, kSB>(i, gbase, p4, mbase, vbase, h, a, lowp ? reinterpret_cast<uint4*>(lowp + origin) : nullptr,
+                                     sr, origin >> 2);
   }
   row_base = (row_base + rows) & (kWarps - 1);
+  gbase += static_cast<int64_t>(pad) * (kBF16 ? 2 : 4);  // the tail below counts from the chunk's start
+  mbase += static_cast<int64_t>(pad) * kStateBytes;
+  if (kOpt == kOptAdamW) vbase += static_cast<int64_t>(pad) * kStateBytes;
   const int t = (n8 << 3) + lane;  // ragged tail (fewer than 8 elements): the next warp in turn takes it
   if (warp == row_base && t < ck.count) {
     float g;
@@ -1033,7 +1068,13 @@ adagc_update_kernel(float* __restrict__ params, const void* __restrict__ grads, 
 // per-tile costs (barrier wait, block barrier, issue) weigh more: measured on the 7B-shaped layout, tiles of
 // 2048 / 4096 / 8192 elements in two stages gave 5060 / 5650 / 6050 GB/s, more stages never helped (4096 x 3:
 // 5700, 4096 x 4: 5670), and rounding with the conversion instruction instead of integer arithmetic took
-// 8192 x 2 to 6650 GB/s.  Partial chunks take the register path afterwards.
+// 8192 x 2 to 6650 GB/s.
+// Partial chunks (a tensor's last, shorter chunk) come after the block's whole tiles.  With fp32 state they take the
+// register path, which on its own reaches the whole tiles' rate down to chunks of about 2000 elements.  With
+// bfloat16 state the register path is the slower one (5300 - 5500 GB/s), so there the partial chunks of at least half a
+// tile go through the same ring, cut into tiles of their own length (measured on layouts of equal tensors of 12288 /
+// 8192 / 6144 / 4096 elements: 6300 / 5950 / 6100 / 5460 GB/s against 5500 / 5380 / 5340 / 5290), and only shorter
+// ones, and every chunk's last count mod 8 elements, are left to the register path.
 // Every wait is bounded: after ~2 s without completion the block records ADAGC_E_TIMEOUT in the
 // status word and leaves its remaining tiles untouched.
 // ------------------------------------------------------------------------------------------------
@@ -1179,19 +1220,99 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     abort_flag = 0;
   }
+  // The larger partial chunks go through the ring too (after the full chunks), in tiles of their own length; the
+  // block lists them here, in table order, one candidate entry per thread.  Entries past the first kRingList
+  // partial chunks, chunks shorter than kRingMin and the last (count mod 8) elements of a listed chunk take the
+  // register path at the end.  (The list is kept small: with fp32 gradients, bfloat16 state and a bfloat16 copy
+  // of the parameters the ring itself takes 224 of the 227 KB a block may have.)
+  constexpr bool kRingPartials = kSB;  // fp32 state: none, the register path is the faster one there (kernel header)
+  constexpr int kRingMin = kTile / 2, kRingList = 256;
+  static_assert(kRingList <= kTmaThreads && kChunkElems <= 65536, "one candidate per thread; lengths fit 16 bits");
+  static_assert(kStages * (kStageBytes + kTile * 2) + kRingList * 10 + 256 <= kMaxDynamicSmem, "ring and list fit");
+  __shared__ uint32_t ring_start4[kRingList];
+  __shared__ uint32_t ring_tensor_or_h[kRingList];  // the owning tensor until the clip factors are read, then the factor
+  __shared__ uint16_t ring_n8[kRingList];
+  __shared__ int ring_warp_count[kTmaThreads / 32];
+  const int listed_end = min(end, mid + kRingList);  // entries [mid, listed_end) are the candidates
+  int n_listed = 0;
+  if (kRingPartials) {
+    const int c = mid + tid;
+    Chunk cand{0u, 0, 0, 0};
+    if (c < listed_end) cand = chunks[c];
+    const bool take = (cand.count & ~7) >= kRingMin;
+    const unsigned takers = __ballot_sync(0xffffffffu, take);
+    if ((tid & 31) == 0) ring_warp_count[tid >> 5] = __popc(takers);
+    __syncthreads();
+    int before = 0;
+    for (int w = 0; w < kTmaThreads / 32; ++w) {
+      const int n_w = ring_warp_count[w];
+      if (w < (tid >> 5)) before += n_w;
+      n_listed += n_w;
+    }
+    if (take) {
+      const int pos = before + __popc(takers & ((1u << (tid & 31)) - 1u));
+      ring_start4[pos] = cand.start4;
+      ring_n8[pos] = static_cast<uint16_t>(cand.count & ~7);
+      ring_tensor_or_h[pos] = static_cast<uint32_t>(cand.tensor);
+    }
+  }
   __syncthreads();
 
   const uint64_t stream_policy = l2_policy_evict_first();  // every byte this kernel moves is used once
-  // thread 0 only: start the loads of one tile (tile `sub` of the chunk that starts at element e0)
-  auto issue_tile = [&](int64_t e0, int sub, int s) {
-    const int64_t e = e0 + static_cast<int64_t>(sub) * kTile;
+  // thread 0 only: start the loads of n elements from arena element e into stage s (n a multiple of 8: every copy
+  // is then a multiple of 16 bytes and starts on a 16-byte boundary)
+  auto issue_span = [&](int64_t e, int n, int s) {
     unsigned char* b = tile_smem + static_cast<size_t>(s) * stage_stride;
-    mbar_arrive_expect_tx(&full_bar[s], kStageBytes);
-    bulk_load_hint(b, params + e, kTile * 4, &full_bar[s], stream_policy);
-    bulk_load_hint(b + kMOff, static_cast<const char*>(m_arena) + e * kSBytes, kTile * kSBytes, &full_bar[s], stream_policy);
+    mbar_arrive_expect_tx(&full_bar[s], static_cast<uint32_t>(n) * tma_elem_bytes(kBF16, kOpt, kSB));
+    bulk_load_hint(b, params + e, n * 4, &full_bar[s], stream_policy);
+    bulk_load_hint(b + kMOff, static_cast<const char*>(m_arena) + e * kSBytes, n * kSBytes, &full_bar[s], stream_policy);
     if (kOpt == kOptAdamW)
-      bulk_load_hint(b + kVOff, static_cast<const char*>(v_arena) + e * kSBytes, kTile * kSBytes, &full_bar[s], stream_policy);
-    bulk_load_hint(b + kGOff, static_cast<const char*>(grads) + e * kGBytes, kTile * kGBytes, &full_bar[s], stream_policy);
+      bulk_load_hint(b + kVOff, static_cast<const char*>(v_arena) + e * kSBytes, n * kSBytes, &full_bar[s], stream_policy);
+    bulk_load_hint(b + kGOff, static_cast<const char*>(grads) + e * kGBytes, n * kGBytes, &full_bar[s], stream_policy);
+  };
+  // tile `sub` of the full chunk that starts at element e0
+  auto issue_tile = [&](int64_t e0, int sub, int s) { issue_span(e0 + static_cast<int64_t>(sub) * kTile, kTile, s); };
+  // thread 0 only: write the updated streams of a stage back and commit them as one group
+  auto store_span = [&](int64_t e, int n, unsigned char* b) {
+    bulk_store_hint(params + e, b, n * 4, stream_policy);
+    bulk_store_hint(static_cast<char*>(m_arena) + e * kSBytes, b + kMOff, n * kSBytes, stream_policy);
+    if (kOpt == kOptAdamW) bulk_store_hint(static_cast<char*>(v_arena) + e * kSBytes, b + kVOff, n * kSBytes, stream_policy);
+    if (lowp) bulk_store_hint(lowp + e, b + kStageBytes, n * 2, stream_policy);
+    bulk_commit();
+  };
+  // all threads: update the groups of four elements of one stage in place.  One copy of the loop per rounding mode,
+  // so that rounding to nearest carries none of the other mode's code, and per tile kind, so that a whole tile's
+  // trip count is a constant.  group0 is the arena index, in groups of four, of the stage's first element.
+  auto update_tile = [&](auto stochastic_tag, auto whole_tag, unsigned char* b, int n_groups, float h, int64_t group0) {
+    constexpr bool kStochastic = decltype(stochastic_tag)::value;
+    constexpr bool kWhole = decltype(whole_tag)::value;
+    const bool fast = kStochastic && use_quotient_approx(&sr, a);
+    float4* p4 = reinterpret_cast<float4*>(b);
+    const int n_q = kWhole ? kTile / 4 : n_groups;
+#pragma unroll
+    for (int q = tid; q < n_q; q += kTmaThreads) {
+      float g0, g1, g2, g3;
+      if (kBF16) {
+        const uint2 w = reinterpret_cast<const uint2*>(b + kGOff)[q];
+        g0 = bf16_lo(w.x); g1 = bf16_hi(w.x); g2 = bf16_lo(w.y); g3 = bf16_hi(w.y);
+      } else {
+        const float4 w = reinterpret_cast<const float4*>(b + kGOff)[q];
+        g0 = w.x; g1 = w.y; g2 = w.z; g3 = w.w;
+      }
+      float4 p = p4[q], m = smem_state4<kSB>(b + kMOff, q), v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (kOpt == kOptAdamW) v = smem_state4<kSB>(b + kVOff, q);
+      adamw_vec4<kOpt>(g0, g1, g2, g3, h, p, m, v, a, fast);
+      p4[q] = p;
+      if (kStochastic) {  // elements 4q .. 4q+3 of this stage: one group of the arenas
+        const uint4 w = rounding_words(group0 + q, sr);
+        reinterpret_cast<uint2*>(b + kMOff)[q] = pack4_stochastic(m, w, 0);
+        if (kOpt == kOptAdamW) reinterpret_cast<uint2*>(b + kVOff)[q] = pack4_stochastic(v, w, 1);
+      } else {
+        smem_state4_store<kSB>(b + kMOff, q, m);
+        if (kOpt == kOptAdamW) smem_state4_store<kSB>(b + kVOff, q, v);
+      }
+      if (lowp) reinterpret_cast<uint2*>(b + kStageBytes)[q] = make_uint2(pack_bf16(p.x, p.y), pack_bf16(p.z, p.w));
+    }
   };
 
   bool healthy = true;
@@ -1229,38 +1350,9 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
       }
       unsigned char* b = tile_smem + static_cast<size_t>(s) * stage_stride;
       if (mbar_wait_bounded(&full_bar[s], phase)) {
-        float4* p4 = reinterpret_cast<float4*>(b);
-        // one copy of the loop per rounding mode, so that rounding to nearest carries none of the other mode's code
-        auto update_tile = [&](auto stochastic_tag) {
-          constexpr bool kStochastic = decltype(stochastic_tag)::value;
-          const bool fast = kStochastic && use_quotient_approx(&sr, a);
-#pragma unroll
-          for (int q = tid; q < kTile / 4; q += kTmaThreads) {
-            float g0, g1, g2, g3;
-            if (kBF16) {
-              const uint2 w = reinterpret_cast<const uint2*>(b + kGOff)[q];
-              g0 = bf16_lo(w.x); g1 = bf16_hi(w.x); g2 = bf16_lo(w.y); g3 = bf16_hi(w.y);
-            } else {
-              const float4 w = reinterpret_cast<const float4*>(b + kGOff)[q];
-              g0 = w.x; g1 = w.y; g2 = w.z; g3 = w.w;
-            }
-            float4 p = p4[q], m = smem_state4<kSB>(b + kMOff, q), v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (kOpt == kOptAdamW) v = smem_state4<kSB>(b + kVOff, q);
-            adamw_vec4<kOpt>(g0, g1, g2, g3, h, p, m, v, a, fast);
-            p4[q] = p;
-            if (kStochastic) {  // elements 4q .. 4q+3 of this tile: one group of the arenas
-              const uint4 w = rounding_words((chunk_start(ck) >> 2) + sub * (kTile / 4) + q, sr);
-              reinterpret_cast<uint2*>(b + kMOff)[q] = pack4_stochastic(m, w, 0);
-              if (kOpt == kOptAdamW) reinterpret_cast<uint2*>(b + kVOff)[q] = pack4_stochastic(v, w, 1);
-            } else {
-              smem_state4_store<kSB>(b + kMOff, q, m);
-              if (kOpt == kOptAdamW) smem_state4_store<kSB>(b + kVOff, q, v);
-            }
-            if (lowp) reinterpret_cast<uint2*>(b + kStageBytes)[q] = make_uint2(pack_bf16(p.x, p.y), pack_bf16(p.z, p.w));
-          }
-        };
-        if (kSB && sr.stochastic) update_tile(std::true_type{});
-        else update_tile(std::false_type{});
+        const int64_t group0 = (chunk_start(ck) >> 2) + sub * (kTile / 4);
+        if (kSB && sr.stochastic) update_tile(std::true_type{}, std::true_type{}, b, 0, h, group0);
+        else update_tile(std::false_type{}, std::true_type{}, b, 0, h, group0);
         fence_generic_to_async_smem();  // the updated tile must be visible to the bulk-copy engine
       } else {
         abort_flag = 1;  // this thread gave up; the barrier below tells every thread
@@ -1271,15 +1363,7 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
         j_fail = j;
         break;
       }
-      if (tid == 0) {
-        const int64_t e = chunk_start(ck) + static_cast<int64_t>(sub) * kTile;
-        bulk_store_hint(params + e, b, kTile * 4, stream_policy);
-        bulk_store_hint(static_cast<char*>(m_arena) + e * kSBytes, b + kMOff, kTile * kSBytes, stream_policy);
-        if (kOpt == kOptAdamW)
-          bulk_store_hint(static_cast<char*>(v_arena) + e * kSBytes, b + kVOff, kTile * kSBytes, stream_policy);
-        if (lowp) bulk_store_hint(lowp + e, b + kStageBytes, kTile * 2, stream_policy);
-        bulk_commit();
-      }
+      if (tid == 0) store_span(chunk_start(ck) + static_cast<int64_t>(sub) * kTile, kTile, b);
       if (last_of_chunk) {
         ck = ck_next;
         h = h_next;
@@ -1312,9 +1396,87 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
   }
   if (!healthy) return;
 
-  // partial chunks: table entry and clip factor are fetched one chunk ahead, so that a warp moving from one small
-  // chunk to the next never waits on two dependent loads with nothing else in flight
   if (mid >= end) return;
+
+  // ---- listed partial chunks: the same ring, continuing its stage and phase count after the n_tiles whole tiles.
+  // A chunk of n8 elements is cut into ceil(n8 / kTile) tiles of (nearly) equal length, each a multiple of 8.
+  if (kRingPartials && n_listed > 0) {
+    if (tid < n_listed) ring_tensor_or_h[tid] = __float_as_uint(h_arr[ring_tensor_or_h[tid]]);
+    __syncthreads();
+    struct Cursor {
+      int i, k, n_t, len, n8;  // listed chunk, tile within it, tiles of the chunk, tile length, elements of the chunk
+      int64_t e0;              // the chunk's first arena element
+    };
+    auto open_chunk = [&](Cursor& cu) {
+      cu.k = 0;
+      if (cu.i < n_listed) {
+        cu.n8 = ring_n8[cu.i];
+        cu.n_t = (cu.n8 + kTile - 1) / kTile;
+        cu.len = ((cu.n8 + cu.n_t - 1) / cu.n_t + 7) & ~7;
+        cu.e0 = static_cast<int64_t>(ring_start4[cu.i]) * 4;
+      }
+    };
+    auto next_tile = [&](Cursor& cu) {
+      if (++cu.k == cu.n_t) {
+        ++cu.i;
+        open_chunk(cu);
+      }
+    };
+    Cursor fetch{0, 0, 0, 0, 0, 0}, work{0, 0, 0, 0, 0, 0};  // thread 0's issue position; every thread's compute position
+    open_chunk(fetch);
+    open_chunk(work);
+    int issued = 0, done = 0;  // tiles of this phase (issued: thread 0 only)
+    auto issue_next = [&]() {
+      const int off = fetch.k * fetch.len;
+      issue_span(fetch.e0 + off, min(fetch.len, fetch.n8 - off), (n_tiles + issued) % kStages);
+      ++issued;
+      next_tile(fetch);
+    };
+    if (tid == 0)
+      for (int k = 0; k < kAhead && fetch.i < n_listed; ++k) issue_next();
+    while (work.i < n_listed) {
+      const int ring_pos = n_tiles + done;
+      const int s = ring_pos % kStages;
+      if (tid == 0 && fetch.i < n_listed) {
+        bulk_wait_smem_read();  // the stores of the previous tile have finished reading the stage that is refilled now
+        issue_next();
+      }
+      unsigned char* b = tile_smem + static_cast<size_t>(s) * stage_stride;
+      const int off = work.k * work.len;
+      const int n = min(work.len, work.n8 - off);
+      if (mbar_wait_bounded(&full_bar[s], (ring_pos / kStages) & 1)) {
+        const float h = __uint_as_float(ring_tensor_or_h[work.i]);
+        const int64_t group0 = (work.e0 + off) >> 2;
+        if (kSB && sr.stochastic) update_tile(std::true_type{}, std::false_type{}, b, n >> 2, h, group0);
+        else update_tile(std::false_type{}, std::false_type{}, b, n >> 2, h, group0);
+        fence_generic_to_async_smem();
+      } else {
+        abort_flag = 1;
+      }
+      __syncthreads();
+      if (abort_flag) {
+        healthy = false;
+        break;
+      }
+      if (tid == 0) store_span(work.e0 + off, n, b);
+      ++done;
+      next_tile(work);
+    }
+    if (tid == 0) {
+      bulk_wait_done();
+      if (!healthy) {
+        atomicOr(status, ADAGC_E_TIMEOUT);
+        for (int jj = n_tiles + done; jj < n_tiles + issued; ++jj)  // loads still in flight into this block's shared memory
+          (void)mbar_wait_bounded(&full_bar[jj % kStages], (jj / kStages) & 1);
+      }
+    }
+    __syncthreads();
+    if (!healthy) return;
+  }
+
+  // ---- what is left, on the register path: short chunks, entries past the listed range, and the last (count mod 8)
+  // elements of the listed chunks.  Table entry and clip factor are fetched one chunk ahead, so that a warp moving
+  // from one small chunk to the next never waits on two dependent loads with nothing else in flight.
   int row_base = 0;
   Chunk ck = chunks[mid];
   float h = h_arr[ck.tensor];
@@ -1325,7 +1487,13 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
       ck_next = chunks[c + 1];
       h_next = h_arr[ck_next.tensor];
     }
-    adamw_partial_chunk<kBF16, kTmaThreads, kOpt, kSB>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp, &sr);
+    const int n8 = ck.count & ~7;
+    if (kRingPartials && c < listed_end && n8 >= kRingMin) {  // listed: all but its ragged tail is done
+      ck.start4 += static_cast<uint32_t>(n8 >> 2);
+      ck.count -= n8;
+    }
+    if (ck.count > 0)
+      adamw_partial_chunk<kBF16, kTmaThreads, kOpt, kSB>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp, &sr);
     ck = ck_next;
     h = h_next;
   }

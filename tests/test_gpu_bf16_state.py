@@ -17,6 +17,8 @@ from test_gpu_parity import _ragged_workload, _report
 
 pytestmark = pytest.mark.gpu
 
+SEED = 0x5EED_0123_4567_89AB      # stochastic rounding of the stored moments
+
 SIZES = [1, 2, 3, 5, 7, 8, 9, 10, 15, 16, 17, 31, 33, 255, 257, 2047, 2049, 4095, 4096, 4097, 16383, 16384, 16385,
          32767, 32768, 32769, 3 * 16384 + 5, 100003, 40 * 16384, 9 * 16384 + 4095]
 
@@ -62,6 +64,21 @@ def test_lion_and_momentum_sgd_all_elements(optimizer, path):
                     H.run_bf16_state(wl, 8, optimizer=optimizer, flags=path))
 
 
+def test_more_partial_chunks_than_a_block_lists():
+    """45 000 tensors, so that every block of the bulk-async update kernel owns about 300 partial chunks: more than it
+    lists for its shared-memory ring.  One tensor in 40 is long enough to go through the ring (with a ragged tail that
+    does not); those among a block's later entries take the register path like the short ones.  Both rounding modes."""
+    sizes = [4100 + (i % 13) if i % 40 == 0 else 8 + (i % 29) for i in range(45000)]
+    sizes[7] = 16383           # a listed chunk of two tiles
+    sizes[11] = 3 * 16384 + 12000
+    wl = _ragged_workload(sizes, "f32")
+    _report("45000 tensors, bf16 state, same state every step",
+            H.run_bf16_state(wl, 3, teacher_forced=True, flags=binding.UPDATE_PATH_BULK))
+    _report("45000 tensors, bf16 state, free running", H.run_bf16_state(wl, 3, flags=binding.UPDATE_PATH_BULK))
+    _report("45000 tensors, bf16 state, stochastic rounding",
+            H.run_bf16_state(wl, 3, flags=binding.UPDATE_PATH_BULK, stochastic_seed=SEED))
+
+
 def test_gpt2_small_all_elements():
     """Config 2 at full size (124 M parameters), every element, 20 free-running steps across the warm-up switch."""
     wl = workloads.build("gpt2_small")
@@ -89,7 +106,6 @@ def test_llama2_7b_sampled():
 
 
 # ------------------------------------------------------------------ stochastic rounding of the stored moments
-SEED = 0x5EED_0123_4567_89AB
 
 
 @pytest.mark.parametrize("path", [binding.UPDATE_PATH_REGISTERS, binding.UPDATE_PATH_BULK, binding.FUSED_SMALL],

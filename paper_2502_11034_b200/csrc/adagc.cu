@@ -363,7 +363,7 @@ __device__ __forceinline__ double block_chunk_sumsq(const uint4* __restrict__ ve
 }
 
 template <bool kBF16>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 8)  // eight resident blocks per SM: the norm and scale grids are sized for that
 adagc_norm_kernel(const void* __restrict__ grads, const Chunk* __restrict__ chunks,
                   const int32_t* __restrict__ block_begin, double* __restrict__ partials, Guard guard) {
   __shared__ double warp_part[kThreads / 32];
@@ -965,30 +965,35 @@ __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, in
   constexpr int kWarps = kBlockThreads / 32;
   constexpr int kStateBytes = kSB ? 2 : 4;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int64_t start = chunk_start(ck);
   // Rows of 256 elements are laid from the last kRowAlign-element boundary at or before the chunk's start, so that a
   // warp's accesses fall on whole lines whatever the tensor's offset; the groups before the start are skipped.
-  const int pad = static_cast<int>(start & (kRowAlign - 1));  // a multiple of 8, like start
+  // A warp that gets no row of this chunk (most warps, for a short chunk) leaves after these few integer operations.
+  const int pad = static_cast<int>(ck.start4 & (kRowAlign / 4 - 1)) << 2;  // a multiple of 8, like the start
+  const int first8 = pad >> 3, n8 = ck.count >> 3;
+  const int rows = (first8 + n8 + 31) >> 5;
+  const int r0 = (warp - row_base) & (kWarps - 1);
+  row_base = (row_base + rows) & (kWarps - 1);
+  const bool has_tail = warp == row_base && (ck.count & 7) != 0;  // the next warp in turn takes the ragged tail
+  if (r0 >= rows && !has_tail) return;
+  const int64_t start = chunk_start(ck);
   const int64_t origin = start - pad;
   float4* __restrict__ p4 = reinterpret_cast<float4*>(params + origin);
   char* __restrict__ mbase = static_cast<char*>(m_arena) + origin * kStateBytes;
   char* __restrict__ vbase = kOpt == kOptAdamW ? static_cast<char*>(v_arena) + origin * kStateBytes : nullptr;
   const char* __restrict__ gbase = static_cast<const char*>(grads) + origin * (kBF16 ? 2 : 4);
-  const int first8 = pad >> 3, n8 = ck.count >> 3;
-  const int rows = (first8 + n8 + 31) >> 5;
 #pragma unroll 2
-  for (int r = (warp - row_base) & (kWarps - 1); r < rows; r += kWarps) {
+  for (int r = r0; r < rows; r += kWarps) {
     const int i = (r << 5) + lane;
     if (i >= first8 && i < first8 + n8)
       adamw_group8<kBF16, kOpt, kSB>(i, gbase, p4, mbase, vbase, h, a, lowp ? reinterpret_cast<uint4*>(lowp + origin) : nullptr,
                                      sr, origin >> 2);
   }
-  row_base = (row_base + rows) & (kWarps - 1);
-  gbase += static_cast<int64_t>(pad) * (kBF16 ? 2 : 4);  // the tail below counts from the chunk's start
+  if (!has_tail) return;
+  gbase += static_cast<int64_t>(pad) * (kBF16 ? 2 : 4);  // the tail counts from the chunk's start
   mbase += static_cast<int64_t>(pad) * kStateBytes;
   if (kOpt == kOptAdamW) vbase += static_cast<int64_t>(pad) * kStateBytes;
-  const int t = (n8 << 3) + lane;  // ragged tail (fewer than 8 elements): the next warp in turn takes it
-  if (warp == row_base && t < ck.count) {
+  const int t = (n8 << 3) + lane;  // ragged tail: fewer than 8 elements
+  if (t < ck.count) {
     float g;
     if (kBF16) {
       g = __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const uint16_t*>(gbase)[t]) << 16);

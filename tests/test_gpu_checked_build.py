@@ -33,6 +33,8 @@ for dtype in ("f32", "bf16"):
     H.run_full_sharded(wl, 4, 3)
 wl = workloads.build("many_small", n_tensors=3000, lo=16, hi=40000)
 H.run_full(wl, 6, hyper_over=dict(lambda_abs=1e4))
+H.run_bf16_state(wl, 3, teacher_forced=True, hyper_over=dict(lambda_abs=1e4))   # partial chunks through the ring
+H.run_bf16_state(wl, 3, hyper_over=dict(lambda_abs=1e4), stochastic_seed=5)
 H.run_full(workloads.build("tiny"), 12)
 print("checked build ok")
 """

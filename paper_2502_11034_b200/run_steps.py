@@ -2,7 +2,10 @@
 
     python -m paper_2502_11034_b200.run_steps --workload gpt2_small --steps 4 [--mode step|clip|lion|sgdm] [--n-layer N]
         [--update-path auto|registers|bulk] [--fused-small] [--state f32|bf16 [--stochastic-seed S]] [--separate-finalize]
-        [--group-mb X [--graph]]
+        [--group-mb X [--graph]] [--equal-tensors N SIZE [--grad-dtype f32|bf16]]
+
+--equal-tensors N SIZE replaces the named layout by N tensors of SIZE elements each (normal gradients): the layouts
+on which the cost per chunk of the norm and update kernels is measured against the tensor size.
 
 A minimal driver of the C ABI (adagc_create / adagc_step / adagc_clip / adagc_get_stats): useful as
 an example and as a small, short-running target for profilers.  Prints the per-phase device times.
@@ -39,11 +42,20 @@ def main():
     ap.add_argument("--state", choices=["f32", "bf16"], default="f32", help="dtype of the m and v arenas (adagc_desc.state_dtype)")
     ap.add_argument("--stochastic-seed", type=int, default=None,
                     help="with --state bf16: round the stored moments stochastically (adagc_set_state_rounding)")
+    ap.add_argument("--equal-tensors", type=int, nargs=2, metavar=("N", "SIZE"), default=None,
+                    help="a layout of N tensors of SIZE elements instead of --workload")
+    ap.add_argument("--grad-dtype", choices=["f32", "bf16"], default="f32", help="gradient dtype of --equal-tensors")
     ap.add_argument("--separate-finalize", action="store_true",
                     help="ADAGC_SEPARATE_FINALIZE: the per-tensor decisions of AdaGC steps in a kernel of their own")
     args = ap.parse_args()
     over = {} if args.n_layer is None else {"n_layer": args.n_layer}
-    wl = workloads.build(args.workload, **over)
+    if args.equal_tensors is not None:
+        n, size = args.equal_tensors
+        specs, total = workloads._layout([(f"t{i}", (size,)) for i in range(n)])
+        wl = workloads.Workload(f"{n}x{size}", 0, specs, args.grad_dtype, dict(workloads.PAPER_DEFAULTS), warmup=args.warmup,
+                                n_steps=args.steps, arena_elems=total)
+    else:
+        wl = workloads.build(args.workload, **over)
     hp = wl.hyper
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)

@@ -534,6 +534,15 @@ def run_ours(args, wl):
                 torch.cuda.empty_cache()
                 per_config[name] = time_layout(binding, workloads, workloads.build(name), dev, 20, 5,
                                                fused_small=(name == "tiny"))
+            for name in ("moe_8x1b", "moe_ernie"):      # expert-parallel-shaped layouts: 747 and 3828 tensors
+                torch.cuda.empty_cache()
+                wl_x = workloads.build(name)
+                need = wl_x.arena_elems * 14 + (6 << 30)       # theta, m, v, bf16 g, and room for the generator's scratch
+                free, _ = torch.cuda.mem_get_info()
+                if free < need:
+                    per_config[name] = {"skipped": f"needs {need >> 30} GiB of free device memory, {free >> 30} GiB free"}
+                else:
+                    per_config[name] = time_layout(binding, workloads, wl_x, dev, 5, 3)
             extra["per_config"] = per_config
 
     if rank == 0:

@@ -312,7 +312,9 @@ __device__ __forceinline__ void sq_acc_rounds(const uint4* __restrict__ vec, int
   for (int u = 0; u < kRounds; ++u) sq_acc_vec<kBF16>(q[u], acc0, acc1);
 }
 
-template <bool kBF16, bool kKeepInL2 = false>
+// kTrailingBarrier = false leaves the second barrier out: the caller then alternates between two `warp_part` arrays
+// from one call to the next (thread 0 reads one while the other warps already fill the other for the next chunk).
+template <bool kBF16, bool kKeepInL2 = false, bool kTrailingBarrier = true>
 __device__ __forceinline__ double block_chunk_sumsq(const uint4* __restrict__ vec, int count, double* warp_part) {
   constexpr int kEPV = kBF16 ? 8 : 4;  // elements per 16-byte vector
   const int tid = threadIdx.x;
@@ -358,29 +360,116 @@ __device__ __forceinline__ double block_chunk_sumsq(const uint4* __restrict__ ve
 #pragma unroll
     for (int k = 1; k < kThreads / 32; ++k) s += warp_part[k];
   }
-  __syncthreads();
+  if (kTrailingBarrier) __syncthreads();
   return s;
+}
+
+// A chunk of at most kThreads vectors gives every thread of block_chunk_sumsq at most one vector, so a single warp can
+// stand in for the whole block with identical bits: in turn k it plays the block's warp k (lane l is thread 32 k + l:
+// its one vector, then -- thread < 8 only -- its element of the ragged tail), takes that warp's shuffle-tree total, and
+// adds the totals in warp order.  Warps of the block that hold no data contribute an exact +0 and are left out.
+// The norm kernels hand such chunks to their warps one each (no block barrier, eight chunks in flight per block): with
+// one short chunk at a time per block they are bound by the latency of a chunk, not by memory.
+template <bool kBF16>
+__device__ __forceinline__ bool warp_sized_chunk(int count) { return count / (kBF16 ? 8 : 4) <= kThreads; }
+
+template <bool kBF16, bool kKeepInL2>
+__device__ __forceinline__ double warp_chunk_sumsq(const uint4* __restrict__ vec, int count) {
+  constexpr int kEPV = kBF16 ? 8 : 4;
+  const int lane = threadIdx.x & 31;
+  const int nvec = count / kEPV;  // <= kThreads
+  const int turns = max(1, (nvec + 31) >> 5);
+  const uint64_t keep = kKeepInL2 ? l2_policy_evict_last() : 0ull;
+  double total = 0.0;
+#pragma unroll 1
+  for (int k0 = 0; k0 < turns; k0 += 4) {  // four turns' loads in flight at a time
+    uint4 q[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = 32 * (k0 + u) + lane;
+      q[u] = i < nvec ? (kKeepInL2 ? ld_nc_l2_hint(vec + i, keep) : __ldg(vec + i)) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int k = k0 + u;
+      if (k >= turns) break;  // uniform
+      double acc0 = 0.0, acc1 = 0.0;
+      if (32 * k + lane < nvec) sq_acc_vec<kBF16>(q[u], acc0, acc1);
+      if (k == 0) {
+        const int t = nvec * kEPV + lane;
+        if (t < count) {
+          const float x = kBF16 ? __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const uint16_t*>(vec)[t]) << 16)
+                                : reinterpret_cast<const float*>(vec)[t];
+          acc0 = sq_acc(acc0, x);
+        }
+      }
+      const double w = warp_sum(acc0 + acc1);
+      total = k == 0 ? w : total + w;
+    }
+  }
+  return total;
+}
+
+// The warp-sized chunks among the table entries [lo, hi), dealt to the block's warps in turn; lane 0 of the warp that
+// summed entry c stores the sum at partials[c] (kIndexIsEntry: the table is in chunk order) or at the entry's partial
+// index.  Not inlined: the streaming loop of the calling kernel keeps its register allocation to itself.
+template <bool kBF16, bool kIndexIsEntry>
+__device__ __noinline__ void sum_warp_sized_chunks(const void* __restrict__ grads, const Chunk* __restrict__ chunks, int lo,
+                                                   int hi, double* __restrict__ partials) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int seen = 0;  // warp-sized chunks before `base`
+  for (int base = lo; base < hi; base += 32) {
+    Chunk e{0u, 0, 0, 0};
+    bool mine_is_small = false;
+    if (base + lane < hi) {
+      e = chunks[base + lane];
+      mine_is_small = warp_sized_chunk<kBF16>(e.count);
+    }
+    const unsigned small = __ballot_sync(0xffffffffu, mine_is_small);
+    for (unsigned rest = small; rest != 0; rest &= rest - 1) {  // uniform over the warp
+      const int j = __ffs(rest) - 1;
+      const int rank = seen + __popc(small & ((1u << j) - 1u));
+      if ((rank & (kThreads / 32 - 1)) != warp) continue;
+      const uint32_t start4 = __shfl_sync(0xffffffffu, e.start4, j);
+      const int count = __shfl_sync(0xffffffffu, e.count, j);
+      const int partial = __shfl_sync(0xffffffffu, e.partial, j);
+      const uint4* vec = reinterpret_cast<const uint4*>(static_cast<const char*>(grads) +
+                                                        static_cast<int64_t>(start4) * 4 * (kBF16 ? 2 : 4));
+      const double s = warp_chunk_sumsq<kBF16, true>(vec, count);
+      if (lane == 0) partials[kIndexIsEntry ? base + j : partial] = s;
+    }
+    seen += __popc(small);
+  }
 }
 
 template <bool kBF16>
 __global__ void __launch_bounds__(kThreads, 8)  // eight resident blocks per SM: the norm and scale grids are sized for that
 adagc_norm_kernel(const void* __restrict__ grads, const Chunk* __restrict__ chunks,
                   const int32_t* __restrict__ block_begin, double* __restrict__ partials, Guard guard) {
-  __shared__ double warp_part[kThreads / 32];
+  __shared__ double warp_part[2][kThreads / 32];  // alternating from chunk to chunk: one barrier per chunk
   const int c_begin = block_begin[blockIdx.x], c_end = block_begin[blockIdx.x + 1];
   ADAGC_CHECK_ENTRIES(chunks, c_begin, c_end, guard);
   if (c_begin >= c_end) return;
   Chunk ck = chunks[c_begin];
+  int flip = 0;
+  bool any_warp_sized = false;
   for (int c = c_begin; c < c_end; ++c) {
     // the next table entry is fetched while this chunk streams: a block of many small chunks would otherwise wait for
     // a dependent load before every chunk's first gradient load
     const Chunk ck_next = c + 1 < c_end ? chunks[c + 1] : ck;
-    const uint4* vec =
-        reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + chunk_start(ck) * (kBF16 ? 2 : 4));
-    const double s = block_chunk_sumsq<kBF16, true>(vec, ck.count, warp_part);
-    if (threadIdx.x == 0) partials[ck.partial] = s;
+    if (warp_sized_chunk<kBF16>(ck.count)) {
+      any_warp_sized = true;  // left to the warps below
+    } else {
+      const uint4* vec =
+          reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + chunk_start(ck) * (kBF16 ? 2 : 4));
+      const double s = block_chunk_sumsq<kBF16, true, false>(vec, ck.count, warp_part[flip]);
+      flip ^= 1;
+      if (threadIdx.x == 0) partials[ck.partial] = s;
+    }
     ck = ck_next;
   }
+  if (any_warp_sized)
+    sum_warp_sized_chunks<kBF16, false>(grads, chunks, c_begin, c_end, partials);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -561,7 +650,7 @@ adagc_norm_decide_kernel(const void* __restrict__ grads, const Chunk* __restrict
                          const int32_t* __restrict__ range_begin, double* partials,
                          const TensorEntry* __restrict__ tensors, unsigned int* tickets, ClipScalars cs,
                          float* __restrict__ ema, StatPtrs st, Guard guard) {
-  __shared__ double warp_part[kThreads / 32];
+  __shared__ double warp_part[2][kThreads / 32];  // alternating from chunk to chunk: one barrier per chunk
   __shared__ int done_list[kDoneListMax];
   __shared__ int n_done;
   griddep_launch_dependents();  // the update kernel may be staged now; it waits for this grid before it needs h
@@ -569,19 +658,26 @@ adagc_norm_decide_kernel(const void* __restrict__ grads, const Chunk* __restrict
   ADAGC_CHECK_ENTRIES(chunks, lo, hi, guard);
   if (lo >= hi) return;
   Chunk ck = chunks[lo];  // original order: entry c is chunk c, its partial is partials[c]
-  const int t_first = ck.tensor;
-  int t_last = t_first;
+  int flip = 0;
+  bool any_warp_sized = false;
   for (int c = lo; c < hi; ++c) {
     const Chunk ck_next = c + 1 < hi ? chunks[c + 1] : ck;  // one entry ahead, as in adagc_norm_kernel
-    const uint4* vec =
-        reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + chunk_start(ck) * (kBF16 ? 2 : 4));
-    const double s = block_chunk_sumsq<kBF16, true>(vec, ck.count, warp_part);
-    if (threadIdx.x == 0) partials[c] = s;
-    t_last = ck.tensor;
+    if (warp_sized_chunk<kBF16>(ck.count)) {
+      any_warp_sized = true;  // left to the warps below
+    } else {
+      const uint4* vec =
+          reinterpret_cast<const uint4*>(static_cast<const char*>(grads) + chunk_start(ck) * (kBF16 ? 2 : 4));
+      const double s = block_chunk_sumsq<kBF16, true, false>(vec, ck.count, warp_part[flip]);
+      flip ^= 1;
+      if (threadIdx.x == 0) partials[c] = s;
+    }
     ck = ck_next;
   }
+  if (any_warp_sized)
+    sum_warp_sized_chunks<kBF16, true>(grads, chunks, lo, hi, partials);
+  const int t_first = chunks[lo].tensor, t_last = chunks[hi - 1].tensor;  // tensors with chunks in this block
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (threadIdx.x == 0) __threadfence();  // this block's partials are visible device-wide before any ticket is
+  if (lane == 0) __threadfence();  // this block's partials (written by lane 0 of its warps) are visible device-wide before any ticket is
   for (int t0 = t_first; t0 <= t_last; t0 += kDoneListMax) {  // (one round, unless a block holds over a thousand tensors)
     const int t1 = min(t_last, t0 + kDoneListMax - 1);
     if (threadIdx.x == 0) n_done = 0;
@@ -600,11 +696,22 @@ adagc_norm_decide_kernel(const void* __restrict__ grads, const Chunk* __restrict
     __syncthreads();
     __threadfence();  // (the partials of the other blocks are read below)
     const int n = n_done;
-    // tensors of a few chunks: one warp each; tensors with very many chunks: the whole block, one after the other
+    // tensors of one chunk: a thread each (the fixed-order sum of a single partial is that partial, and a layout of
+    // many small tensors would otherwise queue their decisions -- three dependent memory round trips each -- behind one
+    // another in eight warps); tensors of a few chunks: one warp each; tensors with very many chunks: the whole block
+    for (int k = threadIdx.x; k < n; k += kThreads) {
+      const int t = done_list[k];
+      const TensorEntry te = tensors[t];
+      if (te.n_chunks != 1) continue;
+      const double total = __ldcg(partials + te.first_chunk);
+      st.sumsq[t] = total;
+      adagc_decide(t, total, cs, ema, st);
+      if (t == 0) *st.steps_done += 1ull;
+    }
     for (int k = warp; k < n; k += kThreads / 32) {
       const int t = done_list[k];
       const TensorEntry te = tensors[t];
-      if (te.n_chunks >= kBigTensorChunks) continue;
+      if (te.n_chunks == 1 || te.n_chunks >= kBigTensorChunks) continue;
       const double total = tensor_partial_sum(partials, te, lane);
       if (lane == 0) {
         st.sumsq[t] = total;
@@ -616,7 +723,7 @@ adagc_norm_decide_kernel(const void* __restrict__ grads, const Chunk* __restrict
       const int t = done_list[k];
       const TensorEntry te = tensors[t];
       if (te.n_chunks < kBigTensorChunks) continue;
-      const double total = tensor_partial_sum_block(partials, te, warp_part);
+      const double total = tensor_partial_sum_block(partials, te, warp_part[0]);
       if (threadIdx.x == 0) {
         st.sumsq[t] = total;
         adagc_decide(t, total, cs, ema, st);

@@ -64,9 +64,22 @@ def test_sharded_global_adaptive_variant():
     assert rep.steps == 10
 
 
-def test_one_rank_equals_the_unsharded_entry_bit_for_bit():
-    """With a single rank the three calls compute exactly what adagc_step computes."""
-    wl = workloads.build("gpt2_small", n_layer=2, d=96, vocab=1031, n_pos=64)
+# sizes around the largest chunk that one warp of the norm kernels sums by itself (256 vectors of 16 bytes: 1024 fp32 or
+# 2048 bfloat16 elements, plus a ragged tail), and a few tiny ones
+WARP_SIZED_EDGE = [1, 3, 4, 5, 8, 31, 33, 1020, 1023, 1024, 1025, 1027, 1028, 1031, 2040, 2047, 2048, 2049, 2055, 2056,
+                   16384 + 1024, 16384 + 1028, 16384 + 2055, 16384 + 2056]
+
+
+@pytest.mark.parametrize("layout", ["gpt2_small", "edge_f32", "edge_bf16"])
+def test_one_rank_equals_the_unsharded_entry_bit_for_bit(layout):
+    """With a single rank the three calls compute exactly what adagc_step computes.  The per-chunk sums of the sharded
+    path come from a kernel that puts a whole block on every chunk, those of adagc_step from the norm kernel that hands
+    short chunks to single warps: the bits must not depend on which of the two summed a chunk."""
+    if layout == "gpt2_small":
+        wl = workloads.build("gpt2_small", n_layer=2, d=96, vocab=1031, n_pos=64)
+    else:
+        from test_gpu_parity import _ragged_workload
+        wl = _ragged_workload(WARP_SIZED_EDGE, layout[5:])
     hp = H.hyper_of(wl, lambda_abs=1e4)
     offs, nums = [t.offset for t in wl.tensors], [t.numel for t in wl.tensors]
     res = []

@@ -1062,8 +1062,30 @@ __device__ __forceinline__ void adamw_group8(int i, const char* __restrict__ gba
 // elements) and the rows of successive chunks go to the block's warps in one continuing round-robin:
 // row_base counts the rows dealt so far.  Restarting at warp 0 for every chunk would give the low warps
 // the extra rows every time and make them the critical path.
+// One element at arena index e, with scalar accesses (the last count mod 8 elements of a chunk).
+template <bool kBF16, int kOpt, bool kSB>
+__device__ __forceinline__ void adamw_single(int64_t e, float h, float* __restrict__ params, const void* __restrict__ grads,
+                                             void* __restrict__ m_arena, void* __restrict__ v_arena, const AdamScalars& a,
+                                             uint16_t* __restrict__ lowp, const StateRounding* sr) {
+  const float g = kBF16 ? __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(grads)[e]) << 16)
+                        : static_cast<const float*>(grads)[e];
+  float p = params[e], m = load_state1<kSB>(m_arena, e), v = 0.0f;
+  if (kOpt == kOptAdamW) v = load_state1<kSB>(v_arena, e);
+  adamw_elem<kOpt>(g, h, p, m, v, a, kSB && use_quotient_approx(sr, a));
+  params[e] = p;
+  if (kSB && sr && sr->stochastic) {
+    store_state1_stochastic(m_arena, e, m, e, *sr, 0);
+    if (kOpt == kOptAdamW) store_state1_stochastic(v_arena, e, v, e, *sr, 1);
+  } else {
+    store_state1<kSB>(m_arena, e, m);
+    if (kOpt == kOptAdamW) store_state1<kSB>(v_arena, e, v);
+  }
+  if (lowp) lowp[e] = static_cast<uint16_t>(f32_to_bf16_bits(p));
+}
+
+// kWithTail = false leaves the chunk's last count mod 8 elements to the caller.
 constexpr int kRowAlign = 256;  // elements
-template <bool kBF16, int kBlockThreads, int kOpt, bool kSB>
+template <bool kBF16, int kBlockThreads, int kOpt, bool kSB, bool kWithTail = true>
 __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, int& row_base, float* __restrict__ params,
                                                     const void* __restrict__ grads, void* __restrict__ m_arena,
                                                     void* __restrict__ v_arena, const AdamScalars& a,
@@ -1080,7 +1102,7 @@ __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, in
   const int rows = (first8 + n8 + 31) >> 5;
   const int r0 = (warp - row_base) & (kWarps - 1);
   row_base = (row_base + rows) & (kWarps - 1);
-  const bool has_tail = warp == row_base && (ck.count & 7) != 0;  // the next warp in turn takes the ragged tail
+  const bool has_tail = kWithTail && warp == row_base && (ck.count & 7) != 0;  // the next warp in turn takes the ragged tail
   if (r0 >= rows && !has_tail) return;
   const int64_t start = chunk_start(ck);
   const int64_t origin = start - pad;
@@ -1096,30 +1118,8 @@ __device__ __forceinline__ void adamw_partial_chunk(const Chunk& ck, float h, in
                                      sr, origin >> 2);
   }
   if (!has_tail) return;
-  gbase += static_cast<int64_t>(pad) * (kBF16 ? 2 : 4);  // the tail counts from the chunk's start
-  mbase += static_cast<int64_t>(pad) * kStateBytes;
-  if (kOpt == kOptAdamW) vbase += static_cast<int64_t>(pad) * kStateBytes;
   const int t = (n8 << 3) + lane;  // ragged tail: fewer than 8 elements
-  if (t < ck.count) {
-    float g;
-    if (kBF16) {
-      g = __uint_as_float(static_cast<uint32_t>(reinterpret_cast<const uint16_t*>(gbase)[t]) << 16);
-    } else {
-      g = reinterpret_cast<const float*>(gbase)[t];
-    }
-    float p = params[start + t], m = load_state1<kSB>(mbase, t), v = 0.0f;
-    if (kOpt == kOptAdamW) v = load_state1<kSB>(vbase, t);
-    adamw_elem<kOpt>(g, h, p, m, v, a, kSB && use_quotient_approx(sr, a));
-    params[start + t] = p;
-    if (kSB && sr && sr->stochastic) {
-      store_state1_stochastic(mbase, t, m, start + t, *sr, 0);
-      if (kOpt == kOptAdamW) store_state1_stochastic(vbase, t, v, start + t, *sr, 1);
-    } else {
-      store_state1<kSB>(mbase, t, m);
-      if (kOpt == kOptAdamW) store_state1<kSB>(vbase, t, v);
-    }
-    if (lowp) lowp[start + t] = static_cast<uint16_t>(f32_to_bf16_bits(p));
-  }
+  if (t < ck.count) adamw_single<kBF16, kOpt, kSB>(start + t, h, params, grads, m_arena, v_arena, a, lowp, sr);
 }
 
 // Register-streaming update kernel: every thread loads eight elements of each stream into registers.
@@ -1599,15 +1599,22 @@ adagc_update_tma_kernel(float* __restrict__ params, const void* __restrict__ gra
       ck_next = chunks[c + 1];
       h_next = h_arr[ck_next.tensor];
     }
-    const int n8 = ck.count & ~7;
-    if (kRingPartials && c < listed_end && n8 >= kRingMin) {  // listed: all but its ragged tail is done
-      ck.start4 += static_cast<uint32_t>(n8 >> 2);
-      ck.count -= n8;
-    }
-    if (ck.count > 0)
-      adamw_partial_chunk<kBF16, kTmaThreads, kOpt, kSB>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp, &sr);
+    const bool listed = kRingPartials && c < listed_end && (ck.count & ~7) >= kRingMin;  // done but for its ragged tail
+    if (!listed)
+      adamw_partial_chunk<kBF16, kTmaThreads, kOpt, kSB, false>(ck, h, row_base, params, grads, m_arena, v_arena, a, lowp, &sr);
     ck = ck_next;
     h = h_next;
+  }
+  // The ragged tails (count mod 8 elements) of all partial chunks, four chunks per warp at a time: lane l takes
+  // element l mod 8 of the tail of entry c0 + l / 8.  One at a time, each tail would cost its warp a memory latency.
+  const int warp = tid >> 5, lane = tid & 31;
+  for (int c0 = mid + warp * 4; c0 < end; c0 += (kTmaThreads / 32) * 4) {
+    const int c = c0 + (lane >> 3);
+    if (c >= end) continue;
+    const Chunk tc = chunks[c];
+    if ((lane & 7) < (tc.count & 7))
+      adamw_single<kBF16, kOpt, kSB>(chunk_start(tc) + (tc.count & ~7) + (lane & 7), h_arr[tc.tensor], params, grads, m_arena,
+                                     v_arena, a, lowp, &sr);
   }
 }
 

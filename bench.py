@@ -48,11 +48,11 @@ NOMINAL_HBM_GBS = 8000.0
 # parameter count because the traffic of this streaming kernel grows in proportion.  None once a kernel has changed
 # since its capture.
 TRAFFIC_BYTES_PER_PARAM = {   # (gradient dtype, state dtype) -> (bytes per parameter, capture)
-    ("bf16", "f32"): ((1742.340e6 + 1435.758e6) / 124439808,
+    ("bf16", "f32"): ((1742.350e6 + 1434.920e6) / 124439808,
                       "profiles/adagc_kernels_gpt2_small_ncu_full.md (GPT-2-small-shaped layout, scaled by N)"),
-    ("bf16", "bf16"): ((1244.601e6 + 938.283e6) / 124439808,
+    ("bf16", "bf16"): ((1244.628e6 + 937.533e6) / 124439808,
                        "profiles/adagc_kernels_gpt2_small_ncu_full.md (GPT-2-small-shaped layout, bfloat16 state, scaled by N)"),
-    ("f32", "f32"): ((3070.694e6 + 2242.556e6) / 191408576,
+    ("f32", "f32"): ((3077.705e6 + 2248.135e6) / 191408576,
                      "profiles/adagc_kernels_many_small_ncu_full.md (20 000 small tensors, scaled by N)"),
 }
 

@@ -355,6 +355,13 @@ int adagc_set_state_rounding(adagc_ctx* ctx, int32_t mode, uint64_t seed);
 /* The update path this context uses: ADAGC_UPDATE_PATH_REGISTERS or ADAGC_UPDATE_PATH_BULK. */
 int adagc_update_path(const adagc_ctx* ctx);
 
+/* Thread blocks that this context launches for its norm / scale kernels (*norm_grid: eight per SM, fewer when the
+ * layout has fewer chunks) and for its update kernel (*update_grid: one per SM on the bulk-async path, two on the
+ * register path).  The kernels' memory behaviour was tuned for exactly these residencies (the paper has no counterpart;
+ * the tests use this to notice a kernel whose register count no longer admits its grid).  Either pointer may be NULL.
+ * Returns ADAGC_OK or ADAGC_E_INVALID_ARG (NULL context). */
+int adagc_launch_grids(const adagc_ctx* ctx, int32_t* norm_grid, int32_t* update_grid);
+
 /* Elements spanned by the arenas: max over tensors of offset + numel. */
 int64_t adagc_arena_elems(const adagc_ctx* ctx);
 

@@ -95,6 +95,8 @@ def lib() -> C.CDLL:
     L.adagc_set_state_rounding.argtypes = [vp, C.c_int32, C.c_uint64]
     L.adagc_update_path.restype = C.c_int
     L.adagc_update_path.argtypes = [vp]
+    L.adagc_launch_grids.restype = C.c_int
+    L.adagc_launch_grids.argtypes = [vp, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     L.adagc_arena_elems.restype = i64
     L.adagc_arena_elems.argtypes = [vp]
     L.adagc_launch_count.restype = C.c_uint64
@@ -370,6 +372,14 @@ class AdaGC:
 
     def launch_count(self) -> int:
         return int(lib().adagc_launch_count(self._h))
+
+    def launch_grids(self):
+        """adagc_launch_grids: (blocks of the norm / scale kernels, blocks of the update kernel)."""
+        n, u = C.c_int32(), C.c_int32()
+        rc = lib().adagc_launch_grids(self._h, C.byref(n), C.byref(u))
+        if rc != 0:
+            raise AdagcError(rc, "adagc_launch_grids")
+        return int(n.value), int(u.value)
 
     def set_phase_timing(self, enabled: bool):
         rc = lib().adagc_set_phase_timing(self._h, 1 if enabled else 0)

@@ -2942,6 +2942,13 @@ int adagc_update_path(const adagc_ctx* ctx) {
   return ctx->update_bulk ? ADAGC_UPDATE_PATH_BULK : ADAGC_UPDATE_PATH_REGISTERS;
 }
 
+int adagc_launch_grids(const adagc_ctx* ctx, int32_t* norm_grid, int32_t* update_grid) {
+  if (!ctx) return ADAGC_E_INVALID_ARG;
+  if (norm_grid) *norm_grid = ctx->grid_wide;
+  if (update_grid) *update_grid = ctx->grid_update;
+  return ADAGC_OK;
+}
+
 int64_t adagc_arena_elems(const adagc_ctx* ctx) { return ctx ? ctx->arena_elems : ADAGC_E_INVALID_ARG; }
 
 uint64_t adagc_launch_count(const adagc_ctx* ctx) { return ctx ? ctx->launches : 0; }

@@ -334,6 +334,24 @@ def test_decisions_in_the_norm_tail_and_in_their_own_kernel(where):
         assert torch.equal(x, y)                                   # bit-identical wherever the decisions are taken
 
 
+def test_launch_grids_match_the_residency_the_kernels_are_tuned_for():
+    """Eight resident 256-thread blocks per SM for the norm / scale kernels, one block per SM for the bulk-async update
+    kernel and two for the register one: a kernel whose register count stops admitting that (the occupancy query at
+    adagc_create then sizes a smaller grid) shows here, not only in a timing."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    wl = workloads.build("gpt2_small", n_layer=4, d=768, vocab=4096, n_pos=64)      # about two thousand chunks
+    offs, nums = [t.offset for t in wl.tensors], [t.numel for t in wl.tensors]
+    for state in (torch.float32, torch.bfloat16):
+        for flags, per_sm in ((binding.UPDATE_PATH_BULK, 1), (binding.UPDATE_PATH_REGISTERS, 2), (0, 1)):
+            opt = binding.AdaGC(nums, offs, wl.torch_grad_dtype, 1.0, flags=flags, state_dtype=state)
+            assert opt.launch_grids() == (8 * sms, per_sm * sms)
+            opt.close()
+    small = binding.AdaGC([100, 20000], [0, 104], torch.float32, 1.0)              # three chunks: one block each
+    assert small.launch_grids() == (3, 3)
+    small.close()
+    assert binding.lib().adagc_launch_grids(None, None, None) == -1
+
+
 def test_single_tensor_and_warmup_zero():
     """T = 1 (the 'global adaptive' view) and T_start = 0 (gamma seeded from the first norm)."""
     wl = _ragged_workload([50000], "bf16")

@@ -1,4 +1,5 @@
-"""Build step: compile csrc/adagc.cu into libadagc.so (next to this file) for sm_100a."""
+"""Build step: compile csrc/adagc.cu (one translation unit; it includes the other files of csrc/) into libadagc.so
+(next to this file) for sm_100a."""
 from __future__ import annotations
 
 import os
@@ -28,7 +29,8 @@ def build(force: bool = False, verbose: bool = False, checked: bool = False) -> 
     checked: the debugging build (-DADAGC_BOUNDS_CHECK, libadagc_checked.so) whose kernels verify every chunk-table entry
     before they use it; select it at run time with ADAGC_LIBRARY=<path>."""
     lib = LIB_CHECKED if checked else LIB
-    newest = max(os.path.getmtime(SRC), os.path.getmtime(HEADER))
+    csrc = os.path.dirname(SRC)
+    newest = max([os.path.getmtime(HEADER)] + [os.path.getmtime(os.path.join(csrc, f)) for f in os.listdir(csrc)])
     if not force and os.path.exists(lib) and os.path.getmtime(lib) >= newest:
         return lib
     cmd = ([nvcc_path()] + NVCC_FLAGS + (["-DADAGC_BOUNDS_CHECK"] if checked else []) +
